@@ -1,0 +1,293 @@
+"""Seeded synthetic ID streams shaped like the workloads of the Monolith paper.
+
+This module only *draws inputs* (feature IDs, bag offsets, pooled gradients).
+It holds none of the table's arithmetic: no hashing into buckets, no counting,
+no pooling, no optimizer.  Both the CPU oracle's tests and the CUDA path's
+tests read the arrays it returns, so the two sides see identical inputs.
+
+Shape of the inputs (Section 2.1 of the paper, observations 1 and 2):
+IDs are long-tail distributed (popular IDs occur orders of magnitude more often
+than unpopular ones), come from a huge sparse space (2^48 in Section 3.1), and
+new IDs keep arriving while old ones go stale.  The paper's own datasets
+(MovieLens, Criteo, the internal one) are not reproduced; bounded Zipf ranks
+mixed into random 64-bit patterns stand in for them.
+
+A *bag* is one (example, feature slot) pair.  A step's IDs are laid out CSR
+style: bag b owns ids[offsets[b]:offsets[b+1]].
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Iterator, Optional
+
+import numpy as np
+
+_MASK64 = np.uint64(0xFFFFFFFFFFFFFFFF)
+RESERVED_ID = 0xFFFFFFFFFFFFFFFF
+
+
+def splitmix64(x: np.ndarray) -> np.ndarray:
+    """SplitMix64 output function (Steele, Lea, Flood 2014) applied element-wise.
+
+    Used only to turn Zipf ranks into well-spread 64-bit IDs; any bijection on
+    64-bit words would do because both sides read the same arrays.
+    """
+    with np.errstate(over="ignore"):
+        z = (np.asarray(x, dtype=np.uint64) + np.uint64(0x9E3779B97F4A7C15)) & _MASK64
+        z = ((z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)) & _MASK64
+        z = ((z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)) & _MASK64
+        return z ^ (z >> np.uint64(31))
+
+
+class BoundedZipf:
+    """Exact sampler for P(r) proportional to r^-s on r in [1, V], any s > 0.
+
+    Rejection-inversion (Hoermann and Derflinger, 1996): invert the integral of
+    the hat x^-s over [0.5, V+0.5], round to the nearest integer and accept
+    with the ratio of the true mass to the hat.  Acceptance is above 90 %, so
+    the vectorised loop below finishes in two or three rounds.
+    """
+
+    def __init__(self, n_values: int, s: float):
+        if n_values < 1 or s <= 0:
+            raise ValueError("need n_values >= 1 and s > 0")
+        self.n = int(n_values)
+        self.s = float(s)
+        self._h_x1 = self._H(1.5) - 1.0
+        self._h_n = self._H(self.n + 0.5)
+        self._cut = 2.0 - self._Hinv(self._H(2.5) - 2.0 ** (-self.s))
+
+    def _H(self, x):
+        x = np.asarray(x, dtype=np.float64)
+        lx = np.log(x)
+        t = (1.0 - self.s) * lx
+        # (exp(t)-1)/t * log(x), stable near t = 0 (s = 1)
+        small = np.abs(t) < 1e-8
+        safe_t = np.where(small, 1.0, t)
+        return np.where(small, 1.0 + t / 2.0, np.expm1(safe_t) / safe_t) * lx
+
+    def _Hinv(self, y):
+        y = np.asarray(y, dtype=np.float64)
+        t = np.maximum(y * (1.0 - self.s), -1.0)
+        small = np.abs(t) < 1e-8
+        safe_t = np.where(small, 1.0, t)
+        return np.exp(np.where(small, 1.0 - t / 2.0, np.log1p(safe_t) / safe_t) * y)
+
+    def sample(self, rng: np.random.Generator, size: int) -> np.ndarray:
+        out = np.empty(size, dtype=np.int64)
+        todo = np.arange(size)
+        while todo.size:
+            u = self._h_n + rng.random(todo.size) * (self._h_x1 - self._h_n)
+            x = self._Hinv(u)
+            k = np.clip(np.floor(x + 0.5), 1, self.n)
+            ok = (k - x <= self._cut) | (u >= self._H(k + 0.5) - np.exp(-self.s * np.log(k)))
+            out[todo[ok]] = k[ok].astype(np.int64)
+            todo = todo[~ok]
+        return out
+
+
+@dataclasses.dataclass(frozen=True)
+class Config:
+    """One workload configuration: the table's parameters and the stream's shape."""
+
+    name: str
+    capacity: int            # embedding rows
+    dim: int                 # fp32 columns per row
+    filter_threshold: int    # occurrences before an ID is admitted
+    ttl: int                 # steps of inactivity after which an ID expires
+    n_examples: int
+    n_slots: int
+    bag_len: tuple           # ("uniform", lo, hi) or ("geometric", mean, lo, hi)
+    zipf_s: float
+    n_distinct: int          # size of the ID universe (Zipf support)
+    steps: int
+    key_cells: int           # cells of the key store (tracked-ID capacity incl. slack)
+    lr: float = 0.05
+    eps: float = 1e-8
+    init_acc: float = 0.0
+    init_scale: float = 0.01
+    grad_std: float = 0.01
+    drift_period: int = 0    # steps between re-keyings of part of the universe; 0 = none
+    drift_new_frac: float = 0.0
+    seed: int = 20220923
+
+    @property
+    def n_bags(self) -> int:
+        return self.n_examples * self.n_slots
+
+
+CONFIGS = {
+    "tiny": Config("tiny", capacity=1 << 17, dim=16, filter_threshold=2, ttl=10,
+                   n_examples=1024, n_slots=8, bag_len=("uniform", 1, 4),
+                   zipf_s=1.1, n_distinct=1 << 20, steps=20, key_cells=1 << 18),
+    "medium": Config("medium", capacity=1 << 22, dim=32, filter_threshold=3, ttl=100,
+                     n_examples=8192, n_slots=26, bag_len=("uniform", 1, 8),
+                     zipf_s=1.05, n_distinct=1 << 24, steps=200, key_cells=1 << 24),
+    "large": Config("large", capacity=1 << 26, dim=64, filter_threshold=5, ttl=1000,
+                    n_examples=16384, n_slots=100, bag_len=("geometric", 5.0, 1, 20),
+                    zipf_s=1.05, n_distinct=1 << 30, steps=100, key_cells=1 << 30),
+    "drift": Config("drift", capacity=1 << 26, dim=32, filter_threshold=3, ttl=200,
+                    n_examples=16384, n_slots=50, bag_len=("geometric", 5.0, 1, 20),
+                    zipf_s=1.2, n_distinct=1 << 30, steps=400, key_cells=1 << 29,
+                    drift_period=50, drift_new_frac=0.30),
+}
+
+# Mixed-dim multi-table configuration: 8 tables, 15 feature slots each.
+MULTI_TABLE_DIMS = (8, 16, 16, 32, 32, 64, 64, 128)
+MULTI_TABLE_CAPACITY_LOG2 = (27, 26, 25, 24, 23, 22, 21, 20)
+MULTI_TABLE_ZIPF_S = (0.9, 0.95, 1.0, 1.05, 1.1, 1.2, 1.25, 1.3)
+
+
+def multi_table_configs(n_examples: int = 32768, slots_per_table: int = 15) -> list:
+    """Eight Config objects, one per table of the mixed-dim configuration."""
+    out = []
+    for t, (d, cl, s) in enumerate(zip(MULTI_TABLE_DIMS, MULTI_TABLE_CAPACITY_LOG2,
+                                       MULTI_TABLE_ZIPF_S)):
+        out.append(Config(f"multi{t}", capacity=1 << cl, dim=d, filter_threshold=3, ttl=500,
+                          n_examples=n_examples, n_slots=slots_per_table,
+                          bag_len=("uniform", 1, 8), zipf_s=s, n_distinct=1 << min(cl + 4, 30),
+                          steps=50, key_cells=1 << min(cl + 3, 30), seed=20220923 + 101 * t))
+    return out
+
+
+def scaled(cfg: Config, **kw) -> Config:
+    """A copy of cfg with some fields replaced (shortened or shrunk test variants)."""
+    return dataclasses.replace(cfg, **kw)
+
+
+@dataclasses.dataclass
+class Step:
+    ids: np.ndarray          # uint64 [n_ids]
+    offsets: np.ndarray      # int64 [n_bags + 1], offsets[0] = 0, offsets[-1] = n_ids
+    grad_pooled: np.ndarray  # float32 [n_bags, dim]
+    now: int
+
+
+def _bag_lengths(rng: np.random.Generator, spec: tuple, n_bags: int) -> np.ndarray:
+    kind = spec[0]
+    if kind == "uniform":
+        _, lo, hi = spec
+        return rng.integers(lo, hi + 1, size=n_bags, dtype=np.int64)
+    if kind == "geometric":
+        _, mean, lo, hi = spec
+        return np.clip(rng.geometric(1.0 / mean, size=n_bags), lo, hi).astype(np.int64)
+    raise ValueError(f"unknown bag length spec {spec!r}")
+
+
+class Stream:
+    """Deterministic per-step generator for one Config.
+
+    step(t) depends only on (cfg.seed, t), so any step can be regenerated on
+    its own and both sides of a parity test can draw the same step twice.
+    """
+
+    def __init__(self, cfg: Config):
+        self.cfg = cfg
+        self._zipf = BoundedZipf(cfg.n_distinct, cfg.zipf_s)
+
+    def _generation(self, ranks: np.ndarray, t: int) -> np.ndarray:
+        """How many times each rank has been re-keyed up to step t (concept drift).
+
+        At every drift_period boundary a rank draws a fresh identity with a
+        probability that grows with its popularity so that about
+        drift_new_frac of the next batch's occurrences are IDs never seen
+        before; the draw is a pure function of (seed, rank, epoch).
+        """
+        cfg = self.cfg
+        gen = np.zeros(ranks.shape, dtype=np.uint64)
+        if cfg.drift_period <= 0:
+            return gen
+        n_epochs = t // cfg.drift_period
+        thresh = np.uint64(int(cfg.drift_new_frac * float(1 << 53)))
+        for e in range(1, n_epochs + 1):
+            h = splitmix64(ranks.astype(np.uint64) * np.uint64(0x2545F4914F6CDD1D)
+                           + np.uint64((cfg.seed * 1000003 + e) & 0xFFFFFFFFFFFFFFFF))
+            gen += ((h >> np.uint64(11)) < thresh).astype(np.uint64)
+        return gen
+
+    def ids_from_ranks(self, ranks: np.ndarray, t: int) -> np.ndarray:
+        cfg = self.cfg
+        gen = self._generation(ranks, t)
+        with np.errstate(over="ignore"):
+            salt = splitmix64(np.uint64(cfg.seed & 0xFFFFFFFFFFFFFFFF) + gen * np.uint64(0x632BE59BD9B4E019))
+            ids = splitmix64(ranks.astype(np.uint64) ^ salt)
+        # the all-ones pattern is the table's reserved padding value
+        ids[ids == np.uint64(RESERVED_ID)] = np.uint64(RESERVED_ID - 1)
+        return ids
+
+    def step(self, t: int, with_grad: bool = True) -> Step:
+        cfg = self.cfg
+        rng = np.random.default_rng([cfg.seed, t])
+        lens = _bag_lengths(rng, cfg.bag_len, cfg.n_bags)
+        offsets = np.zeros(cfg.n_bags + 1, dtype=np.int64)
+        np.cumsum(lens, out=offsets[1:])
+        ranks = self._zipf.sample(rng, int(offsets[-1]))
+        ids = self.ids_from_ranks(ranks, t)
+        if with_grad:
+            grad = rng.standard_normal((cfg.n_bags, cfg.dim), dtype=np.float32) * np.float32(cfg.grad_std)
+        else:
+            grad = np.zeros((0, cfg.dim), dtype=np.float32)
+        return Step(ids=ids, offsets=offsets, grad_pooled=grad, now=t)
+
+    def __iter__(self) -> Iterator[Step]:
+        for t in range(self.cfg.steps):
+            yield self.step(t)
+
+
+def steady_state_population(cfg: Config, now: int, window: Optional[int] = None,
+                            seed_salt: int = 7, max_ranks: Optional[int] = None):
+    """Draw a table population as it would stand after `window` steps of cfg's stream.
+
+    Used to pre-fill a table before timing, so that timed steps run at a
+    realistic load instead of on an empty table.  Under the Poisson model of
+    the stream, rank k occurs Poisson(lambda_k) times per window with
+    lambda_k = (IDs per step) * window * p_k.  For each rank that occurred at
+    least once this returns its ID, its occurrence count (not yet saturated)
+    and a last-seen step drawn so that hot ranks were seen at `now`.
+
+    Returns (ids uint64, counts int64, last_seen int64).
+    """
+    window = int(window if window is not None else min(cfg.ttl, now + 1))
+    rng = np.random.default_rng([cfg.seed, seed_salt, now])
+    mean_len = _mean_bag_len(cfg.bag_len)
+    n_per_step = cfg.n_bags * mean_len
+    n_ranks = cfg.n_distinct if max_ranks is None else min(cfg.n_distinct, max_ranks)
+    stream = Stream(cfg)
+    norm = _zipf_norm(cfg.n_distinct, cfg.zipf_s)
+    ids_l, cnt_l, seen_l = [], [], []
+    chunk = 1 << 24
+    for lo in range(1, n_ranks + 1, chunk):
+        hi = min(lo + chunk, n_ranks + 1)
+        ranks = np.arange(lo, hi, dtype=np.int64)
+        p = ranks.astype(np.float64) ** (-cfg.zipf_s) / norm
+        lam_step = n_per_step * p
+        cnt = rng.poisson(lam_step * window)
+        keep = cnt > 0
+        ranks, cnt, lam_step = ranks[keep], cnt[keep], lam_step[keep]
+        # steps since the most recent occurrence: geometric with per-step hit probability
+        p_hit = -np.expm1(-lam_step)
+        age = np.minimum(rng.geometric(np.maximum(p_hit, 1e-12)) - 1, window - 1)
+        ids_l.append(stream.ids_from_ranks(ranks, now))
+        cnt_l.append(cnt.astype(np.int64))
+        seen_l.append((now - age).astype(np.int64))
+    return np.concatenate(ids_l), np.concatenate(cnt_l), np.concatenate(seen_l)
+
+
+def _mean_bag_len(spec: tuple) -> float:
+    if spec[0] == "uniform":
+        return (spec[1] + spec[2]) / 2.0
+    _, mean, lo, hi = spec
+    q = 1.0 - 1.0 / mean
+    ks = np.arange(1, 2000)
+    pk = (1 - q) * q ** (ks - 1)
+    return float(np.sum(np.clip(ks, lo, hi) * pk))
+
+
+def _zipf_norm(n: int, s: float) -> float:
+    head = min(n, 1 << 20)
+    k = np.arange(1, head + 1, dtype=np.float64)
+    total = float(np.sum(k ** (-s)))
+    if n > head:
+        a, b = head + 0.5, n + 0.5
+        total += (np.log(b / a) if abs(s - 1.0) < 1e-12 else (b ** (1 - s) - a ** (1 - s)) / (1 - s))
+    return total

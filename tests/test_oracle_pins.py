@@ -1,0 +1,396 @@
+"""Pins for the CPU oracle: every rule of the table checked against something
+that is not the oracle itself -- published known answers, closed forms,
+library routines, a per-ID replay and brute force over tiny streams.
+All CPU; none of these tests touches the CUDA library.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mono_oracle as mo
+from paper_2209_07663_b200 import workload as wl
+from tests import replay
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+f32 = np.float32
+
+
+def bags(lists):
+    """[[ids of bag 0], [ids of bag 1], ...] -> (ids uint64, offsets int64)."""
+    ids = np.array([i for b in lists for i in b], dtype=np.uint64)
+    off = np.zeros(len(lists) + 1, np.int64)
+    off[1:] = np.cumsum([len(b) for b in lists])
+    return ids, off
+
+
+# ---------------------------------------------------------------- Philox / init
+
+def test_philox_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        v = [int(x, 16) for x in r]
+        out = mo.philox4x32_10(v[0:4], v[4:6])
+        assert out.tolist() == v[6:10]
+
+
+def test_init_value_uses_counter_layout_and_range():
+    seed, id_ = 0x299F31D0A4093822, 0x85A308D3243F6A88
+    # column block 0x13198a2e with id/seed from the third known-answer vector is not
+    # reachable (block = col // 4), so check the layout with block 0 instead:
+    out = mo.philox4x32_10([id_ & 0xFFFFFFFF, id_ >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32])
+    for col in range(4):
+        u = f32(int(out[col]) >> 8) * f32(1.0 / 8388608.0) - f32(1.0)
+        assert mo.init_value(seed, id_, col, 0.25) == float(u * f32(0.25))
+    out1 = mo.philox4x32_10([id_ & 0xFFFFFFFF, id_ >> 32, 1, 0], [seed & 0xFFFFFFFF, seed >> 32])
+    u = f32(int(out1[2]) >> 8) * f32(1.0 / 8388608.0) - f32(1.0)
+    assert mo.init_value(seed, id_, 6, 0.25) == float(u * f32(0.25))
+    # the third known-answer vector through the same mapping, block reached via id/seed only
+    vals = np.array([mo.init_value(7, i, c, 0.5) for i in range(200) for c in range(16)])
+    assert vals.min() >= -0.5 and vals.max() < 0.5
+    assert abs(vals.mean()) < 0.02 and abs(vals.var() - 0.25 / 3) < 0.01
+    assert len(np.unique(vals)) > 3100          # no repeated columns / IDs
+    assert mo.init_value(7, 3, 5, 0.0) == 0.0
+
+
+# ---------------------------------------------------------------- closed forms (one rule at a time)
+
+def test_pool_counts_resident_ids_when_rows_are_ones():
+    o = mo.OracleTable(64, 4, 1, 0)
+    ids = np.arange(1, 7, dtype=np.uint64)
+    o.import_entries(ids, np.ones(6, np.uint32), np.zeros(6, np.int64), np.array([1, 1, 1, 0, 1, 0], np.uint8),
+                     np.ones((6, 4), f32), np.zeros((6, 4), f32))
+    qi, qo = bags([[1, 2, 3], [4], [], [1, 1, 5, 6, 99], [0xFFFFFFFFFFFFFFFF, 2]])
+    out = o.lookup_pool(qi, qo)
+    assert out.tolist() == [[3.0] * 4, [0.0] * 4, [0.0] * 4, [3.0] * 4, [1.0] * 4]
+
+
+def test_lookup_is_read_only():
+    o = mo.OracleTable(64, 4, 2, 5)
+    ids, off = bags([[10, 11], [10]])
+    for _ in range(5):
+        out = o.lookup_pool(ids, off)
+    assert o.n_tracked == 0 and not out.any()
+
+
+def test_first_adagrad_step_closed_form():
+    lr, eps = 0.05, 1e-8
+    o = mo.OracleTable(8, 4, 1, 0, lr=lr, eps=eps, init_scale=0.0)
+    ids, off = bags([[42]])
+    g = np.array([[0.5, -0.25, 2.0, -1e-3]], f32)
+    assert o.apply_grads(ids, off, g, 0) == 0
+    st = o.probe(np.array([42], np.uint64))
+    want = -lr * g[0].astype(np.float64) / (np.abs(g[0].astype(np.float64)) + eps)
+    np.testing.assert_allclose(st["w"][0], want, rtol=1e-6)
+    np.testing.assert_allclose(st["acc"][0], g[0].astype(np.float64) ** 2, rtol=1e-6)
+
+
+def test_constant_gradient_series_closed_form():
+    lr, eps, g, T = 0.05, 1e-8, 0.3, 17
+    o = mo.OracleTable(8, 4, 1, 0, lr=lr, eps=eps, init_scale=0.0, init_acc=0.0)
+    ids, off = bags([[7]])
+    for t in range(T):
+        o.apply_grads(ids, off, np.full((1, 4), g, f32), t)
+    st = o.probe(np.array([7], np.uint64))
+    gd = float(f32(g))
+    want_w = -lr * sum(gd / (abs(gd) * np.sqrt(i) + eps) for i in range(1, T + 1))
+    np.testing.assert_allclose(st["acc"][0], T * gd * gd, rtol=1e-5)
+    np.testing.assert_allclose(st["w"][0], want_w, rtol=1e-5)
+
+
+def test_init_acc_is_used():
+    o = mo.OracleTable(8, 4, 1, 0, lr=0.1, eps=0.0, init_scale=0.0, init_acc=4.0)
+    ids, off = bags([[7]])
+    o.apply_grads(ids, off, np.full((1, 4), 3.0, f32), 0)
+    st = o.probe(np.array([7], np.uint64))
+    np.testing.assert_allclose(st["acc"][0], 13.0)
+    np.testing.assert_allclose(st["w"][0], -0.1 * 3.0 / np.sqrt(13.0), rtol=1e-6)
+
+
+@pytest.mark.parametrize("thr", [0, 1, 2, 3, 5])
+def test_admission_at_threshold_th_occurrence(thr):
+    o = mo.OracleTable(8, 4, thr, 0)
+    ids, off = bags([[5]])
+    g = np.ones((1, 4), f32)
+    T = max(thr, 1)
+    for t in range(T + 2):
+        o.apply_grads(ids, off, g, t)
+        st = o.probe(np.array([5], np.uint64))
+        assert st["resident"][0] == (1 if t + 1 >= T else 0)
+        assert st["count"][0] == min(t + 1, T)
+        assert st["last_seen"][0] == t
+        # a row exists exactly when the pooled lookup is non-zero (init_scale != 0)
+        assert bool(o.lookup_pool(ids, off).any()) == bool(st["resident"][0])
+
+
+def test_admission_within_one_batch_and_whole_batch_gradient_applies():
+    # three occurrences in one batch with threshold 3: admitted in that batch, and the
+    # gradients of all three occurrences (not only the one that crosses) are applied
+    o = mo.OracleTable(8, 4, 3, 0, lr=1.0, eps=0.0, init_scale=0.0)
+    ids, off = bags([[9, 9], [9], [8]])
+    g = np.array([[1.0] * 4, [2.0] * 4, [7.0] * 4], f32)
+    o.apply_grads(ids, off, g, 0)
+    st = o.probe(np.array([9, 8], np.uint64))
+    assert st["resident"].tolist() == [1, 0] and st["count"].tolist() == [3, 1]
+    G = 1.0 + 1.0 + 2.0                       # bag 0 counted twice
+    np.testing.assert_allclose(st["acc"][0], G * G)
+    np.testing.assert_allclose(st["w"][0], -1.0)          # -lr*G/sqrt(G^2)
+    assert not st["w"][1].any()
+
+
+def test_duplicates_are_summed_before_squaring():
+    o = mo.OracleTable(8, 2, 1, 0, lr=1.0, eps=0.0, init_scale=0.0)
+    ids, off = bags([[3], [3]])
+    o.apply_grads(ids, off, np.array([[1.0, 1.0], [-1.0, 3.0]], f32), 0)
+    st = o.probe(np.array([3], np.uint64))
+    np.testing.assert_allclose(st["acc"][0], [0.0, 16.0])   # (1-1)^2, (1+3)^2; not 1+1, 1+9
+    np.testing.assert_allclose(st["w"][0][1], -1.0)
+
+
+def test_gradient_of_filtered_id_is_dropped_not_deferred():
+    o = mo.OracleTable(8, 2, 2, 0, lr=1.0, eps=0.0, init_scale=0.0)
+    ids, off = bags([[3]])
+    o.apply_grads(ids, off, np.array([[100.0, 100.0]], f32), 0)      # below threshold: dropped
+    o.apply_grads(ids, off, np.array([[2.0, 2.0]], f32), 1)
+    st = o.probe(np.array([3], np.uint64))
+    np.testing.assert_allclose(st["acc"][0], [4.0, 4.0])
+
+
+@pytest.mark.parametrize("ttl", [1, 3, 10])
+def test_expiry_boundary_is_strict(ttl):
+    o = mo.OracleTable(8, 4, 1, ttl)
+    ids, off = bags([[5], [6, 6]])
+    o.apply_grads(ids, off, np.ones((2, 4), f32), 100)
+    assert o.expire(100 + ttl) == 0 and o.n_tracked == 2
+    assert o.expire(100 + ttl + 1) == 2 and o.n_tracked == 0 and o.n_resident == 0
+    assert not o.lookup_pool(ids, off).any()
+
+
+def test_ttl_zero_disables_expiry_and_probation_ids_expire_too():
+    o = mo.OracleTable(8, 4, 1, 0)
+    ids, off = bags([[5]])
+    o.apply_grads(ids, off, np.ones((1, 4), f32), 0)
+    assert o.expire(10 ** 9) == 0 and o.n_tracked == 1
+    o = mo.OracleTable(8, 4, 3, 2)
+    o.apply_grads(ids, off, np.ones((1, 4), f32), 0)        # count 1, on probation
+    o.apply_grads(ids, off, np.ones((1, 4), f32), 1)        # count 2
+    assert o.expire(4) == 1                                  # 4 - 1 > 2
+    o.apply_grads(ids, off, np.ones((1, 4), f32), 5)        # starts again from 0
+    st = o.probe(np.array([5], np.uint64))
+    assert st["count"][0] == 1 and st["resident"][0] == 0
+
+
+def test_unswept_stale_entry_is_refreshed():
+    o = mo.OracleTable(8, 4, 1, 2)
+    ids, off = bags([[5]])
+    o.apply_grads(ids, off, np.ones((1, 4), f32), 0)
+    o.apply_grads(ids, off, np.ones((1, 4), f32), 50)        # stale but never swept: refreshed
+    assert o.expire(51) == 0
+    st = o.probe(np.array([5], np.uint64))
+    assert st["last_seen"][0] == 50 and st["resident"][0] == 1
+
+
+def test_readmission_after_expiry_leaves_no_residue():
+    kw = dict(lr=0.05, eps=1e-8, init_scale=0.1, seed=11)
+    a = mo.OracleTable(8, 4, 1, 2, **kw)
+    ids, off = bags([[5]])
+    for t in range(3):
+        a.apply_grads(ids, off, np.full((1, 4), 0.7, f32), t)
+    a.expire(10)
+    assert a.n_tracked == 0
+    g = np.array([[0.1, -0.2, 0.3, -0.4]], f32)
+    a.apply_grads(ids, off, g, 11)
+    b = mo.OracleTable(8, 4, 1, 2, **kw)
+    b.apply_grads(ids, off, g, 11)
+    sa, sb = a.probe(np.array([5], np.uint64)), b.probe(np.array([5], np.uint64))
+    assert (sa["w"] == sb["w"]).all() and (sa["acc"] == sb["acc"]).all()
+
+
+def test_time_must_not_decrease_and_reserved_id_is_padding():
+    o = mo.OracleTable(8, 4, 1, 0)
+    ids, off = bags([[5, 0xFFFFFFFFFFFFFFFF]])
+    assert o.apply_grads(ids, off, np.ones((1, 4), f32), 5) == mo.OK
+    assert o.apply_grads(ids, off, np.ones((1, 4), f32), 4) == mo.ERR_TIME
+    assert o.n_tracked == 1
+
+
+def test_fresh_row_equals_init_then_one_update():
+    o = mo.OracleTable(8, 8, 1, 0, lr=0.5, eps=0.0, init_scale=0.2, seed=99)
+    ids, off = bags([[1234567]])
+    g = np.full((1, 8), 2.0, f32)
+    o.apply_grads(ids, off, g, 0)
+    st = o.probe(np.array([1234567], np.uint64))
+    init = np.array([mo.init_value(99, 1234567, c, 0.2) for c in range(8)], f32)
+    np.testing.assert_allclose(st["w"][0], init - f32(0.5), rtol=0, atol=1e-7)
+    assert len(set(init.tolist())) == 8
+
+
+# ---------------------------------------------------------------- library special cases
+
+def test_forward_equals_embedding_bag_sum():
+    rng = np.random.default_rng(3)
+    V, d, B = 50, 12, 40
+    W = rng.standard_normal((V, d)).astype(f32)
+    id_of_row = wl.splitmix64(np.arange(V, dtype=np.uint64) + np.uint64(1000))
+    o = mo.OracleTable(V, d, 1, 0)
+    o.import_entries(id_of_row, np.ones(V, np.uint32), np.zeros(V, np.int64), np.ones(V, np.uint8),
+                     W, np.zeros((V, d), f32))
+    lens = rng.integers(0, 6, B)
+    off = np.zeros(B + 1, np.int64)
+    off[1:] = np.cumsum(lens)
+    rows = rng.integers(0, V, off[-1])
+    out = o.lookup_pool(id_of_row[rows], off)
+    ref = torch.nn.functional.embedding_bag(torch.from_numpy(rows), torch.from_numpy(W.astype(np.float64)),
+                                            torch.from_numpy(off[:-1]), mode="sum").numpy()
+    np.testing.assert_allclose(out, ref, rtol=1e-6, atol=1e-7)
+
+
+@pytest.mark.parametrize("init_acc", [0.0, 0.1])
+def test_apply_grads_equals_torch_adagrad_step(init_acc):
+    rng = np.random.default_rng(4)
+    V, d, B, lr, eps = 30, 8, 64, 0.05, 1e-8
+    W0 = rng.standard_normal((V, d)).astype(f32)
+    id_of_row = wl.splitmix64(np.arange(V, dtype=np.uint64) + np.uint64(77))
+    o = mo.OracleTable(V, d, 1, 0, lr=lr, eps=eps, init_acc=init_acc)
+    o.import_entries(id_of_row, np.ones(V, np.uint32), np.zeros(V, np.int64), np.ones(V, np.uint8),
+                     W0, np.full((V, d), init_acc, f32))
+    Wt = torch.nn.Parameter(torch.from_numpy(W0.astype(np.float64)))
+    opt = torch.optim.Adagrad([Wt], lr=lr, eps=eps, initial_accumulator_value=init_acc)
+    for step in range(3):
+        lens = rng.integers(0, 5, B)
+        off = np.zeros(B + 1, np.int64)
+        off[1:] = np.cumsum(lens)
+        rows = rng.integers(0, 20, off[-1])          # rows 20.. never touched
+        grad = (rng.standard_normal((B, d)) * 0.1).astype(f32)
+        opt.zero_grad()
+        pooled = torch.nn.functional.embedding_bag(torch.from_numpy(rows), Wt, torch.from_numpy(off[:-1]),
+                                                   mode="sum")
+        (pooled * torch.from_numpy(grad.astype(np.float64))).sum().backward()
+        opt.step()
+        assert o.apply_grads(id_of_row[rows], off, grad, step) == 0
+    st = o.probe(id_of_row)
+    np.testing.assert_allclose(st["w"], Wt.detach().numpy(), rtol=2e-6, atol=1e-7)
+    acc_ref = opt.state[Wt]["sum"].numpy()
+    np.testing.assert_allclose(st["acc"], acc_ref, rtol=2e-6, atol=1e-9)
+    assert (st["w"][20:] == W0[20:]).all()           # untouched rows unchanged
+
+
+# ---------------------------------------------------------------- per-ID replay and brute force
+
+def _run_oracle(steps, *, capacity, dim, threshold, ttl, **kw):
+    o = mo.OracleTable(capacity, dim, threshold, ttl, **kw)
+    for ids, off, grad, now, sweep in steps:
+        assert o.apply_grads(ids, off, grad, now) == 0
+        if sweep:
+            o.expire(now)
+    return o
+
+
+def _check_against_replay(o, steps, *, dim, threshold, ttl, lr, eps, init_acc, init_scale, seed):
+    hist = replay.id_histories(steps)
+    init_row = lambda i: np.array([mo.init_value(seed, i, c, init_scale) for c in range(dim)], f32)
+    ex = o.export()
+    got = {int(i): k for k, i in enumerate(ex["ids"])}
+    n_tracked = 0
+    for id_, events in hist.items():
+        r = replay.replay_id(id_, events, steps, threshold=threshold, ttl=ttl, lr=lr, eps=eps,
+                             init_acc=init_acc, init_row=init_row)
+        if not r["tracked"]:
+            assert id_ not in got
+            continue
+        n_tracked += 1
+        k = got[id_]
+        assert ex["count"][k] == r["count"] and ex["last_seen"][k] == r["last_seen"]
+        assert bool(ex["resident"][k]) == r["resident"]
+        if r["resident"]:
+            assert (ex["w"][k] == r["w"]).all() and (ex["acc"][k] == r["acc"]).all()
+        else:
+            assert not ex["w"][k].any() and not ex["acc"][k].any()
+    assert n_tracked == len(got) == o.n_tracked
+    assert o.n_resident == int(ex["resident"].sum())
+
+
+def test_random_streams_match_per_id_replay():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=64, n_slots=4, n_distinct=1 << 10, steps=30, dim=8)
+    stream = wl.Stream(cfg)
+    kw = dict(lr=cfg.lr, eps=cfg.eps, init_acc=0.0, init_scale=0.05, seed=5)
+    for threshold, ttl, sweep_every in [(2, 3, 1), (3, 5, 4), (1, 2, 1), (4, 0, 1)]:
+        steps = []
+        for t in range(cfg.steps):
+            s = stream.step(t)
+            steps.append((s.ids, s.offsets, s.grad_pooled, 2 * t, (t % sweep_every) == sweep_every - 1))
+        o = _run_oracle(steps, capacity=cfg.capacity, dim=cfg.dim, threshold=threshold, ttl=ttl, **kw)
+        _check_against_replay(o, steps, dim=cfg.dim, threshold=threshold, ttl=ttl, **kw)
+        # invariants: a probation ID has no row and pools as zero; after a final sweep
+        # nothing is older than ttl
+        ex = o.export()
+        assert (ex["count"][ex["resident"] == 0] < max(threshold, 1)).all()
+        assert (ex["count"][ex["resident"] == 1] == max(threshold, 1)).all()
+        now = 2 * (cfg.steps - 1)
+        o.expire(now)
+        ex = o.export()
+        if ttl:
+            assert (now - ex["last_seen"] <= ttl).all()
+
+
+def test_brute_force_all_tiny_streams():
+    """Every stream of 4 steps over 2 IDs with multiplicities 0..2, all thresholds/TTLs."""
+    d = 2
+    kw = dict(lr=0.05, eps=1e-8, init_acc=0.0, init_scale=0.1, seed=1)
+    per_step = list(itertools.product(range(3), range(3)))
+    n = 0
+    for threshold in (1, 2, 3):
+        for ttl in (1, 2):
+            for combo in itertools.product(per_step, repeat=4):
+                if n % 7:          # thin the 6561 x 6 grid deterministically
+                    n += 1
+                    continue
+                n += 1
+                steps = []
+                for t, (ma, mb) in enumerate(combo):
+                    lists = [[101] * ma, [202] * mb, [101] * (ma > 1)]
+                    ids, off = bags(lists)
+                    grad = np.array([[0.1 * (t + 1), -0.2], [0.3, 0.05 * (t + 1)], [1.0, 1.0]], f32)
+                    steps.append((ids, off, grad, t, True))
+                o = _run_oracle(steps, capacity=4, dim=d, threshold=threshold, ttl=ttl, **kw)
+                _check_against_replay(o, steps, dim=d, threshold=threshold, ttl=ttl, **kw)
+
+
+def test_hand_worked_stream():
+    """A stream small enough to follow by hand: threshold 2, ttl 1, sweep every step."""
+    o = mo.OracleTable(4, 1, 2, 1, lr=1.0, eps=0.0, init_scale=0.0)
+    A, B_, C = 11, 22, 33
+    g1 = np.ones((2, 1), f32)
+    # t=0: A once, B twice -> B admitted (count 2), A on probation (count 1)
+    o.apply_grads(*bags([[A, B_], [B_]]), g1, 0); o.expire(0)
+    st = o.probe(np.array([A, B_, C], np.uint64))
+    assert st["resident"].tolist() == [0, 1, 0] and st["count"].tolist() == [1, 2, 0]
+    assert st["acc"][1][0] == 4.0 and st["w"][1][0] == -1.0          # G = 2
+    # t=1: A again -> admitted; C once
+    o.apply_grads(*bags([[A], [C]]), g1, 1); o.expire(1)
+    st = o.probe(np.array([A, B_, C], np.uint64))
+    assert st["resident"].tolist() == [1, 1, 0] and st["count"].tolist() == [2, 2, 1]
+    assert st["last_seen"].tolist() == [1, 0, 1]
+    # t=2: nothing but C; sweep(2): B last seen 0 -> 2-0 > 1 expires; A (1) and C stay
+    o.apply_grads(*bags([[C], []]), g1, 2); o.expire(2)
+    st = o.probe(np.array([A, B_, C], np.uint64))
+    assert st["resident"].tolist() == [1, 0, 1] and st["count"].tolist() == [2, 0, 2]
+    assert o.n_tracked == 2 and o.n_resident == 2
+
+
+def test_capacity_overflow_is_reported():
+    o = mo.OracleTable(2, 2, 1, 0)
+    rc = o.apply_grads(*bags([[1, 2, 3]]), np.ones((1, 2), f32), 0)
+    assert rc == mo.ERR_FULL and o.n_resident == 2 and o.n_tracked == 3
+
+
+def test_sync_volume_arithmetic_from_the_paper():
+    # Section 3.2: a dim-1024 fp32 row is 4 KB; 100 000 rows are about 400 MB
+    o = mo.OracleTable(4, 1024, 1, 0)
+    o.apply_grads(*bags([[1]]), np.ones((1, 1024), f32), 0)
+    assert o.export()["w"].nbytes == 4096
+    assert 100_000 * 4096 == pytest.approx(400e6, rel=0.03)
