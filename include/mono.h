@@ -1,0 +1,301 @@
+/*
+ * mono.h -- C ABI of the collisionless embedding table for one NVIDIA B200.
+ *
+ * The table is the sparse-parameter store of Monolith (arXiv 2209.07663):
+ * a key-value HashTable from 64-bit feature IDs to fp32 embedding rows that
+ * never lets two IDs share a row (Section 2.1), admits an ID only after it has
+ * occurred a threshold number of times (Section 2.1, filtering heuristic 1),
+ * stamps every ID with its last access so that inactive IDs can be expired
+ * (heuristic 2), and serves the sparse half of a training step (Section 2.2:
+ * pull the parameters, forward, backward, push the updated parameters back).
+ * Sum pooling per bag, gradient de-duplication and the Adagrad row update are
+ * not described in the paper; their definitions are stated at each call.
+ *
+ * Conventions
+ *  - Every call returns an int: MONO_OK or a negative MONO_ERR_* code that the
+ *    host detected before any work was enqueued.  No exception crosses the ABI.
+ *  - Unless a parameter is marked HOST, data pointers are DEVICE pointers owned
+ *    by the caller; the library reads or writes them only through work enqueued
+ *    by the call and never frees or keeps them.
+ *  - All work of a table is enqueued on the CUDA stream given at creation.  The
+ *    hot calls (mono_lookup_pool, mono_apply_grads, mono_expire) return without
+ *    synchronising.  Calls on one table must not overlap on the GPU: issue them
+ *    from one thread, on that stream.
+ *  - Conditions that only the device can see (no free row, key store full,
+ *    malformed offsets) never trap or hang: every device loop is bounded, the
+ *    condition sets a sticky bit and a counter, and mono_status reports them.
+ *  - A "bag" is one (example, feature slot) pair.  Bags are given CSR style:
+ *    bag b owns ids[slot_offsets[b] .. slot_offsets[b+1]).
+ *  - IDs are arbitrary 64-bit patterns except MONO_RESERVED_ID, which is
+ *    padding: it pools as zero and is neither counted nor inserted.
+ *  - Time is the integer `now` the caller passes (a step counter, seconds,
+ *    ...).  It must not decrease and must lie in [0, MONO_MAX_NOW].
+ */
+#ifndef MONO_H_
+#define MONO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MONO_RESERVED_ID 0xFFFFFFFFFFFFFFFFull
+#define MONO_MAX_NOW     0xFFFFFFFEll
+#define MONO_MAX_DIM     1024u
+#define MONO_MAX_CAPACITY (1ull << 30)
+
+enum {
+  MONO_OK = 0,
+  MONO_ERR_ARG = -1,    /* null or misaligned pointer, size out of range, bad option */
+  MONO_ERR_TIME = -2,   /* `now` decreased or is outside [0, MONO_MAX_NOW] */
+  MONO_ERR_CUDA = -3,   /* a CUDA runtime call failed; see mono_last_cuda_error */
+  MONO_ERR_NOMEM = -4,  /* device allocation failed */
+  MONO_ERR_SIZE = -5    /* caller buffer too small (mono_export) */
+};
+
+/* Sticky device-side condition bits reported in mono_status_t.error_bits. */
+enum {
+  MONO_DEV_ROWS_FULL = 1u,    /* an ID reached the threshold but no free row was left;
+                                 it stays tracked without a row and is retried later */
+  MONO_DEV_KEYS_FULL = 2u,    /* an insertion found no cell after the bounded eviction
+                                 chain and the stash was full: one tracked key was lost */
+  MONO_DEV_BAD_OFFSETS = 4u,  /* slot_offsets not monotone or out of [0, n_ids]; the
+                                 offending bag was treated as empty */
+  MONO_DEV_IMPORT_DUP = 8u    /* mono_import met an ID that was already tracked; skipped */
+};
+
+enum { MONO_OPT_ADAGRAD = 1 };
+
+typedef struct mono_table mono_table; /* opaque, owned by the library */
+
+/*
+ * Options of mono_table_create.  Zero-initialise, then set what is needed.
+ *
+ * Row initialisation (the paper does not give one): column c of a newly
+ * admitted ID starts at  (u * 2^-23 - 1) * init_scale  with u the top 24 bits
+ * of word (c mod 4) of Philox4x32-10 (Salmon et al., SC'11) keyed by
+ * (seed low 32 bits, seed high 32 bits) on the counter
+ * (id low 32 bits, id high 32 bits, c / 4, 0).  It depends on nothing but
+ * (seed, id, c), so it is the same whatever the insertion order or row index.
+ */
+typedef struct {
+  int32_t  kind;          /* MONO_OPT_ADAGRAD (0 selects it too) */
+  float    lr;            /* Adagrad learning rate */
+  float    eps;           /* added to sqrt(acc), outside the square root */
+  float    init_acc;      /* initial value of every accumulator element */
+  float    init_scale;    /* rows start uniform in [-init_scale, init_scale); 0 => zeros */
+  uint64_t seed;          /* seeds row initialisation and the table's hash functions */
+  uint64_t key_cells;     /* cells of the key store = how many IDs can be tracked (with or
+                             without a row) at load 1.  Power of two, >= 64.
+                             0 => 4 * capacity rounded up to a power of two. */
+  uint64_t max_ids;       /* scratch is sized for this many IDs per call at creation;
+                             larger calls grow it (an allocation, so not inside a timed
+                             loop).  0 => grown on first use. */
+  uint64_t max_bags;      /* same, for bags per call */
+} mono_opt;
+
+typedef struct {
+  uint32_t error_bits;          /* OR of MONO_DEV_* since creation */
+  uint32_t dim;
+  uint64_t capacity;            /* rows */
+  uint64_t key_cells;
+  uint64_t n_tracked;           /* IDs in the key store (with or without a row) */
+  uint64_t n_resident;          /* IDs that own a row */
+  uint64_t n_admitted_total;    /* rows handed out since creation */
+  uint64_t n_expired_total;     /* IDs removed by mono_expire */
+  uint64_t n_inserted_total;    /* IDs that entered the key store */
+  uint64_t n_rows_refused;      /* admissions refused for lack of a row */
+  uint64_t n_keys_dropped;      /* keys lost to MONO_DEV_KEYS_FULL */
+  uint64_t n_evictions_total;   /* cuckoo displacements performed */
+  uint32_t max_chain;           /* longest eviction chain seen */
+  uint32_t stash_used;          /* occupied stash cells (high-water mark index) */
+  /* totals over all mono_apply_grads calls (for traffic accounting) */
+  uint64_t sum_ids;             /* non-padding ID occurrences */
+  uint64_t sum_unique;          /* distinct IDs per call, summed */
+  uint64_t sum_unique_resident; /* distinct IDs that had (or got) a row, summed */
+  uint64_t sum_new;             /* distinct IDs that were new to the key store, summed */
+} mono_status_t;
+
+typedef struct {
+  uint64_t occupied_cells;      /* occupied key cells incl. stash */
+  uint64_t misplaced;           /* keys found in a bucket that is neither h0(key) nor h1(key) */
+  uint64_t duplicate_keys;      /* keys present in more than one cell */
+  uint64_t resident_cells;
+  uint64_t bad_rows;            /* row index >= capacity */
+  uint64_t shared_rows;         /* rows owned by two cells, or owned and also on the free list */
+  uint64_t free_rows;
+  uint64_t unaccounted_rows;    /* rows neither owned nor free */
+  uint32_t ok;                  /* 1 iff all of the above are consistent with the counters */
+  uint32_t pad_;
+} mono_audit_t;
+
+/*
+ * Create an empty table (Section 2.1: one HashTable per sparse feature group).
+ *  out               HOST, receives the handle
+ *  capacity          number of embedding rows, 1 .. MONO_MAX_CAPACITY
+ *  dim               fp32 columns per row, multiple of 4, 4 .. MONO_MAX_DIM
+ *  filter_threshold  an ID gets a row once its occurrences reach this (0 acts as 1);
+ *                    a per-model hyperparameter in the paper, here set per table
+ *  ttl               an ID unseen for MORE than ttl time units is removed by
+ *                    mono_expire; 0 disables expiry (the paper tunes it per table)
+ *  opt               HOST, may be NULL for defaults (lr 0.05, eps 1e-8, zeros)
+ *  cuda_stream       a cudaStream_t (NULL = the default stream) on the current device
+ * Allocates capacity * dim * 8 bytes of rows+accumulators, key_cells * 16 bytes
+ * of keys, capacity * 4 bytes of free-row bookkeeping and the scratch.
+ */
+int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim,
+                      uint32_t filter_threshold, uint32_t ttl, const mono_opt* opt,
+                      void* cuda_stream);
+
+/* Synchronise the stream and free everything the table owns. */
+int mono_table_destroy(mono_table* t);
+
+/* Grow the scratch so that calls with up to max_ids IDs and max_bags bags
+ * allocate nothing.  Synchronises if it has to reallocate. */
+int mono_reserve(mono_table* t, int64_t max_ids, int64_t max_bags);
+
+/*
+ * Forward (the parameter pull of a training step, Section 2.2; the HashTable
+ * look-up operation of Section 2.1): out[b, :] = sum over the IDs of bag b, in order, of the row of
+ * each ID that owns one; an ID without a row (unknown, below the threshold,
+ * expired) contributes zero; an empty bag gives zeros.  Read-only: counts and
+ * last-access times do not change.
+ *  ids           uint64 [n_ids], 8-byte aligned
+ *  slot_offsets  int64 [n_bags + 1], non-decreasing, slot_offsets[0] >= 0,
+ *                slot_offsets[n_bags] <= n_ids
+ *  out           fp32 [n_bags, dim] row-major, 16-byte aligned, overwritten
+ */
+int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids,
+                     const int64_t* slot_offsets, int64_t n_bags, float* out);
+
+/*
+ * Backward + update (the parameter push of a training step, Section 2.2; the
+ * HashTable update operation with the occurrence filter and the access stamp of Section 2.1).  For the
+ * batch as a whole:
+ *  1. every distinct ID u gets  count(u) += multiplicity of u in ids  (saturating
+ *     at the threshold; the counter only gates admission) and last_seen(u) = now;
+ *     IDs met for the first time enter the key store (cuckoo insertion);
+ *  2. an ID whose count has reached the threshold and that has no row is given a
+ *     free row, initialised as described at mono_opt;
+ *  3. every distinct ID that owns a row takes ONE Adagrad step with
+ *     G = sum over its occurrences j of grad_pooled[bag(j), :]  (summed in fp64,
+ *     rounded once to fp32):   acc += G*G;   w -= lr * G / (sqrt(acc) + eps).
+ *     The whole batch's G applies even when the row was admitted in this call.
+ *     Gradients of IDs without a row are dropped.
+ * The outcome does not depend on the order of IDs or bags.
+ *  grad_pooled   fp32 [n_bags, dim], 16-byte aligned
+ *  now           time of this batch; MONO_ERR_TIME if it decreased
+ */
+int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids,
+                     const int64_t* slot_offsets, int64_t n_bags,
+                     const float* grad_pooled, int64_t now);
+
+/*
+ * Expiry sweep (Section 2.1, heuristic 2): remove every tracked ID, with or
+ * without a row, for which  now - last_seen > ttl; free its row and forget its
+ * count.  Expiry takes effect only here; a stale ID that re-occurs before a
+ * sweep is refreshed.  No-op when ttl == 0.
+ */
+int mono_expire(mono_table* t, int64_t now);
+
+/*
+ * Host-buffer forms of the two hot calls, for callers whose batches live in
+ * host memory (pinned memory makes the copies asynchronous).  They copy the
+ * inputs to library-owned device staging on the table's stream, run the same
+ * kernels as the device-pointer forms, and (lookup) copy the result back.
+ * mono_lookup_pool_host synchronises the stream before returning so that
+ * `out` is readable; mono_apply_grads_host does not synchronise, so the host
+ * buffers must stay valid until the stream has passed the copies.
+ * All pointers HOST.
+ */
+int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids,
+                          const int64_t* slot_offsets, int64_t n_bags, float* out);
+int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids,
+                          const int64_t* slot_offsets, int64_t n_bags,
+                          const float* grad_pooled, int64_t now);
+
+/* ---- inspection and fixtures: not on the hot path, all synchronise ---- */
+
+/* Counters and sticky error bits.  host_out HOST. */
+int mono_status(mono_table* t, mono_status_t* host_out);
+
+/* Clear the sticky error bits (counters are kept). */
+int mono_clear_errors(mono_table* t);
+
+/*
+ * State of n IDs: resident[i] 1/0, count[i] (0 if untracked; equals the
+ * threshold once resident), last_seen[i] (-1 if untracked).  Any output
+ * pointer may be NULL.
+ */
+int mono_probe(mono_table* t, const uint64_t* ids, int64_t n, uint8_t* resident,
+               uint32_t* count, int64_t* last_seen);
+
+/* Rows and accumulators of n IDs, fp32 [n, dim] each; zeros where the ID has
+ * no row.  Either output may be NULL. */
+int mono_read_rows(mono_table* t, const uint64_t* ids, int64_t n, float* w, float* acc);
+
+/*
+ * Dump every tracked ID (any order) into caller buffers of max_n entries:
+ * ids, count, last_seen, resident, and fp32 [max_n, dim] w / acc (zeros for IDs
+ * without a row; w and acc may be NULL).  n_out HOST receives the number
+ * written.  MONO_ERR_SIZE (and *n_out = needed) if max_n is too small.
+ * This is the table's snapshot (Section 2.3) in its simplest form.
+ */
+int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_seen,
+                uint8_t* resident, float* w, float* acc, int64_t max_n, int64_t* n_out);
+
+/*
+ * Insert n entries given as (id, count, last_seen, resident[, w, acc]).  IDs
+ * must be distinct; an ID that is already tracked is skipped and
+ * MONO_DEV_IMPORT_DUP is set.  resident[i] != 0 claims a row; its values come
+ * from w/acc, or from the initialisation rule (and init_acc) when w or acc is
+ * NULL.  count is clamped to the threshold.  Restores a snapshot, or pre-fills
+ * a table to a chosen load.
+ */
+int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count,
+                const int64_t* last_seen, const uint8_t* resident, const float* w,
+                const float* acc, int64_t n);
+
+/*
+ * Structural audit of the cuckoo table (Section 2.1: an element lives in
+ * exactly one of its two candidate positions): every key sits in one of its
+ * two buckets or the stash, no key twice, row indices distinct and disjoint
+ * from the free rows, rows owned + free = capacity.  host_out HOST.
+ */
+int mono_audit(mono_table* t, mono_audit_t* host_out);
+
+/*
+ * Launch accounting for benchmarks (the paper has no counterpart).  Every
+ * kernel the hot calls launch is counted per kernel.  With timing enabled,
+ * each launch is also bracketed by two CUDA events on the table's stream and
+ * mono_timing_read (which synchronises) adds up the elapsed device time per
+ * kernel; the events cost a few microseconds per launch, so leave timing off
+ * when measuring whole-step throughput.  ms is 0 for launches made with timing
+ * off.  reset != 0 zeroes the counts and times after reading.  host_out HOST.
+ */
+#define MONO_MAX_KERNELS 24
+typedef struct {
+  char     name[32];
+  uint64_t launches;
+  double   ms;
+} mono_kernel_time_t;
+typedef struct {
+  uint32_t n_kernels;
+  uint32_t pad_;
+  uint64_t launches_total;
+  mono_kernel_time_t kernel[MONO_MAX_KERNELS];
+} mono_timing_t;
+int mono_timing_enable(mono_table* t, int on);
+int mono_timing_read(mono_table* t, mono_timing_t* host_out, int reset);
+
+/* Text of the last CUDA error seen by this table (HOST string, library-owned). */
+const char* mono_last_cuda_error(mono_table* t);
+
+/* Name of a MONO_* return code. */
+const char* mono_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MONO_H_ */

@@ -1,5 +1,5 @@
 // CPU oracle for the collisionless embedding-table step of Monolith
-// (arXiv 2209.07663, Section 2.1 "Hash Table" and the training step of
+// (arXiv 2209.07663, Section 2.1 on the hash table and the training step of
 // Section 2.2).
 //
 // TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
@@ -114,7 +114,7 @@ void oracle_destroy(void* h) { delete static_cast<Oracle*>(h); }
 
 // Forward: out[b, :] = sum of the rows of the resident IDs of bag b, in the
 // order the IDs appear; IDs without a row contribute nothing (Section 2.2:
-// the worker "requests parameters"; a filtered or unknown ID has none).
+// the worker pulls parameters; a filtered or unknown ID has none).
 // Read-only: neither counts nor times change.
 int oracle_lookup_pool(void* h, const uint64_t* ids, int64_t n_ids, const int64_t* offsets,
                        int64_t n_bags, float* out) {
@@ -136,7 +136,7 @@ int oracle_lookup_pool(void* h, const uint64_t* ids, int64_t n_ids, const int64_
   return ORACLE_OK;
 }
 
-// Backward + update ("push updated parameters", Section 2.2), with the
+// Backward + update (the parameter push of Section 2.2), with the
 // occurrence filter and the last-access stamp of Section 2.1:
 //   1. group the batch's occurrences by ID: multiplicity and the sum, in
 //      double and in occurrence order, of the pooled gradients of their bags;

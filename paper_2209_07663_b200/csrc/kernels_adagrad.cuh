@@ -1,0 +1,192 @@
+// Backward, last phase: per distinct ID that owns a row, sum the pooled
+// gradients of its occurrences' bags (fp64 accumulation, one rounding to fp32)
+// and apply one Adagrad step to the row, in place.  This is the parameter push
+// of Section 2.2 for the sparse rows; the optimizer itself is not
+// named in the paper.
+//
+// Segments of up to kSegChunk occurrences are reduced by one lane group.
+// Longer segments (the head of the Zipf distribution: one ID can own several
+// percent of a batch) are cut into parts of kSegChunk that are reduced by
+// separate groups into fp64 partial sums, then combined by one block per ID in
+// a fixed order.
+#pragma once
+
+#include "kernels_dedup.cuh"
+
+namespace mono {
+
+struct D4 { double x, y, z, w; };
+
+__device__ inline void add4(D4& a, const float4 v) { a.x += (double)v.x; a.y += (double)v.y; a.z += (double)v.z; a.w += (double)v.w; }
+
+// acc += G*G;  w -= lr*G/(sqrt(acc)+eps), each operation rounded to fp32 on its
+// own (no fused multiply-add), so the result does not depend on contraction.
+__device__ inline void adagrad4(float4& w, float4& a, const D4& g, float lr, float eps) {
+  const float gx = (float)g.x, gy = (float)g.y, gz = (float)g.z, gw = (float)g.w;
+  a.x = __fadd_rn(a.x, __fmul_rn(gx, gx));
+  a.y = __fadd_rn(a.y, __fmul_rn(gy, gy));
+  a.z = __fadd_rn(a.z, __fmul_rn(gz, gz));
+  a.w = __fadd_rn(a.w, __fmul_rn(gw, gw));
+  w.x = __fsub_rn(w.x, __fdiv_rn(__fmul_rn(lr, gx), __fadd_rn(__fsqrt_rn(a.x), eps)));
+  w.y = __fsub_rn(w.y, __fdiv_rn(__fmul_rn(lr, gy), __fadd_rn(__fsqrt_rn(a.y), eps)));
+  w.z = __fsub_rn(w.z, __fdiv_rn(__fmul_rn(lr, gz), __fadd_rn(__fsqrt_rn(a.z), eps)));
+  w.w = __fsub_rn(w.w, __fdiv_rn(__fmul_rn(lr, gw), __fadd_rn(__fsqrt_rn(a.w), eps)));
+}
+
+// Load (or, for a row admitted in this call, create) the row, update, store.
+__device__ inline void update_row(const TableView& tv, uint32_t row_word, unsigned long long id,
+                                  uint32_t c4, const D4& g) {
+  const uint32_t row = row_word & ~kFreshBit;
+  float4* pw = reinterpret_cast<float4*>(tv.w_row(row)) + c4;
+  float4* pa = reinterpret_cast<float4*>(tv.acc_row(row)) + c4;
+  float4 w, a;
+  if (row_word & kFreshBit) {
+    w = init_vec(tv, id, c4);
+    a = make_float4(tv.init_acc, tv.init_acc, tv.init_acc, tv.init_acc);
+  } else {
+    w = *pw;
+    a = *pa;
+  }
+  adagrad4(w, a, g, tv.lr, tv.eps);
+  *pw = w;
+  *pa = a;
+}
+
+// Sum of grad rows of bags bag_of_sorted[begin .. end) for the NV column
+// vectors this lane owns.  Four independent loads in flight per step.
+template <int G, int NV>
+__device__ inline void reduce_segment(const Work& wk, const float* __restrict__ grad, long long n_bags,
+                                      uint32_t dim, int gl, uint32_t begin, uint32_t end, D4 (&s)[NV]) {
+  uint32_t i = begin;
+  for (; i + 4 <= end; i += 4) {
+    uint32_t b[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) b[k] = wk.bag_of_sorted[i + k];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint32_t c4 = gl + v * G;
+      if (c4 * 4u < dim) {
+        float4 x[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          x[k] = b[k] < n_bags ? __ldg(reinterpret_cast<const float4*>(grad + (size_t)b[k] * dim) + c4)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) add4(s[v], x[k]);
+      }
+    }
+  }
+  for (; i < end; ++i) {
+    const uint32_t b = wk.bag_of_sorted[i];
+    if (b >= n_bags) continue;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint32_t c4 = gl + v * G;
+      if (c4 * 4u < dim) add4(s[v], __ldg(reinterpret_cast<const float4*>(grad + (size_t)b * dim) + c4));
+    }
+  }
+}
+
+// One lane group per distinct ID with a short segment.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
+  const uint32_t n = tv.st->n_unique;
+  const int gl = threadIdx.x % G;
+  const uint32_t groups = (gridDim.x * blockDim.x) / G;
+  for (uint32_t u = (blockIdx.x * blockDim.x + threadIdx.x) / G; u < n; u += groups) {
+    const uint32_t row_word = wk.urow[u];
+    if (row_word == kNoRow) continue;
+    const uint32_t begin = wk.useg[u], end = wk.useg[u + 1];
+    if (end - begin > kSegChunk) continue;          // handled in parts
+    D4 s[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
+    reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
+    const unsigned long long id = wk.uid[u];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint32_t c4 = gl + v * G;
+      if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
+    }
+  }
+}
+
+// One lane group per part of a long segment: fp64 partial sums to scratch.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+reduce_parts_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
+  uint32_t n_parts = tv.st->n_parts;
+  if (n_parts > wk.max_parts) n_parts = wk.max_parts;
+  const int gl = threadIdx.x % G;
+  const uint32_t groups = (gridDim.x * blockDim.x) / G;
+  for (uint32_t p = (blockIdx.x * blockDim.x + threadIdx.x) / G; p < n_parts; p += groups) {
+    const uint32_t li = wk.part_u[p];
+    const uint32_t u = wk.long_u[li];
+    if (wk.urow[u] == kNoRow) continue;
+    const uint32_t k = p - wk.long_part0[li];
+    const uint32_t seg_end = wk.useg[u + 1];
+    const uint32_t begin = wk.useg[u] + k * kSegChunk;
+    const uint32_t end = begin + kSegChunk < seg_end ? begin + kSegChunk : seg_end;
+    D4 s[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
+    reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
+    double* dst = wk.partials + (size_t)p * tv.dim;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint32_t c4 = gl + v * G;
+      if (c4 * 4u < tv.dim) {
+        reinterpret_cast<double2*>(dst)[c4 * 2] = make_double2(s[v].x, s[v].y);
+        reinterpret_cast<double2*>(dst)[c4 * 2 + 1] = make_double2(s[v].z, s[v].w);
+      }
+    }
+  }
+}
+
+// One block per long ID: thread t owns column t (and t + 256, ...); the parts
+// are added in increasing order, so the combination order is fixed.
+__global__ void __launch_bounds__(256)
+combine_adagrad_kernel(TableView tv, Work wk) {
+  __shared__ double s_sum[8][256];
+  uint32_t n_long = tv.st->n_long;
+  if (n_long > wk.max_long) n_long = wk.max_long;
+  const uint32_t dim = tv.dim;
+  for (uint32_t li = blockIdx.x; li < n_long; li += gridDim.x) {
+    const uint32_t u = wk.long_u[li];
+    const uint32_t row_word = wk.urow[u];
+    if (row_word == kNoRow) continue;                 // block-uniform
+    const uint32_t m = wk.useg[u + 1] - wk.useg[u];
+    const uint32_t parts = (m + kSegChunk - 1) / kSegChunk;
+    const double* src = wk.partials + (size_t)wk.long_part0[li] * dim;
+    const unsigned long long id = wk.uid[u];
+    for (uint32_t cbase = 0; cbase < dim; cbase += 256) {
+      // 256 columns at a time; the 256 threads split into (256 / width) slices of parts
+      const uint32_t width = dim - cbase < 256 ? dim - cbase : 256;      // multiple of 4
+      uint32_t slices = 256 / width;
+      if (slices > 8) slices = 8;
+      const uint32_t col = threadIdx.x % width, slice = threadIdx.x / width;
+      double acc = 0.0;
+      if (slice < slices) {
+        const uint32_t per = (parts + slices - 1) / slices;
+        const uint32_t p_lo = slice * per, p_hi = p_lo + per < parts ? p_lo + per : parts;
+        for (uint32_t p = p_lo; p < p_hi; ++p) acc += src[(size_t)p * dim + cbase + col];
+        s_sum[slice][col] = acc;
+      }
+      __syncthreads();
+      if (threadIdx.x < width / 4) {
+        D4 g = D4{0.0, 0.0, 0.0, 0.0};
+        for (uint32_t s = 0; s < slices; ++s) {
+          g.x += s_sum[s][threadIdx.x * 4 + 0];
+          g.y += s_sum[s][threadIdx.x * 4 + 1];
+          g.z += s_sum[s][threadIdx.x * 4 + 2];
+          g.w += s_sum[s][threadIdx.x * 4 + 3];
+        }
+        update_row(tv, row_word, id, cbase / 4 + threadIdx.x, g);
+      }
+      __syncthreads();
+    }
+  }
+}
+
+}  // namespace mono

@@ -1,0 +1,335 @@
+// Mutating table kernels: count / stamp / admit for IDs that are already
+// tracked, cuckoo insertion of new IDs (Section 2.1: place at h0, displace the
+// occupant to its other bucket, repeat), the expiry sweep, and bulk import.
+#pragma once
+
+#include "kernels_dedup.cuh"
+#include "kernels_forward.cuh"
+
+namespace mono {
+
+// Take a free row.  Returns kNoRow (and records the refusal) when none is left.
+__device__ inline uint32_t alloc_row(const TableView& tv) {
+  const long long old = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top),
+                                              (unsigned long long)(-1LL));
+  if (old <= 0) {
+    atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), 1ull);
+    atomicOr(&tv.st->error_bits, 1u /* MONO_DEV_ROWS_FULL */);
+    atomicAdd(&tv.st->n_rows_refused, 1ull);
+    return kNoRow;
+  }
+  atomicAdd(&tv.st->n_resident, 1ull);
+  atomicAdd(&tv.st->n_admitted_total, 1ull);
+  return tv.free_rows[old - 1];
+}
+
+// Phase 2 of mono_apply_grads: one quad per distinct ID.  Tracked IDs get
+// count += multiplicity (saturating at the threshold), last_seen = now, and a
+// row if the count has reached the threshold; the rest are queued for
+// insertion.  No cell moves during this kernel, so the quad that found a cell
+// owns it.
+__global__ void __launch_bounds__(256)
+table_update_kernel(TableView tv, Work wk, uint32_t now) {
+  const uint32_t n = tv.st->n_unique;
+  const unsigned stash_hw = tv.st->stash_hw;
+  const int lane = threadIdx.x & 31, sub = lane & 3, quad = lane >> 2;
+  const unsigned quad_mask = 0xFu << (lane - sub);
+  const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
+  const uint32_t warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  unsigned int n_res = 0;
+  for (uint32_t u0 = warp_id * 8u; u0 < n; u0 += warps * 8u) {
+    const uint32_t u = u0 + quad;
+    const bool active = u < n;
+    unsigned long long id = kEmptyKey;
+    uint32_t m = 0;
+    if (active) { id = wk.uid[u]; m = wk.useg[u + 1] - wk.useg[u]; }
+
+    // locate the cell (pointer kept on the lane that saw the key)
+    Cell* where = nullptr;
+    unsigned long long meta = 0;
+    bool hit = false;
+    if (active) {
+      Cell* p = tv.cells + tv.bucket0(id) * kCellsPerBucket + sub;
+      const Cell c = *p;
+      if (c.key == id) { hit = true; where = p; meta = c.meta; }
+    }
+    bool found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
+    if (!found) {
+      if (active) {
+        Cell* p = tv.cells + tv.bucket1(id) * kCellsPerBucket + sub;
+        const Cell c = *p;
+        if (c.key == id) { hit = true; where = p; meta = c.meta; }
+      }
+      found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
+      if (!found && stash_hw != 0 && active) {
+        for (unsigned i = sub; i < stash_hw; i += kCellsPerBucket) {
+          const Cell c = tv.stash[i];
+          if (c.key == id) { hit = true; where = tv.stash + i; meta = c.meta; break; }
+        }
+      }
+      found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
+    }
+
+    if (hit) {
+      uint32_t low = meta_low(meta);
+      uint32_t row_word = kNoRow;
+      if (low & kResidentBit) {
+        row_word = low & ~kResidentBit;
+      } else {
+        const unsigned long long c = (unsigned long long)low + m;
+        low = c < tv.threshold ? (uint32_t)c : tv.threshold;
+        if (low >= tv.threshold) {
+          const uint32_t row = alloc_row(tv);
+          if (row != kNoRow) { low = kResidentBit | row; row_word = row | kFreshBit; }
+        }
+      }
+      where->meta = make_meta(now, low);
+      wk.urow[u] = row_word;
+      n_res += row_word != kNoRow;
+    }
+    // queue the IDs that are not tracked yet, one counter update per warp
+    const bool need_insert = active && !found && sub == 0;
+    const unsigned ins_mask = __ballot_sync(0xFFFFFFFFu, need_insert);
+    if (ins_mask) {
+      unsigned base = 0;
+      const int leader = __ffs(ins_mask) - 1;
+      if (lane == leader) base = atomicAdd(&tv.st->n_insert, (unsigned)__popc(ins_mask));
+      base = __shfl_sync(0xFFFFFFFFu, base, leader);
+      if (need_insert) wk.ins_list[base + __popc(ins_mask & ((1u << lane) - 1u))] = u;
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
+  if (lane == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
+}
+
+// Put `item` (a key that is in no cell) into the key store.  Lock-free against
+// other inserters: an empty cell is claimed, and an occupant displaced, with a
+// single 16-byte atomic, so every entry is at all times either in exactly one
+// cell or carried by exactly one thread.  The displacement chain is bounded;
+// what is still carried at the end goes to the stash, and if that is full the
+// entry is dropped and the condition recorded.
+__device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
+  const Cell empty = empty_cell();
+  unsigned long long bkt = tv.bucket0(item.key);
+  uint32_t rnd = (uint32_t)(item.key >> 17) * 2654435761u + 0x9E3779B9u;
+  uint32_t chain = 0;
+  bool placed = false;
+  for (;;) {
+    Cell* base = tv.cells + bkt * kCellsPerBucket;
+    for (uint32_t c = 0; c < kCellsPerBucket && !placed; ++c) {
+      Cell* p = base + ((c + rnd) & 3u);
+      if (*reinterpret_cast<volatile unsigned long long*>(&p->key) == kEmptyKey) {
+        const Cell old = atomicCAS(p, empty, item);
+        placed = old.key == kEmptyKey;
+      }
+    }
+    if (placed) break;
+    if (chain == 0) {
+      // a new ID may take an empty cell of its second bucket before displacing anyone
+      const unsigned long long alt = tv.bucket1(item.key);
+      Cell* abase = tv.cells + alt * kCellsPerBucket;
+      for (uint32_t c = 0; c < kCellsPerBucket && !placed && alt != bkt; ++c) {
+        Cell* p = abase + ((c + rnd) & 3u);
+        if (*reinterpret_cast<volatile unsigned long long*>(&p->key) == kEmptyKey) {
+          const Cell old = atomicCAS(p, empty, item);
+          placed = old.key == kEmptyKey;
+        }
+      }
+      if (placed) break;
+    }
+    if (chain >= kMaxChain) break;
+    ++chain;
+    rnd = rnd * 1664525u + 1013904223u;
+    const Cell old = atomicExch(base + (rnd >> 30), item);
+    if (old.key == kEmptyKey) { placed = true; break; }
+    item = old;
+    const unsigned long long b0 = tv.bucket0(item.key), b1 = tv.bucket1(item.key);
+    bkt = (b0 == bkt) ? b1 : b0;
+  }
+  if (chain) {
+    atomicAdd(&tv.st->n_evictions_total, (unsigned long long)chain);
+    atomicMax(&tv.st->max_chain, chain);
+  }
+  if (placed) return;
+  for (uint32_t i = 0; i < kStashCells; ++i) {
+    if (*reinterpret_cast<volatile unsigned long long*>(&tv.stash[i].key) == kEmptyKey) {
+      const Cell old = atomicCAS(tv.stash + i, empty, item);
+      if (old.key == kEmptyKey) { atomicMax(&tv.st->stash_hw, i + 1u); return; }
+    }
+  }
+  // nowhere to go: the carried entry is lost (its row, if any, stays allocated)
+  atomicOr(&tv.st->error_bits, 2u /* MONO_DEV_KEYS_FULL */);
+  atomicAdd(&tv.st->n_keys_dropped, 1ull);
+  atomicAdd(&tv.st->n_tracked, (unsigned long long)(-1LL));
+  if (meta_resident(item.meta)) atomicAdd(&tv.st->n_resident, (unsigned long long)(-1LL));
+}
+
+// Phase 3 of mono_apply_grads: one thread per new ID.
+__global__ void __launch_bounds__(256)
+table_insert_kernel(TableView tv, Work wk, uint32_t now) {
+  const uint32_t n = tv.st->n_insert;
+  const uint32_t stride = gridDim.x * blockDim.x;
+  const int lane = threadIdx.x & 31;
+  unsigned int n_res = 0, n_done = 0;
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const uint32_t u = wk.ins_list[i];
+    const unsigned long long id = wk.uid[u];
+    const uint32_t m = wk.useg[u + 1] - wk.useg[u];
+    uint32_t low = m < tv.threshold ? m : tv.threshold;
+    uint32_t row_word = kNoRow;
+    if (low >= tv.threshold) {
+      const uint32_t row = alloc_row(tv);
+      if (row != kNoRow) { low = kResidentBit | row; row_word = row | kFreshBit; }
+    }
+    wk.urow[u] = row_word;
+    Cell item; item.key = id; item.meta = make_meta(now, low);
+    cuckoo_insert(tv, item);
+    n_res += row_word != kNoRow;
+    ++n_done;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
+    n_done += __shfl_down_sync(0xFFFFFFFFu, n_done, o);
+  }
+  if (lane == 0) {
+    if (n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
+    if (n_done) {
+      atomicAdd(&tv.st->n_tracked, (unsigned long long)n_done);
+      atomicAdd(&tv.st->n_inserted_total, (unsigned long long)n_done);
+    }
+  }
+}
+
+// End of a mono_apply_grads call: fold the per-call counters into the totals.
+__global__ void finish_apply_kernel(DevState* st) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    st->sum_ids += st->n_valid_ids;
+    st->sum_unique += st->n_unique;
+    st->sum_new += st->n_insert;
+    st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_valid_ids = 0;
+  }
+}
+
+// Expiry sweep (Section 2.1, heuristic 2): a streaming pass over the key
+// store; a cell whose ID has been inactive for longer than ttl is emptied and
+// its row, if it has one, goes back on the free list.
+__global__ void __launch_bounds__(256)
+expire_kernel(TableView tv, unsigned long long n_cells, long long now) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long total = n_cells + kStashCells;
+  const int lane = threadIdx.x & 31;
+  unsigned int n_gone = 0, n_rows = 0;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    Cell* p = i < n_cells ? tv.cells + i : tv.stash + (i - n_cells);
+    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
+    if (v.x == kEmptyKey) continue;
+    if (now - (long long)meta_time(v.y) > (long long)tv.ttl) {
+      ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+      *reinterpret_cast<ulonglong2*>(p) = e;
+      ++n_gone;
+      if (meta_resident(v.y)) {
+        const unsigned long long pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), 1ull);
+        tv.free_rows[pos] = meta_row(v.y);
+        ++n_rows;
+      }
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    n_gone += __shfl_down_sync(0xFFFFFFFFu, n_gone, o);
+    n_rows += __shfl_down_sync(0xFFFFFFFFu, n_rows, o);
+  }
+  if (lane == 0 && n_gone) {
+    atomicAdd(&tv.st->n_tracked, (unsigned long long)(-(long long)n_gone));
+    atomicAdd(&tv.st->n_expired_total, (unsigned long long)n_gone);
+    if (n_rows) atomicAdd(&tv.st->n_resident, (unsigned long long)(-(long long)n_rows));
+  }
+}
+
+// After a sweep: if the stash has become empty, probes may skip it again.
+__global__ void stash_trim_kernel(TableView tv) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    unsigned hw = tv.st->stash_hw;
+    while (hw > 0 && tv.stash[hw - 1].key == kEmptyKey) --hw;
+    tv.st->stash_hw = hw;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+init_table_kernel(TableView tv, unsigned long long n_cells) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+  ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+  for (unsigned long long i = tid; i < n_cells; i += stride) *reinterpret_cast<ulonglong2*>(tv.cells + i) = e;
+  for (unsigned long long i = tid; i < kStashCells; i += stride) *reinterpret_cast<ulonglong2*>(tv.stash + i) = e;
+  // rows are handed out in increasing order from a fresh table
+  for (unsigned long long i = tid; i < tv.capacity; i += stride) tv.free_rows[i] = (uint32_t)(tv.capacity - 1 - i);
+}
+
+__global__ void __launch_bounds__(256)
+init_bset_kernel(BatchSlot* bset, unsigned long long n) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  BatchSlot e; e.key = kEmptyKey; e.count = 0; e.spare = 0;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) bset[i] = e;
+}
+
+// ---- bulk import -----------------------------------------------------------
+
+// One thread per entry: skip IDs that are already tracked, claim a row for
+// resident entries, insert.  row_word[i] tells import_rows_kernel where the
+// entry's values go.
+__global__ void __launch_bounds__(256)
+import_insert_kernel(TableView tv, const unsigned long long* __restrict__ ids, const uint32_t* __restrict__ count,
+                     const long long* __restrict__ last_seen, const uint8_t* __restrict__ resident,
+                     long long n, uint32_t* __restrict__ row_word) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const unsigned stash_hw = tv.st->stash_hw;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const unsigned long long id = ids[i];
+    row_word[i] = kNoRow;
+    if (id == kEmptyKey) continue;
+    bool present = false;
+    const unsigned long long bk[2] = {tv.bucket0(id), tv.bucket1(id)};
+    for (int b = 0; b < 2 && !present; ++b)
+      for (uint32_t c = 0; c < kCellsPerBucket; ++c)
+        present |= load_cell(tv.cells + bk[b] * kCellsPerBucket + c).key == id;
+    for (unsigned s = 0; s < stash_hw && !present; ++s) present |= load_cell(tv.stash + s).key == id;
+    if (present) { atomicOr(&tv.st->error_bits, 8u /* MONO_DEV_IMPORT_DUP */); continue; }
+    long long seen = last_seen[i];
+    if (seen < 0) seen = 0;
+    if (seen > 0xFFFFFFFELL) seen = 0xFFFFFFFELL;
+    uint32_t low = count[i] < tv.threshold ? count[i] : tv.threshold;
+    if (resident[i]) {
+      const uint32_t row = alloc_row(tv);
+      if (row != kNoRow) { low = kResidentBit | row; row_word[i] = row; }
+      else low = tv.threshold;
+    } else if (low >= tv.threshold) {
+      low = tv.threshold - 1;      // "not resident" entries stay below the threshold
+    }
+    Cell item; item.key = id; item.meta = make_meta((uint32_t)seen, low);
+    atomicAdd(&tv.st->n_tracked, 1ull);
+    atomicAdd(&tv.st->n_inserted_total, 1ull);
+    cuckoo_insert(tv, item);
+  }
+}
+
+// One lane group of 8 per entry copies (or initialises) the row and accumulator.
+__global__ void __launch_bounds__(256)
+import_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, const float* __restrict__ w,
+                   const float* __restrict__ acc, long long n, const uint32_t* __restrict__ row_word) {
+  const int gl = threadIdx.x & 7;
+  const long long groups = ((long long)gridDim.x * blockDim.x) >> 3;
+  const uint32_t dim4 = tv.dim / 4;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3; i < n; i += groups) {
+    const uint32_t row = row_word[i];
+    if (row == kNoRow) continue;
+    float4* dw = reinterpret_cast<float4*>(tv.w_row(row));
+    float4* da = reinterpret_cast<float4*>(tv.acc_row(row));
+    for (uint32_t c4 = gl; c4 < dim4; c4 += 8) {
+      dw[c4] = w ? reinterpret_cast<const float4*>(w + i * (long long)tv.dim)[c4] : init_vec(tv, ids[i], c4);
+      da[c4] = acc ? reinterpret_cast<const float4*>(acc + i * (long long)tv.dim)[c4]
+                   : make_float4(tv.init_acc, tv.init_acc, tv.init_acc, tv.init_acc);
+    }
+  }
+}
+
+}  // namespace mono

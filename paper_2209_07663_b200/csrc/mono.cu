@@ -1,0 +1,549 @@
+// Host side of the C ABI declared in include/mono.h: argument checks, memory
+// ownership, and the launch sequence of each call.  Every step of the hot path
+// runs in the kernels included below; nothing here computes on the host.
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/mono.h"
+#include "kernels_adagrad.cuh"
+#include "kernels_dedup.cuh"
+#include "kernels_forward.cuh"
+#include "kernels_inspect.cuh"
+#include "kernels_table.cuh"
+#include "table_layout.cuh"
+
+using namespace mono;
+
+enum KernelId {
+  K_LOOKUP, K_FILL_BAG, K_DEDUP, K_SEG_COUNT, K_SEG_SCAN, K_SEG_OFFSETS, K_PLACE, K_UPDATE, K_INSERT,
+  K_REDUCE, K_PARTS, K_COMBINE, K_RESET, K_FINISH, K_EXPIRE, K_STASH_TRIM, K_COUNT
+};
+static const char* const kKernelNames[K_COUNT] = {
+  "lookup_pool", "fill_occ_bag", "dedup_insert", "seg_count", "seg_scan_blocks", "seg_offsets", "place",
+  "table_update", "table_insert", "reduce_adagrad", "reduce_parts", "combine_adagrad", "dedup_reset",
+  "finish_apply", "expire", "stash_trim"
+};
+
+struct mono_table {
+  // per-kernel launch counts, and (when timing is on) CUDA-event durations
+  uint64_t launches[K_COUNT] = {};
+  double kernel_ms[K_COUNT] = {};
+  bool timing = false;
+  std::vector<cudaEvent_t> spare_events;
+  std::vector<std::pair<int, std::pair<cudaEvent_t, cudaEvent_t>>> pending;
+  cudaEvent_t open_event = nullptr;
+  TableView tv{};
+  Work wk{};
+  cudaStream_t stream = nullptr;
+  int sm_count = 148;
+  uint64_t key_cells = 0;
+  int64_t last_now = -1;
+  int64_t max_ids = 0, max_bags = 0;
+  // device staging for the host-buffer calls
+  unsigned long long* stage_ids = nullptr;
+  long long* stage_off = nullptr;
+  float* stage_vec = nullptr;
+  std::string last_err;
+};
+
+namespace {
+
+#define CUDA_TRY(t, expr)                                                         \
+  do {                                                                            \
+    cudaError_t e__ = (expr);                                                     \
+    if (e__ != cudaSuccess) {                                                     \
+      (t)->last_err = std::string(#expr) + ": " + cudaGetErrorString(e__);        \
+      return e__ == cudaErrorMemoryAllocation ? MONO_ERR_NOMEM : MONO_ERR_CUDA;   \
+    }                                                                             \
+  } while (0)
+
+inline bool is_pow2(uint64_t x) { return x && !(x & (x - 1)); }
+inline uint64_t next_pow2(uint64_t x) { uint64_t p = 1; while (p < x) p <<= 1; return p; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+template <typename T>
+int dev_alloc(mono_table* t, T** p, size_t n) {
+  *p = nullptr;
+  CUDA_TRY(t, cudaMalloc(reinterpret_cast<void**>(p), (n ? n : 1) * sizeof(T)));
+  return MONO_OK;
+}
+
+template <typename T>
+void dev_free(T*& p) { if (p) { cudaFree(p); p = nullptr; } }
+
+void free_scratch(mono_table* t) {
+  Work& w = t->wk;
+  dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
+  dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.urow); dev_free(w.ins_list);
+  dev_free(w.block_sums); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
+  dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec);
+  t->max_ids = t->max_bags = 0;
+}
+
+int grid_for(const mono_table* t, int per_sm) { return t->sm_count * per_sm; }
+
+cudaEvent_t take_event(mono_table* t) {
+  if (!t->spare_events.empty()) { cudaEvent_t e = t->spare_events.back(); t->spare_events.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+void launch_begin(mono_table* t, int kid) {
+  ++t->launches[kid];
+  if (t->timing) { t->open_event = take_event(t); cudaEventRecord(t->open_event, t->stream); }
+}
+void launch_end(mono_table* t, int kid) {
+  if (t->timing) {
+    cudaEvent_t stop = take_event(t);
+    cudaEventRecord(stop, t->stream);
+    t->pending.push_back({kid, {t->open_event, stop}});
+    t->open_event = nullptr;
+  }
+}
+// Every kernel of the hot calls is launched through this, so that launches can
+// be counted and, on request, timed one by one on the table's stream.
+#define LAUNCH(t, kid, ...) do { launch_begin((t), (kid)); __VA_ARGS__; launch_end((t), (kid)); } while (0)
+
+int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
+  if (max_ids <= t->max_ids && max_bags <= t->max_bags) return MONO_OK;
+  if (max_ids < t->max_ids) max_ids = t->max_ids;
+  if (max_bags < t->max_bags) max_bags = t->max_bags;
+  if (max_ids < 1024) max_ids = 1024;
+  if (max_bags < 1024) max_bags = 1024;
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  free_scratch(t);
+  Work& w = t->wk;
+  const size_t n = (size_t)max_ids;
+  const uint64_t slots = next_pow2(2 * (uint64_t)max_ids);
+  int rc;
+#define ALLOC(p, cnt) if ((rc = dev_alloc(t, &(p), (cnt))) != MONO_OK) { free_scratch(t); return rc; }
+  ALLOC(w.bset, slots);
+  ALLOC(w.occ_slot, n); ALLOC(w.occ_rank, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
+  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n + 1); ALLOC(w.urow, n); ALLOC(w.ins_list, n);
+  ALLOC(w.block_sums, (size_t)kScanBlocks + 1);
+  w.max_long = (uint32_t)(n / kSegChunk + 1);
+  w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
+  ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts);
+  ALLOC(w.partials, (size_t)w.max_parts * t->tv.dim);
+  ALLOC(t->stage_ids, n); ALLOC(t->stage_off, (size_t)max_bags + 1);
+  ALLOC(t->stage_vec, (size_t)max_bags * t->tv.dim);
+#undef ALLOC
+  w.bset_mask = slots - 1;
+  init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(w.bset, slots);
+  CUDA_TRY(t, cudaGetLastError());
+  t->max_ids = max_ids;
+  t->max_bags = max_bags;
+  return MONO_OK;
+}
+
+int check_batch(const mono_table* t, const void* ids, int64_t n_ids, const void* off, int64_t n_bags) {
+  if (!t || n_ids < 0 || n_bags < 0) return MONO_ERR_ARG;
+  if (n_ids >= (1ll << 31) || n_bags >= (1ll << 31)) return MONO_ERR_ARG;
+  if (!off || !aligned(off, 8)) return MONO_ERR_ARG;
+  if (n_ids > 0 && (!ids || !aligned(ids, 8))) return MONO_ERR_ARG;
+  return MONO_OK;
+}
+
+// lane-group width and column vectors per lane for a given dim
+template <typename F>
+int dispatch_dim(uint32_t dim, F&& f) {
+  if (dim <= 16) return f(std::integral_constant<int, 4>{}, std::integral_constant<int, 1>{});
+  if (dim <= 32) return f(std::integral_constant<int, 8>{}, std::integral_constant<int, 1>{});
+  if (dim <= 64) return f(std::integral_constant<int, 16>{}, std::integral_constant<int, 1>{});
+  if (dim <= 128) return f(std::integral_constant<int, 32>{}, std::integral_constant<int, 1>{});
+  if (dim <= 256) return f(std::integral_constant<int, 32>{}, std::integral_constant<int, 2>{});
+  if (dim <= 512) return f(std::integral_constant<int, 32>{}, std::integral_constant<int, 4>{});
+  return f(std::integral_constant<int, 32>{}, std::integral_constant<int, 8>{});
+}
+
+int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
+                  int64_t n_bags, float* out) {
+  if (n_bags == 0) return MONO_OK;
+  return dispatch_dim(t->tv.dim, [&](auto g, auto nv) -> int {
+    constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
+    const int64_t groups_per_block = 256 / G;
+    int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 4;
+    if (blocks > cap) blocks = cap;
+    LAUNCH(t, K_LOOKUP, lookup_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, off, n_bags, out));
+    CUDA_TRY(t, cudaGetLastError());
+    return (int)MONO_OK;
+  });
+}
+
+int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
+                 int64_t n_bags, const float* grad, uint32_t now) {
+  if (n_ids == 0 || n_bags == 0) return MONO_OK;
+  cudaStream_t s = t->stream;
+  const TableView& tv = t->tv;
+  const Work& wk = t->wk;
+  const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
+  LAUNCH(t, K_FILL_BAG, fill_occ_bag_kernel<<<g8, 256, 0, s>>>(off, n_bags, n_ids, wk.occ_bag, tv.st));
+  LAUNCH(t, K_DEDUP, dedup_insert_kernel<<<g8, 256, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
+                                                             tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
+  LAUNCH(t, K_SEG_COUNT, seg_count_kernel<<<kScanBlocks, kScanThreads, 0, s>>>(wk, tv.st));
+  LAUNCH(t, K_SEG_SCAN, seg_scan_blocks_kernel<<<1, 32, 0, s>>>(wk));
+  LAUNCH(t, K_SEG_OFFSETS, seg_offsets_kernel<<<kScanBlocks, kScanThreads, 0, s>>>(wk, tv.st));
+  LAUNCH(t, K_PLACE, place_kernel<<<g8, 256, 0, s>>>(wk, n_ids));
+  LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
+  LAUNCH(t, K_INSERT, table_insert_kernel<<<g4, 256, 0, s>>>(tv, wk, now));
+  CUDA_TRY(t, cudaGetLastError());
+  const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
+    constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
+    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
+    LAUNCH(t, K_PARTS, reduce_parts_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
+    return (int)MONO_OK;
+  });
+  if (rc != MONO_OK) return rc;
+  LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g4, 256, 0, s>>>(tv, wk));
+  LAUNCH(t, K_RESET, dedup_reset_kernel<<<g8, 256, 0, s>>>(wk, tv.st));
+  LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 32, 0, s>>>(tv.st));
+  CUDA_TRY(t, cudaGetLastError());
+  return MONO_OK;
+}
+
+int check_now(mono_table* t, int64_t now) {
+  if (now < 0 || now > MONO_MAX_NOW || now < t->last_now) return MONO_ERR_TIME;
+  return MONO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_t filter_threshold,
+                      uint32_t ttl, const mono_opt* opt, void* cuda_stream) {
+  if (!out) return MONO_ERR_ARG;
+  *out = nullptr;
+  if (capacity == 0 || capacity > MONO_MAX_CAPACITY) return MONO_ERR_ARG;
+  if (dim < 4 || dim > MONO_MAX_DIM || (dim & 3u)) return MONO_ERR_ARG;
+  if (filter_threshold >= 0x7FFFFFFFu) return MONO_ERR_ARG;
+  mono_opt o;
+  std::memset(&o, 0, sizeof(o));
+  if (opt) o = *opt; else { o.lr = 0.05f; o.eps = 1e-8f; }
+  if (o.kind != 0 && o.kind != MONO_OPT_ADAGRAD) return MONO_ERR_ARG;
+  uint64_t key_cells = o.key_cells ? o.key_cells : next_pow2(4 * capacity);
+  if (!is_pow2(key_cells) || key_cells < 64 || key_cells > (1ull << 34)) return MONO_ERR_ARG;
+  if (o.max_ids >= (1ull << 31) || o.max_bags >= (1ull << 31)) return MONO_ERR_ARG;
+
+  mono_table* t = new (std::nothrow) mono_table();
+  if (!t) return MONO_ERR_NOMEM;
+  t->stream = static_cast<cudaStream_t>(cuda_stream);
+  t->key_cells = key_cells;
+  int dev = 0, rc = MONO_OK;
+  auto fail = [&](int code) { mono_table_destroy(t); return code; };
+  if (cudaGetDevice(&dev) != cudaSuccess) return fail(MONO_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || t->sm_count < 1)
+    return fail(MONO_ERR_CUDA);
+
+  TableView& tv = t->tv;
+  tv.bucket_mask = key_cells / kCellsPerBucket - 1;
+  tv.seed0 = mix_a(o.seed + 0x1234567ull);
+  tv.seed1 = mix_b(o.seed + 0x89ABCDEFull);
+  tv.capacity = capacity;
+  tv.dim = dim;
+  tv.threshold = filter_threshold ? filter_threshold : 1u;
+  tv.ttl = ttl;
+  tv.lr = o.lr; tv.eps = o.eps; tv.init_acc = o.init_acc; tv.init_scale = o.init_scale;
+  tv.init_key0 = (uint32_t)o.seed;
+  tv.init_key1 = (uint32_t)(o.seed >> 32);
+  if ((rc = dev_alloc(t, &tv.cells, key_cells)) != MONO_OK) return fail(rc);
+  if ((rc = dev_alloc(t, &tv.stash, kStashCells)) != MONO_OK) return fail(rc);
+  if ((rc = dev_alloc(t, &tv.rows, (size_t)capacity * 2 * dim)) != MONO_OK) return fail(rc);
+  if ((rc = dev_alloc(t, &tv.free_rows, capacity)) != MONO_OK) return fail(rc);
+  if ((rc = dev_alloc(t, &tv.st, 1)) != MONO_OK) return fail(rc);
+  DevState init;
+  std::memset(&init, 0, sizeof(init));
+  init.free_top = (long long)capacity;
+  if (cudaMemcpyAsync(tv.st, &init, sizeof(init), cudaMemcpyHostToDevice, t->stream) != cudaSuccess ||
+      cudaStreamSynchronize(t->stream) != cudaSuccess)
+    return fail(MONO_ERR_CUDA);
+  init_table_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(tv, key_cells);
+  if (cudaGetLastError() != cudaSuccess) return fail(MONO_ERR_CUDA);
+  if (o.max_ids || o.max_bags) {
+    if ((rc = reserve(t, (int64_t)o.max_ids, (int64_t)o.max_bags)) != MONO_OK) return fail(rc);
+  }
+  if (cudaStreamSynchronize(t->stream) != cudaSuccess) return fail(MONO_ERR_CUDA);
+  *out = t;
+  return MONO_OK;
+}
+
+int mono_table_destroy(mono_table* t) {
+  if (!t) return MONO_ERR_ARG;
+  cudaStreamSynchronize(t->stream);
+  for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
+  for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
+  free_scratch(t);
+  dev_free(t->tv.cells); dev_free(t->tv.stash); dev_free(t->tv.rows); dev_free(t->tv.free_rows); dev_free(t->tv.st);
+  delete t;
+  return MONO_OK;
+}
+
+int mono_reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
+  if (!t || max_ids < 0 || max_bags < 0 || max_ids >= (1ll << 31) || max_bags >= (1ll << 31)) return MONO_ERR_ARG;
+  return reserve(t, max_ids, max_bags);
+}
+
+int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                     int64_t n_bags, float* out) {
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
+  return launch_lookup(t, reinterpret_cast<const unsigned long long*>(ids), n_ids,
+                       reinterpret_cast<const long long*>(slot_offsets), n_bags, out);
+}
+
+int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                     int64_t n_bags, const float* grad_pooled, int64_t now) {
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if (n_bags > 0 && (!grad_pooled || !aligned(grad_pooled, 16))) return MONO_ERR_ARG;
+  if ((rc = check_now(t, now)) != MONO_OK) return rc;
+  if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  t->last_now = now;
+  return launch_apply(t, reinterpret_cast<const unsigned long long*>(ids), n_ids,
+                      reinterpret_cast<const long long*>(slot_offsets), n_bags, grad_pooled, (uint32_t)now);
+}
+
+int mono_expire(mono_table* t, int64_t now) {
+  if (!t) return MONO_ERR_ARG;
+  int rc = check_now(t, now);
+  if (rc != MONO_OK) return rc;
+  t->last_now = now;
+  if (t->tv.ttl == 0) return MONO_OK;
+  LAUNCH(t, K_EXPIRE, expire_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells, (long long)now));
+  LAUNCH(t, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, t->stream>>>(t->tv));
+  CUDA_TRY(t, cudaGetLastError());
+  return MONO_OK;
+}
+
+int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                          int64_t n_bags, float* out) {
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if (n_bags > 0 && !out) return MONO_ERR_ARG;
+  if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  cudaStream_t s = t->stream;
+  if (n_ids) CUDA_TRY(t, cudaMemcpyAsync(t->stage_ids, ids, (size_t)n_ids * 8, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(t, cudaMemcpyAsync(t->stage_off, slot_offsets, (size_t)(n_bags + 1) * 8, cudaMemcpyHostToDevice, s));
+  if ((rc = launch_lookup(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec)) != MONO_OK) return rc;
+  if (n_bags)
+    CUDA_TRY(t, cudaMemcpyAsync(out, t->stage_vec, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(t, cudaStreamSynchronize(s));
+  return MONO_OK;
+}
+
+int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                          int64_t n_bags, const float* grad_pooled, int64_t now) {
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if (n_bags > 0 && !grad_pooled) return MONO_ERR_ARG;
+  if ((rc = check_now(t, now)) != MONO_OK) return rc;
+  if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  cudaStream_t s = t->stream;
+  if (n_ids) CUDA_TRY(t, cudaMemcpyAsync(t->stage_ids, ids, (size_t)n_ids * 8, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(t, cudaMemcpyAsync(t->stage_off, slot_offsets, (size_t)(n_bags + 1) * 8, cudaMemcpyHostToDevice, s));
+  if (n_bags)
+    CUDA_TRY(t, cudaMemcpyAsync(t->stage_vec, grad_pooled, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyHostToDevice, s));
+  t->last_now = now;
+  return launch_apply(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec, (uint32_t)now);
+}
+
+int mono_status(mono_table* t, mono_status_t* host_out) {
+  if (!t || !host_out) return MONO_ERR_ARG;
+  DevState d;
+  CUDA_TRY(t, cudaMemcpyAsync(&d, t->tv.st, sizeof(d), cudaMemcpyDeviceToHost, t->stream));
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  std::memset(host_out, 0, sizeof(*host_out));
+  host_out->error_bits = d.error_bits;
+  host_out->dim = t->tv.dim;
+  host_out->capacity = t->tv.capacity;
+  host_out->key_cells = t->key_cells;
+  host_out->n_tracked = d.n_tracked;
+  host_out->n_resident = d.n_resident;
+  host_out->n_admitted_total = d.n_admitted_total;
+  host_out->n_expired_total = d.n_expired_total;
+  host_out->n_inserted_total = d.n_inserted_total;
+  host_out->n_rows_refused = d.n_rows_refused;
+  host_out->n_keys_dropped = d.n_keys_dropped;
+  host_out->n_evictions_total = d.n_evictions_total;
+  host_out->max_chain = d.max_chain;
+  host_out->stash_used = d.stash_hw;
+  host_out->sum_ids = d.sum_ids;
+  host_out->sum_unique = d.sum_unique;
+  host_out->sum_unique_resident = d.sum_unique_resident;
+  host_out->sum_new = d.sum_new;
+  return MONO_OK;
+}
+
+int mono_clear_errors(mono_table* t) {
+  if (!t) return MONO_ERR_ARG;
+  CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->error_bits, 0, sizeof(unsigned int), t->stream));
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  return MONO_OK;
+}
+
+int mono_probe(mono_table* t, const uint64_t* ids, int64_t n, uint8_t* resident, uint32_t* count,
+               int64_t* last_seen) {
+  if (!t || n < 0 || (n > 0 && (!ids || !aligned(ids, 8)))) return MONO_ERR_ARG;
+  if (n > 0) {
+    probe_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(t->tv, reinterpret_cast<const unsigned long long*>(ids), n,
+                                                        resident, count, reinterpret_cast<long long*>(last_seen));
+    CUDA_TRY(t, cudaGetLastError());
+  }
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  return MONO_OK;
+}
+
+int mono_read_rows(mono_table* t, const uint64_t* ids, int64_t n, float* w, float* acc) {
+  if (!t || n < 0 || (n > 0 && (!ids || !aligned(ids, 8)))) return MONO_ERR_ARG;
+  if ((w && !aligned(w, 16)) || (acc && !aligned(acc, 16))) return MONO_ERR_ARG;
+  if (n > 0) {
+    read_rows_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(t->tv, reinterpret_cast<const unsigned long long*>(ids),
+                                                            n, w, acc);
+    CUDA_TRY(t, cudaGetLastError());
+  }
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  return MONO_OK;
+}
+
+int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_seen, uint8_t* resident,
+                float* w, float* acc, int64_t max_n, int64_t* n_out) {
+  if (!t || !n_out || max_n < 0 || (max_n > 0 && !ids)) return MONO_ERR_ARG;
+  CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->export_n, 0, sizeof(unsigned long long), t->stream));
+  export_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells,
+                                                       reinterpret_cast<unsigned long long*>(ids), count,
+                                                       reinterpret_cast<long long*>(last_seen), resident, w, acc, max_n);
+  CUDA_TRY(t, cudaGetLastError());
+  unsigned long long n = 0;
+  CUDA_TRY(t, cudaMemcpyAsync(&n, &t->tv.st->export_n, sizeof(n), cudaMemcpyDeviceToHost, t->stream));
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  *n_out = (int64_t)n;
+  return (int64_t)n > max_n ? MONO_ERR_SIZE : MONO_OK;
+}
+
+int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const int64_t* last_seen,
+                const uint8_t* resident, const float* w, const float* acc, int64_t n) {
+  if (!t || n < 0) return MONO_ERR_ARG;
+  if (n == 0) return MONO_OK;
+  if (!ids || !count || !last_seen || !resident || !aligned(ids, 8)) return MONO_ERR_ARG;
+  if ((w && !aligned(w, 16)) || (acc && !aligned(acc, 16))) return MONO_ERR_ARG;
+  uint32_t* row_word = nullptr;
+  const int64_t chunk = n < (1ll << 24) ? n : (1ll << 24);
+  int rc = dev_alloc(t, &row_word, (size_t)chunk);
+  if (rc != MONO_OK) return rc;
+  for (int64_t lo = 0; lo < n; lo += chunk) {
+    const int64_t m = n - lo < chunk ? n - lo : chunk;
+    const size_t ro = (size_t)lo * t->tv.dim;
+    import_insert_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(
+        t->tv, reinterpret_cast<const unsigned long long*>(ids) + lo, count + lo,
+        reinterpret_cast<const long long*>(last_seen) + lo, resident + lo, m, row_word);
+    import_rows_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(
+        t->tv, reinterpret_cast<const unsigned long long*>(ids) + lo, w ? w + ro : nullptr, acc ? acc + ro : nullptr,
+        m, row_word);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaStreamSynchronize(t->stream);
+  cudaFree(row_word);
+  if (e != cudaSuccess) { t->last_err = cudaGetErrorString(e); return MONO_ERR_CUDA; }
+  return MONO_OK;
+}
+
+int mono_audit(mono_table* t, mono_audit_t* host_out) {
+  if (!t || !host_out) return MONO_ERR_ARG;
+  std::memset(host_out, 0, sizeof(*host_out));
+  unsigned int* marks = nullptr;
+  AuditCounters* ctr = nullptr;
+  const size_t words = (size_t)((t->tv.capacity + 31) / 32);
+  int rc = dev_alloc(t, &marks, words);
+  if (rc == MONO_OK) rc = dev_alloc(t, &ctr, 1);
+  AuditCounters h;
+  std::memset(&h, 0, sizeof(h));
+  DevState d;
+  cudaError_t e = cudaSuccess;
+  if (rc == MONO_OK) {
+    cudaStream_t s = t->stream;
+    e = cudaMemsetAsync(marks, 0, words * sizeof(unsigned int), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctr, 0, sizeof(AuditCounters), s);
+    if (e == cudaSuccess) {
+      audit_cells_kernel<<<grid_for(t, 8), 256, 0, s>>>(t->tv, t->key_cells, marks, ctr);
+      audit_free_kernel<<<grid_for(t, 8), 256, 0, s>>>(t->tv, marks, ctr);
+      audit_rows_kernel<<<grid_for(t, 8), 256, 0, s>>>(t->tv, marks, ctr);
+      e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&h, ctr, sizeof(h), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&d, t->tv.st, sizeof(d), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  }
+  if (marks) cudaFree(marks);
+  if (ctr) cudaFree(ctr);
+  if (rc != MONO_OK) return rc;
+  if (e != cudaSuccess) { t->last_err = cudaGetErrorString(e); return MONO_ERR_CUDA; }
+  host_out->occupied_cells = h.occupied;
+  host_out->misplaced = h.misplaced;
+  host_out->duplicate_keys = h.duplicate_keys;
+  host_out->resident_cells = h.resident_cells;
+  host_out->bad_rows = h.bad_rows;
+  host_out->shared_rows = h.shared_rows;
+  host_out->free_rows = h.free_rows;
+  host_out->unaccounted_rows = h.unaccounted_rows;
+  const bool leak_ok = h.unaccounted_rows == 0 || d.n_keys_dropped > 0;   // a dropped key may strand its row
+  host_out->ok = (h.misplaced == 0 && h.duplicate_keys == 0 && h.bad_rows == 0 && h.shared_rows == 0 && leak_ok &&
+                  h.occupied == d.n_tracked && h.resident_cells == d.n_resident &&
+                  h.resident_cells + h.free_rows + h.unaccounted_rows == t->tv.capacity)
+                     ? 1u : 0u;
+  return MONO_OK;
+}
+
+int mono_timing_enable(mono_table* t, int on) {
+  if (!t) return MONO_ERR_ARG;
+  t->timing = on != 0;
+  return MONO_OK;
+}
+
+int mono_timing_read(mono_table* t, mono_timing_t* host_out, int reset) {
+  if (!t || !host_out) return MONO_ERR_ARG;
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  for (auto& p : t->pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p.second.first, p.second.second) == cudaSuccess) t->kernel_ms[p.first] += ms;
+    t->spare_events.push_back(p.second.first);
+    t->spare_events.push_back(p.second.second);
+  }
+  t->pending.clear();
+  std::memset(host_out, 0, sizeof(*host_out));
+  host_out->n_kernels = K_COUNT;
+  for (int k = 0; k < K_COUNT; ++k) {
+    std::strncpy(host_out->kernel[k].name, kKernelNames[k], sizeof(host_out->kernel[k].name) - 1);
+    host_out->kernel[k].launches = t->launches[k];
+    host_out->kernel[k].ms = t->kernel_ms[k];
+    host_out->launches_total += t->launches[k];
+  }
+  if (reset) {
+    for (int k = 0; k < K_COUNT; ++k) { t->launches[k] = 0; t->kernel_ms[k] = 0.0; }
+  }
+  return MONO_OK;
+}
+
+const char* mono_last_cuda_error(mono_table* t) { return t ? t->last_err.c_str() : ""; }
+
+const char* mono_error_string(int code) {
+  switch (code) {
+    case MONO_OK: return "MONO_OK";
+    case MONO_ERR_ARG: return "MONO_ERR_ARG";
+    case MONO_ERR_TIME: return "MONO_ERR_TIME";
+    case MONO_ERR_CUDA: return "MONO_ERR_CUDA";
+    case MONO_ERR_NOMEM: return "MONO_ERR_NOMEM";
+    case MONO_ERR_SIZE: return "MONO_ERR_SIZE";
+    default: return "MONO_ERR_UNKNOWN";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+"""Shared helpers of the GPU parity tests: run the same seeded steps through the
+CPU oracle and the CUDA library and compare the complete table state.
+
+Integer state (tracked set, resident set, counts, last-seen times) must be
+bit-exact.  Floating point is compared per vector (a pooled bag, a row, an
+accumulator row):  max|gpu - oracle| <= TOL * max|oracle|, and an all-zero
+oracle vector must be all-zero on the GPU.  TOL is the 1e-5 the table's
+specification states for fp32 results.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+TOL = 1e-5
+
+
+def assert_vectors_close(got: np.ndarray, want: np.ndarray, what: str, tol: float = TOL):
+    assert got.shape == want.shape, f"{what}: shape {got.shape} vs {want.shape}"
+    if got.size == 0:
+        return
+    got64, want64 = got.astype(np.float64), want.astype(np.float64)
+    err = np.abs(got64 - want64).reshape(got.shape[0], -1).max(axis=1)
+    ref = np.abs(want64).reshape(got.shape[0], -1).max(axis=1)
+    bad = err > tol * ref
+    if bad.any():
+        k = int(np.argmax(err - tol * ref))
+        raise AssertionError(f"{what}: {int(bad.sum())} of {len(bad)} vectors off; worst vector {k}: "
+                             f"err {err[k]:.3e} vs ref {ref[k]:.3e}\n got {got[k][:8]}\nwant {want[k][:8]}")
+
+
+def assert_state_equal(gpu_table, oracle, what: str = "state", rows: bool = True):
+    """Full-table comparison through mono_export / oracle export (both sorted by ID)."""
+    g, o = gpu_table.export(rows=rows), oracle.export()
+    assert len(g["ids"]) == len(o["ids"]), f"{what}: tracked {len(g['ids'])} vs oracle {len(o['ids'])}"
+    assert (g["ids"] == o["ids"]).all(), f"{what}: tracked ID sets differ"
+    assert (g["resident"] == o["resident"]).all(), f"{what}: resident sets differ"
+    assert (g["count"] == o["count"]).all(), f"{what}: counts differ"
+    assert (g["last_seen"] == o["last_seen"]).all(), f"{what}: last_seen differ"
+    st = gpu_table.status()
+    assert st["n_tracked"] == oracle.n_tracked and st["n_resident"] == oracle.n_resident
+    if rows:
+        assert_vectors_close(g["w"], o["w"], f"{what}: rows")
+        assert_vectors_close(g["acc"], o["acc"], f"{what}: accumulators")
+
+
+def assert_audit_ok(gpu_table, what: str = "audit"):
+    a = gpu_table.audit()
+    assert a["ok"] == 1, f"{what}: {a}"
+    return a
+
+
+def run_stream(gpu_table, oracle, stream, steps, *, sweep_every: int = 1, check_every: int = 1,
+               time_scale: int = 1, check_forward: bool = True):
+    """Feed steps [0, steps) of `stream` to both sides; compare as it goes."""
+    for t in range(steps):
+        s = stream.step(t)
+        now = t * time_scale
+        if check_forward:
+            got = gpu_table.lookup_pool(s.ids, s.offsets).cpu().numpy()
+            assert_vectors_close(got, oracle.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+        gpu_table.apply_grads(s.ids, s.offsets, s.grad_pooled, now)
+        assert oracle.apply_grads(s.ids, s.offsets, s.grad_pooled, now) == 0, "stream overflowed the oracle"
+        if sweep_every and t % sweep_every == sweep_every - 1:
+            gpu_table.expire(now)
+            oracle.expire(now)
+        if check_every and (t % check_every == check_every - 1 or t == steps - 1):
+            assert_state_equal(gpu_table, oracle, f"step {t}")
+            assert_audit_ok(gpu_table, f"step {t}")
+    st = gpu_table.status()
+    assert st["error_bits"] == 0, f"device error bits {st['error_bits']}"
+    return st

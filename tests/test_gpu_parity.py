@@ -1,0 +1,358 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded inputs,
+through the C ABI.  Every test here needs a CUDA device.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mono_oracle as mo
+from paper_2209_07663_b200 import binding as mb
+from paper_2209_07663_b200 import workload as wl
+from tests.parity import assert_audit_ok, assert_state_equal, assert_vectors_close, run_stream
+
+pytestmark = pytest.mark.gpu
+f32 = np.float32
+
+
+def make_pair(cfg, **over):
+    kw = dict(lr=cfg.lr, eps=cfg.eps, init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed)
+    kw.update(over)
+    gpu = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, key_cells=cfg.key_cells, **kw)
+    cpu = mo.OracleTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, **kw)
+    return gpu, cpu
+
+
+def bags(lists):
+    ids = np.array([i for b in lists for i in b], dtype=np.uint64)
+    off = np.zeros(len(lists) + 1, np.int64)
+    off[1:] = np.cumsum([len(b) for b in lists])
+    return ids, off
+
+
+# ---------------------------------------------------------------- configured streams
+
+def test_tiny_config_full_stream():
+    cfg = wl.CONFIGS["tiny"]
+    gpu, cpu = make_pair(cfg)
+    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=1)
+    assert st["n_expired_total"] > 0 and st["n_admitted_total"] > 0
+    assert st["n_tracked"] > st["n_resident"] > 0
+
+
+def test_medium_config_prefix():
+    cfg = wl.scaled(wl.CONFIGS["medium"], steps=8)
+    gpu, cpu = make_pair(cfg)
+    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=4, check_every=4)
+
+
+def test_medium_config_short_ttl_churn():
+    # the medium shape with a TTL short enough that rows are recycled many times
+    cfg = wl.scaled(wl.CONFIGS["medium"], steps=10, ttl=2, n_examples=2048, capacity=1 << 18, key_cells=1 << 20)
+    gpu, cpu = make_pair(cfg)
+    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5)
+    assert st["n_expired_total"] > 10000
+
+
+def test_drift_config_scaled_down():
+    cfg = wl.scaled(wl.CONFIGS["drift"], n_examples=512, n_slots=10, n_distinct=1 << 18, capacity=1 << 16,
+                    key_cells=1 << 18, ttl=6, drift_period=4, steps=16)
+    gpu, cpu = make_pair(cfg)
+    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=4)
+
+
+@pytest.mark.parametrize("dim", [4, 8, 12, 16, 32, 48, 64, 128, 200, 256, 512, 1024])
+def test_every_dim_variant(dim):
+    cfg = wl.scaled(wl.CONFIGS["tiny"], dim=dim, n_examples=160, n_slots=5, n_distinct=1 << 12, steps=6,
+                    capacity=1 << 12, key_cells=1 << 13, bag_len=("uniform", 0, 9))
+    gpu, cpu = make_pair(cfg)
+    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=3)
+
+
+def test_multi_table_configs_scaled_down():
+    for cfg in wl.multi_table_configs(n_examples=256, slots_per_table=3):
+        cfg = wl.scaled(cfg, capacity=1 << 13, key_cells=1 << 15, n_distinct=1 << 14, steps=5, ttl=3)
+        gpu, cpu = make_pair(cfg)
+        run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5)
+
+
+# ---------------------------------------------------------------- edge cases
+
+def test_empty_inputs_and_padding():
+    gpu = mb.MonoTable(64, 8, 1, 0, init_scale=0.1, seed=3)
+    cpu = mo.OracleTable(64, 8, 1, 0, init_scale=0.1, seed=3)
+    # no IDs at all, one empty bag
+    ids, off = bags([[]])
+    assert not gpu.lookup_pool(ids, off).cpu().numpy().any()
+    gpu.apply_grads(ids, off, np.ones((1, 8), f32), 0)
+    assert gpu.status()["n_tracked"] == 0
+    # zero bags
+    gpu.apply_grads(np.zeros(0, np.uint64), np.zeros(1, np.int64), np.zeros((0, 8), f32), 0)
+    # padding IDs, empty bags in between, an ID repeated inside one bag
+    lists = [[5, mb.MONO_RESERVED_ID, 5], [], [mb.MONO_RESERVED_ID], [6, 7, 5], []]
+    ids, off = bags(lists)
+    grad = np.arange(40, dtype=f32).reshape(5, 8) / 7
+    for t in range(3):
+        gpu.apply_grads(ids, off, grad, t)
+        cpu.apply_grads(ids, off, grad, t)
+        assert_vectors_close(gpu.lookup_pool(ids, off).cpu().numpy(), cpu.lookup_pool(ids, off), "padding pooled")
+    assert_state_equal(gpu, cpu)
+    assert gpu.status()["n_tracked"] == 3 and gpu.status()["sum_ids"] == 15
+
+
+def test_offsets_that_skip_ids():
+    # offsets may start after 0 and end before n_ids: IDs outside every bag are ignored
+    gpu = mb.MonoTable(64, 4, 1, 0, init_scale=0.1)
+    cpu = mo.OracleTable(64, 4, 1, 0, init_scale=0.1)
+    ids = np.array([1, 2, 3, 4, 5, 6], np.uint64)
+    off = np.array([1, 3, 5], np.int64)
+    grad = np.ones((2, 4), f32)
+    gpu.apply_grads(ids, off, grad, 0)
+    cpu.apply_grads(ids, off, grad, 0)
+    assert_state_equal(gpu, cpu)
+    assert gpu.export()["ids"].tolist() == [2, 3, 4, 5]
+    assert_vectors_close(gpu.lookup_pool(ids, off).cpu().numpy(), cpu.lookup_pool(ids, off), "pooled")
+
+
+@pytest.mark.parametrize("n_occ", [255, 256, 257, 1000, 70000])
+def test_one_hot_id_long_segment(n_occ):
+    # a single ID owning a whole batch: the segment is split into parts and recombined
+    dim = 64
+    rng = np.random.default_rng(n_occ)
+    gpu = mb.MonoTable(64, dim, 3, 0, init_scale=0.05, seed=9)
+    cpu = mo.OracleTable(64, dim, 3, 0, init_scale=0.05, seed=9)
+    n_bags = max(n_occ // 3, 1)
+    lens = np.full(n_bags, 3)
+    lens[-1] += n_occ - lens.sum()
+    off = np.zeros(n_bags + 1, np.int64)
+    off[1:] = np.cumsum(lens)
+    ids = np.full(n_occ, 0xABCDEF0123456789, np.uint64)
+    ids[::97] = 77          # a second, cooler ID mixed in
+    for t in range(2):
+        grad = (rng.standard_normal((n_bags, dim)) * 0.01).astype(f32)
+        gpu.apply_grads(ids, off, grad, t)
+        cpu.apply_grads(ids, off, grad, t)
+    assert_state_equal(gpu, cpu)
+    assert_vectors_close(gpu.lookup_pool(ids[:7], np.array([0, 7], np.int64)).cpu().numpy(),
+                         cpu.lookup_pool(ids[:7], np.array([0, 7], np.int64)), "pooled hot")
+
+
+def test_forward_equals_torch_embedding_bag():
+    rng = np.random.default_rng(5)
+    V, d, B = 3000, 32, 5000
+    W = rng.standard_normal((V, d)).astype(f32)
+    id_of_row = wl.splitmix64(np.arange(V, dtype=np.uint64) + np.uint64(31337))
+    gpu = mb.MonoTable(4096, d, 1, 0)
+    gpu.import_entries(id_of_row, np.ones(V, np.uint32), np.zeros(V, np.int64), np.ones(V, np.uint8), W,
+                       np.zeros((V, d), f32))
+    lens = rng.integers(0, 9, B)
+    off = np.zeros(B + 1, np.int64)
+    off[1:] = np.cumsum(lens)
+    rows = rng.integers(0, V, off[-1])
+    got = gpu.lookup_pool(id_of_row[rows], off).cpu().numpy()
+    ref = torch.nn.functional.embedding_bag(torch.from_numpy(rows), torch.from_numpy(W.astype(np.float64)),
+                                            torch.from_numpy(off[:-1]), mode="sum").numpy()
+    assert_vectors_close(got, ref.astype(f32), "embedding_bag")
+    assert_audit_ok(gpu)
+
+
+def test_host_buffer_calls_match_device_calls():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=256, steps=4)
+    a, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        ids = torch.from_numpy(s.ids.view(np.int64)).pin_memory()
+        off = torch.from_numpy(s.offsets).pin_memory()
+        grad = torch.from_numpy(s.grad_pooled).pin_memory()
+        out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32).pin_memory()
+        mb.mono_lookup_pool_host(a.handle, ids, ids.numel(), off, cfg.n_bags, out)
+        assert_vectors_close(out.numpy(), cpu.lookup_pool(s.ids, s.offsets), f"host pooled {t}")
+        mb.mono_apply_grads_host(a.handle, ids, ids.numel(), off, cfg.n_bags, grad, t)
+        torch.cuda.synchronize()
+        cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+    assert_state_equal(a, cpu)
+
+
+# ---------------------------------------------------------------- expiry, recycling, import/export
+
+def test_expiry_sets_and_row_recycling():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, ttl=2, capacity=1 << 12, key_cells=1 << 15, steps=14,
+                    filter_threshold=1, n_distinct=1 << 14)
+    gpu, cpu = make_pair(cfg)
+    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=1)
+    # more rows were handed out than exist: expired rows were reused, never shared
+    assert st["n_admitted_total"] > cfg.capacity
+    a = assert_audit_ok(gpu)
+    assert a["resident_cells"] + a["free_rows"] == cfg.capacity
+
+
+def test_unswept_entries_survive_and_refresh():
+    gpu = mb.MonoTable(64, 4, 1, 3, init_scale=0.1)
+    cpu = mo.OracleTable(64, 4, 1, 3, init_scale=0.1)
+    g = np.ones((1, 4), f32)
+    for now, lists in [(0, [[1, 2]]), (10, [[1]]), (11, [[3]])]:
+        ids, off = bags(lists)
+        gpu.apply_grads(ids, off, g, now)
+        cpu.apply_grads(ids, off, g, now)
+    assert_state_equal(gpu, cpu, "before sweep")       # 2 is stale but still there
+    gpu.expire(13); cpu.expire(13)
+    assert_state_equal(gpu, cpu, "after sweep(13)")    # 2 gone; 1 (10) and 3 (11) stay
+    gpu.expire(14); cpu.expire(14)
+    assert_state_equal(gpu, cpu, "after sweep(14)")    # 14-10 > 3: 1 gone
+    assert gpu.export()["ids"].tolist() == [3]
+
+
+def test_export_import_roundtrip_into_a_differently_seeded_table():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=6)
+    gpu, cpu = make_pair(cfg)
+    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=0, check_every=0, check_forward=False)
+    snap = gpu.export()
+    other = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, key_cells=cfg.key_cells * 2,
+                         lr=cfg.lr, eps=cfg.eps, init_scale=cfg.init_scale, seed=cfg.seed + 1)
+    other.import_entries(snap["ids"], snap["count"], snap["last_seen"], snap["resident"], snap["w"], snap["acc"])
+    assert_state_equal(other, cpu, "restored")
+    assert_audit_ok(other)
+    # importing the same IDs again changes nothing and is reported
+    other.import_entries(snap["ids"][:10], snap["count"][:10], snap["last_seen"][:10], snap["resident"][:10],
+                         snap["w"][:10], snap["acc"][:10])
+    assert other.status()["error_bits"] & mb.MONO_DEV_IMPORT_DUP
+    assert_state_equal(other, cpu, "after duplicate import")
+
+
+# ---------------------------------------------------------------- cuckoo structure under load
+
+@pytest.mark.parametrize("load", [0.5, 0.8, 0.9])
+@pytest.mark.parametrize("kind", ["random", "sequential", "high_bits", "stride_4096"])
+def test_cuckoo_membership_at_load(load, kind):
+    cells = 1 << 16
+    n = int(cells * load)
+    if kind == "random":
+        ids = wl.splitmix64(np.arange(n, dtype=np.uint64) + np.uint64(12345))
+    elif kind == "sequential":
+        ids = np.arange(1, n + 1, dtype=np.uint64)
+    elif kind == "high_bits":
+        ids = np.arange(1, n + 1, dtype=np.uint64) << np.uint64(40)
+    else:
+        ids = np.arange(1, n + 1, dtype=np.uint64) * np.uint64(4096)
+    gpu = mb.MonoTable(1024, 4, 3, 0, key_cells=cells, seed=17)
+    half = n // 2
+    for part in (ids[:half], ids[half:]):          # second call inserts into an already loaded table
+        gpu.import_entries(part, np.ones(part.size, np.uint32), np.zeros(part.size, np.int64),
+                           np.zeros(part.size, np.uint8))
+    st = gpu.status()
+    assert st["error_bits"] == 0 and st["n_tracked"] == n, st
+    a = assert_audit_ok(gpu)
+    assert a["occupied_cells"] == n
+    absent = wl.splitmix64(np.arange(5000, dtype=np.uint64) + np.uint64(999_999_999))
+    assert gpu.probe(ids, rows=False)["count"].min() == 1
+    assert gpu.probe(absent, rows=False)["count"].max() == 0
+    assert set(gpu.export(rows=False)["ids"].tolist()) == set(ids.tolist())
+
+
+def test_apply_grads_inserts_at_high_load():
+    # the batch path (not import) pushing a small key store to ~0.9 load in a few calls
+    cells = 1 << 14
+    gpu = mb.MonoTable(256, 4, 1000, 0, key_cells=cells, seed=2)
+    cpu = mo.OracleTable(256, 4, 1000, 0, seed=2)
+    per_call = int(cells * 0.09)
+    for t in range(10):
+        ids = wl.splitmix64(np.arange(t * per_call, (t + 1) * per_call, dtype=np.uint64))
+        off = np.arange(0, per_call + 1, 2, dtype=np.int64)
+        grad = np.zeros((off.size - 1, 4), f32)
+        gpu.apply_grads(ids, off, grad, t)
+        cpu.apply_grads(ids, off, grad, t)
+    st = gpu.status()
+    assert st["error_bits"] == 0 and st["n_tracked"] == 10 * (per_call // 2 * 2)
+    assert_state_equal(gpu, cpu)
+    assert_audit_ok(gpu)
+    assert st["n_evictions_total"] > 0          # the displacement path really ran
+
+
+# ---------------------------------------------------------------- overflow conditions (flagged, never fatal)
+
+def test_rows_full_is_flagged_and_table_stays_consistent():
+    gpu = mb.MonoTable(16, 4, 1, 0, key_cells=1 << 10)
+    ids = np.arange(1, 41, dtype=np.uint64)
+    off = np.arange(0, 41, dtype=np.int64)
+    gpu.apply_grads(ids, off, np.ones((40, 4), f32), 0)
+    st = gpu.status()
+    assert st["error_bits"] & mb.MONO_DEV_ROWS_FULL
+    assert st["n_resident"] == 16 and st["n_tracked"] == 40 and st["n_rows_refused"] == 24
+    assert_audit_ok(gpu)
+    pr = gpu.probe(ids)
+    assert pr["resident"].sum() == 16 and (pr["count"] == 1).all()
+    # IDs without a row pool as zero, the others as their row
+    pooled = gpu.lookup_pool(ids, off).cpu().numpy()
+    assert ((np.abs(pooled).max(axis=1) > 0) == (pr["resident"] == 1)).all()
+
+
+def test_key_store_full_is_flagged_without_duplicates():
+    gpu = mb.MonoTable(16, 4, 100, 0, key_cells=64)        # 64 cells + the stash
+    ids = wl.splitmix64(np.arange(2000, dtype=np.uint64))
+    off = np.arange(0, 2001, dtype=np.int64)
+    gpu.apply_grads(ids, off, np.zeros((2000, 4), f32), 0)
+    st = gpu.status()
+    assert st["error_bits"] & mb.MONO_DEV_KEYS_FULL
+    assert st["n_tracked"] + st["n_keys_dropped"] == 2000
+    a = gpu.audit()
+    assert a["duplicate_keys"] == 0 and a["misplaced"] == 0 and a["occupied_cells"] == st["n_tracked"]
+    kept = set(gpu.export(rows=False)["ids"].tolist())
+    assert kept <= set(ids.tolist()) and len(kept) == st["n_tracked"]
+    # the table keeps working: a later call on tracked IDs raises their counts
+    sub = np.array(sorted(kept)[:32], np.uint64)
+    gpu.apply_grads(sub, np.arange(0, 33, dtype=np.int64), np.zeros((32, 4), f32), 1)
+    assert (gpu.probe(sub, rows=False)["count"] == 2).all()
+
+
+def test_malformed_offsets_are_flagged_not_followed():
+    gpu = mb.MonoTable(64, 4, 1, 0)
+    ids = np.arange(1, 9, dtype=np.uint64)
+    off = np.array([0, 4, 2, 100], np.int64)           # decreasing, then past the end
+    out = gpu.lookup_pool(ids, off).cpu().numpy()
+    assert out.shape == (3, 4)
+    gpu.apply_grads(ids, off, np.ones((3, 4), f32), 0)
+    assert gpu.status()["error_bits"] & mb.MONO_DEV_BAD_OFFSETS
+    assert_audit_ok(gpu)
+
+
+def test_host_detected_errors():
+    with pytest.raises(mb.MonoError) as e:
+        mb.mono_table_create(64, 6, 1, 0)                 # dim not a multiple of 4
+    assert e.value.code == mb.MONO_ERR_ARG
+    with pytest.raises(mb.MonoError):
+        mb.mono_table_create(64, 8, 1, 0, key_cells=1000)  # not a power of two
+    with pytest.raises(mb.MonoError):
+        mb.mono_table_create(0, 8, 1, 0)
+    gpu = mb.MonoTable(64, 8, 1, 5)
+    ids = torch.arange(1, 9, dtype=torch.int64, device="cuda")
+    off = torch.tensor([0, 8], dtype=torch.int64, device="cuda")
+    grad = torch.ones((1, 8), device="cuda")
+    mb.mono_apply_grads(gpu.handle, ids, 8, off, 1, grad, 7)
+    for bad_now in (6, -1, mb.MONO_MAX_NOW + 1):
+        with pytest.raises(mb.MonoError) as e:
+            mb.mono_apply_grads(gpu.handle, ids, 8, off, 1, grad, bad_now)
+        assert e.value.code == mb.MONO_ERR_TIME
+    with pytest.raises(mb.MonoError) as e:
+        mb.mono_expire(gpu.handle, 3)
+    assert e.value.code == mb.MONO_ERR_TIME
+    with pytest.raises(mb.MonoError) as e:                 # misaligned output
+        mb.mono_lookup_pool(gpu.handle, ids, 8, off, 1, grad.data_ptr() + 4)
+    assert e.value.code == mb.MONO_ERR_ARG
+    with pytest.raises(mb.MonoError):
+        mb.mono_lookup_pool(gpu.handle, None, 8, off, 1, grad)
+    with pytest.raises(mb.MonoError):
+        mb.mono_lookup_pool(gpu.handle, ids, -1, off, 1, grad)
+    assert gpu.status()["n_tracked"] == 8 and gpu.status()["error_bits"] == 0
+
+
+def test_large_times_near_the_limit():
+    gpu = mb.MonoTable(64, 4, 1, 10, init_scale=0.1)
+    cpu = mo.OracleTable(64, 4, 1, 10, init_scale=0.1)
+    base = mb.MONO_MAX_NOW - 30
+    for k, lists in enumerate([[[1, 2]], [[2, 3]], [[3]]]):
+        ids, off = bags(lists)
+        gpu.apply_grads(ids, off, np.ones((1, 4), f32), base + 10 * k)
+        cpu.apply_grads(ids, off, np.ones((1, 4), f32), base + 10 * k)
+    gpu.expire(mb.MONO_MAX_NOW); cpu.expire(mb.MONO_MAX_NOW)
+    assert_state_equal(gpu, cpu)
+    assert gpu.export()["ids"].tolist() == [3]
