@@ -176,8 +176,8 @@ def test_host_buffer_calls_match_device_calls():
 # ---------------------------------------------------------------- expiry, recycling, import/export
 
 def test_expiry_sets_and_row_recycling():
-    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, ttl=2, capacity=1 << 12, key_cells=1 << 15, steps=14,
-                    filter_threshold=1, n_distinct=1 << 14)
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, ttl=2, capacity=1 << 14, key_cells=1 << 16, steps=14,
+                    filter_threshold=1, n_distinct=1 << 18)
     gpu, cpu = make_pair(cfg)
     st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=1)
     # more rows were handed out than exist: expired rows were reused, never shared
