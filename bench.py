@@ -1,0 +1,449 @@
+#!/usr/bin/env python
+"""Benchmark of the collisionless embedding-table step on B200.
+
+One "step" is one pass of the whole hot path over one fresh synthetic batch:
+mono_lookup_pool (probe, gather, sum pooling) + mono_apply_grads (dedup,
+count/stamp/admit, cuckoo insert, segmented gradient reduce, Adagrad), with
+mono_expire called once every `sweep_period` steps inside the timed region.
+The table is pre-filled to the steady state of the configured stream, so the
+timed steps run at the load the stream would reach, not on an empty table.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large]
+    python bench.py --impl reference ...     # the CPU oracle, timed on the host
+
+Prints one JSON line (rank 0).  With N > 1 (under torchrun) every rank owns an
+independent table and its own batches (weak scaling, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import concurrent.futures
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2209_07663_b200 import workload as wl  # noqa: E402
+
+METRIC = "feature IDs/sec (lookup+pool+update) on 1 B200; % of HBM roofline"
+UNIT = "IDs/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# --------------------------------------------------------------------------- helpers
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_source_digest() -> str:
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2209_07663_b200", "csrc")
+    for name in sorted(os.listdir(d)):
+        with open(os.path.join(d, name), "rb") as f:
+            h.update(name.encode())
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu summary of this kernel, or None when
+    there is none or the kernels have changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", f"traffic_{kernel}_{workload}.txt")
+    if not os.path.exists(path):
+        return None
+    kv = {}
+    for line in open(path):
+        if "=" in line and not line.lstrip().startswith("#"):
+            k, v = line.split("=", 1)
+            kv[k.strip()] = v.strip()
+    if kv.get("source_digest") != kernel_source_digest():
+        return None
+    try:
+        return float(kv["dram_bytes_per_launch_scaled"])
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """nvidia-smi in the background while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    smax.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def sample_of_step(step: wl.Step, n_bags: int) -> wl.Step:
+    """The first n_bags bags of a step (a bounded sample for the CPU oracle)."""
+    n_bags = min(n_bags, step.offsets.size - 1)
+    n_ids = int(step.offsets[n_bags])
+    return wl.Step(ids=step.ids[:n_ids], offsets=step.offsets[:n_bags + 1],
+                   grad_pooled=step.grad_pooled[:n_bags], now=step.now)
+
+
+def time_oracle(cfg: wl.Config, steps: int, warmup: int, sample_bags: int, first_step: int = 0):
+    """lookup_pool + apply_grads of the CPU oracle on the first `sample_bags` bags of each
+    step, from an empty table.  Returns (ids_per_second, ms_per_step, ids_per_step)."""
+    from oracle import mono_oracle as mo
+    o = mo.OracleTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
+                       init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed)
+    stream = wl.Stream(cfg)
+    batches = [sample_of_step(stream.step(first_step + t), sample_bags) for t in range(warmup + steps)]
+    n_ids, elapsed = 0, 0.0
+    for t, s in enumerate(batches):
+        t0 = time.perf_counter()
+        o.lookup_pool(s.ids, s.offsets)
+        o.apply_grads(s.ids, s.offsets, s.grad_pooled, first_step + t)
+        dt = time.perf_counter() - t0
+        if t >= warmup:
+            elapsed += dt
+            n_ids += s.ids.size
+    return n_ids / elapsed, 1e3 * elapsed / steps, n_ids / steps
+
+
+# --------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = wl.CONFIGS[args.workload]
+    sample_bags = max(cfg.n_bags // args.oracle_fraction, 1)
+    ids_s, ms_step, ids_step = time_oracle(cfg, args.steps, args.warmup, sample_bags)
+    sample = (f"first {sample_bags} of {cfg.n_bags} bags of each step (~{int(ids_step)} IDs), "
+              f"lookup_pool + apply_grads, from an empty table")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ids_s, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "capacity": cfg.capacity, "dim": cfg.dim,
+                   "bags_per_step": cfg.n_bags, "sample": sample},
+        "cpu_baseline": {"value": ids_s, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": ids_s, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- our arm
+
+def algorithmic_bytes(n, b, u, ur, unew, d):
+    """Bytes the method itself must move per step, per kernel group (each distinct datum
+    once per phase; 32-byte sector as the smallest random access)."""
+    fwd = 8 * n + 8 * (b + 1) + 32 * n + 4 * d * ur + 4 * d * b
+    dedup = 8 * n + 8 * (b + 1) + 24 * n
+    table = 64 * u + (16 + 8 * d) * unew
+    adagrad = 4 * d * b + 16 * d * ur
+    return {"lookup_pool": fwd, "dedup": dedup, "table": table, "adagrad": adagrad,
+            "total": fwd + dedup + table + adagrad}
+
+
+KERNEL_GROUP = {
+    "lookup_pool": "lookup_pool",
+    "fill_occ_bag": "dedup", "dedup_insert": "dedup", "seg_count": "dedup", "seg_scan_blocks": "dedup",
+    "seg_offsets": "dedup", "place": "dedup", "dedup_reset": "dedup", "finish_apply": "dedup",
+    "table_update": "table", "table_insert": "table",
+    "reduce_adagrad": "adagrad", "combine_adagrad": "adagrad",
+}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2209_07663_b200 import binding as mb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the table has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+
+    base = wl.CONFIGS[args.workload]
+    cfg = wl.scaled(base, seed=base.seed + 7919 * rank)          # every rank its own stream and table
+    K, W, E = args.steps, args.warmup, args.e2e_steps
+    sweep_period = args.sweep_period or K
+    now0 = cfg.ttl - 1 if args.prefill else 0
+    stream = wl.Stream(cfg)
+
+    # ---- table, pre-filled to the steady state of the stream
+    t_setup = time.time()
+    table = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
+                         init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed,
+                         key_cells=cfg.key_cells, max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1),
+                         max_bags=cfg.n_bags)
+    if args.prefill:
+        for ids, cnt, seen in wl.steady_state_population_torch(cfg, now0, dev):
+            res = (cnt >= cfg.filter_threshold).to(torch.uint8)
+            mb.mono_import(table.handle, ids, cnt, seen, res, None, None, ids.numel())
+            del ids, cnt, seen, res
+    st0 = table.status()
+    if st0["error_bits"]:
+        raise SystemExit(f"pre-fill overflowed the table: {st0}")
+
+    # ---- batches: ids/offsets from the seeded host generator, gradients drawn on the device
+    n_batches = W + 2 * K + E
+
+    def make(i):
+        return stream.step(now0 + 1 + i, with_grad=False)
+
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        host_batches = list(pool.map(make, range(n_batches)))
+    gg = torch.Generator(device=dev)
+    gg.manual_seed(cfg.seed)
+    dev_batches = []
+    for t, s in enumerate(host_batches[:W + 2 * K]):
+        ids = torch.from_numpy(s.ids.view(np.int64)).to(dev)
+        off = torch.from_numpy(s.offsets).to(dev)
+        grad = torch.randn((cfg.n_bags, cfg.dim), device=dev, generator=gg).mul_(cfg.grad_std)
+        dev_batches.append((ids, off, grad))
+    out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+    setup_s = time.time() - t_setup
+
+    def step(i, sweep=False):
+        """Step i of the stream (time now0 + 1 + i) on its own fresh batch."""
+        ids, off, grad = dev_batches[i]
+        mb.mono_lookup_pool(table.handle, ids, ids.numel(), off, cfg.n_bags, out)
+        mb.mono_apply_grads(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0 + 1 + i)
+        if sweep:
+            mb.mono_expire(table.handle, now0 + 1 + i)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up, then the timed region
+    for t in range(W):
+        step(t)
+    barrier()
+    st_a = table.status()
+    mb.mono_timing_read(table.handle, reset=True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for t in range(K):
+        step(W + t, sweep=(t + 1) % sweep_period == 0)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    st_b = table.status()
+    launches = mb.mono_timing_read(table.handle, reset=True)["launches_total"]
+    n_ids_timed = st_b["sum_ids"] - st_a["sum_ids"]
+
+    # ---- the same steps on fresh batches with every kernel bracketed by CUDA events
+    mb.mono_timing_enable(table.handle, True)
+    for t in range(K):
+        step(W + K + t, sweep=(t + 1) % sweep_period == 0)
+    torch.cuda.synchronize()
+    tim = mb.mono_timing_read(table.handle, reset=True)
+    mb.mono_timing_enable(table.handle, False)
+    st_c = table.status()
+
+    # ---- end to end: host buffers in, pooled output back out, through the host-buffer calls
+    e2e = None
+    if E > 0:
+        pinned = []
+        for s in host_batches[W + 2 * K:]:
+            ids = torch.from_numpy(s.ids.view(np.int64)).pin_memory()
+            off = torch.from_numpy(s.offsets).pin_memory()
+            grad = torch.randn((cfg.n_bags, cfg.dim)).mul_(cfg.grad_std).pin_memory()
+            pinned.append((ids, off, grad))
+        out_h = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32).pin_memory()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e_ids, h2d, d2h = 0, 0, 0
+        e0.record()
+        for t, (ids, off, grad) in enumerate(pinned):
+            now = now0 + 1 + W + 2 * K + t
+            mb.mono_lookup_pool_host(table.handle, ids, ids.numel(), off, cfg.n_bags, out_h)
+            mb.mono_apply_grads_host(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now)
+            n_e2e_ids += ids.numel()
+            h2d += 2 * (ids.numel() * 8 + off.numel() * 8) + grad.numel() * 4
+            d2h += out_h.numel() * 4
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e = {"ids": n_e2e_ids, "ms": e2e_ms, "h2d": h2d // E, "d2h": d2h // E}
+    st_end = table.status()
+
+    # ---- aggregate over ranks: max time, summed work
+    agg = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], dtype=torch.float64, device=dev)
+    work = torch.tensor([float(n_ids_timed), float(e2e["ids"]) if e2e else 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(agg, op=dist.ReduceOp.MAX)
+        dist.all_reduce(work, op=dist.ReduceOp.SUM)
+    ms_max, e2e_ms_max = agg.tolist()
+    ids_all, e2e_ids_all = work.tolist()
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        d = cfg.dim
+        # per-step averages over the per-kernel pass (the steps the kernel times belong to)
+        n = (st_c["sum_ids"] - st_b["sum_ids"]) / K
+        u = (st_c["sum_unique"] - st_b["sum_unique"]) / K
+        ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / K
+        unew = (st_c["sum_new"] - st_b["sum_new"]) / K
+        alg = algorithmic_bytes(n, cfg.n_bags, u, ur, unew, d)
+        per_kernel = {}
+        for name, v in tim["kernels"].items():
+            if v["launches"] and name in KERNEL_GROUP:
+                per_kernel[name] = {"ms_per_launch": v["ms"] / v["launches"], "launches": v["launches"]}
+        group_ms = {}
+        for name, v in per_kernel.items():
+            group_ms[KERNEL_GROUP[name]] = group_ms.get(KERNEL_GROUP[name], 0.0) + v["ms_per_launch"]
+        # the kernel group that takes the most device time, and its largest kernel
+        dom_group = max(group_ms, key=group_ms.get)
+        dom_kernels = sorted((k for k in per_kernel if KERNEL_GROUP[k] == dom_group),
+                             key=lambda k: -per_kernel[k]["ms_per_launch"])
+        dom_bytes, dom_ms = alg[dom_group], group_ms[dom_group]
+        achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+        step_ms = ms_max / K
+        line = {
+            "metric": METRIC, "value": ids_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": args.workload, "capacity": cfg.capacity, "dim": d, "key_cells": cfg.key_cells,
+                "bags_per_step": cfg.n_bags, "ids_per_step": n, "unique_per_step": u,
+                "unique_resident_per_step": ur, "new_per_step": unew, "zipf_s": cfg.zipf_s,
+                "id_universe": cfg.n_distinct, "filter_threshold": cfg.filter_threshold, "ttl": cfg.ttl,
+                "prefill": "steady state of the stream" if args.prefill else "empty table",
+                "rows_resident_at_start": st0["n_resident"], "ids_tracked_at_start": st0["n_tracked"],
+                "row_load": st0["n_resident"] / cfg.capacity, "key_load": st0["n_tracked"] / cfg.key_cells,
+                "sweep_period_steps": sweep_period, "l2": "every step reads a fresh batch larger than L2",
+                "parallelism": f"{world} independent table(s), one per GPU",
+            },
+            "bags_per_s": world * cfg.n_bags * K / (ms_max * 1e-3),
+            "gpu_launches": launches,
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
+                       "reasons": clocks["reasons"], "samples": clocks["samples"]},
+            "roofline": {
+                "bound": "hbm", "kernel": dom_kernels[0], "kernels_timed_together": dom_kernels,
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": dom_bytes,
+                "ms_per_launch": dom_ms,
+                "traffic": recorded_traffic(dom_kernels[0], args.workload),
+            },
+            "whole_step": {
+                "algorithmic_bytes": alg["total"], "achieved_gbs": alg["total"] / (step_ms * 1e-3) / 1e9,
+                "frac_of_measured_peak": alg["total"] / (step_ms * 1e-3) / 1e9 / peak,
+                "frac_of_8tbs": alg["total"] / (step_ms * 1e-3) / 1e9 / 8000.0,
+                "bytes_by_group": {k: v for k, v in alg.items() if k != "total"},
+                "ms_by_kernel": {k: round(v["ms_per_launch"], 4) for k, v in per_kernel.items()},
+                "expire_ms_per_launch": (tim["kernels"]["expire"]["ms"] / tim["kernels"]["expire"]["launches"]
+                                         if tim["kernels"]["expire"]["launches"] else None),
+            },
+            "table_after": {"n_tracked": st_end["n_tracked"], "n_resident": st_end["n_resident"],
+                            "error_bits": st_end["error_bits"], "max_chain": st_end["max_chain"],
+                            "evictions": st_end["n_evictions_total"], "stash_used": st_end["stash_used"]},
+            "setup_s": round(setup_s, 1),
+        }
+        if e2e:
+            line["e2e"] = {"value": e2e_ids_all / (e2e_ms_max * 1e-3), "unit": UNIT,
+                           "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "ms_per_step": e2e_ms_max / E, "steps": E}
+        if world == 1 and args.oracle_steps > 0:
+            sample_bags = max(cfg.n_bags // args.oracle_fraction, 1)
+            ids_s, _, ids_step = time_oracle(cfg, args.oracle_steps, 1, sample_bags, first_step=now0 + 1)
+            line["cpu_baseline"] = {
+                "value": ids_s, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": (f"{args.oracle_steps} steps of the first {sample_bags} of {cfg.n_bags} bags "
+                           f"(~{int(ids_step)} IDs each), lookup_pool + apply_grads, from an empty table; "
+                           f"host has {os.cpu_count()} cores, the oracle uses one thread")}
+        print(json.dumps(line), flush=True)
+    table.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--sweep-period", type=int, default=0, help="steps between expiry sweeps (0 = --steps)")
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--no-prefill", dest="prefill", action="store_false")
+    ap.add_argument("--oracle-steps", type=int, default=4)
+    ap.add_argument("--oracle-fraction", type=int, default=8, help="the oracle runs on 1/this of each step's bags")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

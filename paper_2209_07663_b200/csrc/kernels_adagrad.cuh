@@ -87,58 +87,55 @@ __device__ inline void reduce_segment(const Work& wk, const float* __restrict__ 
   }
 }
 
-// One lane group per distinct ID with a short segment.
+// One lane group per work item.  Items [0, n_unique) are the distinct IDs: a
+// group reduces an ID's whole segment and updates its row when the segment is
+// short.  Items [n_unique, n_unique + n_parts) are the parts of the long
+// segments: a group reduces one part into fp64 partial sums in scratch, which
+// combine_adagrad_kernel adds up afterwards.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
   const uint32_t n = tv.st->n_unique;
-  const int gl = threadIdx.x % G;
-  const uint32_t groups = (gridDim.x * blockDim.x) / G;
-  for (uint32_t u = (blockIdx.x * blockDim.x + threadIdx.x) / G; u < n; u += groups) {
-    const uint32_t row_word = wk.urow[u];
-    if (row_word == kNoRow) continue;
-    const uint32_t begin = wk.useg[u], end = wk.useg[u + 1];
-    if (end - begin > kSegChunk) continue;          // handled in parts
-    D4 s[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
-    reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
-    const unsigned long long id = wk.uid[u];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-      const uint32_t c4 = gl + v * G;
-      if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
-    }
-  }
-}
-
-// One lane group per part of a long segment: fp64 partial sums to scratch.
-template <int G, int NV>
-__global__ void __launch_bounds__(256)
-reduce_parts_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
   uint32_t n_parts = tv.st->n_parts;
   if (n_parts > wk.max_parts) n_parts = wk.max_parts;
+  const uint32_t n_items = n + n_parts;
   const int gl = threadIdx.x % G;
   const uint32_t groups = (gridDim.x * blockDim.x) / G;
-  for (uint32_t p = (blockIdx.x * blockDim.x + threadIdx.x) / G; p < n_parts; p += groups) {
-    const uint32_t li = wk.part_u[p];
-    const uint32_t u = wk.long_u[li];
-    if (wk.urow[u] == kNoRow) continue;
-    const uint32_t k = p - wk.long_part0[li];
-    const uint32_t seg_end = wk.useg[u + 1];
-    const uint32_t begin = wk.useg[u] + k * kSegChunk;
-    const uint32_t end = begin + kSegChunk < seg_end ? begin + kSegChunk : seg_end;
+  for (uint32_t item = (blockIdx.x * blockDim.x + threadIdx.x) / G; item < n_items; item += groups) {
     D4 s[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
-    reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
-    double* dst = wk.partials + (size_t)p * tv.dim;
+    if (item < n) {
+      const uint32_t u = item;
+      const uint32_t row_word = wk.urow[u];
+      if (row_word == kNoRow) continue;
+      const uint32_t begin = wk.useg[u], end = wk.useg[u + 1];
+      if (end - begin > kSegChunk) continue;          // reduced in parts
+      reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
+      const unsigned long long id = wk.uid[u];
 #pragma unroll
-    for (int v = 0; v < NV; ++v) {
-      const uint32_t c4 = gl + v * G;
-      if (c4 * 4u < tv.dim) {
-        reinterpret_cast<double2*>(dst)[c4 * 2] = make_double2(s[v].x, s[v].y);
-        reinterpret_cast<double2*>(dst)[c4 * 2 + 1] = make_double2(s[v].z, s[v].w);
+      for (int v = 0; v < NV; ++v) {
+        const uint32_t c4 = gl + v * G;
+        if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
+      }
+    } else {
+      const uint32_t p = item - n;
+      const uint32_t li = wk.part_u[p];
+      const uint32_t u = wk.long_u[li];
+      if (wk.urow[u] == kNoRow) continue;
+      const uint32_t k = p - wk.long_part0[li];
+      const uint32_t seg_end = wk.useg[u + 1];
+      const uint32_t begin = wk.useg[u] + k * kSegChunk;
+      const uint32_t end = begin + kSegChunk < seg_end ? begin + kSegChunk : seg_end;
+      reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
+      double* dst = wk.partials + (size_t)p * tv.dim;
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const uint32_t c4 = gl + v * G;
+        if (c4 * 4u < tv.dim) {
+          reinterpret_cast<double2*>(dst)[c4 * 2] = make_double2(s[v].x, s[v].y);
+          reinterpret_cast<double2*>(dst)[c4 * 2 + 1] = make_double2(s[v].z, s[v].w);
+        }
       }
     }
   }

@@ -23,11 +23,11 @@ using namespace mono;
 
 enum KernelId {
   K_LOOKUP, K_FILL_BAG, K_DEDUP, K_SEG_COUNT, K_SEG_SCAN, K_SEG_OFFSETS, K_PLACE, K_UPDATE, K_INSERT,
-  K_REDUCE, K_PARTS, K_COMBINE, K_RESET, K_FINISH, K_EXPIRE, K_STASH_TRIM, K_COUNT
+  K_REDUCE, K_COMBINE, K_RESET, K_FINISH, K_EXPIRE, K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
   "lookup_pool", "fill_occ_bag", "dedup_insert", "seg_count", "seg_scan_blocks", "seg_offsets", "place",
-  "table_update", "table_insert", "reduce_adagrad", "reduce_parts", "combine_adagrad", "dedup_reset",
+  "table_update", "table_insert", "reduce_adagrad", "combine_adagrad", "dedup_reset",
   "finish_apply", "expire", "stash_trim"
 };
 
@@ -198,7 +198,6 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
-    LAUNCH(t, K_PARTS, reduce_parts_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;

@@ -264,13 +264,22 @@ def steady_state_population(cfg: Config, now: int, window: Optional[int] = None,
         cnt = rng.poisson(lam_step * window)
         keep = cnt > 0
         ranks, cnt, lam_step = ranks[keep], cnt[keep], lam_step[keep]
-        # steps since the most recent occurrence: geometric with per-step hit probability
-        p_hit = -np.expm1(-lam_step)
-        age = np.minimum(rng.geometric(np.maximum(p_hit, 1e-12)) - 1, window - 1)
+        # steps since the most recent occurrence: geometric with the per-step hit
+        # probability, conditioned on falling inside the window
+        age = _truncated_geometric(rng.random(ranks.size), -np.expm1(-lam_step), window)
         ids_l.append(stream.ids_from_ranks(ranks, now))
         cnt_l.append(cnt.astype(np.int64))
         seen_l.append((now - age).astype(np.int64))
     return np.concatenate(ids_l), np.concatenate(cnt_l), np.concatenate(seen_l)
+
+
+def _truncated_geometric(u, p_hit, window: int):
+    """Inverse CDF of P(a) ~ (1-p)^a p on a in [0, window): uniform for tiny p."""
+    p_hit = np.clip(p_hit, 1e-12, 1 - 1e-12)
+    log_q = np.log1p(-p_hit)
+    mass = -np.expm1(window * log_q)                  # 1 - q^window
+    a = np.floor(np.log1p(-u * mass) / log_q)
+    return np.clip(a, 0, window - 1).astype(np.int64)
 
 
 def _mean_bag_len(spec: tuple) -> float:
@@ -291,3 +300,67 @@ def _zipf_norm(n: int, s: float) -> float:
         a, b = head + 0.5, n + 0.5
         total += (np.log(b / a) if abs(s - 1.0) < 1e-12 else (b ** (1 - s) - a ** (1 - s)) / (1 - s))
     return total
+
+
+# ---------------------------------------------------------------------------
+# Device-side twins of the generators above (torch), for benchmarks that need a
+# table population of hundreds of millions of IDs without a slow host loop.
+# They reproduce the numpy functions bit for bit (checked in the CPU tests).
+# ---------------------------------------------------------------------------
+
+def _signed64(c: int) -> int:
+    c &= 0xFFFFFFFFFFFFFFFF
+    return c - (1 << 64) if c >= (1 << 63) else c
+
+
+def _lsr(x, k: int):
+    """Logical shift right of an int64 tensor."""
+    return (x >> k) & ((1 << (64 - k)) - 1)
+
+
+def splitmix64_torch(x):
+    """splitmix64() on an int64 torch tensor holding uint64 bit patterns."""
+    z = x + _signed64(0x9E3779B97F4A7C15)
+    z = (z ^ _lsr(z, 30)) * _signed64(0xBF58476D1CE4E5B9)
+    z = (z ^ _lsr(z, 27)) * _signed64(0x94D049BB133111EB)
+    return z ^ _lsr(z, 31)
+
+
+def ids_from_ranks_torch(cfg: Config, ranks):
+    """Stream.ids_from_ranks for a config without drift, on an int64 tensor of ranks."""
+    import torch
+    if cfg.drift_period > 0:
+        raise ValueError("the device twin covers configs without drift")
+    salt = int(splitmix64(np.array([cfg.seed & 0xFFFFFFFFFFFFFFFF], dtype=np.uint64))[0])
+    ids = splitmix64_torch(ranks ^ _signed64(salt))
+    return torch.where(ids == -1, torch.full_like(ids, -2), ids)
+
+
+def steady_state_population_torch(cfg: Config, now: int, device, window: Optional[int] = None,
+                                  chunk: int = 1 << 26, seed_salt: int = 7):
+    """Device twin of steady_state_population: yields (ids int64, counts int32,
+    last_seen int64) chunk by chunk, each a torch tensor on `device`.
+    Same model (Poisson occurrences per rank over the window); its own random
+    stream (torch's), so it is reproducible for a given seed but does not match
+    the numpy draw element by element.
+    """
+    import torch
+    window = int(window if window is not None else min(cfg.ttl, now + 1))
+    gen = torch.Generator(device=device)
+    gen.manual_seed((cfg.seed * 1000003 + seed_salt * 7919 + now) & 0x7FFFFFFFFFFFFFFF)
+    n_per_step = cfg.n_bags * _mean_bag_len(cfg.bag_len)
+    norm = _zipf_norm(cfg.n_distinct, cfg.zipf_s)
+    for lo in range(1, cfg.n_distinct + 1, chunk):
+        hi = min(lo + chunk, cfg.n_distinct + 1)
+        ranks = torch.arange(lo, hi, dtype=torch.int64, device=device)
+        lam_step = ranks.to(torch.float64).pow(-cfg.zipf_s).mul_(n_per_step / norm)
+        cnt = torch.poisson((lam_step * window).to(torch.float32), generator=gen)
+        keep = cnt > 0
+        ranks, cnt, lam_step = ranks[keep], cnt[keep], lam_step[keep]
+        # steps since the last occurrence: geometric, conditioned on lying inside the window
+        p_hit = (-torch.expm1(-lam_step)).clamp_(1e-12, 1 - 1e-12)
+        u = torch.rand(ranks.shape, dtype=torch.float64, device=device, generator=gen)
+        log_q = torch.log1p(-p_hit)
+        mass = -torch.expm1(window * log_q)
+        age = torch.floor(torch.log1p(-u * mass) / log_q).clamp_(0, window - 1)
+        yield ids_from_ranks_torch(cfg, ranks), cnt.to(torch.int32), (now - age).to(torch.int64)

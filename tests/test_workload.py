@@ -81,3 +81,28 @@ def test_steady_state_population_is_consistent():
     assert cnt.min() >= 1 and seen.max() <= 99 and seen.min() >= 0
     # hot ranks were seen in the very last step
     assert seen[0] == 99 and cnt[0] > cnt[-1]
+    # cold IDs are spread over the whole window instead of piling up at its far end
+    cold = seen[cnt == 1]
+    assert (cold == 0).mean() < 0.05 and abs(cold.mean() - 49.5) < 5
+
+
+def test_torch_twins_reproduce_the_numpy_generators():
+    import torch
+    x = np.array([0, 1, 2**63, 2**64 - 1, 0x9E3779B97F4A7C15, 123456789], dtype=np.uint64)
+    got = wl.splitmix64_torch(torch.from_numpy(x.view(np.int64))).numpy().view(np.uint64)
+    assert (got == wl.splitmix64(x)).all()
+    cfg = wl.CONFIGS["medium"]
+    ranks = np.array([1, 2, 3, 1000, 2**24], dtype=np.int64)
+    want = wl.Stream(cfg).ids_from_ranks(ranks, 5)
+    got = wl.ids_from_ranks_torch(cfg, torch.from_numpy(ranks)).numpy().view(np.uint64)
+    assert (got == want).all()
+    small = wl.scaled(cfg, n_distinct=1 << 14)
+    chunks = list(wl.steady_state_population_torch(small, now=99, device="cpu", chunk=1 << 12))
+    ids = torch.cat([c[0] for c in chunks]).numpy()
+    cnt = torch.cat([c[1] for c in chunks]).numpy()
+    seen = torch.cat([c[2] for c in chunks]).numpy()
+    assert len(np.unique(ids)) == ids.size and cnt.min() >= 1
+    assert seen.max() == 99 and seen.min() >= 0 and seen[0] == 99
+    ref_ids, ref_cnt, _ = wl.steady_state_population(small, now=99)
+    assert abs(ids.size - ref_ids.size) < 0.05 * ref_ids.size          # same model, different draws
+    assert abs(int(cnt.sum()) - int(ref_cnt.sum())) < 0.05 * ref_cnt.sum()
