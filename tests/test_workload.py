@@ -82,7 +82,10 @@ def test_steady_state_population_is_consistent():
     # hot ranks were seen in the very last step
     assert seen[0] == 99 and cnt[0] > cnt[-1]
     # cold IDs are spread over the whole window instead of piling up at its far end
+    sparse = wl.scaled(cfg, n_examples=8, n_slots=4)
+    _, cnt, seen = wl.steady_state_population(sparse, now=99)
     cold = seen[cnt == 1]
+    assert cold.size > 1000
     assert (cold == 0).mean() < 0.05 and abs(cold.mean() - 49.5) < 5
 
 
