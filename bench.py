@@ -199,11 +199,10 @@ def algorithmic_bytes(n, b, u, ur, unew, d):
 
 
 KERNEL_GROUP = {
-    "lookup_pool": "lookup_pool",
-    "fill_occ_bag": "dedup", "dedup_insert": "dedup", "seg_count": "dedup", "seg_scan_blocks": "dedup",
-    "seg_offsets": "dedup", "place": "dedup", "dedup_reset": "dedup", "finish_apply": "dedup",
+    "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
+    "fill_occ_bag": "dedup", "dedup_tile": "dedup", "dedup_reset": "dedup", "finish_apply": "dedup",
     "table_update": "table", "table_insert": "table",
-    "reduce_adagrad": "adagrad", "combine_adagrad": "adagrad",
+    "scatter_singletons": "adagrad", "reduce_adagrad": "adagrad", "combine_adagrad": "adagrad",
 }
 
 

@@ -1,14 +1,21 @@
 // Backward, last phase: per distinct ID that owns a row, sum the pooled
 // gradients of its occurrences' bags (fp64 accumulation, one rounding to fp32)
 // and apply one Adagrad step to the row, in place.  This is the parameter push
-// of Section 2.2 for the sparse rows; the optimizer itself is not
-// named in the paper.
+// of Section 2.2 for the sparse rows; the optimizer itself is not named in the
+// paper.
 //
-// Segments of up to kSegChunk occurrences are reduced by one lane group.
-// Longer segments (the head of the Zipf distribution: one ID can own several
-// percent of a batch) are cut into parts of kSegChunk that are reduced by
-// separate groups into fp64 partial sums, then combined by one block per ID in
-// a fixed order.
+// Three cases, by how often the ID occurs in the batch:
+//  - once (most distinct IDs of a long-tailed batch): its gradient is the
+//    pooled gradient of its one bag, so scatter_singletons_kernel updates the
+//    row straight from the occurrence, in bag order, and the gradient rows
+//    stream through once;
+//  - 2 .. kSegChunk times: scatter_singletons_kernel drops each occurrence's
+//    bag into the ID's segment of bag_of_sorted[], and one lane group of
+//    reduce_adagrad_kernel gathers the segment's gradient rows;
+//  - more (the head of the Zipf distribution: one ID can own several percent of
+//    a batch): the segment is cut into parts of kSegChunk that separate groups
+//    reduce into fp64 partial sums, combined by one block per ID in a fixed
+//    order.
 #pragma once
 
 #include "kernels_dedup.cuh"
@@ -87,11 +94,72 @@ __device__ inline void reduce_segment(const Work& wk, const float* __restrict__ 
   }
 }
 
+// One warp per 32 consecutive occurrences.  Each lane looks its occurrence up in
+// the per-call set: an occurrence of a repeated ID that has a row is filed
+// under its ID; the lanes whose ID occurs once and has a row are then served
+// in turn by lane groups of G, which read the bag's gradient row, the table
+// row and its accumulator, and write both back updated.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_ids, long long n_bags) {
+  constexpr int kGroups = 32 / G;
+  const int lane = threadIdx.x & 31;
+  const int gl = lane % G, grp = lane / G;
+  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long n_rounds = (n_ids + 31) / 32;
+  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rounds; r += n_warps) {
+    const long long j = r * 32 + lane;
+    uint32_t row_word = kNoRow, bag = 0;
+    unsigned long long id = 0;
+    bool single = false;
+    if (j < n_ids) {
+      const uint32_t s = wk.occ_slot[j];
+      if (s != kNoSlot) {
+        const BatchSlot bs = wk.bset[s];
+        bag = wk.occ_bag[j];
+        if (bs.b != kNoRow && bag < n_bags) {
+          if (bs.a == kSingleton) { single = true; row_word = bs.b; id = bs.key; }
+          else wk.bag_of_sorted[bs.a + wk.occ_rank[j]] = bag;
+        }
+      }
+    }
+    unsigned todo = __ballot_sync(0xFFFFFFFFu, single);
+    while (todo) {
+      // the next kGroups flagged lanes, one per lane group
+      int src = -1;
+      unsigned rest = todo;
+#pragma unroll
+      for (int g = 0; g < kGroups; ++g) {
+        const int l = rest ? __ffs(rest) - 1 : -1;
+        if (l >= 0) rest &= rest - 1;
+        if (g == grp) src = l;
+      }
+      todo = rest;
+      const int from = src < 0 ? 0 : src;
+      const uint32_t rw = __shfl_sync(0xFFFFFFFFu, row_word, from);
+      const uint32_t bg = __shfl_sync(0xFFFFFFFFu, bag, from);
+      const unsigned long long key = __shfl_sync(0xFFFFFFFFu, id, from);
+      if (src >= 0) {
+        const float4* g4 = reinterpret_cast<const float4*>(grad + (size_t)bg * tv.dim);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+          const uint32_t c4 = gl + v * G;
+          if (c4 * 4u < tv.dim) {
+            const float4 x = __ldg(g4 + c4);
+            const D4 g = D4{(double)x.x, (double)x.y, (double)x.z, (double)x.w};
+            update_row(tv, rw, key, c4, g);
+          }
+        }
+      }
+    }
+  }
+}
+
 // One lane group per work item.  Items [0, n_unique) are the distinct IDs: a
-// group reduces an ID's whole segment and updates its row when the segment is
-// short.  Items [n_unique, n_unique + n_parts) are the parts of the long
-// segments: a group reduces one part into fp64 partial sums in scratch, which
-// combine_adagrad_kernel adds up afterwards.
+// group reduces the whole segment of a repeated ID and updates its row when
+// the segment is short.  Items [n_unique, n_unique + n_parts) are the parts of
+// the long segments: a group reduces one part into fp64 partial sums in
+// scratch, which combine_adagrad_kernel adds up afterwards.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
@@ -107,11 +175,12 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
     for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
     if (item < n) {
       const uint32_t u = item;
+      const uint32_t m = wk.ulen[u];
+      if (m < 2 || m > kSegChunk) continue;           // single occurrence: done already; long: in parts
       const uint32_t row_word = wk.urow[u];
       if (row_word == kNoRow) continue;
-      const uint32_t begin = wk.useg[u], end = wk.useg[u + 1];
-      if (end - begin > kSegChunk) continue;          // reduced in parts
-      reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
+      const uint32_t begin = wk.useg[u];
+      reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, begin + m, s);
       const unsigned long long id = wk.uid[u];
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
@@ -122,9 +191,8 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
       const uint32_t p = item - n;
       const uint32_t li = wk.part_u[p];
       const uint32_t u = wk.long_u[li];
-      if (wk.urow[u] == kNoRow) continue;
       const uint32_t k = p - wk.long_part0[li];
-      const uint32_t seg_end = wk.useg[u + 1];
+      const uint32_t seg_end = wk.useg[u] + wk.ulen[u];
       const uint32_t begin = wk.useg[u] + k * kSegChunk;
       const uint32_t end = begin + kSegChunk < seg_end ? begin + kSegChunk : seg_end;
       reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
@@ -153,7 +221,7 @@ combine_adagrad_kernel(TableView tv, Work wk) {
     const uint32_t u = wk.long_u[li];
     const uint32_t row_word = wk.urow[u];
     if (row_word == kNoRow) continue;                 // block-uniform
-    const uint32_t m = wk.useg[u + 1] - wk.useg[u];
+    const uint32_t m = wk.ulen[u];
     const uint32_t parts = (m + kSegChunk - 1) / kSegChunk;
     const double* src = wk.partials + (size_t)wk.long_part0[li] * dim;
     const unsigned long long id = wk.uid[u];

@@ -1,5 +1,5 @@
-// Forward: cuckoo look-up of every ID of a bag, gather of the rows that exist,
-// sum in ID order (the HashTable look-up operation of Section 2.1 serving the
+// Forward: cuckoo look-up of every ID of a batch, gather of the rows that
+// exist, sum per bag in ID order (the HashTable look-up operation of Section 2.1 serving the
 // parameter pull of Section 2.2; sum pooling per bag).
 #pragma once
 
@@ -39,26 +39,38 @@ __device__ inline bool quad_find(const TableView& tv, unsigned long long id, boo
   return hit;
 }
 
-// One group of G lanes per bag (G = 4, 8, 16 or 32 chosen from dim so that a
-// lane owns NV 16-byte column vectors).  Per round the group resolves G/4 IDs
-// at once -- each quad probes one ID -- then every lane adds its columns of
-// the rows found, in ID order, so the fp32 sum has one fixed order.
-template <int G, int NV>
+// Forward, step 1: one quad per ID occurrence resolves the ID to its row index
+// (kNoRow when the ID has none).  Every occurrence is independent, so the
+// random bucket reads of a whole batch are in flight together.
 __global__ void __launch_bounds__(256)
-lookup_pool_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
-                   const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out) {
-  constexpr int kIdsPerRound = G / 4;
-  const int lane = threadIdx.x & 31;
-  const int gl = lane % G;
-  const int sub = gl & 3;
-  const int quad = gl >> 2;
-  const unsigned group_mask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane - gl));
+probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
+                  uint32_t* __restrict__ occ_row) {
+  const int lane = threadIdx.x & 31, sub = lane & 3;
   const unsigned quad_mask = 0xFu << (lane - sub);
   const unsigned stash_hw = tv.st->stash_hw;
+  const long long n_quads = ((long long)gridDim.x * blockDim.x) >> 2;
+  for (long long j = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 2; j < n_ids; j += n_quads) {
+    const unsigned long long id = ids[j];
+    unsigned long long meta;
+    const bool hit = quad_find(tv, id, id != kEmptyKey, sub, quad_mask, stash_hw, &meta);
+    const bool any = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
+    if (hit) occ_row[j] = meta_resident(meta) ? meta_row(meta) : kNoRow;
+    else if (!any && sub == 0) occ_row[j] = kNoRow;
+  }
+}
+
+// Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
+// dim so that a lane owns NV 16-byte column vectors) adds up the rows of the
+// bag's IDs, in ID order, so the fp32 sum has one fixed order.  The row
+// indices are known, so the loads of up to four rows are issued together.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long n_ids,
+                   const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out) {
+  const int gl = threadIdx.x % G;
   const uint32_t dim = tv.dim;
   const long long groups_per_block = blockDim.x / G;
   const long long stride = (long long)gridDim.x * groups_per_block;
-
   for (long long bag = (long long)blockIdx.x * groups_per_block + threadIdx.x / G; bag < n_bags; bag += stride) {
     long long lo = offsets[bag], hi = offsets[bag + 1];
     if (lo < 0 || hi < lo || hi > n_ids) {
@@ -68,36 +80,22 @@ lookup_pool_kernel(TableView tv, const unsigned long long* __restrict__ ids, lon
     float4 sum[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) sum[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-
-    for (long long base = lo; base < hi; base += kIdsPerRound) {
-      const long long j = base + quad;
-      unsigned long long id = kEmptyKey;
-      if (j < hi) id = ids[j];
-      const bool active = id != kEmptyKey;
-      unsigned long long meta;
-      const bool hit = quad_find(tv, id, active, sub, quad_mask, stash_hw, &meta);
-      const uint32_t my_row = (hit && meta_resident(meta)) ? meta_row(meta) : kNoRow;
-      // lanes that hold a row, as a bit per lane of the group
-      const unsigned holders = (__ballot_sync(group_mask, my_row != kNoRow) & group_mask) >> (lane - gl);
-      uint32_t row_of[kIdsPerRound];
+    for (long long base = lo; base < hi; base += 4) {
+      uint32_t row[4];
 #pragma unroll
-      for (int i = 0; i < kIdsPerRound; ++i) {
-        const unsigned nib = (holders >> (4 * i)) & 0xFu;
-        const int src = 4 * i + (nib ? (__ffs(nib) - 1) : 0);
-        const uint32_t r = __shfl_sync(group_mask, my_row, src, G);
-        row_of[i] = nib ? r : kNoRow;
-      }
+      for (int k = 0; k < 4; ++k) row[k] = base + k < hi ? __ldg(occ_row + base + k) : kNoRow;
 #pragma unroll
-      for (int i = 0; i < kIdsPerRound; ++i) {
-        if (row_of[i] != kNoRow) {
-          const float4* src = reinterpret_cast<const float4*>(tv.w_row(row_of[i]));
+      for (int v = 0; v < NV; ++v) {
+        const uint32_t c4 = gl + v * G;
+        if (c4 * 4u < dim) {
+          float4 x[4];
 #pragma unroll
-          for (int v = 0; v < NV; ++v) {
-            const uint32_t c4 = gl + v * G;
-            if (c4 * 4u < dim) {
-              const float4 x = __ldg(src + c4);
-              sum[v].x += x.x; sum[v].y += x.y; sum[v].z += x.z; sum[v].w += x.w;
-            }
+          for (int k = 0; k < 4; ++k)
+            x[k] = row[k] != kNoRow ? __ldg(reinterpret_cast<const float4*>(tv.w_row(row[k])) + c4)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            if (row[k] != kNoRow) { sum[v].x += x[k].x; sum[v].y += x[k].y; sum[v].z += x[k].z; sum[v].w += x[k].w; }
           }
         }
       }

@@ -8,7 +8,8 @@
 
 namespace mono {
 
-// Take a free row.  Returns kNoRow (and records the refusal) when none is left.
+// Take a free row (one at a time: the bulk-import path).  Returns kNoRow (and
+// records the refusal) when none is left.
 __device__ inline uint32_t alloc_row(const TableView& tv) {
   const long long old = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top),
                                               (unsigned long long)(-1LL));
@@ -23,26 +24,89 @@ __device__ inline uint32_t alloc_row(const TableView& tv) {
   return tv.free_rows[old - 1];
 }
 
+// Block-wide reservation for the batch path: every thread states whether it
+// needs a row and how many entries of bag_of_sorted[] its ID's segment takes;
+// one thread does the two counter updates for the whole block, so counters that
+// every admission would otherwise hit are touched once per block and round.
+// Returns the row (kNoRow if refused or not asked for) and, in *seg_start, the
+// start of the reserved segment.  All threads of the block must call.
+struct BlockAlloc {
+  unsigned long long warp_sums[8];
+  long long row_base;       // free_top before this block's reservation
+  unsigned int rows_granted;
+  unsigned int seg_base;
+};
+
+__device__ inline uint32_t block_reserve(const TableView& tv, BlockAlloc* sh, bool need_row, uint32_t seg_len,
+                                         uint32_t* seg_start) {
+  unsigned long long total = 0;
+  const unsigned long long mine = ((unsigned long long)(need_row ? 1u : 0u) << 32) | seg_len;
+  const unsigned long long before = block_exclusive_scan(mine, sh->warp_sums, &total);
+  const unsigned int rows_wanted = (unsigned int)(total >> 32), seg_total = (unsigned int)total;
+  if (threadIdx.x == 0) {
+    unsigned int granted = 0;
+    long long old = 0;
+    if (rows_wanted) {
+      old = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top),
+                                 (unsigned long long)(-(long long)rows_wanted));
+      const long long avail = old > 0 ? old : 0;
+      granted = avail >= (long long)rows_wanted ? rows_wanted : (unsigned int)avail;
+      if (granted < rows_wanted) {
+        atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)(rows_wanted - granted));
+        atomicOr(&tv.st->error_bits, 1u /* MONO_DEV_ROWS_FULL */);
+        atomicAdd(&tv.st->n_rows_refused, (unsigned long long)(rows_wanted - granted));
+      }
+      if (granted) {
+        atomicAdd(&tv.st->n_resident, (unsigned long long)granted);
+        atomicAdd(&tv.st->n_admitted_total, (unsigned long long)granted);
+      }
+    }
+    sh->row_base = old;
+    sh->rows_granted = granted;
+    sh->seg_base = seg_total ? atomicAdd(&tv.st->seg_cursor, seg_total) : 0u;
+  }
+  __syncthreads();
+  *seg_start = sh->seg_base + (unsigned int)before;
+  const unsigned int my_row_index = (unsigned int)(before >> 32);
+  uint32_t row = kNoRow;
+  if (need_row && my_row_index < sh->rows_granted) row = tv.free_rows[sh->row_base - 1 - my_row_index];
+  return row;
+}
+
+// A distinct ID whose segment is longer than kSegChunk is reduced in parts:
+// register it and its parts.  Rare (the few hottest IDs of a batch).
+__device__ inline void register_long(const TableView& tv, const Work& wk, uint32_t u, uint32_t m) {
+  const uint32_t parts = (m + kSegChunk - 1) / kSegChunk;
+  const uint32_t li = atomicAdd(&tv.st->n_long, 1u);
+  const uint32_t p0 = atomicAdd(&tv.st->n_parts, parts);
+  if (li < wk.max_long && p0 + parts <= wk.max_parts) {
+    wk.long_u[li] = u;
+    wk.long_part0[li] = p0;
+    for (uint32_t p = 0; p < parts; ++p) wk.part_u[p0 + p] = li;
+  }
+}
+
 // Phase 2 of mono_apply_grads: one quad per distinct ID.  Tracked IDs get
 // count += multiplicity (saturating at the threshold), last_seen = now, and a
-// row if the count has reached the threshold; the rest are queued for
+// row if the count has reached the threshold; the rest are marked for
 // insertion.  No cell moves during this kernel, so the quad that found a cell
-// owns it.
+// owns it.  IDs that end up with a row and occur more than once also get their
+// segment of bag_of_sorted[] here.
 __global__ void __launch_bounds__(256)
 table_update_kernel(TableView tv, Work wk, uint32_t now) {
+  __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_unique;
   const unsigned stash_hw = tv.st->stash_hw;
-  const int lane = threadIdx.x & 31, sub = lane & 3, quad = lane >> 2;
+  const int lane = threadIdx.x & 31, sub = lane & 3;
   const unsigned quad_mask = 0xFu << (lane - sub);
-  const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
-  const uint32_t warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t per_block = blockDim.x / 4;
   unsigned int n_res = 0;
-  for (uint32_t u0 = warp_id * 8u; u0 < n; u0 += warps * 8u) {
-    const uint32_t u = u0 + quad;
+  for (uint32_t base = blockIdx.x * per_block; base < n; base += gridDim.x * per_block) {   // block-uniform
+    const uint32_t u = base + threadIdx.x / 4;
     const bool active = u < n;
     unsigned long long id = kEmptyKey;
-    uint32_t m = 0;
-    if (active) { id = wk.uid[u]; m = wk.useg[u + 1] - wk.useg[u]; }
+    uint32_t m = 0, slot = 0;
+    if (active) { id = wk.uid[u]; slot = wk.uslot[u]; m = wk.bset[slot].a; }
 
     // locate the cell (pointer kept on the lane that saw the key)
     Cell* where = nullptr;
@@ -70,32 +134,40 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
       found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
     }
 
+    // what the owning lane wants from the block-wide reservation
+    uint32_t low = meta_low(meta);
+    bool resident = false, need_row = false;
     if (hit) {
-      uint32_t low = meta_low(meta);
-      uint32_t row_word = kNoRow;
-      if (low & kResidentBit) {
-        row_word = low & ~kResidentBit;
-      } else {
+      resident = (low & kResidentBit) != 0;
+      if (!resident) {
         const unsigned long long c = (unsigned long long)low + m;
         low = c < tv.threshold ? (uint32_t)c : tv.threshold;
-        if (low >= tv.threshold) {
-          const uint32_t row = alloc_row(tv);
-          if (row != kNoRow) { low = kResidentBit | row; row_word = row | kFreshBit; }
-        }
+        need_row = low >= tv.threshold;
       }
+    }
+    // a segment is reserved for every repeated ID that may end up with a row
+    // (if the row is refused, the segment stays unused)
+    const uint32_t seg_len = (hit && (resident || need_row) && m > 1) ? m : 0u;
+    uint32_t seg_start = 0;
+    const uint32_t new_row = block_reserve(tv, &sh, need_row, seg_len, &seg_start);
+
+    if (hit) {
+      uint32_t row_word = kNoRow;
+      if (resident) row_word = low & ~kResidentBit;
+      else if (new_row != kNoRow) { low = kResidentBit | new_row; row_word = new_row | kFreshBit; }
       where->meta = make_meta(now, low);
       wk.urow[u] = row_word;
-      n_res += row_word != kNoRow;
-    }
-    // queue the IDs that are not tracked yet, one counter update per warp
-    const bool need_insert = active && !found && sub == 0;
-    const unsigned ins_mask = __ballot_sync(0xFFFFFFFFu, need_insert);
-    if (ins_mask) {
-      unsigned base = 0;
-      const int leader = __ffs(ins_mask) - 1;
-      if (lane == leader) base = atomicAdd(&tv.st->n_insert, (unsigned)__popc(ins_mask));
-      base = __shfl_sync(0xFFFFFFFFu, base, leader);
-      if (need_insert) wk.ins_list[base + __popc(ins_mask & ((1u << lane) - 1u))] = u;
+      wk.ulen[u] = m;
+      wk.useg[u] = seg_start;
+      BatchSlot bs; bs.key = id; bs.a = m > 1 ? seg_start : kSingleton; bs.b = row_word;
+      wk.bset[slot] = bs;
+      if (row_word != kNoRow) {
+        ++n_res;
+        if (m > kSegChunk) register_long(tv, wk, u, m);
+      }
+    } else if (active && !found && sub == 0) {
+      wk.urow[u] = kNeedsInsert;
+      wk.ulen[u] = m;
     }
   }
   for (int o = 16; o > 0; o >>= 1) n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
@@ -164,27 +236,38 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
   if (meta_resident(item.meta)) atomicAdd(&tv.st->n_resident, (unsigned long long)(-1LL));
 }
 
-// Phase 3 of mono_apply_grads: one thread per new ID.
+// Phase 3 of mono_apply_grads: one thread per distinct ID; the ones marked by
+// phase 2 as unknown to the key store are inserted (with a row straight away
+// when the batch alone reaches the threshold).
 __global__ void __launch_bounds__(256)
 table_insert_kernel(TableView tv, Work wk, uint32_t now) {
-  const uint32_t n = tv.st->n_insert;
-  const uint32_t stride = gridDim.x * blockDim.x;
+  __shared__ BlockAlloc sh;
+  const uint32_t n = tv.st->n_unique;
   const int lane = threadIdx.x & 31;
   unsigned int n_res = 0, n_done = 0;
-  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-    const uint32_t u = wk.ins_list[i];
+  for (uint32_t base = blockIdx.x * blockDim.x; base < n; base += gridDim.x * blockDim.x) {   // block-uniform
+    const uint32_t u = base + threadIdx.x;
+    const bool todo = u < n && wk.urow[u] == kNeedsInsert;
+    uint32_t m = 0;
+    if (todo) m = wk.ulen[u];
+    const uint32_t count = m < tv.threshold ? m : tv.threshold;
+    const bool need_row = todo && count >= tv.threshold;
+    uint32_t seg_start = 0;
+    const uint32_t row = block_reserve(tv, &sh, need_row, (need_row && m > 1) ? m : 0u, &seg_start);
+    if (!todo) continue;
     const unsigned long long id = wk.uid[u];
-    const uint32_t m = wk.useg[u + 1] - wk.useg[u];
-    uint32_t low = m < tv.threshold ? m : tv.threshold;
-    uint32_t row_word = kNoRow;
-    if (low >= tv.threshold) {
-      const uint32_t row = alloc_row(tv);
-      if (row != kNoRow) { low = kResidentBit | row; row_word = row | kFreshBit; }
-    }
+    uint32_t low = count, row_word = kNoRow;
+    if (row != kNoRow) { low = kResidentBit | row; row_word = row | kFreshBit; }
     wk.urow[u] = row_word;
+    wk.useg[u] = seg_start;
+    BatchSlot bs; bs.key = id; bs.a = m > 1 ? seg_start : kSingleton; bs.b = row_word;
+    wk.bset[wk.uslot[u]] = bs;
+    if (row_word != kNoRow) {
+      ++n_res;
+      if (m > kSegChunk) register_long(tv, wk, u, m);
+    }
     Cell item; item.key = id; item.meta = make_meta(now, low);
     cuckoo_insert(tv, item);
-    n_res += row_word != kNoRow;
     ++n_done;
   }
   for (int o = 16; o > 0; o >>= 1) {
@@ -196,6 +279,7 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     if (n_done) {
       atomicAdd(&tv.st->n_tracked, (unsigned long long)n_done);
       atomicAdd(&tv.st->n_inserted_total, (unsigned long long)n_done);
+      atomicAdd(&tv.st->n_insert, n_done);
     }
   }
 }
@@ -207,31 +291,43 @@ __global__ void finish_apply_kernel(DevState* st) {
     st->sum_unique += st->n_unique;
     st->sum_new += st->n_insert;
     st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_valid_ids = 0;
+    st->seg_cursor = 0;
   }
 }
 
 // Expiry sweep (Section 2.1, heuristic 2): a streaming pass over the key
 // store; a cell whose ID has been inactive for longer than ttl is emptied and
-// its row, if it has one, goes back on the free list.
+// its row, if it has one, goes back on the free list (one counter update per
+// warp and round).
 __global__ void __launch_bounds__(256)
 expire_kernel(TableView tv, unsigned long long n_cells, long long now) {
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long total = n_cells + kStashCells;
+  const unsigned long long rounds = (total + stride - 1) / stride;        // same for every thread
   const int lane = threadIdx.x & 31;
   unsigned int n_gone = 0, n_rows = 0;
-  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-    Cell* p = i < n_cells ? tv.cells + i : tv.stash + (i - n_cells);
-    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
-    if (v.x == kEmptyKey) continue;
-    if (now - (long long)meta_time(v.y) > (long long)tv.ttl) {
-      ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
-      *reinterpret_cast<ulonglong2*>(p) = e;
-      ++n_gone;
-      if (meta_resident(v.y)) {
-        const unsigned long long pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), 1ull);
-        tv.free_rows[pos] = meta_row(v.y);
-        ++n_rows;
+  for (unsigned long long r = 0; r < rounds; ++r) {
+    const unsigned long long i = r * stride + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    bool frees_row = false;
+    uint32_t row = 0;
+    if (i < total) {
+      Cell* p = i < n_cells ? tv.cells + i : tv.stash + (i - n_cells);
+      const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
+      if (v.x != kEmptyKey && now - (long long)meta_time(v.y) > (long long)tv.ttl) {
+        ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+        *reinterpret_cast<ulonglong2*>(p) = e;
+        ++n_gone;
+        if (meta_resident(v.y)) { frees_row = true; row = meta_row(v.y); ++n_rows; }
       }
+    }
+    const unsigned mask = __ballot_sync(0xFFFFFFFFu, frees_row);
+    if (mask) {
+      unsigned long long pos = 0;
+      const int leader = __ffs(mask) - 1;
+      if (lane == leader)
+        pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)__popc(mask));
+      pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
+      if (frees_row) tv.free_rows[pos + __popc(mask & ((1u << lane) - 1u))] = row;
     }
   }
   for (int o = 16; o > 0; o >>= 1) {
@@ -268,7 +364,7 @@ init_table_kernel(TableView tv, unsigned long long n_cells) {
 __global__ void __launch_bounds__(256)
 init_bset_kernel(BatchSlot* bset, unsigned long long n) {
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-  BatchSlot e; e.key = kEmptyKey; e.count = 0; e.spare = 0;
+  BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
   for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) bset[i] = e;
 }
 

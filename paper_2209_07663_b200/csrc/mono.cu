@@ -22,12 +22,11 @@
 using namespace mono;
 
 enum KernelId {
-  K_LOOKUP, K_FILL_BAG, K_DEDUP, K_SEG_COUNT, K_SEG_SCAN, K_SEG_OFFSETS, K_PLACE, K_UPDATE, K_INSERT,
-  K_REDUCE, K_COMBINE, K_RESET, K_FINISH, K_EXPIRE, K_STASH_TRIM, K_COUNT
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_COMBINE, K_RESET, K_FINISH, K_EXPIRE, K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
-  "lookup_pool", "fill_occ_bag", "dedup_insert", "seg_count", "seg_scan_blocks", "seg_offsets", "place",
-  "table_update", "table_insert", "reduce_adagrad", "combine_adagrad", "dedup_reset",
+  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "table_insert",
+  "scatter_singletons", "reduce_adagrad", "combine_adagrad", "dedup_reset",
   "finish_apply", "expire", "stash_trim"
 };
 
@@ -81,8 +80,8 @@ void dev_free(T*& p) { if (p) { cudaFree(p); p = nullptr; } }
 void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
-  dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.urow); dev_free(w.ins_list);
-  dev_free(w.block_sums); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
+  dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
+  dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec);
   t->max_ids = t->max_bags = 0;
 }
@@ -126,8 +125,7 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
 #define ALLOC(p, cnt) if ((rc = dev_alloc(t, &(p), (cnt))) != MONO_OK) { free_scratch(t); return rc; }
   ALLOC(w.bset, slots);
   ALLOC(w.occ_slot, n); ALLOC(w.occ_rank, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
-  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n + 1); ALLOC(w.urow, n); ALLOC(w.ins_list, n);
-  ALLOC(w.block_sums, (size_t)kScanBlocks + 1);
+  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
   ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts);
@@ -166,13 +164,21 @@ int dispatch_dim(uint32_t dim, F&& f) {
 int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
                   int64_t n_bags, float* out) {
   if (n_bags == 0) return MONO_OK;
+  uint32_t* occ_row = t->wk.occ_rank;      // scratch shared with the backward call (calls never overlap)
+  if (n_ids > 0) {
+    int64_t blocks = (n_ids * 4 + 255) / 256;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
+    if (blocks > cap) blocks = cap;
+    LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, occ_row));
+  }
   return dispatch_dim(t->tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     const int64_t groups_per_block = 256 / G;
     int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
-    const int64_t cap = (int64_t)grid_for(t, 8) * 4;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
     if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_LOOKUP, lookup_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, off, n_bags, out));
+    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, occ_row, n_ids, off,
+                                                                                    n_bags, out));
     CUDA_TRY(t, cudaGetLastError());
     return (int)MONO_OK;
   });
@@ -186,17 +192,15 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   const Work& wk = t->wk;
   const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
   LAUNCH(t, K_FILL_BAG, fill_occ_bag_kernel<<<g8, 256, 0, s>>>(off, n_bags, n_ids, wk.occ_bag, tv.st));
-  LAUNCH(t, K_DEDUP, dedup_insert_kernel<<<g8, 256, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
-                                                             tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
-  LAUNCH(t, K_SEG_COUNT, seg_count_kernel<<<kScanBlocks, kScanThreads, 0, s>>>(wk, tv.st));
-  LAUNCH(t, K_SEG_SCAN, seg_scan_blocks_kernel<<<1, 32, 0, s>>>(wk));
-  LAUNCH(t, K_SEG_OFFSETS, seg_offsets_kernel<<<kScanBlocks, kScanThreads, 0, s>>>(wk, tv.st));
-  LAUNCH(t, K_PLACE, place_kernel<<<g8, 256, 0, s>>>(wk, n_ids));
+  const int tiles = (int)((n_ids + kTileIds - 1) / kTileIds);
+  LAUNCH(t, K_DEDUP, dedup_tile_kernel<<<tiles, 256, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
+                                                            tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
-  LAUNCH(t, K_INSERT, table_insert_kernel<<<g4, 256, 0, s>>>(tv, wk, now));
+  LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   CUDA_TRY(t, cudaGetLastError());
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
+    LAUNCH(t, K_SCATTER, scatter_singletons_kernel<G, NV><<<g8 * 2, 256, 0, s>>>(tv, wk, grad, n_ids, n_bags));
     LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
@@ -295,6 +299,7 @@ int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
+  if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
   return launch_lookup(t, reinterpret_cast<const unsigned long long*>(ids), n_ids,
                        reinterpret_cast<const long long*>(slot_offsets), n_bags, out);
 }

@@ -87,7 +87,7 @@ struct DevState {
   unsigned int n_long;                   // distinct IDs whose segment is split into parts
   unsigned int n_parts;
   unsigned int n_valid_ids;
-  unsigned int pad1;
+  unsigned int seg_cursor;               // entries of bag_of_sorted[] handed out so far
   // export / audit scratch
   unsigned long long export_n;
 };
