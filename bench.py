@@ -200,7 +200,7 @@ def algorithmic_bytes(n, b, u, ur, unew, d):
 
 KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
-    "fill_occ_bag": "dedup", "dedup_tile": "dedup", "dedup_reset": "dedup", "finish_apply": "dedup",
+    "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
     "table_update": "table", "table_insert": "table",
     "scatter_singletons": "adagrad", "reduce_adagrad": "adagrad", "combine_adagrad": "adagrad",
 }

@@ -60,36 +60,47 @@ __device__ inline void update_row(const TableView& tv, uint32_t row_word, unsign
 }
 
 // Sum of grad rows of bags bag_of_sorted[begin .. end) for the NV column
-// vectors this lane owns.  Four independent loads in flight per step.
+// vectors this lane owns.  Eight independent row loads in flight per step.
 template <int G, int NV>
 __device__ inline void reduce_segment(const Work& wk, const float* __restrict__ grad, long long n_bags,
                                       uint32_t dim, int gl, uint32_t begin, uint32_t end, D4 (&s)[NV]) {
+  constexpr int kDepth = NV == 1 ? 8 : 4;
   uint32_t i = begin;
-  for (; i + 4 <= end; i += 4) {
-    uint32_t b[4];
+  for (; i + kDepth <= end; i += kDepth) {
+    uint32_t b[kDepth];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) b[k] = wk.bag_of_sorted[i + k];
+    for (int k = 0; k < kDepth; ++k) b[k] = wk.bag_of_sorted[i + k];
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const uint32_t c4 = gl + v * G;
       if (c4 * 4u < dim) {
-        float4 x[4];
+        float4 x[kDepth];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < kDepth; ++k)
           x[k] = b[k] < n_bags ? __ldg(reinterpret_cast<const float4*>(grad + (size_t)b[k] * dim) + c4)
                                : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) add4(s[v], x[k]);
+        for (int k = 0; k < kDepth; ++k) add4(s[v], x[k]);
       }
     }
   }
-  for (; i < end; ++i) {
-    const uint32_t b = wk.bag_of_sorted[i];
-    if (b >= n_bags) continue;
+  if (i < end) {
+    // the ragged tail, again with all its loads issued before the adds
+    uint32_t b[kDepth];
+#pragma unroll
+    for (int k = 0; k < kDepth; ++k) b[k] = i + k < end ? wk.bag_of_sorted[i + k] : 0xFFFFFFFFu;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const uint32_t c4 = gl + v * G;
-      if (c4 * 4u < dim) add4(s[v], __ldg(reinterpret_cast<const float4*>(grad + (size_t)b * dim) + c4));
+      if (c4 * 4u < dim) {
+        float4 x[kDepth];
+#pragma unroll
+        for (int k = 0; k < kDepth; ++k)
+          x[k] = b[k] < n_bags ? __ldg(reinterpret_cast<const float4*>(grad + (size_t)b[k] * dim) + c4)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < kDepth; ++k) add4(s[v], x[k]);
+      }
     }
   }
 }
@@ -117,6 +128,11 @@ scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad,
       if (s != kNoSlot) {
         const BatchSlot bs = wk.bset[s];
         bag = wk.occ_bag[j];
+        if (bs.a == kSingleton) {
+          // the only occurrence of its ID: nobody else needs the slot, empty it for the next call
+          BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
+          wk.bset[s] = e;
+        }
         if (bs.b != kNoRow && bag < n_bags) {
           if (bs.a == kSingleton) { single = true; row_word = bs.b; id = bs.key; }
           else wk.bag_of_sorted[bs.a + wk.occ_rank[j]] = bag;
@@ -155,15 +171,16 @@ scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad,
   }
 }
 
-// One lane group per work item.  Items [0, n_unique) are the distinct IDs: a
-// group reduces the whole segment of a repeated ID and updates its row when
-// the segment is short.  Items [n_unique, n_unique + n_parts) are the parts of
-// the long segments: a group reduces one part into fp64 partial sums in
+// One lane group per work item.  Items [0, n_multi) are the repeated IDs: a
+// group empties the ID's slot of the per-call set (every occurrence has been
+// filed by now), reduces the whole segment and updates the row when the
+// segment is short.  Items [n_multi, n_multi + n_parts) are the parts of the
+// long segments: a group reduces one part into fp64 partial sums in
 // scratch, which combine_adagrad_kernel adds up afterwards.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
-  const uint32_t n = tv.st->n_unique;
+  const uint32_t n = tv.st->n_multi;
   uint32_t n_parts = tv.st->n_parts;
   if (n_parts > wk.max_parts) n_parts = wk.max_parts;
   const uint32_t n_items = n + n_parts;
@@ -174,11 +191,14 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
 #pragma unroll
     for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
     if (item < n) {
-      const uint32_t u = item;
+      const uint32_t u = wk.multi_list[item];
+      if (gl == 0) {
+        BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
+        wk.bset[wk.uslot[u]] = e;
+      }
       const uint32_t m = wk.ulen[u];
-      if (m < 2 || m > kSegChunk) continue;           // single occurrence: done already; long: in parts
       const uint32_t row_word = wk.urow[u];
-      if (row_word == kNoRow) continue;
+      if (row_word == kNoRow || m > kSegChunk) continue;      // no row: gradient dropped; long: in parts
       const uint32_t begin = wk.useg[u];
       reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, begin + m, s);
       const unsigned long long id = wk.uid[u];

@@ -35,11 +35,17 @@ constexpr uint32_t kNeedsInsert = 0xFFFFFFFEu; // urow[] of an ID that is not in
 constexpr uint32_t kSegChunk = 256;            // longest segment one lane group reduces alone
 constexpr int kTileIds = 1024;                 // occurrences per block of dedup_tile_kernel
 constexpr int kTileSlots = 2048;               // shared-memory table of one tile
+constexpr int kPrimaryProbes = 16;             // positions tried in the primary tier of the per-call set
 
 // Scratch of one mono_apply_grads call.
 struct Work {
-  BatchSlot* bset;           // [bset_mask + 1], all keys empty between calls
-  unsigned long long bset_mask;
+  // The per-call set has two tiers, both empty between calls.  The primary tier
+  // is small enough to stay in L2 for a batch with the usual share of repeats;
+  // an ID that finds no free slot among its first kPrimaryProbes positions there
+  // goes to the secondary tier, which alone can hold a batch of all-distinct IDs.
+  BatchSlot* bset;           // [primary_mask + 1 + secondary_mask + 1]
+  uint32_t primary_mask;     // primary tier: slots [0, primary_mask]
+  uint32_t secondary_mask;   // secondary tier: slots primary_mask + 1 + [0, secondary_mask]
   uint32_t* occ_slot;        // [max_ids] slot of each occurrence, kNoSlot if padding / outside bags
   uint32_t* occ_rank;        // [max_ids] rank of the occurrence among those of its ID
   uint32_t* occ_bag;         // [max_ids] bag of each occurrence
@@ -49,6 +55,7 @@ struct Work {
   uint32_t* useg;            // [max_ids] start of the ID's segment in bag_of_sorted
   uint32_t* ulen;            // [max_ids] multiplicity of the ID in this batch
   uint32_t* urow;            // [max_ids] row word per distinct ID (kNoRow / kNeedsInsert / row | kFreshBit)
+  uint32_t* multi_list;      // [max_ids / 2 + 1] distinct IDs that occur more than once
   uint32_t* long_u;          // [max_long] distinct IDs whose segment is reduced in parts
   uint32_t* long_part0;      // [max_long] first part of each
   uint32_t* part_u;          // [max_parts] owner (index into long_u) of each part
@@ -136,34 +143,62 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   }
   __syncthreads();
 
-  // 2. one visit of the global set per distinct ID of the tile
-  unsigned long long new_id[kSlotsPerThread];
-  uint32_t new_gslot[kSlotsPerThread];
+  // 2. one visit of the global set per distinct ID of the tile.  The first
+  //    probes of a thread's slots are issued together, then resolved, then the
+  //    counter updates are issued together, so their latencies overlap.
+  unsigned long long tid_[kSlotsPerThread], seen[kSlotsPerThread];
+  uint32_t g[kSlotsPerThread], base_rank[kSlotsPerThread];
+  bool is_new[kSlotsPerThread];
+#pragma unroll
+  for (int k = 0; k < kSlotsPerThread; ++k) {
+    tid_[k] = s_key[k * 256 + threadIdx.x];
+    g[k] = (uint32_t)(mix_b(tid_[k] ^ seed) >> 20) & wk.primary_mask;
+    seen[k] = tid_[k] == kEmptyKey ? 0ull : *reinterpret_cast<volatile unsigned long long*>(&wk.bset[g[k]].key);
+  }
   unsigned int n_new = 0;
 #pragma unroll
   for (int k = 0; k < kSlotsPerThread; ++k) {
-    const int s = k * 256 + threadIdx.x;
-    const unsigned long long id = s_key[s];
-    new_id[k] = kEmptyKey;
-    new_gslot[k] = 0;
-    if (id == kEmptyKey) continue;
-    unsigned long long g = (mix_b(id ^ seed) >> 20) & wk.bset_mask;
-    bool is_new = false;
-    // the set has at least twice as many slots as a call has IDs, so an empty
-    // slot is always reached; the bound only guards against misuse
-    for (unsigned long long probe = 0; probe <= wk.bset_mask; ++probe) {
-      unsigned long long kk = *reinterpret_cast<volatile unsigned long long*>(&wk.bset[g].key);
+    is_new[k] = false;
+    if (tid_[k] == kEmptyKey) continue;
+    const unsigned long long id = tid_[k];
+    unsigned long long kk = seen[k];
+    bool placed = false;
+    // primary tier: a short window of consecutive positions
+    for (int probe = 0; probe < kPrimaryProbes; ++probe) {
       if (kk == kEmptyKey) {
-        kk = atomicCAS(&wk.bset[g].key, kEmptyKey, id);
-        if (kk == kEmptyKey) { is_new = true; break; }
+        kk = atomicCAS(&wk.bset[g[k]].key, kEmptyKey, id);
+        if (kk == kEmptyKey) { is_new[k] = true; placed = true; break; }
       }
-      if (kk == id) break;
-      g = (g + 1) & wk.bset_mask;
+      if (kk == id) { placed = true; break; }
+      g[k] = (g[k] + 1) & wk.primary_mask;
+      kk = *reinterpret_cast<volatile unsigned long long*>(&wk.bset[g[k]].key);
     }
-    const unsigned int base = atomicAdd(&wk.bset[g].a, s_cnt[s]);
-    s_cnt[s] = base;
-    s_gslot[s] = (uint32_t)g;
-    if (is_new) { new_id[k] = id; new_gslot[k] = (uint32_t)g; ++n_new; }
+    if (!placed) {
+      // secondary tier: it has at least twice as many slots as a call has IDs, so
+      // an empty slot is always reached; the bound only guards against misuse
+      const uint32_t base2 = wk.primary_mask + 1u;
+      uint32_t q = (uint32_t)(mix_a(id ^ seed) >> 24) & wk.secondary_mask;
+      for (uint32_t probe = 0; probe <= wk.secondary_mask; ++probe) {
+        kk = *reinterpret_cast<volatile unsigned long long*>(&wk.bset[base2 + q].key);
+        if (kk == kEmptyKey) {
+          kk = atomicCAS(&wk.bset[base2 + q].key, kEmptyKey, id);
+          if (kk == kEmptyKey) { is_new[k] = true; break; }
+        }
+        if (kk == id) break;
+        q = (q + 1) & wk.secondary_mask;
+      }
+      g[k] = base2 + q;
+    }
+    n_new += is_new[k];
+  }
+#pragma unroll
+  for (int k = 0; k < kSlotsPerThread; ++k)
+    base_rank[k] = tid_[k] == kEmptyKey ? 0u : atomicAdd(&wk.bset[g[k]].a, s_cnt[k * 256 + threadIdx.x]);
+#pragma unroll
+  for (int k = 0; k < kSlotsPerThread; ++k) {
+    if (tid_[k] == kEmptyKey) continue;
+    s_cnt[k * 256 + threadIdx.x] = base_rank[k];
+    s_gslot[k * 256 + threadIdx.x] = g[k];
   }
   // number the IDs this tile saw first: one counter update per tile
   // (new IDs in the low word, valid occurrences in the high word of one scan)
@@ -178,9 +213,9 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   my_u += s_ubase;
 #pragma unroll
   for (int k = 0; k < kSlotsPerThread; ++k) {
-    if (new_id[k] != kEmptyKey) {
-      wk.uid[my_u] = new_id[k];
-      wk.uslot[my_u] = new_gslot[k];
+    if (is_new[k]) {
+      wk.uid[my_u] = tid_[k];
+      wk.uslot[my_u] = g[k];
       ++my_u;
     }
   }
@@ -194,17 +229,6 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
       wk.occ_slot[j] = s == kNoSlot ? kNoSlot : s_gslot[s];
       wk.occ_rank[j] = s == kNoSlot ? 0u : s_cnt[s] + my_rank[k];
     }
-  }
-}
-
-// Empty the set again (only the slots that were used) for the next call.
-__global__ void __launch_bounds__(256)
-dedup_reset_kernel(Work wk, const DevState* st) {
-  const uint32_t n = st->n_unique;
-  const uint32_t stride = gridDim.x * blockDim.x;
-  for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < n; u += stride) {
-    BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
-    wk.bset[wk.uslot[u]] = e;
   }
 }
 

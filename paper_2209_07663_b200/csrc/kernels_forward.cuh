@@ -39,23 +39,45 @@ __device__ inline bool quad_find(const TableView& tv, unsigned long long id, boo
   return hit;
 }
 
-// Forward, step 1: one quad per ID occurrence resolves the ID to its row index
-// (kNoRow when the ID has none).  Every occurrence is independent, so the
-// random bucket reads of a whole batch are in flight together.
+// Read-only look-up by one thread: the four cells of the first bucket are
+// read together (one 64-byte piece of a line), the second bucket and the stash
+// only on a miss.  Returns true and the metadata when the ID is tracked.
+__device__ inline bool thread_lookup(const TableView& tv, unsigned long long id, unsigned stash_hw,
+                                     unsigned long long* meta) {
+  const Cell* b = tv.cells + tv.bucket0(id) * kCellsPerBucket;
+  Cell c[kCellsPerBucket];
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+    if (c[k].key == id) { *meta = c[k].meta; return true; }
+  b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+    if (c[k].key == id) { *meta = c[k].meta; return true; }
+  for (unsigned i = 0; i < stash_hw; ++i) {
+    const Cell s = load_cell_ro(tv.stash + i);
+    if (s.key == id) { *meta = s.meta; return true; }
+  }
+  return false;
+}
+
+// Forward, step 1: one thread per ID occurrence resolves the ID to its row
+// index (kNoRow when the ID has none).  Every occurrence is independent, so
+// the random bucket reads of a whole batch are in flight together.
 __global__ void __launch_bounds__(256)
 probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
                   uint32_t* __restrict__ occ_row) {
-  const int lane = threadIdx.x & 31, sub = lane & 3;
-  const unsigned quad_mask = 0xFu << (lane - sub);
   const unsigned stash_hw = tv.st->stash_hw;
-  const long long n_quads = ((long long)gridDim.x * blockDim.x) >> 2;
-  for (long long j = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 2; j < n_ids; j += n_quads) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
     const unsigned long long id = ids[j];
-    unsigned long long meta;
-    const bool hit = quad_find(tv, id, id != kEmptyKey, sub, quad_mask, stash_hw, &meta);
-    const bool any = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
-    if (hit) occ_row[j] = meta_resident(meta) ? meta_row(meta) : kNoRow;
-    else if (!any && sub == 0) occ_row[j] = kNoRow;
+    unsigned long long meta = 0;
+    uint32_t row = kNoRow;
+    if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) row = meta_row(meta);
+    occ_row[j] = row;
   }
 }
 

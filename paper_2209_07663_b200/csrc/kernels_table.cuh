@@ -24,26 +24,36 @@ __device__ inline uint32_t alloc_row(const TableView& tv) {
   return tv.free_rows[old - 1];
 }
 
-// Block-wide reservation for the batch path: every thread states whether it
-// needs a row and how many entries of bag_of_sorted[] its ID's segment takes;
-// one thread does the two counter updates for the whole block, so counters that
-// every admission would otherwise hit are touched once per block and round.
-// Returns the row (kNoRow if refused or not asked for) and, in *seg_start, the
-// start of the reserved segment.  All threads of the block must call.
+// Block-wide reservation for the batch path: every thread states whether its
+// ID needs a row, whether it occurs more than once in the batch (it then gets a
+// place in multi_list[]) and how many entries of bag_of_sorted[] its segment
+// takes; one thread does the counter updates for the whole block, so counters
+// that every admission would otherwise hit are touched once per block and
+// round.  All threads of the block must call.
 struct BlockAlloc {
   unsigned long long warp_sums[8];
   long long row_base;       // free_top before this block's reservation
   unsigned int rows_granted;
   unsigned int seg_base;
+  unsigned int multi_base;
 };
 
-__device__ inline uint32_t block_reserve(const TableView& tv, BlockAlloc* sh, bool need_row, uint32_t seg_len,
-                                         uint32_t* seg_start) {
+struct Reservation {
+  uint32_t row;             // kNoRow if refused or not asked for
+  uint32_t seg_start;
+  uint32_t multi_pos;
+};
+
+__device__ inline Reservation block_reserve(const TableView& tv, BlockAlloc* sh, bool need_row, bool is_multi,
+                                            uint32_t seg_len) {
+  // rows in bits 48.., repeated IDs in bits 32..47, segment entries in the low word
   unsigned long long total = 0;
-  const unsigned long long mine = ((unsigned long long)(need_row ? 1u : 0u) << 32) | seg_len;
+  const unsigned long long mine =
+      ((unsigned long long)(need_row ? 1u : 0u) << 48) | ((unsigned long long)(is_multi ? 1u : 0u) << 32) | seg_len;
   const unsigned long long before = block_exclusive_scan(mine, sh->warp_sums, &total);
-  const unsigned int rows_wanted = (unsigned int)(total >> 32), seg_total = (unsigned int)total;
   if (threadIdx.x == 0) {
+    const unsigned int rows_wanted = (unsigned int)(total >> 48), multi_total = (unsigned int)(total >> 32) & 0xFFFFu,
+                       seg_total = (unsigned int)total;
     unsigned int granted = 0;
     long long old = 0;
     if (rows_wanted) {
@@ -64,13 +74,16 @@ __device__ inline uint32_t block_reserve(const TableView& tv, BlockAlloc* sh, bo
     sh->row_base = old;
     sh->rows_granted = granted;
     sh->seg_base = seg_total ? atomicAdd(&tv.st->seg_cursor, seg_total) : 0u;
+    sh->multi_base = multi_total ? atomicAdd(&tv.st->n_multi, multi_total) : 0u;
   }
   __syncthreads();
-  *seg_start = sh->seg_base + (unsigned int)before;
-  const unsigned int my_row_index = (unsigned int)(before >> 32);
-  uint32_t row = kNoRow;
-  if (need_row && my_row_index < sh->rows_granted) row = tv.free_rows[sh->row_base - 1 - my_row_index];
-  return row;
+  Reservation r;
+  r.seg_start = sh->seg_base + (unsigned int)before;
+  r.multi_pos = sh->multi_base + ((unsigned int)(before >> 32) & 0xFFFFu);
+  const unsigned int my_row_index = (unsigned int)(before >> 48);
+  r.row = kNoRow;
+  if (need_row && my_row_index < sh->rows_granted) r.row = tv.free_rows[sh->row_base - 1 - my_row_index];
+  return r;
 }
 
 // A distinct ID whose segment is longer than kSegChunk is reduced in parts:
@@ -86,55 +99,59 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
   }
 }
 
-// Phase 2 of mono_apply_grads: one quad per distinct ID.  Tracked IDs get
+// Thread-level look-up that keeps the cell's address: the four cells of the
+// first bucket are read together, the second bucket and the stash only on a miss.
+__device__ inline Cell* thread_find(const TableView& tv, unsigned long long id, unsigned stash_hw,
+                                    unsigned long long* meta) {
+  Cell* b = tv.cells + tv.bucket0(id) * kCellsPerBucket;
+  Cell c[kCellsPerBucket];
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) {
+    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(b + k);
+    c[k].key = v.x; c[k].meta = v.y;
+  }
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+    if (c[k].key == id) { *meta = c[k].meta; return b + k; }
+  b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) {
+    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(b + k);
+    c[k].key = v.x; c[k].meta = v.y;
+  }
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+    if (c[k].key == id) { *meta = c[k].meta; return b + k; }
+  for (unsigned i = 0; i < stash_hw; ++i)
+    if (tv.stash[i].key == id) { *meta = tv.stash[i].meta; return tv.stash + i; }
+  return nullptr;
+}
+
+// Phase 2 of mono_apply_grads: one thread per distinct ID.  Tracked IDs get
 // count += multiplicity (saturating at the threshold), last_seen = now, and a
 // row if the count has reached the threshold; the rest are marked for
-// insertion.  No cell moves during this kernel, so the quad that found a cell
-// owns it.  IDs that end up with a row and occur more than once also get their
-// segment of bag_of_sorted[] here.
+// insertion.  No cell moves during this kernel, so the thread that found a
+// cell owns it.  IDs that end up with a row and occur more than once also get
+// their segment of bag_of_sorted[] here.
 __global__ void __launch_bounds__(256)
 table_update_kernel(TableView tv, Work wk, uint32_t now) {
   __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_unique;
   const unsigned stash_hw = tv.st->stash_hw;
-  const int lane = threadIdx.x & 31, sub = lane & 3;
-  const unsigned quad_mask = 0xFu << (lane - sub);
-  const uint32_t per_block = blockDim.x / 4;
   unsigned int n_res = 0;
-  for (uint32_t base = blockIdx.x * per_block; base < n; base += gridDim.x * per_block) {   // block-uniform
-    const uint32_t u = base + threadIdx.x / 4;
+  for (uint32_t base = blockIdx.x * blockDim.x; base < n; base += gridDim.x * blockDim.x) {   // block-uniform
+    const uint32_t u = base + threadIdx.x;
     const bool active = u < n;
-    unsigned long long id = kEmptyKey;
+    unsigned long long id = kEmptyKey, meta = 0;
     uint32_t m = 0, slot = 0;
-    if (active) { id = wk.uid[u]; slot = wk.uslot[u]; m = wk.bset[slot].a; }
-
-    // locate the cell (pointer kept on the lane that saw the key)
     Cell* where = nullptr;
-    unsigned long long meta = 0;
-    bool hit = false;
     if (active) {
-      Cell* p = tv.cells + tv.bucket0(id) * kCellsPerBucket + sub;
-      const Cell c = *p;
-      if (c.key == id) { hit = true; where = p; meta = c.meta; }
+      id = wk.uid[u];
+      slot = wk.uslot[u];
+      m = wk.bset[slot].a;
+      where = thread_find(tv, id, stash_hw, &meta);
     }
-    bool found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
-    if (!found) {
-      if (active) {
-        Cell* p = tv.cells + tv.bucket1(id) * kCellsPerBucket + sub;
-        const Cell c = *p;
-        if (c.key == id) { hit = true; where = p; meta = c.meta; }
-      }
-      found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
-      if (!found && stash_hw != 0 && active) {
-        for (unsigned i = sub; i < stash_hw; i += kCellsPerBucket) {
-          const Cell c = tv.stash[i];
-          if (c.key == id) { hit = true; where = tv.stash + i; meta = c.meta; break; }
-        }
-      }
-      found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
-    }
-
-    // what the owning lane wants from the block-wide reservation
+    const bool hit = where != nullptr;
     uint32_t low = meta_low(meta);
     bool resident = false, need_row = false;
     if (hit) {
@@ -148,30 +165,29 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
     // a segment is reserved for every repeated ID that may end up with a row
     // (if the row is refused, the segment stays unused)
     const uint32_t seg_len = (hit && (resident || need_row) && m > 1) ? m : 0u;
-    uint32_t seg_start = 0;
-    const uint32_t new_row = block_reserve(tv, &sh, need_row, seg_len, &seg_start);
-
+    const Reservation rv = block_reserve(tv, &sh, need_row, hit && m > 1, seg_len);
+    if (!active) continue;
+    wk.ulen[u] = m;
     if (hit) {
       uint32_t row_word = kNoRow;
       if (resident) row_word = low & ~kResidentBit;
-      else if (new_row != kNoRow) { low = kResidentBit | new_row; row_word = new_row | kFreshBit; }
+      else if (rv.row != kNoRow) { low = kResidentBit | rv.row; row_word = rv.row | kFreshBit; }
       where->meta = make_meta(now, low);
       wk.urow[u] = row_word;
-      wk.ulen[u] = m;
-      wk.useg[u] = seg_start;
-      BatchSlot bs; bs.key = id; bs.a = m > 1 ? seg_start : kSingleton; bs.b = row_word;
+      wk.useg[u] = rv.seg_start;
+      BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kSingleton; bs.b = row_word;
       wk.bset[slot] = bs;
+      if (m > 1) wk.multi_list[rv.multi_pos] = u;
       if (row_word != kNoRow) {
         ++n_res;
         if (m > kSegChunk) register_long(tv, wk, u, m);
       }
-    } else if (active && !found && sub == 0) {
+    } else {
       wk.urow[u] = kNeedsInsert;
-      wk.ulen[u] = m;
     }
   }
   for (int o = 16; o > 0; o >>= 1) n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
-  if (lane == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
+  if ((threadIdx.x & 31) == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
 }
 
 // Put `item` (a key that is in no cell) into the key store.  Lock-free against
@@ -252,16 +268,16 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     if (todo) m = wk.ulen[u];
     const uint32_t count = m < tv.threshold ? m : tv.threshold;
     const bool need_row = todo && count >= tv.threshold;
-    uint32_t seg_start = 0;
-    const uint32_t row = block_reserve(tv, &sh, need_row, (need_row && m > 1) ? m : 0u, &seg_start);
+    const Reservation rv = block_reserve(tv, &sh, need_row, todo && m > 1, (need_row && m > 1) ? m : 0u);
     if (!todo) continue;
     const unsigned long long id = wk.uid[u];
     uint32_t low = count, row_word = kNoRow;
-    if (row != kNoRow) { low = kResidentBit | row; row_word = row | kFreshBit; }
+    if (rv.row != kNoRow) { low = kResidentBit | rv.row; row_word = rv.row | kFreshBit; }
     wk.urow[u] = row_word;
-    wk.useg[u] = seg_start;
-    BatchSlot bs; bs.key = id; bs.a = m > 1 ? seg_start : kSingleton; bs.b = row_word;
+    wk.useg[u] = rv.seg_start;
+    BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kSingleton; bs.b = row_word;
     wk.bset[wk.uslot[u]] = bs;
+    if (m > 1) wk.multi_list[rv.multi_pos] = u;
     if (row_word != kNoRow) {
       ++n_res;
       if (m > kSegChunk) register_long(tv, wk, u, m);
@@ -291,7 +307,7 @@ __global__ void finish_apply_kernel(DevState* st) {
     st->sum_unique += st->n_unique;
     st->sum_new += st->n_insert;
     st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_valid_ids = 0;
-    st->seg_cursor = 0;
+    st->seg_cursor = 0; st->n_multi = 0;
   }
 }
 

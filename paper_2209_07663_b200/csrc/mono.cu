@@ -22,11 +22,12 @@
 using namespace mono;
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_COMBINE, K_RESET, K_FINISH, K_EXPIRE, K_STASH_TRIM, K_COUNT
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
   "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "table_insert",
-  "scatter_singletons", "reduce_adagrad", "combine_adagrad", "dedup_reset",
+  "scatter_singletons", "reduce_adagrad", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
 
@@ -81,7 +82,7 @@ void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
   dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
-  dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
+  dev_free(w.multi_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec);
   t->max_ids = t->max_bags = 0;
 }
@@ -120,12 +121,16 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   free_scratch(t);
   Work& w = t->wk;
   const size_t n = (size_t)max_ids;
-  const uint64_t slots = next_pow2(2 * (uint64_t)max_ids);
+  uint64_t primary = next_pow2(((uint64_t)max_ids * 2) / 5);
+  if (primary < 1024) primary = 1024;
+  const uint64_t secondary = next_pow2(2 * (uint64_t)max_ids);
+  const uint64_t slots = primary + secondary;
   int rc;
 #define ALLOC(p, cnt) if ((rc = dev_alloc(t, &(p), (cnt))) != MONO_OK) { free_scratch(t); return rc; }
   ALLOC(w.bset, slots);
   ALLOC(w.occ_slot, n); ALLOC(w.occ_rank, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
   ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n);
+  ALLOC(w.multi_list, n / 2 + 1);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
   ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts);
@@ -133,7 +138,8 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   ALLOC(t->stage_ids, n); ALLOC(t->stage_off, (size_t)max_bags + 1);
   ALLOC(t->stage_vec, (size_t)max_bags * t->tv.dim);
 #undef ALLOC
-  w.bset_mask = slots - 1;
+  w.primary_mask = (uint32_t)(primary - 1);
+  w.secondary_mask = (uint32_t)(secondary - 1);
   init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(w.bset, slots);
   CUDA_TRY(t, cudaGetLastError());
   t->max_ids = max_ids;
@@ -166,8 +172,8 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
   if (n_bags == 0) return MONO_OK;
   uint32_t* occ_row = t->wk.occ_rank;      // scratch shared with the backward call (calls never overlap)
   if (n_ids > 0) {
-    int64_t blocks = (n_ids * 4 + 255) / 256;
-    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
+    int64_t blocks = (n_ids + 255) / 256;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 4;
     if (blocks > cap) blocks = cap;
     LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, occ_row));
   }
@@ -206,7 +212,6 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   });
   if (rc != MONO_OK) return rc;
   LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g4, 256, 0, s>>>(tv, wk));
-  LAUNCH(t, K_RESET, dedup_reset_kernel<<<g8, 256, 0, s>>>(wk, tv.st));
   LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 32, 0, s>>>(tv.st));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;

@@ -88,6 +88,8 @@ struct DevState {
   unsigned int n_parts;
   unsigned int n_valid_ids;
   unsigned int seg_cursor;               // entries of bag_of_sorted[] handed out so far
+  unsigned int n_multi;                  // distinct IDs that occur more than once in the batch
+  unsigned int pad1;
   // export / audit scratch
   unsigned long long export_n;
 };
