@@ -31,10 +31,10 @@ struct __align__(16) BatchSlot {
 
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
 constexpr uint32_t kSingleton = 0xFFFFFFFFu;   // BatchSlot::a of an ID that occurs once in the batch
-constexpr uint32_t kNeedsInsert = 0xFFFFFFFEu; // urow[] of an ID that is not in the key store yet
 constexpr uint32_t kSegChunk = 256;            // longest segment one lane group reduces alone
 constexpr int kTileIds = 1024;                 // occurrences per block of dedup_tile_kernel
 constexpr int kTileSlots = 2048;               // shared-memory table of one tile
+constexpr int kTileThreads = 512;              // block size of dedup_tile_kernel
 constexpr int kPrimaryProbes = 16;             // positions tried in the primary tier of the per-call set
 
 // Scratch of one mono_apply_grads call.
@@ -54,7 +54,8 @@ struct Work {
   uint32_t* uslot;           // [max_ids] slot of each distinct ID
   uint32_t* useg;            // [max_ids] start of the ID's segment in bag_of_sorted
   uint32_t* ulen;            // [max_ids] multiplicity of the ID in this batch
-  uint32_t* urow;            // [max_ids] row word per distinct ID (kNoRow / kNeedsInsert / row | kFreshBit)
+  uint32_t* urow;            // [max_ids] row word per distinct ID (kNoRow / row | kFreshBit)
+  uint32_t* ins_list;        // [max_ids] distinct IDs that are not in the key store yet
   uint32_t* multi_list;      // [max_ids / 2 + 1] distinct IDs that occur more than once
   uint32_t* long_u;          // [max_long] distinct IDs whose segment is reduced in parts
   uint32_t* long_part0;      // [max_long] first part of each
@@ -100,19 +101,19 @@ __device__ inline unsigned long long block_exclusive_scan(unsigned long long v, 
 }
 
 // One block per tile of kTileIds consecutive occurrences.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kTileThreads, 3)
 dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long n_ids,
                   const long long* __restrict__ offsets, long long n_bags, DevState* st,
                   unsigned long long seed) {
-  constexpr int kPerThread = kTileIds / 256;
-  constexpr int kSlotsPerThread = kTileSlots / 256;
+  constexpr int kPerThread = kTileIds / kTileThreads;
+  constexpr int kSlotsPerThread = kTileSlots / kTileThreads;
   __shared__ unsigned long long s_key[kTileSlots];
   __shared__ unsigned int s_cnt[kTileSlots];     // multiplicity in the tile, then base rank
   __shared__ unsigned int s_gslot[kTileSlots];   // the ID's slot in the global set
-  __shared__ unsigned long long s_warp[8];
+  __shared__ unsigned long long s_warp[kTileThreads / 32];
   __shared__ unsigned int s_ubase;
 
-  for (int i = threadIdx.x; i < kTileSlots; i += 256) { s_key[i] = kEmptyKey; s_cnt[i] = 0; }
+  for (int i = threadIdx.x; i < kTileSlots; i += kTileThreads) { s_key[i] = kEmptyKey; s_cnt[i] = 0; }
   long long first = offsets[0], last = offsets[n_bags];
   if (first < 0) first = 0;
   if (last > n_ids) last = n_ids;
@@ -124,7 +125,7 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   unsigned int n_valid = 0;
 #pragma unroll
   for (int k = 0; k < kPerThread; ++k) {
-    const long long j = tile0 + k * 256 + threadIdx.x;
+    const long long j = tile0 + k * kTileThreads + threadIdx.x;
     unsigned long long id = kEmptyKey;
     if (j >= first && j < last) id = ids[j];
     my_slot[k] = kNoSlot;
@@ -151,7 +152,7 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   bool is_new[kSlotsPerThread];
 #pragma unroll
   for (int k = 0; k < kSlotsPerThread; ++k) {
-    tid_[k] = s_key[k * 256 + threadIdx.x];
+    tid_[k] = s_key[k * kTileThreads + threadIdx.x];
     g[k] = (uint32_t)(mix_b(tid_[k] ^ seed) >> 20) & wk.primary_mask;
     seen[k] = tid_[k] == kEmptyKey ? 0ull : *reinterpret_cast<volatile unsigned long long*>(&wk.bset[g[k]].key);
   }
@@ -193,12 +194,12 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   }
 #pragma unroll
   for (int k = 0; k < kSlotsPerThread; ++k)
-    base_rank[k] = tid_[k] == kEmptyKey ? 0u : atomicAdd(&wk.bset[g[k]].a, s_cnt[k * 256 + threadIdx.x]);
+    base_rank[k] = tid_[k] == kEmptyKey ? 0u : atomicAdd(&wk.bset[g[k]].a, s_cnt[k * kTileThreads + threadIdx.x]);
 #pragma unroll
   for (int k = 0; k < kSlotsPerThread; ++k) {
     if (tid_[k] == kEmptyKey) continue;
-    s_cnt[k * 256 + threadIdx.x] = base_rank[k];
-    s_gslot[k * 256 + threadIdx.x] = g[k];
+    s_cnt[k * kTileThreads + threadIdx.x] = base_rank[k];
+    s_gslot[k * kTileThreads + threadIdx.x] = g[k];
   }
   // number the IDs this tile saw first: one counter update per tile
   // (new IDs in the low word, valid occurrences in the high word of one scan)
@@ -223,7 +224,7 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   // 3. every occurrence learns its ID's slot and its rank
 #pragma unroll
   for (int k = 0; k < kPerThread; ++k) {
-    const long long j = tile0 + k * 256 + threadIdx.x;
+    const long long j = tile0 + k * kTileThreads + threadIdx.x;
     if (j < n_ids) {
       const uint32_t s = my_slot[k];
       wk.occ_slot[j] = s == kNoSlot ? kNoSlot : s_gslot[s];

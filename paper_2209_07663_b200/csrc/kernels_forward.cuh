@@ -39,45 +39,92 @@ __device__ inline bool quad_find(const TableView& tv, unsigned long long id, boo
   return hit;
 }
 
-// Read-only look-up by one thread: the four cells of the first bucket are
-// read together (one 64-byte piece of a line), the second bucket and the stash
-// only on a miss.  Returns true and the metadata when the ID is tracked.
-__device__ inline bool thread_lookup(const TableView& tv, unsigned long long id, unsigned stash_hw,
-                                     unsigned long long* meta) {
-  const Cell* b = tv.cells + tv.bucket0(id) * kCellsPerBucket;
-  Cell c[kCellsPerBucket];
+// Look-up of four IDs by one quad.  Each lane brings its own ID (hashed once,
+// by its owner); the quad then resolves the four IDs in turn, every lane
+// reading one cell of the ID's bucket, so a bucket costs one coalesced 64-byte
+// request.  On return every lane knows, for its own ID, whether it is tracked,
+// its metadata and the index of its cell (in cells[], or n_cells + i for stash
+// cell i).  All four lanes must call; `active` false skips the lane's ID.
+struct Found {
+  bool hit;
+  unsigned long long meta;
+  unsigned long long cell;
+};
+
+__device__ inline Found quad4_find(const TableView& tv, unsigned long long id, bool active, int lane,
+                                   unsigned stash_hw) {
+  const int sub = lane & 3, q0 = lane - sub;
+  const unsigned quad_mask = 0xFu << q0;
+  const unsigned long long n_cells = (tv.bucket_mask + 1) * kCellsPerBucket;
+  const unsigned long long b0 = active ? tv.bucket0(id) : 0ull;
+  Found mine;
+  mine.hit = false; mine.meta = 0; mine.cell = 0;
+  // first buckets of the four IDs: all four reads are issued before any is examined
+  unsigned long long id_k[4], bkt[4];
+  Cell c[4];
+  unsigned act = __ballot_sync(quad_mask, active) >> q0;
 #pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
-    if (c[k].key == id) { *meta = c[k].meta; return true; }
-  b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
-    if (c[k].key == id) { *meta = c[k].meta; return true; }
-  for (unsigned i = 0; i < stash_hw; ++i) {
-    const Cell s = load_cell_ro(tv.stash + i);
-    if (s.key == id) { *meta = s.meta; return true; }
+  for (int k = 0; k < 4; ++k) {
+    id_k[k] = __shfl_sync(quad_mask, id, q0 + k);
+    bkt[k] = __shfl_sync(quad_mask, b0, q0 + k);
+    c[k] = (act >> k) & 1u ? load_cell_ro(tv.cells + bkt[k] * kCellsPerBucket + sub) : empty_cell();
   }
-  return false;
+  unsigned bal[4];
+  unsigned miss = 0;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    bal[k] = __ballot_sync(quad_mask, ((act >> k) & 1u) && c[k].key == id_k[k]) & quad_mask;
+    if (((act >> k) & 1u) && !bal[k]) miss |= 1u << k;
+  }
+  if (miss) {                                                    // quad-uniform
+    // second buckets of the IDs that missed, again read together
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if ((miss >> k) & 1u) {
+        bkt[k] = tv.bucket1(id_k[k]);
+        c[k] = load_cell_ro(tv.cells + bkt[k] * kCellsPerBucket + sub);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if ((miss >> k) & 1u) bal[k] = __ballot_sync(quad_mask, c[k].key == id_k[k]) & quad_mask;
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (!((act >> k) & 1u)) continue;
+    unsigned long long cell = bkt[k] * kCellsPerBucket;
+    if (!bal[k] && stash_hw != 0) {
+      for (unsigned base = 0; base < stash_hw && !bal[k]; base += kCellsPerBucket) {
+        c[k] = base + sub < stash_hw ? load_cell_ro(tv.stash + base + sub) : empty_cell();
+        bal[k] = __ballot_sync(quad_mask, c[k].key == id_k[k]) & quad_mask;
+        cell = n_cells + base;
+      }
+    }
+    if (bal[k]) {
+      const int src = __ffs(bal[k]) - 1;                         // absolute lane that saw the key
+      const unsigned long long m = __shfl_sync(quad_mask, c[k].meta, src);
+      if (sub == k) { mine.hit = true; mine.meta = m; mine.cell = cell + (unsigned)(src - q0); }
+    }
+  }
+  return mine;
 }
 
-// Forward, step 1: one thread per ID occurrence resolves the ID to its row
-// index (kNoRow when the ID has none).  Every occurrence is independent, so
-// the random bucket reads of a whole batch are in flight together.
+// Forward, step 1: every ID occurrence is resolved to its row index (kNoRow
+// when the ID has none).  Every occurrence is independent, so the random
+// bucket reads of a whole batch are in flight together.
 __global__ void __launch_bounds__(256)
 probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
                   uint32_t* __restrict__ occ_row) {
   const unsigned stash_hw = tv.st->stash_hw;
+  const int lane = threadIdx.x & 31;
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
-    const unsigned long long id = ids[j];
-    unsigned long long meta = 0;
-    uint32_t row = kNoRow;
-    if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) row = meta_row(meta);
-    occ_row[j] = row;
+  const long long rounds = (n_ids + stride - 1) / stride;       // same trip count for every lane
+  for (long long r = 0; r < rounds; ++r) {
+    const long long j = r * stride + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long id = kEmptyKey;
+    if (j < n_ids) id = ids[j];
+    const Found f = quad4_find(tv, id, id != kEmptyKey, lane, stash_hw);
+    if (j < n_ids) occ_row[j] = (f.hit && meta_resident(f.meta)) ? meta_row(f.meta) : kNoRow;
   }
 }
 

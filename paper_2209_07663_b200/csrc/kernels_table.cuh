@@ -25,7 +25,8 @@ __device__ inline uint32_t alloc_row(const TableView& tv) {
 }
 
 // Block-wide reservation for the batch path: every thread states whether its
-// ID needs a row, whether it occurs more than once in the batch (it then gets a
+// ID needs a row, whether it must be inserted into the key store (it then gets
+// a place in ins_list[]), whether it occurs more than once in the batch (a
 // place in multi_list[]) and how many entries of bag_of_sorted[] its segment
 // takes; one thread does the counter updates for the whole block, so counters
 // that every admission would otherwise hit are touched once per block and
@@ -36,24 +37,27 @@ struct BlockAlloc {
   unsigned int rows_granted;
   unsigned int seg_base;
   unsigned int multi_base;
+  unsigned int ins_base;
 };
 
 struct Reservation {
   uint32_t row;             // kNoRow if refused or not asked for
   uint32_t seg_start;
   uint32_t multi_pos;
+  uint32_t ins_pos;
 };
 
 __device__ inline Reservation block_reserve(const TableView& tv, BlockAlloc* sh, bool need_row, bool is_multi,
-                                            uint32_t seg_len) {
-  // rows in bits 48.., repeated IDs in bits 32..47, segment entries in the low word
+                                            bool need_insert, uint32_t seg_len) {
+  // segment entries in bits 0..31, repeated IDs in 32..41, inserts in 42..51, rows in 52..61
   unsigned long long total = 0;
-  const unsigned long long mine =
-      ((unsigned long long)(need_row ? 1u : 0u) << 48) | ((unsigned long long)(is_multi ? 1u : 0u) << 32) | seg_len;
+  const unsigned long long mine = ((unsigned long long)(need_row ? 1u : 0u) << 52) |
+                                  ((unsigned long long)(need_insert ? 1u : 0u) << 42) |
+                                  ((unsigned long long)(is_multi ? 1u : 0u) << 32) | seg_len;
   const unsigned long long before = block_exclusive_scan(mine, sh->warp_sums, &total);
   if (threadIdx.x == 0) {
-    const unsigned int rows_wanted = (unsigned int)(total >> 48), multi_total = (unsigned int)(total >> 32) & 0xFFFFu,
-                       seg_total = (unsigned int)total;
+    const unsigned int rows_wanted = (unsigned int)(total >> 52) & 0x3FFu, ins_total = (unsigned int)(total >> 42) & 0x3FFu,
+                       multi_total = (unsigned int)(total >> 32) & 0x3FFu, seg_total = (unsigned int)total;
     unsigned int granted = 0;
     long long old = 0;
     if (rows_wanted) {
@@ -75,12 +79,14 @@ __device__ inline Reservation block_reserve(const TableView& tv, BlockAlloc* sh,
     sh->rows_granted = granted;
     sh->seg_base = seg_total ? atomicAdd(&tv.st->seg_cursor, seg_total) : 0u;
     sh->multi_base = multi_total ? atomicAdd(&tv.st->n_multi, multi_total) : 0u;
+    sh->ins_base = ins_total ? atomicAdd(&tv.st->n_insert, ins_total) : 0u;
   }
   __syncthreads();
   Reservation r;
   r.seg_start = sh->seg_base + (unsigned int)before;
-  r.multi_pos = sh->multi_base + ((unsigned int)(before >> 32) & 0xFFFFu);
-  const unsigned int my_row_index = (unsigned int)(before >> 48);
+  r.multi_pos = sh->multi_base + ((unsigned int)(before >> 32) & 0x3FFu);
+  r.ins_pos = sh->ins_base + ((unsigned int)(before >> 42) & 0x3FFu);
+  const unsigned int my_row_index = (unsigned int)(before >> 52) & 0x3FFu;
   r.row = kNoRow;
   if (need_row && my_row_index < sh->rows_granted) r.row = tv.free_rows[sh->row_base - 1 - my_row_index];
   return r;
@@ -99,60 +105,33 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
   }
 }
 
-// Thread-level look-up that keeps the cell's address: the four cells of the
-// first bucket are read together, the second bucket and the stash only on a miss.
-__device__ inline Cell* thread_find(const TableView& tv, unsigned long long id, unsigned stash_hw,
-                                    unsigned long long* meta) {
-  Cell* b = tv.cells + tv.bucket0(id) * kCellsPerBucket;
-  Cell c[kCellsPerBucket];
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) {
-    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(b + k);
-    c[k].key = v.x; c[k].meta = v.y;
-  }
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
-    if (c[k].key == id) { *meta = c[k].meta; return b + k; }
-  b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) {
-    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(b + k);
-    c[k].key = v.x; c[k].meta = v.y;
-  }
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
-    if (c[k].key == id) { *meta = c[k].meta; return b + k; }
-  for (unsigned i = 0; i < stash_hw; ++i)
-    if (tv.stash[i].key == id) { *meta = tv.stash[i].meta; return tv.stash + i; }
-  return nullptr;
-}
-
-// Phase 2 of mono_apply_grads: one thread per distinct ID.  Tracked IDs get
-// count += multiplicity (saturating at the threshold), last_seen = now, and a
-// row if the count has reached the threshold; the rest are marked for
-// insertion.  No cell moves during this kernel, so the thread that found a
-// cell owns it.  IDs that end up with a row and occur more than once also get
-// their segment of bag_of_sorted[] here.
+// Phase 2 of mono_apply_grads: one thread per distinct ID (look-ups shared
+// within quads).  Tracked IDs get count += multiplicity (saturating at the
+// threshold), last_seen = now, and a row if the count has reached the
+// threshold; the rest are queued for insertion.  No cell moves during this
+// kernel, so the thread whose ID sits in a cell owns it.  IDs that end up with a
+// row and occur more than once also get their segment of bag_of_sorted[] here.
 __global__ void __launch_bounds__(256)
 table_update_kernel(TableView tv, Work wk, uint32_t now) {
   __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_unique;
   const unsigned stash_hw = tv.st->stash_hw;
+  const unsigned long long n_cells = (tv.bucket_mask + 1) * kCellsPerBucket;
+  const int lane = threadIdx.x & 31;
   unsigned int n_res = 0;
   for (uint32_t base = blockIdx.x * blockDim.x; base < n; base += gridDim.x * blockDim.x) {   // block-uniform
     const uint32_t u = base + threadIdx.x;
     const bool active = u < n;
-    unsigned long long id = kEmptyKey, meta = 0;
+    unsigned long long id = kEmptyKey;
     uint32_t m = 0, slot = 0;
-    Cell* where = nullptr;
     if (active) {
       id = wk.uid[u];
       slot = wk.uslot[u];
       m = wk.bset[slot].a;
-      where = thread_find(tv, id, stash_hw, &meta);
     }
-    const bool hit = where != nullptr;
-    uint32_t low = meta_low(meta);
+    const Found f = quad4_find(tv, id, active, lane, stash_hw);
+    const bool hit = f.hit;
+    uint32_t low = meta_low(f.meta);
     bool resident = false, need_row = false;
     if (hit) {
       resident = (low & kResidentBit) != 0;
@@ -165,13 +144,14 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
     // a segment is reserved for every repeated ID that may end up with a row
     // (if the row is refused, the segment stays unused)
     const uint32_t seg_len = (hit && (resident || need_row) && m > 1) ? m : 0u;
-    const Reservation rv = block_reserve(tv, &sh, need_row, hit && m > 1, seg_len);
+    const Reservation rv = block_reserve(tv, &sh, need_row, hit && m > 1, active && !hit, seg_len);
     if (!active) continue;
     wk.ulen[u] = m;
     if (hit) {
       uint32_t row_word = kNoRow;
       if (resident) row_word = low & ~kResidentBit;
       else if (rv.row != kNoRow) { low = kResidentBit | rv.row; row_word = rv.row | kFreshBit; }
+      Cell* where = f.cell < n_cells ? tv.cells + f.cell : tv.stash + (f.cell - n_cells);
       where->meta = make_meta(now, low);
       wk.urow[u] = row_word;
       wk.useg[u] = rv.seg_start;
@@ -183,11 +163,11 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
         if (m > kSegChunk) register_long(tv, wk, u, m);
       }
     } else {
-      wk.urow[u] = kNeedsInsert;
+      wk.ins_list[rv.ins_pos] = u;
     }
   }
   for (int o = 16; o > 0; o >>= 1) n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
-  if ((threadIdx.x & 31) == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
+  if (lane == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
 }
 
 // Put `item` (a key that is in no cell) into the key store.  Lock-free against
@@ -252,23 +232,22 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
   if (meta_resident(item.meta)) atomicAdd(&tv.st->n_resident, (unsigned long long)(-1LL));
 }
 
-// Phase 3 of mono_apply_grads: one thread per distinct ID; the ones marked by
-// phase 2 as unknown to the key store are inserted (with a row straight away
-// when the batch alone reaches the threshold).
+// Phase 3 of mono_apply_grads: one thread per ID that phase 2 found unknown to
+// the key store; it is inserted (with a row straight away when the batch alone
+// reaches the threshold).
 __global__ void __launch_bounds__(256)
 table_insert_kernel(TableView tv, Work wk, uint32_t now) {
   __shared__ BlockAlloc sh;
-  const uint32_t n = tv.st->n_unique;
+  const uint32_t n = tv.st->n_insert;
   const int lane = threadIdx.x & 31;
   unsigned int n_res = 0, n_done = 0;
   for (uint32_t base = blockIdx.x * blockDim.x; base < n; base += gridDim.x * blockDim.x) {   // block-uniform
-    const uint32_t u = base + threadIdx.x;
-    const bool todo = u < n && wk.urow[u] == kNeedsInsert;
-    uint32_t m = 0;
-    if (todo) m = wk.ulen[u];
+    const bool todo = base + threadIdx.x < n;
+    uint32_t u = 0, m = 0;
+    if (todo) { u = wk.ins_list[base + threadIdx.x]; m = wk.ulen[u]; }
     const uint32_t count = m < tv.threshold ? m : tv.threshold;
     const bool need_row = todo && count >= tv.threshold;
-    const Reservation rv = block_reserve(tv, &sh, need_row, todo && m > 1, (need_row && m > 1) ? m : 0u);
+    const Reservation rv = block_reserve(tv, &sh, need_row, todo && m > 1, false, (need_row && m > 1) ? m : 0u);
     if (!todo) continue;
     const unsigned long long id = wk.uid[u];
     uint32_t low = count, row_word = kNoRow;
@@ -295,7 +274,6 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     if (n_done) {
       atomicAdd(&tv.st->n_tracked, (unsigned long long)n_done);
       atomicAdd(&tv.st->n_inserted_total, (unsigned long long)n_done);
-      atomicAdd(&tv.st->n_insert, n_done);
     }
   }
 }

@@ -82,7 +82,7 @@ void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
   dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
-  dev_free(w.multi_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
+  dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec);
   t->max_ids = t->max_bags = 0;
 }
@@ -130,7 +130,7 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   ALLOC(w.bset, slots);
   ALLOC(w.occ_slot, n); ALLOC(w.occ_rank, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
   ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n);
-  ALLOC(w.multi_list, n / 2 + 1);
+  ALLOC(w.multi_list, n / 2 + 1); ALLOC(w.ins_list, n);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
   ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts);
@@ -199,7 +199,7 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
   LAUNCH(t, K_FILL_BAG, fill_occ_bag_kernel<<<g8, 256, 0, s>>>(off, n_bags, n_ids, wk.occ_bag, tv.st));
   const int tiles = (int)((n_ids + kTileIds - 1) / kTileIds);
-  LAUNCH(t, K_DEDUP, dedup_tile_kernel<<<tiles, 256, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
+  LAUNCH(t, K_DEDUP, dedup_tile_kernel<<<tiles, kTileThreads, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
                                                             tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
