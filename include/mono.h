@@ -51,7 +51,9 @@ enum {
   MONO_ERR_TIME = -2,   /* `now` decreased or is outside [0, MONO_MAX_NOW] */
   MONO_ERR_CUDA = -3,   /* a CUDA runtime call failed; see mono_last_cuda_error */
   MONO_ERR_NOMEM = -4,  /* device allocation failed */
-  MONO_ERR_SIZE = -5    /* caller buffer too small (mono_export) */
+  MONO_ERR_SIZE = -5,   /* caller buffer too small (mono_export) */
+  MONO_ERR_LIMIT = -6   /* the call is larger than the fixed maximum of an entry point that
+                           never allocates (mono_lookup_pool_noalloc) */
 };
 
 /* Sticky device-side condition bits reported in mono_status_t.error_bits. */
@@ -214,6 +216,37 @@ int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids,
 int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids,
                           const int64_t* slot_offsets, int64_t n_bags,
                           const float* grad_pooled, int64_t now);
+
+/*
+ * mono_lookup_pool for callers that must not allocate device memory.  (The
+ * paper has no counterpart; this is a deployment variant of the forward call.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * serving loop whose memory budget was fixed at start-up, under an allocator
+ * that owns the whole device, or in a process that has handed every spare
+ * byte to other tenants.  mono_lookup_pool keeps its per-ID scratch (the row
+ * index of every ID of the batch) in a buffer it grows with cudaMalloc when a
+ * larger batch arrives; this entry point keeps the same scratch in a fixed
+ * array that is part of the library image instead, so it never calls
+ * cudaMalloc, cudaFree or anything else that allocates.
+ *
+ *  - Same arguments, same result and same error codes as mono_lookup_pool.
+ *  - n_ids may be at most MONO_NOALLOC_MAX_IDS; a larger batch is refused with
+ *    MONO_ERR_LIMIT before anything is enqueued (split it into several calls).
+ *  - The array (MONO_NOALLOC_MAX_IDS * 4 bytes = 4 MiB) is reserved on every
+ *    GPU that loads the library, from load until the process exits.
+ *  - The first call on a device looks up the array's device address once
+ *    (no allocation, but a runtime query): make that first call before any
+ *    CUDA stream capture begins on that device.
+ *  - All tables and all calls on a device share the one array, and it keeps
+ *    whatever the previous call left in it.  Nothing in it needs clearing --
+ *    each call overwrites the entries it reads -- but two calls that are in
+ *    flight on the GPU at the same time (different streams, different tables)
+ *    would overwrite each other's entries: serialise them.
+ */
+#define MONO_NOALLOC_MAX_IDS (1u << 20)
+int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids,
+                             const int64_t* slot_offsets, int64_t n_bags, float* out);
 
 /* ---- inspection and fixtures: not on the hot path, all synchronise ---- */
 

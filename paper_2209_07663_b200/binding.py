@@ -15,6 +15,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmono.so")
 
 MONO_OK, MONO_ERR_ARG, MONO_ERR_TIME, MONO_ERR_CUDA, MONO_ERR_NOMEM, MONO_ERR_SIZE = 0, -1, -2, -3, -4, -5
+MONO_ERR_LIMIT = -6
+MONO_NOALLOC_MAX_IDS = 1 << 20
 MONO_DEV_ROWS_FULL, MONO_DEV_KEYS_FULL, MONO_DEV_BAD_OFFSETS, MONO_DEV_IMPORT_DUP = 1, 2, 4, 8
 MONO_RESERVED_ID = 0xFFFFFFFFFFFFFFFF
 MONO_MAX_NOW = 0xFFFFFFFE
@@ -23,7 +25,7 @@ EXPORTS = [
     "mono_table_create", "mono_table_destroy", "mono_reserve", "mono_lookup_pool", "mono_apply_grads",
     "mono_expire", "mono_lookup_pool_host", "mono_apply_grads_host", "mono_status", "mono_clear_errors",
     "mono_probe", "mono_read_rows", "mono_export", "mono_import", "mono_audit", "mono_last_cuda_error",
-    "mono_error_string", "mono_timing_enable", "mono_timing_read",
+    "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc",
 ]
 
 
@@ -102,6 +104,7 @@ def load_library(path: Optional[str] = None):
         "mono_audit": (ci, [vp, ctypes.POINTER(mono_audit_t)]),
         "mono_last_cuda_error": (ctypes.c_char_p, [vp]),
         "mono_error_string": (ctypes.c_char_p, [ci]),
+        "mono_lookup_pool_noalloc": (ci, [vp, vp, i64, vp, i64, vp]),
         "mono_timing_enable": (ci, [vp, ci]),
         "mono_timing_read": (ci, [vp, ctypes.POINTER(mono_timing_t), ci]),
     }
@@ -170,6 +173,14 @@ def mono_reserve(t: int, max_ids: int, max_bags: int) -> None:
 def mono_lookup_pool(t: int, ids, n_ids: int, slot_offsets, n_bags: int, out) -> None:
     _check("mono_lookup_pool", load_library().mono_lookup_pool(t, _ptr(ids), n_ids, _ptr(slot_offsets), n_bags,
                                                                _ptr(out)), t)
+
+
+def mono_lookup_pool_noalloc(t: int, ids, n_ids: int, slot_offsets, n_bags: int, out) -> None:
+    """mono_lookup_pool for callers that may not allocate device memory: the per-ID scratch
+    lives in a fixed array inside the library, so at most MONO_NOALLOC_MAX_IDS IDs per call,
+    and calls must not overlap on the GPU."""
+    _check("mono_lookup_pool_noalloc", load_library().mono_lookup_pool_noalloc(t, _ptr(ids), n_ids, _ptr(slot_offsets),
+                                                                               n_bags, _ptr(out)), t)
 
 
 def mono_apply_grads(t: int, ids, n_ids: int, slot_offsets, n_bags: int, grad_pooled, now: int) -> None:

@@ -4,6 +4,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <utility>
@@ -20,6 +21,11 @@
 #include "table_layout.cuh"
 
 using namespace mono;
+
+// Scratch of mono_lookup_pool_noalloc: part of the library image, so the entry
+// point never allocates.  In host code this name is only a handle for
+// cudaGetSymbolAddress; kernels get the device address that call returns.
+static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
   K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_COMBINE, K_FINISH, K_EXPIRE,
@@ -333,6 +339,54 @@ int mono_expire(mono_table* t, int64_t now) {
   return MONO_OK;
 }
 
+// Device address of g_noalloc_occ_row on the current device, looked up once per
+// device (with that device current) and remembered.
+static int noalloc_scratch(mono_table* t, uint32_t** out) {
+  static std::mutex mu;
+  static uint32_t* addr[64] = {};
+  int dev = 0;
+  CUDA_TRY(t, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return MONO_ERR_ARG;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[dev]) {
+    uint32_t* p = nullptr;
+    CUDA_TRY(t, cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_occ_row));
+    addr[dev] = p;
+  }
+  *out = addr[dev];
+  return MONO_OK;
+}
+
+int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                             int64_t n_bags, float* out) {
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
+  if (n_ids > (int64_t)MONO_NOALLOC_MAX_IDS) return MONO_ERR_LIMIT;
+  if (n_bags == 0) return MONO_OK;
+  uint32_t* occ_row = nullptr;
+  if ((rc = noalloc_scratch(t, &occ_row)) != MONO_OK) return rc;
+  const unsigned long long* d_ids = reinterpret_cast<const unsigned long long*>(ids);
+  const long long* d_off = reinterpret_cast<const long long*>(slot_offsets);
+  if (n_ids > 0) {
+    int64_t blocks = (n_ids + 255) / 256;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 4;
+    if (blocks > cap) blocks = cap;
+    LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, d_ids, n_ids, occ_row));
+  }
+  return dispatch_dim(t->tv.dim, [&](auto g, auto nv) -> int {
+    constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
+    const int64_t groups_per_block = 256 / G;
+    int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
+    if (blocks > cap) blocks = cap;
+    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, occ_row, n_ids, d_off,
+                                                                                    n_bags, out));
+    CUDA_TRY(t, cudaGetLastError());
+    return (int)MONO_OK;
+  });
+}
+
 int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                           int64_t n_bags, float* out) {
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
@@ -551,6 +605,7 @@ const char* mono_error_string(int code) {
     case MONO_ERR_CUDA: return "MONO_ERR_CUDA";
     case MONO_ERR_NOMEM: return "MONO_ERR_NOMEM";
     case MONO_ERR_SIZE: return "MONO_ERR_SIZE";
+    case MONO_ERR_LIMIT: return "MONO_ERR_LIMIT";
     default: return "MONO_ERR_UNKNOWN";
   }
 }
