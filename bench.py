@@ -206,6 +206,24 @@ KERNEL_GROUP = {
 }
 
 
+def rank_config(base: wl.Config, rank: int) -> wl.Config:
+    """Every rank owns an independent table and draws its own stream (weak scaling)."""
+    return wl.scaled(base, seed=base.seed + 7919 * rank)
+
+
+def aggregate_over_ranks(times_ms, work_units, device="cpu"):
+    """Job-level figures from per-rank ones: the slowest rank's time for each timed region
+    (MAX), the work of all ranks together (SUM).  Works without a process group (N = 1)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    w = torch.tensor(list(work_units), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    return t.tolist(), w.tolist()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -222,8 +240,9 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
 
     base = wl.CONFIGS[args.workload]
-    cfg = wl.scaled(base, seed=base.seed + 7919 * rank)          # every rank its own stream and table
+    cfg = rank_config(base, rank)
     K, W, E = args.steps, args.warmup, args.e2e_steps
+    KT = min(K, args.kernel_steps)            # steps of the per-kernel timing pass
     sweep_period = args.sweep_period or K
     now0 = cfg.ttl - 1 if args.prefill else 0
     stream = wl.Stream(cfg)
@@ -244,7 +263,7 @@ def run_ours(args):
         raise SystemExit(f"pre-fill overflowed the table: {st0}")
 
     # ---- batches: ids/offsets from the seeded host generator, gradients drawn on the device
-    n_batches = W + 2 * K + E
+    n_batches = W + K + KT + E
 
     def make(i):
         return stream.step(now0 + 1 + i, with_grad=False)
@@ -254,7 +273,7 @@ def run_ours(args):
     gg = torch.Generator(device=dev)
     gg.manual_seed(cfg.seed)
     dev_batches = []
-    for t, s in enumerate(host_batches[:W + 2 * K]):
+    for t, s in enumerate(host_batches[:W + K + KT]):
         ids = torch.from_numpy(s.ids.view(np.int64)).to(dev)
         off = torch.from_numpy(s.offsets).to(dev)
         grad = torch.randn((cfg.n_bags, cfg.dim), device=dev, generator=gg).mul_(cfg.grad_std)
@@ -299,8 +318,8 @@ def run_ours(args):
 
     # ---- the same steps on fresh batches with every kernel bracketed by CUDA events
     mb.mono_timing_enable(table.handle, True)
-    for t in range(K):
-        step(W + K + t, sweep=(t + 1) % sweep_period == 0)
+    for t in range(KT):
+        step(W + K + t, sweep=(t == KT - 1))
     torch.cuda.synchronize()
     tim = mb.mono_timing_read(table.handle, reset=True)
     mb.mono_timing_enable(table.handle, False)
@@ -310,7 +329,7 @@ def run_ours(args):
     e2e = None
     if E > 0:
         pinned = []
-        for s in host_batches[W + 2 * K:]:
+        for s in host_batches[W + K + KT:]:
             ids = torch.from_numpy(s.ids.view(np.int64)).pin_memory()
             off = torch.from_numpy(s.offsets).pin_memory()
             grad = torch.randn((cfg.n_bags, cfg.dim)).mul_(cfg.grad_std).pin_memory()
@@ -321,7 +340,7 @@ def run_ours(args):
         n_e2e_ids, h2d, d2h = 0, 0, 0
         e0.record()
         for t, (ids, off, grad) in enumerate(pinned):
-            now = now0 + 1 + W + 2 * K + t
+            now = now0 + 1 + W + K + KT + t
             mb.mono_lookup_pool_host(table.handle, ids, ids.numel(), off, cfg.n_bags, out_h)
             mb.mono_apply_grads_host(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now)
             n_e2e_ids += ids.numel()
@@ -334,22 +353,17 @@ def run_ours(args):
     st_end = table.status()
 
     # ---- aggregate over ranks: max time, summed work
-    agg = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], dtype=torch.float64, device=dev)
-    work = torch.tensor([float(n_ids_timed), float(e2e["ids"]) if e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(agg, op=dist.ReduceOp.MAX)
-        dist.all_reduce(work, op=dist.ReduceOp.SUM)
-    ms_max, e2e_ms_max = agg.tolist()
-    ids_all, e2e_ids_all = work.tolist()
+    (ms_max, e2e_ms_max), (ids_all, e2e_ids_all) = aggregate_over_ranks(
+        [ms_total, e2e["ms"] if e2e else 0.0], [float(n_ids_timed), float(e2e["ids"]) if e2e else 0.0], dev)
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
         d = cfg.dim
         # per-step averages over the per-kernel pass (the steps the kernel times belong to)
-        n = (st_c["sum_ids"] - st_b["sum_ids"]) / K
-        u = (st_c["sum_unique"] - st_b["sum_unique"]) / K
-        ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / K
-        unew = (st_c["sum_new"] - st_b["sum_new"]) / K
+        n = (st_c["sum_ids"] - st_b["sum_ids"]) / KT
+        u = (st_c["sum_unique"] - st_b["sum_unique"]) / KT
+        ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / KT
+        unew = (st_c["sum_new"] - st_b["sum_new"]) / KT
         alg = algorithmic_bytes(n, cfg.n_bags, u, ur, unew, d)
         per_kernel = {}
         for name, v in tim["kernels"].items():
@@ -426,12 +440,13 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS))
     ap.add_argument("--sweep-period", type=int, default=0, help="steps between expiry sweeps (0 = --steps)")
     ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--kernel-steps", type=int, default=8, help="steps of the per-kernel CUDA-event pass")
     ap.add_argument("--no-prefill", dest="prefill", action="store_false")
     ap.add_argument("--oracle-steps", type=int, default=4)
     ap.add_argument("--oracle-fraction", type=int, default=8, help="the oracle runs on 1/this of each step's bags")
