@@ -171,12 +171,12 @@ scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad,
   }
 }
 
-// One lane group per work item.  Items [0, n_multi) are the repeated IDs: a
+// One lane group per work item.  Items [0, n_parts) are the parts of the long
+// segments (the heaviest items, so they are started first): a group reduces
+// one part into fp64 partial sums in scratch, which combine_adagrad_kernel adds
+// up afterwards.  Items [n_parts, n_parts + n_multi) are the repeated IDs: a
 // group empties the ID's slot of the per-call set (every occurrence has been
-// filed by now), reduces the whole segment and updates the row when the
-// segment is short.  Items [n_multi, n_multi + n_parts) are the parts of the
-// long segments: a group reduces one part into fp64 partial sums in
-// scratch, which combine_adagrad_kernel adds up afterwards.
+// filed by now), and when the segment is short reduces it and updates the row.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
@@ -190,8 +190,8 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
     D4 s[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
-    if (item < n) {
-      const uint32_t u = wk.multi_list[item];
+    if (item >= n_parts) {
+      const uint32_t u = wk.multi_list[item - n_parts];
       if (gl == 0) {
         BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
         wk.bset[wk.uslot[u]] = e;
@@ -208,7 +208,7 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
         if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
       }
     } else {
-      const uint32_t p = item - n;
+      const uint32_t p = item;
       const uint32_t li = wk.part_u[p];
       const uint32_t u = wk.long_u[li];
       const uint32_t k = p - wk.long_part0[li];
@@ -229,11 +229,14 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
   }
 }
 
-// One block per long ID: thread t owns column t (and t + 256, ...); the parts
-// are added in increasing order, so the combination order is fixed.
-__global__ void __launch_bounds__(256)
+// One block per long ID: the block's threads split into slices of the parts,
+// one column each; the slices' sums are added in increasing order, so the
+// combination order is fixed.
+constexpr int kCombineThreads = 1024;
+__global__ void __launch_bounds__(kCombineThreads)
 combine_adagrad_kernel(TableView tv, Work wk) {
-  __shared__ double s_sum[8][256];
+  constexpr int kMaxSlices = 16;
+  __shared__ double s_sum[kMaxSlices][256];
   uint32_t n_long = tv.st->n_long;
   if (n_long > wk.max_long) n_long = wk.max_long;
   const uint32_t dim = tv.dim;
@@ -246,17 +249,23 @@ combine_adagrad_kernel(TableView tv, Work wk) {
     const double* src = wk.partials + (size_t)wk.long_part0[li] * dim;
     const unsigned long long id = wk.uid[u];
     for (uint32_t cbase = 0; cbase < dim; cbase += 256) {
-      // 256 columns at a time; the 256 threads split into (256 / width) slices of parts
+      // 256 columns at a time; the threads split into (kCombineThreads / width) slices of parts
       const uint32_t width = dim - cbase < 256 ? dim - cbase : 256;      // multiple of 4
-      uint32_t slices = 256 / width;
-      if (slices > 8) slices = 8;
+      uint32_t slices = kCombineThreads / width;
+      if (slices > kMaxSlices) slices = kMaxSlices;
       const uint32_t col = threadIdx.x % width, slice = threadIdx.x / width;
-      double acc = 0.0;
       if (slice < slices) {
         const uint32_t per = (parts + slices - 1) / slices;
         const uint32_t p_lo = slice * per, p_hi = p_lo + per < parts ? p_lo + per : parts;
-        for (uint32_t p = p_lo; p < p_hi; ++p) acc += src[(size_t)p * dim + cbase + col];
-        s_sum[slice][col] = acc;
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+        uint32_t p = p_lo;
+        for (; p + 4 <= p_hi; p += 4) {               // four loads in flight, added in a fixed order
+          const double x0 = src[(size_t)p * dim + cbase + col], x1 = src[(size_t)(p + 1) * dim + cbase + col];
+          const double x2 = src[(size_t)(p + 2) * dim + cbase + col], x3 = src[(size_t)(p + 3) * dim + cbase + col];
+          a0 += x0; a1 += x1; a2 += x2; a3 += x3;
+        }
+        for (; p < p_hi; ++p) a0 += src[(size_t)p * dim + cbase + col];
+        s_sum[slice][col] = (a0 + a1) + (a2 + a3);
       }
       __syncthreads();
       if (threadIdx.x < width / 4) {

@@ -109,22 +109,47 @@ __device__ inline Found quad4_find(const TableView& tv, unsigned long long id, b
   return mine;
 }
 
-// Forward, step 1: every ID occurrence is resolved to its row index (kNoRow
-// when the ID has none).  Every occurrence is independent, so the random
-// bucket reads of a whole batch are in flight together.
+// Read-only look-up by one thread: the four cells of the first bucket are read
+// together, the second bucket and the stash only on a miss.  Returns true and
+// the metadata when the ID is tracked.
+__device__ inline bool thread_lookup(const TableView& tv, unsigned long long id, unsigned stash_hw,
+                                     unsigned long long* meta) {
+  const Cell* b = tv.cells + tv.bucket0(id) * kCellsPerBucket;
+  Cell c[kCellsPerBucket];
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+    if (c[k].key == id) { *meta = c[k].meta; return true; }
+  b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+    if (c[k].key == id) { *meta = c[k].meta; return true; }
+  for (unsigned i = 0; i < stash_hw; ++i) {
+    const Cell s = load_cell_ro(tv.stash + i);
+    if (s.key == id) { *meta = s.meta; return true; }
+  }
+  return false;
+}
+
+// Forward, step 1: one thread per ID occurrence resolves the ID to its row
+// index (kNoRow when the ID has none).  Every occurrence is independent, so
+// the random bucket reads of a whole batch are in flight together.  (Measured
+// against quad-cooperative variants: the shuffles those need cost more issue
+// slots than the extra L1 wavefronts of four 16-byte loads per thread.)
 __global__ void __launch_bounds__(256)
 probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
                   uint32_t* __restrict__ occ_row) {
   const unsigned stash_hw = tv.st->stash_hw;
-  const int lane = threadIdx.x & 31;
   const long long stride = (long long)gridDim.x * blockDim.x;
-  const long long rounds = (n_ids + stride - 1) / stride;       // same trip count for every lane
-  for (long long r = 0; r < rounds; ++r) {
-    const long long j = r * stride + (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    unsigned long long id = kEmptyKey;
-    if (j < n_ids) id = ids[j];
-    const Found f = quad4_find(tv, id, id != kEmptyKey, lane, stash_hw);
-    if (j < n_ids) occ_row[j] = (f.hit && meta_resident(f.meta)) ? meta_row(f.meta) : kNoRow;
+  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
+    const unsigned long long id = ids[j];
+    unsigned long long meta = 0;
+    uint32_t row = kNoRow;
+    if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) row = meta_row(meta);
+    occ_row[j] = row;
   }
 }
 

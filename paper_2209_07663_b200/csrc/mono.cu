@@ -217,7 +217,7 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
-  LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g4, 256, 0, s>>>(tv, wk));
+  LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g4, kCombineThreads, 0, s>>>(tv, wk));
   LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 32, 0, s>>>(tv.st));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
