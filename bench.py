@@ -51,10 +51,24 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def kernel_source_digest() -> str:
+KERNEL_SOURCES = {
+    "probe_rows": ("kernels_forward.cuh", "table_layout.cuh"),
+    "gather_pool": ("kernels_forward.cuh", "table_layout.cuh"),
+    "fill_occ_bag": ("kernels_dedup.cuh", "table_layout.cuh"),
+    "dedup_tile": ("kernels_dedup.cuh", "table_layout.cuh"),
+    "table_update": ("kernels_table.cuh", "kernels_forward.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "table_insert": ("kernels_table.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "scatter_singletons": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "reduce_adagrad": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "combine_adagrad": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+}
+
+
+def kernel_source_digest(kernel: str) -> str:
+    """Digest of the source files a kernel is compiled from (its own file and what it includes)."""
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2209_07663_b200", "csrc")
-    for name in sorted(os.listdir(d)):
+    for name in KERNEL_SOURCES.get(kernel, sorted(os.listdir(d))):
         with open(os.path.join(d, name), "rb") as f:
             h.update(name.encode())
             h.update(f.read())
@@ -72,7 +86,7 @@ def recorded_traffic(kernel: str, workload: str):
         if "=" in line and not line.lstrip().startswith("#"):
             k, v = line.split("=", 1)
             kv[k.strip()] = v.strip()
-    if kv.get("source_digest") != kernel_source_digest():
+    if kv.get("source_digest") != kernel_source_digest(kernel):
         return None
     try:
         return float(kv["dram_bytes_per_launch_scaled"])
@@ -187,15 +201,22 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- our arm
 
-def algorithmic_bytes(n, b, u, ur, unew, d):
-    """Bytes the method itself must move per step, per kernel group (each distinct datum
-    once per phase; 32-byte sector as the smallest random access)."""
-    fwd = 8 * n + 8 * (b + 1) + 32 * n + 4 * d * ur + 4 * d * b
-    dedup = 8 * n + 8 * (b + 1) + 24 * n
-    table = 64 * u + (16 + 8 * d) * unew
-    adagrad = 4 * d * b + 16 * d * ur
-    return {"lookup_pool": fwd, "dedup": dedup, "table": table, "adagrad": adagrad,
-            "total": fwd + dedup + table + adagrad}
+def algorithmic_bytes(n, b, u, ur, ur1, unew, d):
+    """Bytes the method itself must move per step, per kernel (each distinct datum once per
+    phase; 32-byte sector as the smallest random access).  n occurrences, b bags, u distinct
+    IDs, ur of them with a row, ur1 of those occurring once in the batch, unew new IDs."""
+    per_kernel = {
+        "probe_rows": 8 * n + 32 * n,                        # ids + one bucket sector per occurrence
+        "gather_pool": 8 * (b + 1) + 4 * d * ur + 4 * d * b,  # offsets, each distinct row once, out
+        "fill_occ_bag": 8 * (b + 1),                         # offsets
+        "dedup_tile": 8 * n + 24 * n,                        # ids + (key, index) pairs written and read
+        "table_update": 64 * u,                              # probe + count/stamp read-modify-write
+        "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
+        "scatter_singletons": 4 * d * b + 16 * d * ur1,      # gradients once + rows of IDs seen once
+        "reduce_adagrad": 16 * d * (ur - ur1),               # rows of repeated IDs (gradients counted above)
+        "combine_adagrad": 0, "finish_apply": 0,
+    }
+    return per_kernel, sum(per_kernel.values())
 
 
 KERNEL_GROUP = {
@@ -364,19 +385,20 @@ def run_ours(args):
         u = (st_c["sum_unique"] - st_b["sum_unique"]) / KT
         ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / KT
         unew = (st_c["sum_new"] - st_b["sum_new"]) / KT
-        alg = algorithmic_bytes(n, cfg.n_bags, u, ur, unew, d)
+        ur1 = (st_c["sum_single_resident"] - st_b["sum_single_resident"]) / KT
+        alg_kernel, alg_total = algorithmic_bytes(n, cfg.n_bags, u, ur, ur1, unew, d)
         per_kernel = {}
         for name, v in tim["kernels"].items():
             if v["launches"] and name in KERNEL_GROUP:
                 per_kernel[name] = {"ms_per_launch": v["ms"] / v["launches"], "launches": v["launches"]}
-        group_ms = {}
+        group_bytes, group_ms = {}, {}
         for name, v in per_kernel.items():
-            group_ms[KERNEL_GROUP[name]] = group_ms.get(KERNEL_GROUP[name], 0.0) + v["ms_per_launch"]
-        # the kernel group that takes the most device time, and its largest kernel
-        dom_group = max(group_ms, key=group_ms.get)
-        dom_kernels = sorted((k for k in per_kernel if KERNEL_GROUP[k] == dom_group),
-                             key=lambda k: -per_kernel[k]["ms_per_launch"])
-        dom_bytes, dom_ms = alg[dom_group], group_ms[dom_group]
+            g = KERNEL_GROUP[name]
+            group_ms[g] = group_ms.get(g, 0.0) + v["ms_per_launch"]
+            group_bytes[g] = group_bytes.get(g, 0) + alg_kernel[name]
+        # the kernel that takes the most device time
+        dom = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_launch"])
+        dom_bytes, dom_ms = alg_kernel[dom], per_kernel[dom]["ms_per_launch"]
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
         step_ms = ms_max / K
         line = {
@@ -386,7 +408,7 @@ def run_ours(args):
             "config": {
                 "workload": args.workload, "capacity": cfg.capacity, "dim": d, "key_cells": cfg.key_cells,
                 "bags_per_step": cfg.n_bags, "ids_per_step": n, "unique_per_step": u,
-                "unique_resident_per_step": ur, "new_per_step": unew, "zipf_s": cfg.zipf_s,
+                "unique_resident_per_step": ur, "unique_resident_once_per_step": ur1, "new_per_step": unew, "zipf_s": cfg.zipf_s,
                 "id_universe": cfg.n_distinct, "filter_threshold": cfg.filter_threshold, "ttl": cfg.ttl,
                 "prefill": "steady state of the stream" if args.prefill else "empty table",
                 "rows_resident_at_start": st0["n_resident"], "ids_tracked_at_start": st0["n_tracked"],
@@ -399,17 +421,20 @@ def run_ours(args):
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
                        "reasons": clocks["reasons"], "samples": clocks["samples"]},
             "roofline": {
-                "bound": "hbm", "kernel": dom_kernels[0], "kernels_timed_together": dom_kernels,
+                "bound": "hbm", "kernel": dom + "_kernel",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": dom_bytes,
                 "ms_per_launch": dom_ms,
-                "traffic": recorded_traffic(dom_kernels[0], args.workload),
+                "traffic": recorded_traffic(dom, args.workload),
             },
             "whole_step": {
-                "algorithmic_bytes": alg["total"], "achieved_gbs": alg["total"] / (step_ms * 1e-3) / 1e9,
-                "frac_of_measured_peak": alg["total"] / (step_ms * 1e-3) / 1e9 / peak,
-                "frac_of_8tbs": alg["total"] / (step_ms * 1e-3) / 1e9 / 8000.0,
-                "bytes_by_group": {k: v for k, v in alg.items() if k != "total"},
+                "algorithmic_bytes": alg_total, "achieved_gbs": alg_total / (step_ms * 1e-3) / 1e9,
+                "frac_of_measured_peak": alg_total / (step_ms * 1e-3) / 1e9 / peak,
+                "frac_of_8tbs": alg_total / (step_ms * 1e-3) / 1e9 / 8000.0,
+                "bytes_by_kernel": alg_kernel,
+                "frac_by_kernel": {k: round(alg_kernel[k] / (v["ms_per_launch"] * 1e-3) / 1e9 / peak, 3)
+                                   for k, v in per_kernel.items()},
+                "frac_by_phase": {g: round(group_bytes[g] / (group_ms[g] * 1e-3) / 1e9 / peak, 3) for g in group_ms},
                 "ms_by_kernel": {k: round(v["ms_per_launch"], 4) for k, v in per_kernel.items()},
                 "expire_ms_per_launch": (tim["kernels"]["expire"]["ms"] / tim["kernels"]["expire"]["launches"]
                                          if tim["kernels"]["expire"]["launches"] else None),

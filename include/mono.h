@@ -117,6 +117,7 @@ typedef struct {
   uint64_t sum_unique;          /* distinct IDs per call, summed */
   uint64_t sum_unique_resident; /* distinct IDs that had (or got) a row, summed */
   uint64_t sum_new;             /* distinct IDs that were new to the key store, summed */
+  uint64_t sum_single_resident; /* distinct IDs with a row that occurred once in their batch, summed */
 } mono_status_t;
 
 typedef struct {

@@ -49,7 +49,7 @@ class mono_status_t(ctypes.Structure):
                 ("n_keys_dropped", ctypes.c_uint64), ("n_evictions_total", ctypes.c_uint64),
                 ("max_chain", ctypes.c_uint32), ("stash_used", ctypes.c_uint32), ("sum_ids", ctypes.c_uint64),
                 ("sum_unique", ctypes.c_uint64), ("sum_unique_resident", ctypes.c_uint64),
-                ("sum_new", ctypes.c_uint64)]
+                ("sum_new", ctypes.c_uint64), ("sum_single_resident", ctypes.c_uint64)]
 
 
 class mono_audit_t(ctypes.Structure):

@@ -118,6 +118,7 @@ scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad,
   const int gl = lane % G, grp = lane / G;
   const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const long long n_rounds = (n_ids + 31) / 32;
+  unsigned int n_single = 0;
   for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rounds; r += n_warps) {
     const long long j = r * 32 + lane;
     uint32_t row_word = kNoRow, bag = 0;
@@ -140,6 +141,7 @@ scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad,
       }
     }
     unsigned todo = __ballot_sync(0xFFFFFFFFu, single);
+    n_single += __popc(todo);
     while (todo) {
       // the next kGroups flagged lanes, one per lane group
       int src = -1;
@@ -169,6 +171,7 @@ scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad,
       }
     }
   }
+  if (lane == 0 && n_single) atomicAdd(&tv.st->sum_single_resident, (unsigned long long)n_single);
 }
 
 // One lane group per work item.  Items [0, n_parts) are the parts of the long

@@ -443,6 +443,7 @@ int mono_status(mono_table* t, mono_status_t* host_out) {
   host_out->sum_unique = d.sum_unique;
   host_out->sum_unique_resident = d.sum_unique_resident;
   host_out->sum_new = d.sum_new;
+  host_out->sum_single_resident = d.sum_single_resident;
   return MONO_OK;
 }
 

@@ -81,6 +81,7 @@ struct DevState {
   unsigned long long sum_unique;
   unsigned long long sum_unique_resident;
   unsigned long long sum_new;
+  unsigned long long sum_single_resident;
   // per-call work counters, reset at the end of every mono_apply_grads
   unsigned int n_unique;
   unsigned int n_insert;
