@@ -32,9 +32,9 @@ struct __align__(16) BatchSlot {
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
 constexpr uint32_t kSingleton = 0xFFFFFFFFu;   // BatchSlot::a of an ID that occurs once in the batch
 constexpr uint32_t kSegChunk = 256;            // longest segment one lane group reduces alone
-constexpr int kTileIds = 1024;                 // occurrences per block of dedup_tile_kernel
-constexpr int kTileSlots = 2048;               // shared-memory table of one tile
-constexpr int kTileThreads = 512;              // block size of dedup_tile_kernel
+constexpr int kTileIds = 512;                  // occurrences per block of dedup_tile_kernel
+constexpr int kTileSlots = 1024;               // shared-memory table of one tile
+constexpr int kTileThreads = 256;              // block size of dedup_tile_kernel
 constexpr int kPrimaryProbes = 16;             // positions tried in the primary tier of the per-call set
 
 // Scratch of one mono_apply_grads call.
@@ -101,7 +101,7 @@ __device__ inline unsigned long long block_exclusive_scan(unsigned long long v, 
 }
 
 // One block per tile of kTileIds consecutive occurrences.
-__global__ void __launch_bounds__(kTileThreads, 3)
+__global__ void __launch_bounds__(kTileThreads, 6)
 dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long n_ids,
                   const long long* __restrict__ offsets, long long n_bags, DevState* st,
                   unsigned long long seed) {

@@ -109,24 +109,30 @@ __device__ inline Found quad4_find(const TableView& tv, unsigned long long id, b
   return mine;
 }
 
-// Read-only look-up by one thread: the four cells of the first bucket are read
-// together, the second bucket and the stash only on a miss.  Returns true and
-// the metadata when the ID is tracked.
+// Read-only look-up by one thread.  An insertion tries the cell named by the
+// top bits of the hash first, so that cell is read first and alone; the other
+// three cells of the bucket, the second bucket and the stash follow only on a
+// miss.  Returns true and the metadata when the ID is tracked.
 __device__ inline bool thread_lookup(const TableView& tv, unsigned long long id, unsigned stash_hw,
                                      unsigned long long* meta) {
-  const Cell* b = tv.cells + tv.bucket0(id) * kCellsPerBucket;
-  Cell c[kCellsPerBucket];
+  const unsigned long long h0 = tv.hash0(id);
+  const Cell* b = tv.cells + (h0 & tv.bucket_mask) * kCellsPerBucket;
+  const uint32_t first = (uint32_t)(h0 >> 62);
+  Cell c[kCellsPerBucket - 1];
+  const Cell c0 = load_cell_ro(b + first);
+  if (c0.key == id) { *meta = c0.meta; return true; }
 #pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
+  for (uint32_t k = 1; k < kCellsPerBucket; ++k) c[k - 1] = load_cell_ro(b + ((first + k) & 3u));
 #pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
+  for (uint32_t k = 0; k < kCellsPerBucket - 1; ++k)
     if (c[k].key == id) { *meta = c[k].meta; return true; }
+  Cell d[kCellsPerBucket];
   b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
 #pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) c[k] = load_cell_ro(b + k);
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) d[k] = load_cell_ro(b + k);
 #pragma unroll
   for (uint32_t k = 0; k < kCellsPerBucket; ++k)
-    if (c[k].key == id) { *meta = c[k].meta; return true; }
+    if (d[k].key == id) { *meta = d[k].meta; return true; }
   for (unsigned i = 0; i < stash_hw; ++i) {
     const Cell s = load_cell_ro(tv.stash + i);
     if (s.key == id) { *meta = s.meta; return true; }

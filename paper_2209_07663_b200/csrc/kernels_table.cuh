@@ -106,7 +106,8 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
 }
 
 // Phase 2 of mono_apply_grads: one thread per distinct ID (look-ups shared
-// within quads).  Tracked IDs get count += multiplicity (saturating at the
+// within quads: measured faster here than per-thread look-ups, because IDs new
+// to the table miss both buckets).  Tracked IDs get count += multiplicity (saturating at the
 // threshold), last_seen = now, and a row if the count has reached the
 // threshold; the rest are queued for insertion.  No cell moves during this
 // kernel, so the thread whose ID sits in a cell owns it.  IDs that end up with a
@@ -178,14 +179,16 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
 // entry is dropped and the condition recorded.
 __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
   const Cell empty = empty_cell();
-  unsigned long long bkt = tv.bucket0(item.key);
+  unsigned long long h0 = tv.hash0(item.key), h1 = tv.hash1(item.key);
+  unsigned long long bkt = h0 & tv.bucket_mask;
+  uint32_t first = (uint32_t)(h0 >> 62);            // the cell of this bucket the entry prefers
   uint32_t rnd = (uint32_t)(item.key >> 17) * 2654435761u + 0x9E3779B9u;
   uint32_t chain = 0;
   bool placed = false;
   for (;;) {
     Cell* base = tv.cells + bkt * kCellsPerBucket;
     for (uint32_t c = 0; c < kCellsPerBucket && !placed; ++c) {
-      Cell* p = base + ((c + rnd) & 3u);
+      Cell* p = base + ((c + first) & 3u);
       if (*reinterpret_cast<volatile unsigned long long*>(&p->key) == kEmptyKey) {
         const Cell old = atomicCAS(p, empty, item);
         placed = old.key == kEmptyKey;
@@ -194,10 +197,10 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
     if (placed) break;
     if (chain == 0) {
       // a new ID may take an empty cell of its second bucket before displacing anyone
-      const unsigned long long alt = tv.bucket1(item.key);
+      const unsigned long long alt = h1 & tv.bucket_mask;
       Cell* abase = tv.cells + alt * kCellsPerBucket;
       for (uint32_t c = 0; c < kCellsPerBucket && !placed && alt != bkt; ++c) {
-        Cell* p = abase + ((c + rnd) & 3u);
+        Cell* p = abase + ((c + (uint32_t)(h1 >> 62)) & 3u);
         if (*reinterpret_cast<volatile unsigned long long*>(&p->key) == kEmptyKey) {
           const Cell old = atomicCAS(p, empty, item);
           placed = old.key == kEmptyKey;
@@ -211,8 +214,11 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
     const Cell old = atomicExch(base + (rnd >> 30), item);
     if (old.key == kEmptyKey) { placed = true; break; }
     item = old;
-    const unsigned long long b0 = tv.bucket0(item.key), b1 = tv.bucket1(item.key);
-    bkt = (b0 == bkt) ? b1 : b0;
+    h0 = tv.hash0(item.key);
+    h1 = tv.hash1(item.key);
+    const bool to_second = (h0 & tv.bucket_mask) == bkt;
+    bkt = (to_second ? h1 : h0) & tv.bucket_mask;
+    first = (uint32_t)((to_second ? h1 : h0) >> 62);
   }
   if (chain) {
     atomicAdd(&tv.st->n_evictions_total, (unsigned long long)chain);

@@ -111,8 +111,12 @@ struct TableView {
   float lr, eps, init_acc, init_scale;
   uint32_t init_key0, init_key1;    // Philox key = table seed
 
-  __device__ inline unsigned long long bucket0(unsigned long long id) const { return mix_a(id ^ seed0) & bucket_mask; }
-  __device__ inline unsigned long long bucket1(unsigned long long id) const { return mix_b(id ^ seed1) & bucket_mask; }
+  // h0 / h1: the low bits pick the bucket, the top two bits the cell of that bucket an
+  // insertion tries first, so a look-up that reads that one cell first usually needs no more
+  __device__ inline unsigned long long hash0(unsigned long long id) const { return mix_a(id ^ seed0); }
+  __device__ inline unsigned long long hash1(unsigned long long id) const { return mix_b(id ^ seed1); }
+  __device__ inline unsigned long long bucket0(unsigned long long id) const { return hash0(id) & bucket_mask; }
+  __device__ inline unsigned long long bucket1(unsigned long long id) const { return hash1(id) & bucket_mask; }
   __device__ inline float* w_row(uint32_t row) const { return rows + (size_t)row * 2u * dim; }
   __device__ inline float* acc_row(uint32_t row) const { return rows + (size_t)row * 2u * dim + dim; }
 };
