@@ -232,13 +232,57 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
   }
 }
 
-// One block per long ID: the block's threads split into slices of the parts,
+// First level of the combination for very long segments: one block adds up one
+// group of kFoldWidth consecutive parts of one ID, column by column, and leaves
+// the sum in the group's first part.  Fixed order within the block.
+__global__ void __launch_bounds__(256)
+fold_partials_kernel(TableView tv, Work wk) {
+  __shared__ double s_sum[8][256];
+  uint32_t n_folds = tv.st->n_folds;
+  if (n_folds > wk.max_folds) n_folds = wk.max_folds;
+  const uint32_t dim = tv.dim;
+  for (uint32_t fi = blockIdx.x; fi < n_folds; fi += gridDim.x) {
+    const uint32_t li = wk.fold_li[fi], f = wk.fold_idx[fi];
+    const uint32_t u = wk.long_u[li];
+    if (wk.urow[u] == kNoRow) continue;               // block-uniform
+    const uint32_t parts = (wk.ulen[u] + kSegChunk - 1) / kSegChunk;
+    const uint32_t p_begin = f * kFoldWidth;
+    const uint32_t p_end = p_begin + kFoldWidth < parts ? p_begin + kFoldWidth : parts;
+    double* base = wk.partials + ((size_t)wk.long_part0[li] + p_begin) * dim;
+    for (uint32_t cbase = 0; cbase < dim; cbase += 256) {
+      const uint32_t width = dim - cbase < 256 ? dim - cbase : 256;
+      uint32_t slices = 256 / width;
+      if (slices > 8) slices = 8;
+      const uint32_t col = threadIdx.x % width, slice = threadIdx.x / width;
+      const uint32_t n = p_end - p_begin;
+      if (slice < slices) {
+        const uint32_t per = (n + slices - 1) / slices;
+        const uint32_t lo = slice * per, hi = lo + per < n ? lo + per : n;
+        double a0 = 0.0, a1 = 0.0;
+        uint32_t p = lo;
+        for (; p + 2 <= hi; p += 2) { a0 += base[(size_t)p * dim + cbase + col]; a1 += base[(size_t)(p + 1) * dim + cbase + col]; }
+        if (p < hi) a0 += base[(size_t)p * dim + cbase + col];
+        s_sum[slice][col] = a0 + a1;
+      }
+      __syncthreads();                                // every read of this group's parts is done
+      if (threadIdx.x < width) {
+        double g = 0.0;
+        for (uint32_t s = 0; s < slices; ++s) g += s_sum[s][threadIdx.x];
+        base[cbase + threadIdx.x] = g;
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// One block per long ID: the block's threads split into slices of the parts
+// (or, for a very long segment, of the group sums fold_partials_kernel left),
 // one column each; the slices' sums are added in increasing order, so the
 // combination order is fixed.
-constexpr int kCombineThreads = 1024;
+constexpr int kCombineThreads = 256;
 __global__ void __launch_bounds__(kCombineThreads)
 combine_adagrad_kernel(TableView tv, Work wk) {
-  constexpr int kMaxSlices = 16;
+  constexpr int kMaxSlices = 8;
   __shared__ double s_sum[kMaxSlices][256];
   uint32_t n_long = tv.st->n_long;
   if (n_long > wk.max_long) n_long = wk.max_long;
@@ -248,11 +292,12 @@ combine_adagrad_kernel(TableView tv, Work wk) {
     const uint32_t row_word = wk.urow[u];
     if (row_word == kNoRow) continue;                 // block-uniform
     const uint32_t m = wk.ulen[u];
-    const uint32_t parts = (m + kSegChunk - 1) / kSegChunk;
+    uint32_t parts = (m + kSegChunk - 1) / kSegChunk;
+    size_t stride = dim;                              // distance between the sums to add
+    if (parts > kFoldWidth) { parts = (parts + kFoldWidth - 1) / kFoldWidth; stride = (size_t)kFoldWidth * dim; }
     const double* src = wk.partials + (size_t)wk.long_part0[li] * dim;
     const unsigned long long id = wk.uid[u];
     for (uint32_t cbase = 0; cbase < dim; cbase += 256) {
-      // 256 columns at a time; the threads split into (kCombineThreads / width) slices of parts
       const uint32_t width = dim - cbase < 256 ? dim - cbase : 256;      // multiple of 4
       uint32_t slices = kCombineThreads / width;
       if (slices > kMaxSlices) slices = kMaxSlices;
@@ -260,15 +305,11 @@ combine_adagrad_kernel(TableView tv, Work wk) {
       if (slice < slices) {
         const uint32_t per = (parts + slices - 1) / slices;
         const uint32_t p_lo = slice * per, p_hi = p_lo + per < parts ? p_lo + per : parts;
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+        double a0 = 0.0, a1 = 0.0;
         uint32_t p = p_lo;
-        for (; p + 4 <= p_hi; p += 4) {               // four loads in flight, added in a fixed order
-          const double x0 = src[(size_t)p * dim + cbase + col], x1 = src[(size_t)(p + 1) * dim + cbase + col];
-          const double x2 = src[(size_t)(p + 2) * dim + cbase + col], x3 = src[(size_t)(p + 3) * dim + cbase + col];
-          a0 += x0; a1 += x1; a2 += x2; a3 += x3;
-        }
-        for (; p < p_hi; ++p) a0 += src[(size_t)p * dim + cbase + col];
-        s_sum[slice][col] = (a0 + a1) + (a2 + a3);
+        for (; p + 2 <= p_hi; p += 2) { a0 += src[p * stride + cbase + col]; a1 += src[(p + 1) * stride + cbase + col]; }
+        if (p < p_hi) a0 += src[p * stride + cbase + col];
+        s_sum[slice][col] = a0 + a1;
       }
       __syncthreads();
       if (threadIdx.x < width / 4) {

@@ -31,7 +31,8 @@ struct __align__(16) BatchSlot {
 
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
 constexpr uint32_t kSingleton = 0xFFFFFFFFu;   // BatchSlot::a of an ID that occurs once in the batch
-constexpr uint32_t kSegChunk = 256;            // longest segment one lane group reduces alone
+constexpr uint32_t kSegChunk = 64;             // longest segment one lane group reduces alone
+constexpr uint32_t kFoldWidth = 64;           // parts added up by one block of fold_partials_kernel
 constexpr int kTileIds = 512;                  // occurrences per block of dedup_tile_kernel
 constexpr int kTileSlots = 1024;               // shared-memory table of one tile
 constexpr int kTileThreads = 256;              // block size of dedup_tile_kernel
@@ -61,7 +62,9 @@ struct Work {
   uint32_t* long_part0;      // [max_long] first part of each
   uint32_t* part_u;          // [max_parts] owner (index into long_u) of each part
   double* partials;          // [max_parts][dim]
-  uint32_t max_long, max_parts;
+  uint32_t* fold_li;         // [max_folds] owner (index into long_u) of each fold
+  uint32_t* fold_idx;        // [max_folds] which group of kFoldWidth parts of that owner
+  uint32_t max_long, max_parts, max_folds;
 };
 
 // bag -> occurrences: every occurrence learns which bag it belongs to.

@@ -102,6 +102,13 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
     wk.long_u[li] = u;
     wk.long_part0[li] = p0;
     for (uint32_t p = 0; p < parts; ++p) wk.part_u[p0 + p] = li;
+    if (parts > kFoldWidth) {
+      // very long segment: its parts are first added up in groups of kFoldWidth
+      const uint32_t nf = (parts + kFoldWidth - 1) / kFoldWidth;
+      const uint32_t f0 = atomicAdd(&tv.st->n_folds, nf);
+      if (f0 + nf <= wk.max_folds)
+        for (uint32_t f = 0; f < nf; ++f) { wk.fold_li[f0 + f] = li; wk.fold_idx[f0 + f] = f; }
+    }
   }
 }
 
@@ -290,7 +297,7 @@ __global__ void finish_apply_kernel(DevState* st) {
     st->sum_ids += st->n_valid_ids;
     st->sum_unique += st->n_unique;
     st->sum_new += st->n_insert;
-    st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_valid_ids = 0;
+    st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_folds = 0; st->n_valid_ids = 0;
     st->seg_cursor = 0; st->n_multi = 0;
   }
 }

@@ -28,12 +28,12 @@ using namespace mono;
 static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
   K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
   "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "table_insert",
-  "scatter_singletons", "reduce_adagrad", "combine_adagrad",
+  "scatter_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
 
@@ -88,7 +88,7 @@ void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
   dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
-  dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials);
+  dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec);
   t->max_ids = t->max_bags = 0;
 }
@@ -141,6 +141,8 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
   ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts);
   ALLOC(w.partials, (size_t)w.max_parts * t->tv.dim);
+  w.max_folds = w.max_parts / kFoldWidth + w.max_long + 1;
+  ALLOC(w.fold_li, w.max_folds); ALLOC(w.fold_idx, w.max_folds);
   ALLOC(t->stage_ids, n); ALLOC(t->stage_off, (size_t)max_bags + 1);
   ALLOC(t->stage_vec, (size_t)max_bags * t->tv.dim);
 #undef ALLOC
@@ -217,7 +219,8 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
-  LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g4, kCombineThreads, 0, s>>>(tv, wk));
+  LAUNCH(t, K_FOLD, fold_partials_kernel<<<g4, 256, 0, s>>>(tv, wk));
+  LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g8, kCombineThreads, 0, s>>>(tv, wk));
   LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 32, 0, s>>>(tv.st));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;

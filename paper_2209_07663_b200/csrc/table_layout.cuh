@@ -87,6 +87,8 @@ struct DevState {
   unsigned int n_insert;
   unsigned int n_long;                   // distinct IDs whose segment is split into parts
   unsigned int n_parts;
+  unsigned int n_folds;                  // groups of kFoldWidth parts that are added up before the final combine
+  unsigned int pad2;
   unsigned int n_valid_ids;
   unsigned int seg_cursor;               // entries of bag_of_sorted[] handed out so far
   unsigned int n_multi;                  // distinct IDs that occur more than once in the batch

@@ -113,7 +113,7 @@ def test_offsets_that_skip_ids():
     assert_vectors_close(gpu.lookup_pool(ids, off).cpu().numpy(), cpu.lookup_pool(ids, off), "pooled")
 
 
-@pytest.mark.parametrize("n_occ", [255, 256, 257, 1000, 70000])
+@pytest.mark.parametrize("n_occ", [63, 64, 65, 255, 257, 1000, 4096, 4097, 4200, 70000])
 def test_one_hot_id_long_segment(n_occ):
     # a single ID owning a whole batch: the segment is split into parts and recombined
     dim = 64
