@@ -215,7 +215,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d):
         "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
         "scatter_singletons": 4 * d * b + 16 * d * ur1,      # gradients once + rows of IDs seen once
         "reduce_adagrad": 16 * d * (ur - ur1),               # rows of repeated IDs (gradients counted above)
-        "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
+        "expand_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
     }
     return per_kernel, sum(per_kernel.values())
 
@@ -223,7 +223,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d):
 KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
     "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
-    "table_update": "table", "table_insert": "table",
+    "table_update": "table", "table_insert": "table", "expand_parts": "table",
     "scatter_singletons": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
     "combine_adagrad": "adagrad",
 }

@@ -101,7 +101,7 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
   if (li < wk.max_long && p0 + parts <= wk.max_parts) {
     wk.long_u[li] = u;
     wk.long_part0[li] = p0;
-    for (uint32_t p = 0; p < parts; ++p) wk.part_u[p0 + p] = li;
+    // (part_u[] is filled by expand_parts_kernel: a segment can have thousands of parts)
     if (parts > kFoldWidth) {
       // very long segment: its parts are first added up in groups of kFoldWidth
       const uint32_t nf = (parts + kFoldWidth - 1) / kFoldWidth;
@@ -288,6 +288,20 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
       atomicAdd(&tv.st->n_tracked, (unsigned long long)n_done);
       atomicAdd(&tv.st->n_inserted_total, (unsigned long long)n_done);
     }
+  }
+}
+
+// After phases 2 and 3: every part of a long segment learns which ID it belongs to
+// (one block per long ID, its threads share the parts).
+__global__ void __launch_bounds__(128)
+expand_parts_kernel(TableView tv, Work wk) {
+  uint32_t n_long = tv.st->n_long;
+  if (n_long > wk.max_long) n_long = wk.max_long;
+  for (uint32_t li = blockIdx.x; li < n_long; li += gridDim.x) {
+    const uint32_t parts = (wk.ulen[wk.long_u[li]] + kSegChunk - 1) / kSegChunk;
+    const uint32_t p0 = wk.long_part0[li];
+    if (p0 + parts > wk.max_parts) continue;
+    for (uint32_t p = threadIdx.x; p < parts; p += blockDim.x) wk.part_u[p0 + p] = li;
   }
 }
 

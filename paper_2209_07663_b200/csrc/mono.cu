@@ -28,11 +28,11 @@ using namespace mono;
 static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_EXPAND, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
   K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
-  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "table_insert",
+  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "table_insert", "expand_parts",
   "scatter_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
@@ -211,6 +211,7 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
                                                             tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
+  LAUNCH(t, K_EXPAND, expand_parts_kernel<<<g4, 128, 0, s>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
