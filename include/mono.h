@@ -280,6 +280,30 @@ int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_see
                 uint8_t* resident, float* w, float* acc, int64_t max_n, int64_t* n_out);
 
 /*
+ * Rebuild the key store with new hash functions and, optionally, a new size (Section 2.1:
+ * cuckoo hashing rehashes when an insertion runs into a cycle; on a fixed-size device table
+ * that moment is reported as MONO_DEV_KEYS_FULL or a filling stash, and the caller rehashes
+ * between batches).  Every tracked ID keeps its count, last-access time and row; only its
+ * position changes.  new_key_cells: power of two >= 64, 0 keeps the size.  new_seed seeds the
+ * two bucket hash functions (row initialisation keeps the seed given at creation).
+ * Allocates the new store before freeing the old one; synchronises.  Keys that were dropped
+ * earlier are not brought back; if the new store is too small the usual overflow bits are set.
+ */
+int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed);
+
+/*
+ * Incremental export for parameter synchronisation (Section 2.2.3: the training side keeps
+ * the set of touched keys -- IDs whose embeddings were trained since the last
+ * synchronisation -- and pushes only those rows to the serving side).  Every ID whose row
+ * mono_apply_grads has updated since the previous call is written to ids / w (fp32
+ * [max_n, dim], any order) and leaves the set.  n_out HOST receives how many touched IDs
+ * there were.  If that is more than max_n, the first max_n found are exported, the rest stay
+ * in the set for the next call, and the return code is MONO_ERR_SIZE.  An ID that expired
+ * before the call is not exported.  One pass over the key store; synchronises.
+ */
+int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, int64_t* n_out);
+
+/*
  * Insert n entries given as (id, count, last_seen, resident[, w, acc]).  IDs
  * must be distinct; an ID that is already tracked is skipped and
  * MONO_DEV_IMPORT_DUP is set.  resident[i] != 0 claims a row; its values come

@@ -38,6 +38,7 @@ struct Entry {
   uint32_t count = 0;        // occurrences so far, saturating at the threshold
   int64_t last_seen = 0;     // `now` of the last apply_grads that contained the ID
   bool resident = false;     // owns an embedding row
+  bool touched = false;      // row trained since the last export of touched keys
   std::vector<float> w;      // embedding row (empty unless resident)
   std::vector<float> acc;    // Adagrad accumulator (empty unless resident)
 };
@@ -196,6 +197,7 @@ int oracle_apply_grads(void* h, const uint64_t* ids, int64_t n_ids, const int64_
         e.acc[col] = a;
         e.w[col] = e.w[col] - o->lr * G / (sqrtf(a) + o->eps);
       }
+      e.touched = true;      // Section 2.2.3: the ID joins the set of touched keys
     }
   }
   return rc;
@@ -223,6 +225,31 @@ int64_t oracle_expire(void* h, int64_t now) {
 
 int64_t oracle_n_tracked(void* h) { return (int64_t)static_cast<Oracle*>(h)->map.size(); }
 int64_t oracle_n_resident(void* h) { return (int64_t)static_cast<Oracle*>(h)->n_resident; }
+
+// Parameter synchronisation (Section 2.2.3): the touched keys are the IDs whose
+// embeddings were trained since the last synchronisation.  Writes them in
+// increasing ID order with their rows and empties the set.  An ID that expired
+// in between is simply gone.  Buffers sized by oracle_n_touched.
+int64_t oracle_n_touched(void* h) {
+  Oracle* o = static_cast<Oracle*>(h);
+  int64_t n = 0;
+  for (auto& kv : o->map) n += kv.second.touched ? 1 : 0;
+  return n;
+}
+
+int64_t oracle_export_touched(void* h, uint64_t* ids, float* w) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::vector<uint64_t> keys;
+  for (auto& kv : o->map) if (kv.second.touched) keys.push_back(kv.first);
+  std::sort(keys.begin(), keys.end());
+  for (size_t i = 0; i < keys.size(); ++i) {
+    Entry& e = o->map[keys[i]];
+    ids[i] = keys[i];
+    for (uint32_t c = 0; c < o->dim; ++c) w[i * (size_t)o->dim + c] = e.w[c];
+    e.touched = false;
+  }
+  return (int64_t)keys.size();
+}
 
 // State of n given IDs.  Untracked: resident 0, count 0, last_seen -1, zeros.
 int oracle_probe(void* h, const uint64_t* ids, int64_t n, uint8_t* resident, uint32_t* count,

@@ -56,6 +56,10 @@ def lib():
         L.oracle_probe.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp]
         L.oracle_export.restype = i64
         L.oracle_export.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.oracle_n_touched.restype = i64
+        L.oracle_n_touched.argtypes = [vp]
+        L.oracle_export_touched.restype = i64
+        L.oracle_export_touched.argtypes = [vp, vp, vp]
         L.oracle_import.restype = ctypes.c_int
         L.oracle_import.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64]
         L.oracle_philox4x32_10.restype = None
@@ -149,6 +153,15 @@ class OracleTable:
         m = lib().oracle_export(self._h, _p(ids), _p(cnt), _p(seen), _p(res), _p(w), _p(acc))
         assert m == n
         return {"ids": ids, "resident": res, "count": cnt, "last_seen": seen, "w": w, "acc": acc}
+
+    def export_touched(self):
+        """IDs trained since the last call (sorted) and their rows; empties the set."""
+        n = int(lib().oracle_n_touched(self._h))
+        ids = np.empty(n, np.uint64)
+        w = np.empty((n, self.dim), np.float32)
+        m = lib().oracle_export_touched(self._h, _p(ids), _p(w))
+        assert m == n
+        return {"ids": ids, "w": w}
 
     def import_entries(self, ids, count, last_seen, resident, w=None, acc=None) -> int:
         ids = _c(ids, np.uint64)

@@ -25,7 +25,7 @@ EXPORTS = [
     "mono_table_create", "mono_table_destroy", "mono_reserve", "mono_lookup_pool", "mono_apply_grads",
     "mono_expire", "mono_lookup_pool_host", "mono_apply_grads_host", "mono_status", "mono_clear_errors",
     "mono_probe", "mono_read_rows", "mono_export", "mono_import", "mono_audit", "mono_last_cuda_error",
-    "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc",
+    "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc", "mono_export_touched", "mono_rehash",
 ]
 
 
@@ -101,6 +101,8 @@ def load_library(path: Optional[str] = None):
         "mono_read_rows": (ci, [vp, vp, i64, vp, vp]),
         "mono_export": (ci, [vp, vp, vp, vp, vp, vp, vp, i64, ctypes.POINTER(i64)]),
         "mono_import": (ci, [vp, vp, vp, vp, vp, vp, vp, i64]),
+        "mono_export_touched": (ci, [vp, vp, vp, i64, ctypes.POINTER(i64)]),
+        "mono_rehash": (ci, [vp, u64, u64]),
         "mono_audit": (ci, [vp, ctypes.POINTER(mono_audit_t)]),
         "mono_last_cuda_error": (ctypes.c_char_p, [vp]),
         "mono_error_string": (ctypes.c_char_p, [ci]),
@@ -227,6 +229,20 @@ def mono_export(t: int, ids, count, last_seen, resident, w, acc, max_n: int) -> 
     if rc == MONO_ERR_SIZE:
         raise MonoError("mono_export", rc, f"{n.value} entries needed, {max_n} given")
     _check("mono_export", rc, t)
+    return n.value
+
+
+def mono_rehash(t: int, new_key_cells: int = 0, new_seed: int = 0) -> None:
+    _check("mono_rehash", load_library().mono_rehash(t, new_key_cells, new_seed), t)
+
+
+def mono_export_touched(t: int, ids, w, max_n: int) -> int:
+    """Export and clear the touched set; returns how many touched IDs there were (if that is more
+    than max_n only the first max_n were exported and the rest stay touched)."""
+    n = ctypes.c_int64(0)
+    rc = load_library().mono_export_touched(t, _ptr(ids), _ptr(w), max_n, ctypes.byref(n))
+    if rc != MONO_ERR_SIZE:
+        _check("mono_export_touched", rc, t)
     return n.value
 
 
@@ -359,6 +375,22 @@ class MonoTable:
         if rows:
             out["w"], out["acc"] = w[:m].cpu().numpy()[order], acc[:m].cpu().numpy()[order]
         return out
+
+    def rehash(self, new_key_cells: int = 0, new_seed: int = 0):
+        mono_rehash(self.handle, new_key_cells, new_seed)
+
+    def export_touched(self, max_n=None) -> dict:
+        """IDs trained since the last call and their rows, sorted by ID; clears the set."""
+        torch = self._torch
+        import numpy as np
+        n = int(self.status()["n_resident"]) + 8 if max_n is None else int(max_n)
+        ids = torch.empty(n, dtype=torch.int64, device="cuda")
+        w = torch.empty((n, self.dim), dtype=torch.float32, device="cuda")
+        found = mono_export_touched(self.handle, ids, w, n)
+        m = min(found, n)
+        ids_h = ids[:m].cpu().numpy().view(np.uint64)
+        order = np.argsort(ids_h, kind="stable")
+        return {"ids": ids_h[order], "w": w[:m].cpu().numpy()[order], "found": found}
 
     def import_entries(self, ids, count, last_seen, resident, w=None, acc=None):
         torch = self._torch

@@ -79,6 +79,39 @@ export_kernel(TableView tv, unsigned long long n_cells, unsigned long long* ids,
   }
 }
 
+// Incremental export (Section 2.2.3 of the paper: the set of touched keys, the IDs whose
+// embeddings were trained since the last synchronisation).  A streaming pass over the key
+// store: every row marked as trained is appended to the caller's buffers and its mark is
+// cleared; when the buffers are full the remaining marks stay for the next call.
+__global__ void __launch_bounds__(256)
+export_touched_kernel(TableView tv, unsigned long long n_cells, unsigned long long* ids, float* w, long long max_n) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long total = n_cells + kStashCells;
+  const unsigned long long rounds = (total + stride - 1) / stride;
+  const int lane = threadIdx.x & 31;
+  for (unsigned long long r = 0; r < rounds; ++r) {
+    const unsigned long long i = r * stride + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    Cell* p = nullptr;
+    Cell c = empty_cell();
+    if (i < total) { p = i < n_cells ? tv.cells + i : tv.stash + (i - n_cells); c = *p; }
+    const bool mine = c.key != kEmptyKey && meta_touched(c.meta);
+    const unsigned mask = __ballot_sync(0xFFFFFFFFu, mine);
+    if (!mask) continue;
+    unsigned long long base = 0;
+    const int leader = __ffs(mask) - 1;
+    if (lane == leader) base = atomicAdd(&tv.st->export_n, (unsigned long long)__popc(mask));
+    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (!mine) continue;
+    const long long k = (long long)(base + __popc(mask & ((1u << lane) - 1u)));
+    if (k >= max_n) continue;
+    ids[k] = c.key;
+    p->meta = c.meta & ~(unsigned long long)kTouchedBit;
+    const float4* src = reinterpret_cast<const float4*>(tv.w_row(meta_row(c.meta)));
+    float4* dst = reinterpret_cast<float4*>(w + k * (long long)tv.dim);
+    for (uint32_t c4 = 0; c4 < tv.dim / 4; ++c4) dst[c4] = src[c4];
+  }
+}
+
 struct AuditCounters {
   unsigned long long occupied, misplaced, duplicate_keys, resident_cells, bad_rows, shared_rows, free_rows,
       unaccounted_rows;

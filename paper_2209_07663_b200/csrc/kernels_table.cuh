@@ -157,8 +157,9 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
     wk.ulen[u] = m;
     if (hit) {
       uint32_t row_word = kNoRow;
-      if (resident) row_word = low & ~kResidentBit;
-      else if (rv.row != kNoRow) { low = kResidentBit | rv.row; row_word = rv.row | kFreshBit; }
+      // every ID of the batch that has a row is trained in this call: mark it for the next sync
+      if (resident) { row_word = low & kRowMask; low |= kTouchedBit; }
+      else if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
       Cell* where = f.cell < n_cells ? tv.cells + f.cell : tv.stash + (f.cell - n_cells);
       where->meta = make_meta(now, low);
       wk.urow[u] = row_word;
@@ -264,7 +265,7 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     if (!todo) continue;
     const unsigned long long id = wk.uid[u];
     uint32_t low = count, row_word = kNoRow;
-    if (rv.row != kNoRow) { low = kResidentBit | rv.row; row_word = rv.row | kFreshBit; }
+    if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
     wk.urow[u] = row_word;
     wk.useg[u] = rv.seg_start;
     BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kSingleton; bs.b = row_word;
@@ -387,6 +388,20 @@ init_bset_kernel(BatchSlot* bset, unsigned long long n) {
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
   BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
   for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) bset[i] = e;
+}
+
+// Rehash (Section 2.1: cuckoo hashing rehashes when an insertion runs into a cycle; here the
+// caller asks for it, between batches): every entry of the old key store is inserted into a
+// new, empty one that has its own size and hash seeds.
+__global__ void __launch_bounds__(256)
+rehash_kernel(TableView fresh, const Cell* __restrict__ old_cells, unsigned long long n_old_cells,
+              const Cell* __restrict__ old_stash) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long total = n_old_cells + kStashCells;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const Cell c = i < n_old_cells ? old_cells[i] : old_stash[i - n_old_cells];
+    if (c.key != kEmptyKey) cuckoo_insert(fresh, c);
+  }
 }
 
 // ---- bulk import -----------------------------------------------------------

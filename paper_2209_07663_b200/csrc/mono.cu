@@ -497,6 +497,56 @@ int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_see
   return (int64_t)n > max_n ? MONO_ERR_SIZE : MONO_OK;
 }
 
+int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
+  if (!t) return MONO_ERR_ARG;
+  if (new_key_cells == 0) new_key_cells = t->key_cells;
+  if (!is_pow2(new_key_cells) || new_key_cells < 64 || new_key_cells > (1ull << 34)) return MONO_ERR_ARG;
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  TableView fresh = t->tv;
+  fresh.cells = nullptr;
+  fresh.stash = nullptr;
+  int rc = dev_alloc(t, &fresh.cells, new_key_cells);
+  if (rc == MONO_OK) rc = dev_alloc(t, &fresh.stash, kStashCells);
+  if (rc != MONO_OK) { dev_free(fresh.cells); dev_free(fresh.stash); return rc; }
+  fresh.bucket_mask = new_key_cells / kCellsPerBucket - 1;
+  fresh.seed0 = mix_a(new_seed + 0x1234567ull);
+  fresh.seed1 = mix_b(new_seed + 0x89ABCDEFull);
+  const unsigned long long old_n = t->key_cells;
+  // the new store starts empty (capacity 0 keeps the kernel away from the free-row list)
+  TableView init_view = fresh;
+  init_view.capacity = 0;
+  init_table_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(init_view, new_key_cells);
+  cudaError_t e = cudaMemsetAsync(&t->tv.st->stash_hw, 0, sizeof(unsigned int), t->stream);
+  if (e == cudaSuccess) {
+    rehash_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(fresh, t->tv.cells, old_n, t->tv.stash);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(t->stream);
+  if (e != cudaSuccess) {
+    t->last_err = cudaGetErrorString(e);
+    dev_free(fresh.cells); dev_free(fresh.stash);
+    return MONO_ERR_CUDA;
+  }
+  dev_free(t->tv.cells);
+  dev_free(t->tv.stash);
+  t->tv = fresh;
+  t->key_cells = new_key_cells;
+  return MONO_OK;
+}
+
+int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, int64_t* n_out) {
+  if (!t || !n_out || max_n < 0 || (max_n > 0 && (!ids || !w || !aligned(w, 16) || !aligned(ids, 8)))) return MONO_ERR_ARG;
+  CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->export_n, 0, sizeof(unsigned long long), t->stream));
+  export_touched_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells,
+                                                               reinterpret_cast<unsigned long long*>(ids), w, max_n);
+  CUDA_TRY(t, cudaGetLastError());
+  unsigned long long n = 0;
+  CUDA_TRY(t, cudaMemcpyAsync(&n, &t->tv.st->export_n, sizeof(n), cudaMemcpyDeviceToHost, t->stream));
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  *n_out = (int64_t)n;
+  return (int64_t)n > max_n ? MONO_ERR_SIZE : MONO_OK;
+}
+
 int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const int64_t* last_seen,
                 const uint8_t* resident, const float* w, const float* acc, int64_t n) {
   if (!t || n < 0) return MONO_ERR_ARG;

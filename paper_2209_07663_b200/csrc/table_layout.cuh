@@ -18,7 +18,8 @@ namespace mono {
 //
 // meta, high 32 bits: last_seen (time of the last mono_apply_grads that held
 //                     the ID);
-// meta, low 32 bits : bit 31 set   -> the ID owns row (low 31 bits);
+// meta, low 32 bits : bit 31 set   -> the ID owns row (low 30 bits); bit 30 then marks a row
+//                     trained since the last mono_export_touched;
 //                     bit 31 clear -> still filtered, low 31 bits = occurrences
 //                     so far (< threshold unless no row was free).
 // ---------------------------------------------------------------------------
@@ -29,6 +30,8 @@ struct __align__(16) Cell {
 
 constexpr unsigned long long kEmptyKey = 0xFFFFFFFFFFFFFFFFull;
 constexpr uint32_t kResidentBit = 0x80000000u;
+constexpr uint32_t kTouchedBit = 0x40000000u;    // set with kResidentBit only
+constexpr uint32_t kRowMask = 0x3FFFFFFFu;
 constexpr uint32_t kCellsPerBucket = 4;
 constexpr uint32_t kStashCells = 256;      // overflow area scanned only when non-empty
 constexpr uint32_t kMaxChain = 96;         // bound on one insertion's displacement chain
@@ -44,7 +47,8 @@ __host__ __device__ inline unsigned long long make_meta(uint32_t time, uint32_t 
   return ((unsigned long long)time << 32) | low;
 }
 __host__ __device__ inline bool meta_resident(unsigned long long m) { return (meta_low(m) & kResidentBit) != 0; }
-__host__ __device__ inline uint32_t meta_row(unsigned long long m) { return meta_low(m) & ~kResidentBit; }
+__host__ __device__ inline uint32_t meta_row(unsigned long long m) { return meta_low(m) & kRowMask; }
+__host__ __device__ inline bool meta_touched(unsigned long long m) { return (meta_low(m) & (kResidentBit | kTouchedBit)) == (kResidentBit | kTouchedBit); }
 
 // Two unrelated 64-bit finalisers (multiply / xor-shift).  Both differ from the
 // mixer the workload generator uses for IDs, so structured inputs of one do not

@@ -219,6 +219,80 @@ def test_export_import_roundtrip_into_a_differently_seeded_table():
     assert_state_equal(other, cpu, "after duplicate import")
 
 
+def test_rehash_moves_keys_but_changes_no_state():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=12)
+    gpu, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        if t == 3:
+            gpu.rehash(new_seed=12345)                       # same size, new hash functions
+        if t == 6:
+            gpu.rehash(cfg.key_cells * 4, new_seed=7)        # grow
+        if t == 9:
+            gpu.rehash(cfg.key_cells // 2, new_seed=99)      # shrink (still fits)
+        if t in (3, 6, 9):
+            assert_state_equal(gpu, cpu, f"after rehash at step {t}")
+            a = assert_audit_ok(gpu)
+            assert gpu.status()["key_cells"] in (cfg.key_cells, cfg.key_cells * 4, cfg.key_cells // 2)
+            assert_vectors_close(gpu.lookup_pool(s.ids, s.offsets).cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets),
+                                 "pooled after rehash")
+        gpu.expire(t); cpu.expire(t)
+    assert_state_equal(gpu, cpu)
+    assert gpu.status()["error_bits"] == 0
+
+
+def test_rehash_into_a_larger_store_empties_the_stash():
+    # a 64-cell store pushed to its limit: entries end up in the stash; a larger store takes them all back
+    gpu = mb.MonoTable(16, 4, 100, 0, key_cells=64, seed=5)
+    cpu = mo.OracleTable(16, 4, 100, 0, seed=5)
+    ids = wl.splitmix64(np.arange(150, dtype=np.uint64))
+    off = np.arange(0, 151, dtype=np.int64)
+    gpu.apply_grads(ids, off, np.zeros((150, 4), f32), 0)
+    cpu.apply_grads(ids, off, np.zeros((150, 4), f32), 0)
+    st = gpu.status()
+    assert st["stash_used"] > 0 and st["n_keys_dropped"] == 0 and st["n_tracked"] == 150
+    gpu.rehash(1024, new_seed=1)
+    st = gpu.status()
+    assert st["stash_used"] == 0 and st["n_tracked"] == 150 and st["key_cells"] == 1024
+    assert_state_equal(gpu, cpu)
+    assert_audit_ok(gpu)
+    with pytest.raises(mb.MonoError):
+        gpu.rehash(1000)                                     # not a power of two
+
+
+def test_touched_key_export_matches_the_oracle():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=12, ttl=3)
+    gpu, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        if t % 2 == 1:
+            gpu.expire(t); cpu.expire(t)
+        if t % 3 == 2:
+            g, o = gpu.export_touched(), cpu.export_touched()
+            assert g["found"] == o["ids"].size > 0 and (g["ids"] == o["ids"]).all()
+            assert_vectors_close(g["w"], o["w"], f"touched rows at step {t}")
+            assert gpu.export_touched()["found"] == 0               # the set is empty afterwards
+    assert_state_equal(gpu, cpu)
+    assert_audit_ok(gpu)
+    # a buffer that is too small exports what fits and keeps the rest for the next call
+    s = stream.step(cfg.steps)
+    gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, cfg.steps)
+    cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, cfg.steps)
+    want = cpu.export_touched()
+    first = gpu.export_touched(max_n=100)
+    assert first["found"] == want["ids"].size and first["ids"].size == 100
+    rest = gpu.export_touched()
+    assert rest["found"] == want["ids"].size - 100
+    both = np.sort(np.concatenate([first["ids"], rest["ids"]]))
+    assert (both == want["ids"]).all()
+
+
 # ---------------------------------------------------------------- cuckoo structure under load
 
 @pytest.mark.parametrize("load", [0.5, 0.8, 0.9])

@@ -388,9 +388,30 @@ def test_capacity_overflow_is_reported():
     assert rc == mo.ERR_FULL and o.n_resident == 2 and o.n_tracked == 3
 
 
+def test_touched_keys_are_the_ids_trained_since_the_last_export():
+    o = mo.OracleTable(16, 2, 2, 3, lr=1.0, eps=0.0, init_scale=0.0)
+    g = np.ones((2, 2), f32)
+    o.apply_grads(*bags([[1, 1], [2]]), g, 0)          # 1 admitted and trained; 2 still filtered
+    t = o.export_touched()
+    assert t["ids"].tolist() == [1] and t["w"].tolist() == [[-1.0, -1.0]]
+    assert o.export_touched()["ids"].size == 0        # the export empties the set
+    o.lookup_pool(*bags([[1, 2]]))                     # look-ups do not touch
+    assert o.export_touched()["ids"].size == 0
+    o.apply_grads(*bags([[2], [3, 3]]), g, 1)          # 2 reaches the threshold, 3 admitted at once
+    o.apply_grads(*bags([[3], []]), g, 2)
+    t = o.export_touched()
+    assert t["ids"].tolist() == [2, 3]
+    np.testing.assert_allclose(t["w"], o.probe(np.array([2, 3], np.uint64))["w"])
+    # a touched ID that expires before the export is not exported
+    o.apply_grads(*bags([[1], []]), g, 3)
+    o.expire(3 + 3 + 1)
+    assert o.export_touched()["ids"].size == 0
+
+
 def test_sync_volume_arithmetic_from_the_paper():
     # Section 3.2: a dim-1024 fp32 row is 4 KB; 100 000 rows are about 400 MB
     o = mo.OracleTable(4, 1024, 1, 0)
     o.apply_grads(*bags([[1]]), np.ones((1, 1024), f32), 0)
     assert o.export()["w"].nbytes == 4096
+    assert o.export_touched()["w"].nbytes == 4096      # one touched ID of dim 1024 is a 4 KB push
     assert 100_000 * 4096 == pytest.approx(400e6, rel=0.03)
