@@ -464,13 +464,141 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_multi(args):
+    """The mixed-dim multi-table configuration: 8 independent tables, each on its own CUDA
+    stream, so that the latency-bound kernels of one table overlap the bandwidth-bound kernels
+    of another.  A step = lookup_pool + apply_grads on every table."""
+    import torch
+    from paper_2209_07663_b200 import binding as mb
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the table has no CPU path")
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    K, W = args.steps, args.warmup
+    cfgs = [rank_config(c, rank) for c in wl.multi_table_configs()]
+    streams = [torch.cuda.Stream(device=dev) for _ in cfgs]
+    tables, now0 = [], []
+    for cfg, st in zip(cfgs, streams):
+        t = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
+                         init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed, key_cells=cfg.key_cells,
+                         max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1), max_bags=cfg.n_bags,
+                         stream=st.cuda_stream)
+        n0 = cfg.ttl - 1
+        for ids, cnt, seen in wl.steady_state_population_torch(cfg, n0, dev):
+            res = (cnt >= cfg.filter_threshold).to(torch.uint8)
+            torch.cuda.synchronize()
+            mb.mono_import(t.handle, ids, cnt, seen, res, None, None, ids.numel())
+            del ids, cnt, seen, res
+        s0 = t.status()
+        if s0["error_bits"]:
+            raise SystemExit(f"pre-fill overflowed table {cfg.name}: {s0}")
+        tables.append(t)
+        now0.append(n0)
+
+    n_batches = W + 2 * K
+    jobs = [(ti, i) for ti in range(len(cfgs)) for i in range(n_batches)]
+    gens = [wl.Stream(c) for c in cfgs]
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+        host = list(pool.map(lambda j: gens[j[0]].step(now0[j[0]] + 1 + j[1], with_grad=False), jobs))
+    gg = torch.Generator(device=dev)
+    gg.manual_seed(cfgs[0].seed)
+    batches = [[None] * n_batches for _ in cfgs]
+    outs = []
+    for (ti, i), st in zip(jobs, host):
+        cfg = cfgs[ti]
+        batches[ti][i] = (torch.from_numpy(st.ids.view(np.int64)).to(dev), torch.from_numpy(st.offsets).to(dev),
+                          torch.randn((cfg.n_bags, cfg.dim), device=dev, generator=gg).mul_(cfg.grad_std))
+    for cfg in cfgs:
+        outs.append(torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device=dev))
+    torch.cuda.synchronize()
+
+    def step(i, serial):
+        for ti, (cfg, t) in enumerate(zip(cfgs, tables)):
+            ids, off, grad = batches[ti][i]
+            mb.mono_lookup_pool(t.handle, ids, ids.numel(), off, cfg.n_bags, outs[ti])
+            mb.mono_apply_grads(t.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0[ti] + 1 + i)
+            if serial:
+                streams[ti].synchronize()
+
+    def timed(first, serial):
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for st in streams:
+            st.wait_event(ev0)
+        for i in range(first, first + K):
+            step(i, serial)
+        for st in streams:
+            done = torch.cuda.Event()
+            done.record(st)
+            torch.cuda.current_stream().wait_event(done)
+        ev1.record()
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1)
+
+    for i in range(W):
+        step(i, False)
+    before = [t.status() for t in tables]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms = timed(W, False)
+    clocks = sampler.stop()
+    mid = [t.status() for t in tables]
+    ms_serial = timed(W + K, True)
+    after = [t.status() for t in tables]
+    n_ids = sum(b["sum_ids"] - a["sum_ids"] for a, b in zip(before, mid))
+    n_ids_serial = sum(b["sum_ids"] - a["sum_ids"] for a, b in zip(mid, after))
+    launches = sum(mb.mono_timing_read(t.handle)["launches_total"] for t in tables)
+    (ms_max,), (ids_all,) = aggregate_over_ranks([ms], [float(n_ids)], dev)
+    alg = 0
+    for cfg, a, b in zip(cfgs, before, mid):
+        n = b["sum_ids"] - a["sum_ids"]
+        u, ur = b["sum_unique"] - a["sum_unique"], b["sum_unique_resident"] - a["sum_unique_resident"]
+        ur1, unew = b["sum_single_resident"] - a["sum_single_resident"], b["sum_new"] - a["sum_new"]
+        alg += algorithmic_bytes(n, cfg.n_bags * K, u, ur, ur1, unew, cfg.dim)[1]
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        achieved = alg / (ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": ids_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "multi", "tables": [{"name": c.name, "capacity": c.capacity, "dim": c.dim,
+                                                         "slots": c.n_slots, "zipf_s": c.zipf_s,
+                                                         "row_load": s0["n_resident"] / c.capacity,
+                                                         "key_load": s0["n_tracked"] / c.key_cells}
+                                                        for c, s0 in zip(cfgs, before)],
+                       "examples_per_step": cfgs[0].n_examples, "slots_total": sum(c.n_slots for c in cfgs),
+                       "ids_per_step": n_ids / K, "prefill": "steady state of each stream", "sweep": "none",
+                       "l2": "every step reads fresh batches larger than L2",
+                       "parallelism": "8 tables on 8 CUDA streams of one GPU"},
+            "serial": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,
+                       "what": "the same calls with each table's stream drained before the next table starts"},
+            "gpu_launches": launches, "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
+                                                 "reasons": clocks["reasons"], "samples": clocks["samples"]},
+            "roofline": {"bound": "hbm", "kernel": "all kernels of the 8 tables (whole step)", "achieved": achieved,
+                         "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                         "traffic": None},
+            "error_bits": [s["error_bits"] for s in after],
+        }
+        print(json.dumps(line), flush=True)
+    for t in tables:
+        t.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS) + ["multi"])
     ap.add_argument("--sweep-period", type=int, default=0, help="steps between expiry sweeps (0 = --steps)")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--kernel-steps", type=int, default=8, help="steps of the per-kernel CUDA-event pass")
@@ -481,7 +609,11 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
+        if args.workload == "multi":
+            args.workload = "large"
         run_reference(args)
+    elif args.workload == "multi":
+        run_multi(args)
     else:
         run_ours(args)
 

@@ -132,22 +132,49 @@ CONFIGS = {
                     drift_period=50, drift_new_frac=0.30),
 }
 
-# Mixed-dim multi-table configuration: 8 tables, 15 feature slots each.
+# Mixed-dim multi-table configuration: 8 tables, 120 feature slots spread over them so that
+# every table settles near (and below) 0.9 row load under its own Zipf exponent.
 MULTI_TABLE_DIMS = (8, 16, 16, 32, 32, 64, 64, 128)
 MULTI_TABLE_CAPACITY_LOG2 = (27, 26, 25, 24, 23, 22, 21, 20)
 MULTI_TABLE_ZIPF_S = (0.9, 0.95, 1.0, 1.05, 1.1, 1.2, 1.25, 1.3)
+MULTI_TABLE_SLOTS = (33, 23, 16, 12, 9, 11, 9, 7)
+MULTI_TABLE_UNIVERSE_LOG2_EXTRA = (2, 2, 2, 2, 2, 2, 1, 1)
 
 
-def multi_table_configs(n_examples: int = 32768, slots_per_table: int = 15) -> list:
-    """Eight Config objects, one per table of the mixed-dim configuration."""
+def multi_table_configs(n_examples: int = 32768, slots=MULTI_TABLE_SLOTS) -> list:
+    """Eight Config objects, one per table of the mixed-dim configuration.
+    `slots` is the number of feature slots per table (an int gives every table the same)."""
+    if isinstance(slots, int):
+        slots = (slots,) * 8
     out = []
-    for t, (d, cl, s) in enumerate(zip(MULTI_TABLE_DIMS, MULTI_TABLE_CAPACITY_LOG2,
-                                       MULTI_TABLE_ZIPF_S)):
+    for t, (d, cl, s, sl, ex) in enumerate(zip(MULTI_TABLE_DIMS, MULTI_TABLE_CAPACITY_LOG2, MULTI_TABLE_ZIPF_S,
+                                               slots, MULTI_TABLE_UNIVERSE_LOG2_EXTRA)):
         out.append(Config(f"multi{t}", capacity=1 << cl, dim=d, filter_threshold=3, ttl=500,
-                          n_examples=n_examples, n_slots=slots_per_table,
-                          bag_len=("uniform", 1, 8), zipf_s=s, n_distinct=1 << min(cl + 4, 30),
-                          steps=50, key_cells=1 << min(cl + 3, 30), seed=20220923 + 101 * t))
+                          n_examples=n_examples, n_slots=sl,
+                          bag_len=("uniform", 1, 8), zipf_s=s, n_distinct=1 << min(cl + ex, 30),
+                          steps=50, key_cells=1 << min(cl + 2, 30), seed=20220923 + 101 * t))
     return out
+
+
+def expected_steady_state(cfg: Config, window: Optional[int] = None):
+    """Expected (tracked IDs, IDs with a row) after `window` steps of cfg's stream under the
+    Poisson model of steady_state_population (ranks binned geometrically beyond the head)."""
+    from math import lgamma
+    window = cfg.ttl if window is None else window
+    v = cfg.n_distinct
+    head = np.arange(1, min(v, 2_000_000) + 1, dtype=np.float64)
+    k, w = head, np.ones_like(head)
+    if v > 2_000_000:
+        e = np.unique(np.floor(np.geomspace(2_000_000, v, 200_000)).astype(np.int64))
+        lo, hi = e[:-1] + 1, e[1:]
+        k, w = np.concatenate([head, (lo + hi) / 2.0]), np.concatenate([w, (hi - lo + 1).astype(np.float64)])
+    p = k ** (-cfg.zipf_s)
+    p /= (p * w).sum()
+    lam = cfg.n_bags * _mean_bag_len(cfg.bag_len) * window * p
+    cdf = np.zeros_like(lam)
+    for j in range(max(cfg.filter_threshold, 1)):
+        cdf += np.exp(-lam + j * np.log(np.maximum(lam, 1e-300)) - lgamma(j + 1))
+    return float((w * -np.expm1(-lam)).sum()), float((w * (1.0 - np.minimum(cdf, 1.0))).sum())
 
 
 def scaled(cfg: Config, **kw) -> Config:

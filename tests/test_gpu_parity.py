@@ -69,7 +69,7 @@ def test_every_dim_variant(dim):
 
 
 def test_multi_table_configs_scaled_down():
-    for cfg in wl.multi_table_configs(n_examples=256, slots_per_table=3):
+    for cfg in wl.multi_table_configs(n_examples=256, slots=3):
         cfg = wl.scaled(cfg, capacity=1 << 13, key_cells=1 << 15, n_distinct=1 << 14, steps=5, ttl=3)
         gpu, cpu = make_pair(cfg)
         run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5)

@@ -109,3 +109,16 @@ def test_torch_twins_reproduce_the_numpy_generators():
     ref_ids, ref_cnt, _ = wl.steady_state_population(small, now=99)
     assert abs(ids.size - ref_ids.size) < 0.05 * ref_ids.size          # same model, different draws
     assert abs(int(cnt.sum()) - int(ref_cnt.sum())) < 0.05 * ref_cnt.sum()
+
+
+def test_configured_streams_fit_their_tables():
+    # steady state of every configured stream under the Poisson model: rows and keys fit
+    for cfg in [wl.CONFIGS["tiny"], wl.CONFIGS["medium"], wl.CONFIGS["large"]] + wl.multi_table_configs():
+        tracked, admitted = wl.expected_steady_state(cfg)
+        assert admitted <= 0.93 * cfg.capacity, (cfg.name, admitted / cfg.capacity)
+        assert tracked <= 0.80 * cfg.key_cells, (cfg.name, tracked / cfg.key_cells)
+    assert sum(wl.MULTI_TABLE_SLOTS) == 120
+    total = sum(c.capacity * c.dim * 8 + c.key_cells * 16 + c.capacity * 4 for c in wl.multi_table_configs())
+    assert total < 120e9                                  # rows + accumulators + key stores + free lists
+    t, a = wl.expected_steady_state(wl.CONFIGS["large"])
+    assert 4.2e8 < t < 5.0e8 and 5.5e7 < a < 6.5e7        # the pre-fill the benchmark starts from
