@@ -53,7 +53,56 @@ struct Oracle {
   int64_t last_now = INT64_MIN;
   uint64_t n_resident = 0;
   std::unordered_map<uint64_t, Entry> map;
+  // probabilistic filter (count-min sketch) in place of exact per-ID counters; depth 0 = off
+  uint32_t sketch_depth = 0;
+  uint64_t sketch_width = 0;        // power of two
+  std::vector<uint64_t> sketch;     // [depth][width]
+  int64_t sketch_epoch = 0;         // time of the last reset
 };
+
+// SplitMix64 output function (Steele, Lea, Flood 2014); the sketch's row hashes are
+// built from it so that both sides index the same counters.
+inline uint64_t splitmix64_mix(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// Counter of row r that ID `id` maps to.
+inline uint64_t sketch_index(const Oracle* o, uint32_t r, uint64_t id) {
+  return splitmix64_mix(id ^ (o->seed + (uint64_t)(r + 1) * 0x9E3779B97F4A7C15ull)) & (o->sketch_width - 1);
+}
+
+inline uint64_t sketch_estimate(const Oracle* o, uint64_t id) {
+  uint64_t est = UINT64_MAX;
+  for (uint32_t r = 0; r < o->sketch_depth; ++r)
+    est = std::min(est, o->sketch[(size_t)r * o->sketch_width + sketch_index(o, r, id)]);
+  return est;
+}
+
+// One Adagrad step of a row with the summed gradient g (fp64 sums rounded once to fp32).
+inline void adagrad_row(const Oracle* o, Entry& e, const std::vector<double>& g) {
+  for (uint32_t col = 0; col < o->dim; ++col) {
+    const float G = (float)g[col];
+    const float a = e.acc[col] + G * G;
+    e.acc[col] = a;
+    e.w[col] = e.w[col] - o->lr * G / (sqrtf(a) + o->eps);
+  }
+  e.touched = true;      // Section 2.2.3: the ID joins the set of touched keys
+}
+
+inline float init_value(uint64_t seed, uint64_t id, uint32_t col, float scale);   // defined below
+
+inline void give_row(Oracle* o, Entry& e, uint64_t id) {
+  e.resident = true;
+  ++o->n_resident;
+  e.w.resize(o->dim); e.acc.resize(o->dim);
+  for (uint32_t col = 0; col < o->dim; ++col) {
+    e.w[col] = init_value(o->seed, id, col, o->init_scale);
+    e.acc[col] = o->init_acc;
+  }
+}
 
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy
 // as 1, 2, 3", SC'11).  Counter-based, so a row's initial value depends only
@@ -110,6 +159,19 @@ void* oracle_create(uint64_t capacity, uint32_t dim, uint32_t filter_threshold, 
   o->seed = seed;
   return o;
 }
+
+// Switch the admission filter to a count-min sketch of `depth` rows of `width` counters
+// (width a power of two).  Call before the first batch.
+int oracle_enable_sketch(void* h, uint32_t depth, uint64_t width) {
+  Oracle* o = static_cast<Oracle*>(h);
+  if (!o || depth == 0 || width == 0 || (width & (width - 1)) || !o->map.empty()) return ORACLE_ERR_ARG;
+  o->sketch_depth = depth;
+  o->sketch_width = width;
+  o->sketch.assign((size_t)depth * width, 0ull);
+  return ORACLE_OK;
+}
+
+uint64_t oracle_sketch_index(void* h, uint32_t r, uint64_t id) { return sketch_index(static_cast<Oracle*>(h), r, id); }
 
 void oracle_destroy(void* h) { delete static_cast<Oracle*>(h); }
 
@@ -174,6 +236,34 @@ int oracle_apply_grads(void* h, const uint64_t* ids, int64_t n_ids, const int64_
   }
 
   int rc = ORACLE_OK;
+  if (o->sketch_depth) {
+    // Probabilistic filter (Section 2.1, heuristic 1, second method): a count-min sketch
+    // stands in for the per-ID counters, so an ID without a row costs no entry at all.
+    //  a. every distinct ID without a row adds its multiplicity to one counter per sketch row;
+    //  b. after all additions of the batch, an ID whose smallest counter has reached the
+    //     threshold is given a row (it may get there early through collisions, never late);
+    //  c. IDs with a row are stamped and updated as in the exact mode.
+    for (size_t u = 0; u < order.size(); ++u) {
+      auto it = o->map.find(order[u]);
+      if (it != o->map.end() && it->second.resident) continue;
+      for (uint32_t r = 0; r < o->sketch_depth; ++r)
+        o->sketch[(size_t)r * o->sketch_width + sketch_index(o, r, order[u])] += groups[u].mult;
+    }
+    for (size_t u = 0; u < order.size(); ++u) {
+      const uint64_t id = order[u];
+      auto it = o->map.find(id);
+      if (it == o->map.end()) {
+        if (sketch_estimate(o, id) < o->threshold) continue;
+        if (o->n_resident >= o->capacity) { rc = ORACLE_ERR_FULL; continue; }
+        it = o->map.emplace(id, Entry()).first;
+        it->second.count = o->threshold;
+        give_row(o, it->second, id);
+      }
+      it->second.last_seen = now;
+      adagrad_row(o, it->second, groups[u].g);
+    }
+    return rc;
+  }
   for (size_t u = 0; u < order.size(); ++u) {
     const uint64_t id = order[u];
     Entry& e = o->map[id];             // creates {count 0, not resident} if untracked
@@ -182,23 +272,9 @@ int oracle_apply_grads(void* h, const uint64_t* ids, int64_t n_ids, const int64_
     e.last_seen = now;
     if (!e.resident && e.count >= o->threshold) {
       if (o->n_resident >= o->capacity) { rc = ORACLE_ERR_FULL; continue; }
-      e.resident = true;
-      ++o->n_resident;
-      e.w.resize(d); e.acc.resize(d);
-      for (uint32_t col = 0; col < d; ++col) {
-        e.w[col] = init_value(o->seed, id, col, o->init_scale);
-        e.acc[col] = o->init_acc;
-      }
+      give_row(o, e, id);
     }
-    if (e.resident) {
-      for (uint32_t col = 0; col < d; ++col) {
-        const float G = (float)groups[u].g[col];
-        const float a = e.acc[col] + G * G;
-        e.acc[col] = a;
-        e.w[col] = e.w[col] - o->lr * G / (sqrtf(a) + o->eps);
-      }
-      e.touched = true;      // Section 2.2.3: the ID joins the set of touched keys
-    }
+    if (e.resident) adagrad_row(o, e, groups[u].g);
   }
   return rc;
 }
@@ -210,6 +286,12 @@ int64_t oracle_expire(void* h, int64_t now) {
   Oracle* o = static_cast<Oracle*>(h);
   if (!o) return ORACLE_ERR_ARG;
   if (o->ttl == 0) return 0;
+  // the sketch forgets in whole windows: it is cleared when more than ttl has passed since
+  // it was last cleared (time 0 at creation)
+  if (o->sketch_depth && now - o->sketch_epoch > (int64_t)o->ttl) {
+    std::fill(o->sketch.begin(), o->sketch.end(), 0ull);
+    o->sketch_epoch = now;
+  }
   int64_t removed = 0;
   for (auto it = o->map.begin(); it != o->map.end();) {
     if (now - it->second.last_seen > (int64_t)o->ttl) {
@@ -262,7 +344,11 @@ int oracle_probe(void* h, const uint64_t* ids, int64_t n, uint8_t* resident, uin
     const bool tracked = it != o->map.end() && ids[i] != kReservedId;
     const bool res = tracked && it->second.resident;
     if (resident) resident[i] = res ? 1 : 0;
-    if (count) count[i] = tracked ? it->second.count : 0;
+    if (count) {
+      count[i] = tracked ? it->second.count : 0;
+      if (!tracked && o->sketch_depth && ids[i] != kReservedId)     // sketch mode: the estimate, capped
+        count[i] = (uint32_t)std::min<uint64_t>(sketch_estimate(o, ids[i]), o->threshold);
+    }
     if (last_seen) last_seen[i] = tracked ? it->second.last_seen : -1;
     for (uint32_t c = 0; c < d; ++c) {
       if (w) w[i * (int64_t)d + c] = res ? it->second.w[c] : 0.0f;

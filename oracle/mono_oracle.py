@@ -40,6 +40,10 @@ def lib():
                                   ctypes.c_int64, ctypes.c_float)
         L.oracle_create.restype = vp
         L.oracle_create.argtypes = [u64, u32, u32, u32, f32, f32, f32, f32, u64]
+        L.oracle_enable_sketch.restype = ctypes.c_int
+        L.oracle_enable_sketch.argtypes = [vp, u32, u64]
+        L.oracle_sketch_index.restype = u64
+        L.oracle_sketch_index.argtypes = [vp, u32, u64]
         L.oracle_destroy.restype = None
         L.oracle_destroy.argtypes = [vp]
         L.oracle_lookup_pool.restype = ctypes.c_int
@@ -82,7 +86,8 @@ class OracleTable:
     """The plain map-based table: one entry per tracked ID."""
 
     def __init__(self, capacity: int, dim: int, filter_threshold: int, ttl: int, *, lr: float = 0.05,
-                 eps: float = 1e-8, init_acc: float = 0.0, init_scale: float = 0.01, seed: int = 0):
+                 eps: float = 1e-8, init_acc: float = 0.0, init_scale: float = 0.01, seed: int = 0,
+                 sketch_depth: int = 0, sketch_width: int = 0):
         self.dim = int(dim)
         self.capacity = int(capacity)
         self.threshold = max(int(filter_threshold), 1)
@@ -91,6 +96,9 @@ class OracleTable:
                                       init_scale, seed)
         if not self._h:
             raise ValueError("oracle_create rejected its arguments")
+        if sketch_depth:
+            if lib().oracle_enable_sketch(self._h, sketch_depth, sketch_width) != OK:
+                raise ValueError("sketch needs depth >= 1 and a power-of-two width")
 
     def close(self):
         if self._h:
@@ -102,6 +110,9 @@ class OracleTable:
             self.close()
         except Exception:
             pass
+
+    def sketch_index(self, r: int, id_: int) -> int:
+        return int(lib().oracle_sketch_index(self._h, r, id_))
 
     def lookup_pool(self, ids, offsets) -> np.ndarray:
         ids, offsets = _c(ids, np.uint64), _c(offsets, np.int64)

@@ -415,3 +415,95 @@ def test_sync_volume_arithmetic_from_the_paper():
     assert o.export()["w"].nbytes == 4096
     assert o.export_touched()["w"].nbytes == 4096      # one touched ID of dim 1024 is a 4 KB push
     assert 100_000 * 4096 == pytest.approx(400e6, rel=0.03)
+
+
+# ---------------------------------------------------------------- probabilistic (count-min) filter
+
+def _stream_steps(cfg, n, time_scale=1):
+    st = wl.Stream(cfg)
+    out = []
+    for t in range(n):
+        s = st.step(t)
+        out.append((s.ids, s.offsets, s.grad_pooled, t * time_scale))
+    return out
+
+
+def test_sketch_index_uses_splitmix64_of_id_and_row():
+    o = mo.OracleTable(8, 4, 2, 0, seed=77, sketch_depth=3, sketch_width=1 << 10)
+    gamma = 0x9E3779B97F4A7C15
+    for r in range(3):
+        for id_ in (0, 1, 12345678901234567, 2**64 - 2):
+            x = np.array([id_ ^ ((77 + (r + 1) * gamma) & (2**64 - 1))], dtype=np.uint64)
+            assert o.sketch_index(r, id_) == int(wl.splitmix64(x)[0]) & 1023      # workload's copy is pinned
+    rows = {(o.sketch_index(0, i), o.sketch_index(1, i)) for i in range(200)}
+    assert len(rows) > 190                                                         # rows hash independently
+
+
+def test_sketch_without_collisions_equals_exact_counters():
+    # with no expiry and a sketch so wide that no two IDs of the stream share a counter, the
+    # sketch is an exact counter per ID: same admissions, same rows, step by step
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=64, n_slots=4, n_distinct=1 << 9, dim=4, ttl=0)
+    kw = dict(lr=cfg.lr, eps=cfg.eps, init_scale=0.05, seed=3)
+    exact = mo.OracleTable(cfg.capacity, cfg.dim, 3, 0, **kw)
+    sk = mo.OracleTable(cfg.capacity, cfg.dim, 3, 0, sketch_depth=2, sketch_width=1 << 24, **kw)
+    steps = _stream_steps(cfg, 15)
+    all_ids = np.unique(np.concatenate([s[0] for s in steps]))
+    for r in range(2):
+        assert len({sk.sketch_index(r, int(i)) for i in all_ids}) == all_ids.size    # really collision-free
+    for ids, off, grad, now in steps:
+        assert exact.apply_grads(ids, off, grad, now) == 0 and sk.apply_grads(ids, off, grad, now) == 0
+        a, b = exact.probe(all_ids), sk.probe(all_ids)
+        assert (a["resident"] == b["resident"]).all() and (a["count"] == b["count"]).all()
+        assert (a["w"] == b["w"]).all() and (a["acc"] == b["acc"]).all()
+        assert (a["last_seen"][a["resident"] == 1] == b["last_seen"][b["resident"] == 1]).all()
+    assert sk.n_tracked == sk.n_resident == exact.n_resident       # IDs without a row cost no entry
+    assert exact.n_tracked > exact.n_resident
+
+
+def test_sketch_errs_only_towards_admitting():
+    # a narrow sketch: whatever the exact filter has admitted, the sketch has admitted too
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=128, n_slots=4, n_distinct=1 << 12, dim=4, ttl=0)
+    exact = mo.OracleTable(cfg.capacity, cfg.dim, 4, 0, seed=1)
+    sk = mo.OracleTable(cfg.capacity, cfg.dim, 4, 0, seed=1, sketch_depth=2, sketch_width=256)
+    steps = _stream_steps(cfg, 10)
+    all_ids = np.unique(np.concatenate([s[0] for s in steps]))
+    early = 0
+    for ids, off, grad, now in steps:
+        exact.apply_grads(ids, off, grad, now)
+        sk.apply_grads(ids, off, grad, now)
+        a, b = exact.probe(all_ids, rows=False), sk.probe(all_ids, rows=False)
+        assert (b["resident"] >= a["resident"]).all()
+        assert (b["count"] >= a["count"]).all()                    # estimates never undercount
+        early += int((b["resident"] > a["resident"]).sum())
+    assert early > 0                                               # and with 256 counters it does over-admit
+
+
+def test_sketch_with_one_counter_counts_everything():
+    # width 1: every ID shares the counter, so the estimate is the number of occurrences so far
+    o = mo.OracleTable(8, 2, 5, 0, lr=1.0, eps=0.0, init_scale=0.0, sketch_depth=1, sketch_width=1)
+    g = np.ones((2, 2), f32)
+    o.apply_grads(*bags([[1, 2], [3]]), g, 0)                      # 3 occurrences: nobody admitted
+    assert o.n_tracked == 0 and o.probe(np.array([9], np.uint64))["count"][0] == 3
+    o.apply_grads(*bags([[4], [5]]), g, 1)                         # 5 occurrences: 4 and 5 admitted now
+    assert sorted(o.export()["ids"].tolist()) == [4, 5]
+    o.apply_grads(*bags([[4], [1]]), g, 2)                         # 4 has a row and adds nothing; 1 brings it to 6
+    st = o.probe(np.array([1, 4, 5], np.uint64))
+    assert st["resident"].tolist() == [1, 1, 1] and st["last_seen"].tolist() == [2, 2, 1]
+    assert st["acc"][1][0] == 2.0 and st["acc"][0][0] == 1.0       # 4 trained twice, 1 once
+    assert o.probe(np.array([77], np.uint64))["count"][0] == 5     # capped at the threshold (estimate is 6)
+
+
+def test_sketch_is_cleared_in_whole_windows():
+    o = mo.OracleTable(8, 2, 3, 10, sketch_depth=2, sketch_width=1 << 16)
+    g = np.ones((1, 2), f32)
+    o.apply_grads(*bags([[1, 1]]), g, 0)
+    o.expire(10)                                                   # 10 - 0 > 10 is false: kept
+    assert o.probe(np.array([1], np.uint64))["count"][0] == 2
+    o.expire(11)                                                   # cleared, window restarts at 11
+    assert o.probe(np.array([1], np.uint64))["count"][0] == 0
+    o.apply_grads(*bags([[1, 1]]), g, 12)
+    o.expire(21)                                                   # 21 - 11 > 10 is false
+    o.apply_grads(*bags([[1]]), g, 21)                             # third occurrence inside the window
+    assert o.probe(np.array([1], np.uint64))["resident"][0] == 1
+    o.expire(40)                                                   # the row's own expiry still works
+    assert o.n_tracked == 0
