@@ -95,7 +95,28 @@ typedef struct {
                              larger calls grow it (an allocation, so not inside a timed
                              loop).  0 => grown on first use. */
   uint64_t max_bags;      /* same, for bags per call */
+  uint64_t sketch_width;  /* counters per sketch row, power of two (see sketch_depth) */
+  uint32_t sketch_depth;  /* 0: exact per-ID counters (default).  1..8: probabilistic filter, a
+                             count-min sketch of sketch_depth rows; see below */
+  uint32_t pad_;
 } mono_opt;
+
+/*
+ * Probabilistic admission filter (Section 2.1, heuristic 1: besides filtering by occurrence
+ * count the paper uses a probabilistic filter to save more memory; it does not say which).
+ * With sketch_depth > 0 an ID without a row has no entry in the key store at all.  Instead,
+ * per batch: (a) every distinct ID without a row adds its multiplicity to one 32-bit counter
+ * in each sketch row -- row r (0-based) uses counter
+ *     SplitMix64(id XOR (seed + (r + 1) * 0x9E3779B97F4A7C15)) AND (sketch_width - 1),
+ * SplitMix64 being the output function of Steele, Lea and Flood's generator;  (b) once all
+ * additions of the batch are done, an ID whose smallest counter has reached filter_threshold
+ * is given a row and enters the key store.  Collisions can only raise an estimate, so the
+ * sketch never rejects an ID the exact filter would admit, but it may admit one early.
+ * mono_expire clears the whole sketch when more than ttl has passed since it was last cleared
+ * (time 0 at creation), and expires rows as usual.  mono_probe reports, for an ID without an
+ * entry, count = min(estimate, filter_threshold).  Counters must not reach 2^32 between two
+ * clearings.  mono_import skips entries that are not resident.
+ */
 
 typedef struct {
   uint32_t error_bits;          /* OR of MONO_DEV_* since creation */

@@ -38,7 +38,8 @@ class MonoError(RuntimeError):
 class mono_opt(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int32), ("lr", ctypes.c_float), ("eps", ctypes.c_float),
                 ("init_acc", ctypes.c_float), ("init_scale", ctypes.c_float), ("seed", ctypes.c_uint64),
-                ("key_cells", ctypes.c_uint64), ("max_ids", ctypes.c_uint64), ("max_bags", ctypes.c_uint64)]
+                ("key_cells", ctypes.c_uint64), ("max_ids", ctypes.c_uint64), ("max_bags", ctypes.c_uint64),
+                ("sketch_width", ctypes.c_uint64), ("sketch_depth", ctypes.c_uint32), ("pad_", ctypes.c_uint32)]
 
 
 class mono_status_t(ctypes.Structure):
@@ -153,10 +154,12 @@ def _check(fn: str, rc: int, handle=None):
 
 def mono_table_create(capacity: int, dim: int, filter_threshold: int, ttl: int, *, lr: float = 0.05,
                       eps: float = 1e-8, init_acc: float = 0.0, init_scale: float = 0.0, seed: int = 0,
-                      key_cells: int = 0, max_ids: int = 0, max_bags: int = 0, stream: int = 0) -> int:
+                      key_cells: int = 0, max_ids: int = 0, max_bags: int = 0, stream: int = 0,
+                      sketch_depth: int = 0, sketch_width: int = 0) -> int:
     """Returns the table handle (an integer address)."""
     opt = mono_opt(kind=1, lr=lr, eps=eps, init_acc=init_acc, init_scale=init_scale, seed=seed,
-                   key_cells=key_cells, max_ids=max_ids, max_bags=max_bags)
+                   key_cells=key_cells, max_ids=max_ids, max_bags=max_bags, sketch_width=sketch_width,
+                   sketch_depth=sketch_depth)
     h = ctypes.c_void_p()
     rc = load_library().mono_table_create(ctypes.byref(h), capacity, dim, filter_threshold, ttl,
                                           ctypes.byref(opt), stream or None)

@@ -31,7 +31,14 @@ probe_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long
     const unsigned long long meta = p ? p->meta : 0ull;
     const bool res = p && meta_resident(meta);
     if (resident) resident[i] = res ? 1 : 0;
-    if (count) count[i] = !p ? 0u : (res ? tv.threshold : meta_low(meta));
+    if (count) {
+      uint32_t c = !p ? 0u : (res ? tv.threshold : meta_low(meta));
+      if (!p && tv.sketch_depth != 0 && ids[i] != kEmptyKey) {        // probabilistic filter: the estimate, capped
+        const unsigned int est = tv.sketch_estimate(ids[i]);
+        c = est < tv.threshold ? est : tv.threshold;
+      }
+      count[i] = c;
+    }
     if (last_seen) last_seen[i] = p ? (long long)meta_time(meta) : -1LL;
   }
 }

@@ -246,9 +246,26 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
   if (meta_resident(item.meta)) atomicAdd(&tv.st->n_resident, (unsigned long long)(-1LL));
 }
 
+// Probabilistic filter, between phases 2 and 3: every distinct ID that is not in the key
+// store adds its multiplicity to one counter per sketch row.  All additions of a batch are
+// done before any estimate is read (next kernel), so the outcome does not depend on order.
+__global__ void __launch_bounds__(256)
+sketch_add_kernel(TableView tv, Work wk) {
+  const uint32_t n = tv.st->n_insert;
+  const uint32_t stride = gridDim.x * blockDim.x;
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const uint32_t u = wk.ins_list[i];
+    const unsigned long long id = wk.uid[u];
+    const uint32_t m = wk.ulen[u];
+    for (uint32_t r = 0; r < tv.sketch_depth; ++r) atomicAdd(tv.sketch_counter(r, id), m);
+  }
+}
+
 // Phase 3 of mono_apply_grads: one thread per ID that phase 2 found unknown to
-// the key store; it is inserted (with a row straight away when the batch alone
-// reaches the threshold).
+// the key store.  Exact filter: it is inserted (with a row straight away when
+// the batch alone reaches the threshold).  Probabilistic filter: it is inserted,
+// with a row, only if its sketch estimate has reached the threshold; otherwise
+// nothing is stored for it.
 __global__ void __launch_bounds__(256)
 table_insert_kernel(TableView tv, Work wk, uint32_t now) {
   __shared__ BlockAlloc sh;
@@ -259,7 +276,12 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     const bool todo = base + threadIdx.x < n;
     uint32_t u = 0, m = 0;
     if (todo) { u = wk.ins_list[base + threadIdx.x]; m = wk.ulen[u]; }
-    const uint32_t count = m < tv.threshold ? m : tv.threshold;
+    const bool sketch = tv.sketch_depth != 0;
+    uint32_t count = m < tv.threshold ? m : tv.threshold;
+    if (sketch && todo) {
+      const unsigned int est = tv.sketch_estimate(wk.uid[u]);
+      count = est < tv.threshold ? est : tv.threshold;
+    }
     const bool need_row = todo && count >= tv.threshold;
     const Reservation rv = block_reserve(tv, &sh, need_row, todo && m > 1, false, (need_row && m > 1) ? m : 0u);
     if (!todo) continue;
@@ -275,6 +297,7 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
       ++n_res;
       if (m > kSegChunk) register_long(tv, wk, u, m);
     }
+    if (sketch && row_word == kNoRow) continue;      // below the estimate (or no row left): not stored
     Cell item; item.key = id; item.meta = make_meta(now, low);
     cuckoo_insert(tv, item);
     ++n_done;
@@ -426,6 +449,7 @@ import_insert_kernel(TableView tv, const unsigned long long* __restrict__ ids, c
         present |= load_cell(tv.cells + bk[b] * kCellsPerBucket + c).key == id;
     for (unsigned s = 0; s < stash_hw && !present; ++s) present |= load_cell(tv.stash + s).key == id;
     if (present) { atomicOr(&tv.st->error_bits, 8u /* MONO_DEV_IMPORT_DUP */); continue; }
+    if (tv.sketch_depth != 0 && !resident[i]) continue;     // probabilistic filter: IDs without a row have no entry
     long long seen = last_seen[i];
     if (seen < 0) seen = 0;
     if (seen > 0xFFFFFFFELL) seen = 0xFFFFFFFELL;

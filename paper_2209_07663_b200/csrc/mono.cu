@@ -28,11 +28,11 @@ using namespace mono;
 static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_INSERT, K_EXPAND, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
   K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
-  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "table_insert", "expand_parts",
+  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "sketch_add", "table_insert", "expand_parts",
   "scatter_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
@@ -51,6 +51,7 @@ struct mono_table {
   int sm_count = 148;
   uint64_t key_cells = 0;
   int64_t last_now = -1;
+  int64_t sketch_epoch = 0;       // time the sketch was last cleared
   int64_t max_ids = 0, max_bags = 0;
   // device staging for the host-buffer calls
   unsigned long long* stage_ids = nullptr;
@@ -210,6 +211,7 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   LAUNCH(t, K_DEDUP, dedup_tile_kernel<<<tiles, kTileThreads, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
                                                             tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
+  if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   LAUNCH(t, K_EXPAND, expand_parts_kernel<<<g4, 128, 0, s>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
@@ -250,6 +252,7 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   uint64_t key_cells = o.key_cells ? o.key_cells : next_pow2(4 * capacity);
   if (!is_pow2(key_cells) || key_cells < 64 || key_cells > (1ull << 34)) return MONO_ERR_ARG;
   if (o.max_ids >= (1ull << 31) || o.max_bags >= (1ull << 31)) return MONO_ERR_ARG;
+  if (o.sketch_depth > 8 || (o.sketch_depth && (!is_pow2(o.sketch_width) || o.sketch_width > (1ull << 32)))) return MONO_ERR_ARG;
 
   mono_table* t = new (std::nothrow) mono_table();
   if (!t) return MONO_ERR_NOMEM;
@@ -277,6 +280,14 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   if ((rc = dev_alloc(t, &tv.rows, (size_t)capacity * 2 * dim)) != MONO_OK) return fail(rc);
   if ((rc = dev_alloc(t, &tv.free_rows, capacity)) != MONO_OK) return fail(rc);
   if ((rc = dev_alloc(t, &tv.st, 1)) != MONO_OK) return fail(rc);
+  tv.sketch_depth = o.sketch_depth;
+  tv.sketch_seed = o.seed;
+  if (o.sketch_depth) {
+    tv.sketch_mask = o.sketch_width - 1;
+    const size_t counters = (size_t)o.sketch_depth * o.sketch_width;
+    if ((rc = dev_alloc(t, &tv.sketch, counters)) != MONO_OK) return fail(rc);
+    if (cudaMemsetAsync(tv.sketch, 0, counters * sizeof(unsigned int), t->stream) != cudaSuccess) return fail(MONO_ERR_CUDA);
+  }
   DevState init;
   std::memset(&init, 0, sizeof(init));
   init.free_top = (long long)capacity;
@@ -299,7 +310,7 @@ int mono_table_destroy(mono_table* t) {
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
   free_scratch(t);
-  dev_free(t->tv.cells); dev_free(t->tv.stash); dev_free(t->tv.rows); dev_free(t->tv.free_rows); dev_free(t->tv.st);
+  dev_free(t->tv.cells); dev_free(t->tv.stash); dev_free(t->tv.rows); dev_free(t->tv.free_rows); dev_free(t->tv.st); dev_free(t->tv.sketch);
   delete t;
   return MONO_OK;
 }
@@ -337,6 +348,12 @@ int mono_expire(mono_table* t, int64_t now) {
   if (rc != MONO_OK) return rc;
   t->last_now = now;
   if (t->tv.ttl == 0) return MONO_OK;
+  if (t->tv.sketch_depth && now - t->sketch_epoch > (int64_t)t->tv.ttl) {
+    // the sketch forgets in whole windows: cleared when more than ttl has passed since the last clearing
+    CUDA_TRY(t, cudaMemsetAsync(t->tv.sketch, 0, (size_t)t->tv.sketch_depth * (t->tv.sketch_mask + 1) * sizeof(unsigned int),
+                                t->stream));
+    t->sketch_epoch = now;
+  }
   LAUNCH(t, K_EXPIRE, expire_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells, (long long)now));
   LAUNCH(t, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, t->stream>>>(t->tv));
   CUDA_TRY(t, cudaGetLastError());

@@ -66,6 +66,15 @@ __host__ __device__ inline unsigned long long mix_b(unsigned long long x) {
   return x;
 }
 
+// SplitMix64 output function (Steele, Lea, Flood 2014): the sketch's row hashes are
+// defined through it in the ABI header, so the CPU oracle indexes the same counters.
+__host__ __device__ inline unsigned long long splitmix64_mix(unsigned long long z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
 // Counters and sticky condition bits, one block per table in device memory.
 struct DevState {
   unsigned int error_bits;
@@ -116,6 +125,11 @@ struct TableView {
   uint32_t ttl;
   float lr, eps, init_acc, init_scale;
   uint32_t init_key0, init_key1;    // Philox key = table seed
+  // probabilistic admission filter (count-min sketch); sketch_depth 0 = exact counters
+  unsigned int* sketch;             // [sketch_depth][sketch_mask + 1]
+  unsigned long long sketch_mask;
+  unsigned long long sketch_seed;
+  uint32_t sketch_depth;
 
   // h0 / h1: the low bits pick the bucket, the top two bits the cell of that bucket an
   // insertion tries first, so a look-up that reads that one cell first usually needs no more
@@ -123,6 +137,20 @@ struct TableView {
   __device__ inline unsigned long long hash1(unsigned long long id) const { return mix_b(id ^ seed1); }
   __device__ inline unsigned long long bucket0(unsigned long long id) const { return hash0(id) & bucket_mask; }
   __device__ inline unsigned long long bucket1(unsigned long long id) const { return hash1(id) & bucket_mask; }
+  // counter of sketch row r that `id` maps to
+  __device__ inline unsigned int* sketch_counter(uint32_t r, unsigned long long id) const {
+    const unsigned long long i = splitmix64_mix(id ^ (sketch_seed + (unsigned long long)(r + 1) * 0x9E3779B97F4A7C15ull)) & sketch_mask;
+    return sketch + (size_t)r * (sketch_mask + 1) + i;
+  }
+  // count-min estimate of the occurrences of `id`: the smallest of its counters
+  __device__ inline unsigned int sketch_estimate(unsigned long long id) const {
+    unsigned int est = 0xFFFFFFFFu;
+    for (uint32_t r = 0; r < sketch_depth; ++r) {
+      const unsigned int c = *reinterpret_cast<const volatile unsigned int*>(sketch_counter(r, id));
+      est = c < est ? c : est;
+    }
+    return est;
+  }
   __device__ inline float* w_row(uint32_t row) const { return rows + (size_t)row * 2u * dim; }
   __device__ inline float* acc_row(uint32_t row) const { return rows + (size_t)row * 2u * dim + dim; }
 };

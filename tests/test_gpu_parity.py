@@ -219,6 +219,31 @@ def test_export_import_roundtrip_into_a_differently_seeded_table():
     assert_state_equal(other, cpu, "after duplicate import")
 
 
+@pytest.mark.parametrize("depth,width", [(1, 1), (2, 1 << 10), (3, 1 << 14), (4, 1 << 22)])
+def test_probabilistic_filter_matches_the_sketch_oracle(depth, width):
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=14, ttl=4, filter_threshold=3)
+    kw = dict(sketch_depth=depth, sketch_width=width)
+    gpu, cpu = make_pair(cfg, **kw)
+    stream = wl.Stream(cfg)
+    seen = []
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        seen.append(np.unique(s.ids))
+        got = gpu.lookup_pool(s.ids, s.offsets).cpu().numpy()
+        assert_vectors_close(got, cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+        gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
+        if t % 3 == 2:
+            gpu.expire(t); cpu.expire(t)                  # clears the sketch every other sweep (ttl 4)
+        assert_state_equal(gpu, cpu, f"step {t}")         # only IDs with a row have entries
+        ids = np.unique(np.concatenate(seen[-3:]))
+        g, o = gpu.probe(ids, rows=False), cpu.probe(ids, rows=False)
+        assert (g["count"] == o["count"]).all() and (g["resident"] == o["resident"]).all(), f"estimates at step {t}"
+    st = gpu.status()
+    assert st["error_bits"] == 0 and st["n_tracked"] == st["n_resident"] > 0
+    assert_audit_ok(gpu)
+
+
 def test_rehash_moves_keys_but_changes_no_state():
     cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=12)
     gpu, cpu = make_pair(cfg)
