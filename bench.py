@@ -3,8 +3,9 @@
 
 One "step" is one pass of the whole hot path over one fresh synthetic batch:
 mono_lookup_pool (probe, gather, sum pooling) + mono_apply_grads (dedup,
-count/stamp/admit, cuckoo insert, segmented gradient reduce, Adagrad), with
-mono_expire called once every `sweep_period` steps inside the timed region.
+count/stamp/admit, cuckoo insert, segmented gradient reduce, Adagrad), followed
+by one slice of the expiry sweep (mono_expire_slice: 1/`sweep_slices` of the key
+store per step, so every step carries the same share of the sweep).
 The table is pre-filled to the steady state of the configured stream, so the
 timed steps run at the load the stream would reach, not on an empty table.
 
@@ -202,7 +203,7 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- our arm
 
-def algorithmic_bytes(n, b, u, ur, ur1, unew, d):
+def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0):
     """Bytes the method itself must move per step, per kernel (each distinct datum once per
     phase; 32-byte sector as the smallest random access).  n occurrences, b bags, u distinct
     IDs, ur of them with a row, ur1 of those occurring once in the batch, unew new IDs."""
@@ -216,6 +217,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d):
         "scatter_singletons": 4 * d * b + 16 * d * ur1,      # gradients once + rows of IDs seen once
         "reduce_adagrad": 16 * d * (ur - ur1),               # rows of repeated IDs (gradients counted above)
         "expand_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
+        "expire": 16 * sweep_cells,                          # one streaming read of the swept cells
     }
     return per_kernel, sum(per_kernel.values())
 
@@ -225,7 +227,7 @@ KERNEL_GROUP = {
     "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
     "table_update": "table", "table_insert": "table", "expand_parts": "table",
     "scatter_singletons": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
-    "combine_adagrad": "adagrad",
+    "combine_adagrad": "adagrad", "expire": "expire",
 }
 
 
@@ -266,7 +268,7 @@ def run_ours(args):
     cfg = rank_config(base, rank)
     K, W, E = args.steps, args.warmup, args.e2e_steps
     KT = min(K, args.kernel_steps)            # steps of the per-kernel timing pass
-    sweep_period = args.sweep_period or K
+    S = args.sweep_slices
     now0 = cfg.ttl - 1 if args.prefill else 0
     stream = wl.Stream(cfg)
 
@@ -305,13 +307,13 @@ def run_ours(args):
     torch.cuda.synchronize()
     setup_s = time.time() - t_setup
 
-    def step(i, sweep=False):
+    def step(i):
         """Step i of the stream (time now0 + 1 + i) on its own fresh batch."""
         ids, off, grad = dev_batches[i]
         mb.mono_lookup_pool(table.handle, ids, ids.numel(), off, cfg.n_bags, out)
         mb.mono_apply_grads(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0 + 1 + i)
-        if sweep:
-            mb.mono_expire(table.handle, now0 + 1 + i)
+        if S > 0:
+            mb.mono_expire_slice(table.handle, now0 + 1 + i, i % S, S)
 
     def barrier():
         if world > 1:
@@ -330,7 +332,7 @@ def run_ours(args):
     barrier()
     ev0.record()
     for t in range(K):
-        step(W + t, sweep=(t + 1) % sweep_period == 0)
+        step(W + t)
     ev1.record()
     barrier()
     ms_total = ev0.elapsed_time(ev1)
@@ -342,7 +344,7 @@ def run_ours(args):
     # ---- the same steps on fresh batches with every kernel bracketed by CUDA events
     mb.mono_timing_enable(table.handle, True)
     for t in range(KT):
-        step(W + K + t, sweep=(t == KT - 1))
+        step(W + K + t)
     torch.cuda.synchronize()
     tim = mb.mono_timing_read(table.handle, reset=True)
     mb.mono_timing_enable(table.handle, False)
@@ -366,6 +368,8 @@ def run_ours(args):
             now = now0 + 1 + W + K + KT + t
             mb.mono_lookup_pool_host(table.handle, ids, ids.numel(), off, cfg.n_bags, out_h)
             mb.mono_apply_grads_host(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now)
+            if S > 0:
+                mb.mono_expire_slice(table.handle, now, (W + K + KT + t) % S, S)
             n_e2e_ids += ids.numel()
             h2d += 2 * (ids.numel() * 8 + off.numel() * 8) + grad.numel() * 4
             d2h += out_h.numel() * 4
@@ -388,7 +392,7 @@ def run_ours(args):
         ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / KT
         unew = (st_c["sum_new"] - st_b["sum_new"]) / KT
         ur1 = (st_c["sum_single_resident"] - st_b["sum_single_resident"]) / KT
-        alg_kernel, alg_total = algorithmic_bytes(n, cfg.n_bags, u, ur, ur1, unew, d)
+        alg_kernel, alg_total = algorithmic_bytes(n, cfg.n_bags, u, ur, ur1, unew, d, cfg.key_cells // S if S > 0 else 0)
         per_kernel = {}
         for name, v in tim["kernels"].items():
             if v["launches"] and name in KERNEL_GROUP:
@@ -415,7 +419,8 @@ def run_ours(args):
                 "prefill": "steady state of the stream" if args.prefill else "empty table",
                 "rows_resident_at_start": st0["n_resident"], "ids_tracked_at_start": st0["n_tracked"],
                 "row_load": st0["n_resident"] / cfg.capacity, "key_load": st0["n_tracked"] / cfg.key_cells,
-                "sweep_period_steps": sweep_period, "l2": "every step reads a fresh batch larger than L2",
+                "sweep": (f"every step sweeps 1/{S} of the key store (a full sweep every {S} steps)" if S > 0
+                          else "none"), "l2": "every step reads a fresh batch larger than L2",
                 "parallelism": f"{world} independent table(s), one per GPU",
             },
             "bags_per_s": world * cfg.n_bags * K / (ms_max * 1e-3),
@@ -599,7 +604,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS) + ["multi"])
-    ap.add_argument("--sweep-period", type=int, default=0, help="steps between expiry sweeps (0 = --steps)")
+    ap.add_argument("--sweep-slices", type=int, default=32,
+                    help="every step sweeps 1/S of the key store for expired IDs (0 = no sweep)")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--kernel-steps", type=int, default=8, help="steps of the per-kernel CUDA-event pass")
     ap.add_argument("--no-prefill", dest="prefill", action="store_false")

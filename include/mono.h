@@ -224,6 +224,16 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids,
 int mono_expire(mono_table* t, int64_t now);
 
 /*
+ * Incremental form of mono_expire: sweeps slice `slice` of `n_slices` equal parts of the key
+ * store (the last slice also covers the overflow stash), so that the cost of a full sweep can
+ * be spread over n_slices training steps.  Calling it for slice = 0 .. n_slices-1 with the
+ * same `now` (and no other call in between) has exactly the effect of mono_expire(now).
+ * 1 <= n_slices <= 65536, slice < n_slices.  With the probabilistic filter, slice 0 is the
+ * one that clears the sketch when its window has passed.
+ */
+int mono_expire_slice(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices);
+
+/*
  * Host-buffer forms of the two hot calls, for callers whose batches live in
  * host memory (pinned memory makes the copies asynchronous).  They copy the
  * inputs to library-owned device staging on the table's stream, run the same

@@ -7,38 +7,6 @@
 
 namespace mono {
 
-// Find `id` in its two candidate buckets (and the stash when it is in use) with
-// the four lanes `sub` = 0..3 of a quad reading one cell each.  Returns, on the
-// lane that saw the key, hit = true and the cell's metadata.  `quad_mask` names
-// the four lanes; all four must call together.
-__device__ inline bool quad_find(const TableView& tv, unsigned long long id, bool active, int sub,
-                                 unsigned quad_mask, unsigned stash_hw, unsigned long long* meta_out) {
-  bool hit = false;
-  unsigned long long meta = 0;
-  if (active) {
-    const Cell c = load_cell_ro(tv.cells + tv.bucket0(id) * kCellsPerBucket + sub);
-    hit = c.key == id;
-    meta = c.meta;
-  }
-  bool found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
-  if (!found) {
-    if (active) {
-      const Cell c = load_cell_ro(tv.cells + tv.bucket1(id) * kCellsPerBucket + sub);
-      hit = c.key == id;
-      meta = c.meta;
-    }
-    found = (__ballot_sync(quad_mask, hit) & quad_mask) != 0;
-    if (!found && stash_hw != 0 && active) {
-      for (unsigned i = sub; i < stash_hw; i += kCellsPerBucket) {
-        const Cell c = load_cell_ro(tv.stash + i);
-        if (c.key == id) { hit = true; meta = c.meta; break; }
-      }
-    }
-  }
-  *meta_out = meta;
-  return hit;
-}
-
 // Look-up of four IDs by one quad.  Each lane brings its own ID (hashed once,
 // by its owner); the quad then resolves the four IDs in turn, every lane
 // reading one cell of the ID's bucket, so a bucket costs one coalesced 64-byte

@@ -345,34 +345,44 @@ __global__ void finish_apply_kernel(DevState* st) {
 // its row, if it has one, goes back on the free list (one counter update per
 // warp and round).
 __global__ void __launch_bounds__(256)
-expire_kernel(TableView tv, unsigned long long n_cells, long long now) {
+expire_kernel(TableView tv, unsigned long long n_cells, unsigned long long first, unsigned long long last,
+              long long now) {
+  // sweeps cells [first, last) of the sequence "key store, then stash" (total n_cells + kStashCells)
+  constexpr int kDepth = 4;                                                // independent loads per thread and round
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-  const unsigned long long total = n_cells + kStashCells;
-  const unsigned long long rounds = (total + stride - 1) / stride;        // same for every thread
+  const unsigned long long rounds = (last - first + stride * kDepth - 1) / (stride * kDepth);  // same for every thread
   const int lane = threadIdx.x & 31;
   unsigned int n_gone = 0, n_rows = 0;
   for (unsigned long long r = 0; r < rounds; ++r) {
-    const unsigned long long i = r * stride + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-    bool frees_row = false;
-    uint32_t row = 0;
-    if (i < total) {
-      Cell* p = i < n_cells ? tv.cells + i : tv.stash + (i - n_cells);
-      const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
-      if (v.x != kEmptyKey && now - (long long)meta_time(v.y) > (long long)tv.ttl) {
-        ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
-        *reinterpret_cast<ulonglong2*>(p) = e;
-        ++n_gone;
-        if (meta_resident(v.y)) { frees_row = true; row = meta_row(v.y); ++n_rows; }
-      }
+    const unsigned long long i0 = first + r * kDepth * stride + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    Cell* p[kDepth];
+    ulonglong2 v[kDepth];
+#pragma unroll
+    for (int k = 0; k < kDepth; ++k) {
+      const unsigned long long i = i0 + k * stride;
+      p[k] = i < last ? (i < n_cells ? tv.cells + i : tv.stash + (i - n_cells)) : nullptr;
+      v[k].x = kEmptyKey; v[k].y = 0ull;
+      if (p[k]) v[k] = *reinterpret_cast<const ulonglong2*>(p[k]);
     }
-    const unsigned mask = __ballot_sync(0xFFFFFFFFu, frees_row);
-    if (mask) {
-      unsigned long long pos = 0;
-      const int leader = __ffs(mask) - 1;
-      if (lane == leader)
-        pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)__popc(mask));
-      pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
-      if (frees_row) tv.free_rows[pos + __popc(mask & ((1u << lane) - 1u))] = row;
+#pragma unroll
+    for (int k = 0; k < kDepth; ++k) {
+      bool frees_row = false;
+      uint32_t row = 0;
+      if (v[k].x != kEmptyKey && now - (long long)meta_time(v[k].y) > (long long)tv.ttl) {
+        ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+        *reinterpret_cast<ulonglong2*>(p[k]) = e;
+        ++n_gone;
+        if (meta_resident(v[k].y)) { frees_row = true; row = meta_row(v[k].y); ++n_rows; }
+      }
+      const unsigned mask = __ballot_sync(0xFFFFFFFFu, frees_row);
+      if (mask) {
+        unsigned long long pos = 0;
+        const int leader = __ffs(mask) - 1;
+        if (lane == leader)
+          pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)__popc(mask));
+        pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
+        if (frees_row) tv.free_rows[pos + __popc(mask & ((1u << lane) - 1u))] = row;
+      }
     }
   }
   for (int o = 16; o > 0; o >>= 1) {

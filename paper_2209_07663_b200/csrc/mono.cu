@@ -342,22 +342,36 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
                       reinterpret_cast<const long long*>(slot_offsets), n_bags, grad_pooled, (uint32_t)now);
 }
 
-int mono_expire(mono_table* t, int64_t now) {
-  if (!t) return MONO_ERR_ARG;
+static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices) {
+  if (!t || n_slices == 0 || slice >= n_slices) return MONO_ERR_ARG;
   int rc = check_now(t, now);
   if (rc != MONO_OK) return rc;
   t->last_now = now;
   if (t->tv.ttl == 0) return MONO_OK;
-  if (t->tv.sketch_depth && now - t->sketch_epoch > (int64_t)t->tv.ttl) {
+  if (slice == 0 && t->tv.sketch_depth && now - t->sketch_epoch > (int64_t)t->tv.ttl) {
     // the sketch forgets in whole windows: cleared when more than ttl has passed since the last clearing
     CUDA_TRY(t, cudaMemsetAsync(t->tv.sketch, 0, (size_t)t->tv.sketch_depth * (t->tv.sketch_mask + 1) * sizeof(unsigned int),
                                 t->stream));
     t->sketch_epoch = now;
   }
-  LAUNCH(t, K_EXPIRE, expire_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells, (long long)now));
-  LAUNCH(t, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, t->stream>>>(t->tv));
+  const unsigned long long total = t->key_cells + kStashCells;
+  const unsigned long long first = t->key_cells / n_slices * slice;             // key_cells is a power of two >= 64
+  const unsigned long long last = slice + 1 == n_slices ? total : t->key_cells / n_slices * (slice + 1);
+  if (last > first) {
+    unsigned long long blocks = (last - first + 255) / 256;
+    if (blocks > (unsigned long long)grid_for(t, 8)) blocks = grid_for(t, 8);
+    LAUNCH(t, K_EXPIRE, expire_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, t->key_cells, first, last, (long long)now));
+  }
+  if (slice + 1 == n_slices) LAUNCH(t, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, t->stream>>>(t->tv));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
+}
+
+int mono_expire(mono_table* t, int64_t now) { return expire_range(t, now, 0, 1); }
+
+int mono_expire_slice(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices) {
+  if (n_slices > 65536) return MONO_ERR_ARG;
+  return expire_range(t, now, slice, n_slices);
 }
 
 // Device address of g_noalloc_occ_row on the current device, looked up once per

@@ -199,8 +199,5 @@ __device__ inline Cell load_cell_ro(const Cell* p) {
   Cell c; c.key = v.x; c.meta = v.y; return c;
 }
 
-__device__ inline void warp_add(unsigned long long* ctr, unsigned int pred_count_mask_popc) {
-  if (pred_count_mask_popc) atomicAdd(ctr, (unsigned long long)pred_count_mask_popc);
-}
 
 }  // namespace mono

@@ -1,7 +1,8 @@
 """Parity at the full size of the `large` configuration, in the launch configuration the
 benchmark times: table pre-filled to the stream's steady state (hundreds of millions of
 tracked IDs, ~0.9 row load), whole batches of 1.6 M bags through mono_lookup_pool and
-mono_apply_grads, then mono_expire.
+mono_apply_grads, then the sweep in the 32 slices the benchmark spreads over its steps
+(here all at one time, which makes them equal to one mono_expire).
 
 The oracle cannot hold that table, so it is checked on a sample: a few hundred bags and
 every ID they contain, plus IDs drawn from the head, the middle and the tail of the batch.
@@ -95,7 +96,8 @@ def test_large_config_full_size_sampled_parity():
         assert cpu.apply_grads(masked, s.offsets, s.grad_pooled, now) == 0
         del ids, off, grad
     last = now0 + n_steps
-    gpu.expire(last)
+    for k in range(32):
+        mb.mono_expire_slice(gpu.handle, last, k, 32)
     cpu.expire(last)
 
     g, o = gpu.probe(sample_ids), cpu.probe(sample_ids)

@@ -186,6 +186,72 @@ def test_expiry_sets_and_row_recycling():
     assert a["resident_cells"] + a["free_rows"] == cfg.capacity
 
 
+@pytest.mark.parametrize("n_slices", [1, 3, 7, 64])
+def test_sliced_sweep_equals_one_full_sweep(n_slices):
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=8, ttl=2, key_cells=1 << 16)
+    gpu, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        for k in range(n_slices):
+            mb.mono_expire_slice(gpu.handle, t, k, n_slices)
+        cpu.expire(t)
+        assert_state_equal(gpu, cpu, f"step {t}")
+    assert gpu.status()["n_expired_total"] > 0
+    assert_audit_ok(gpu)
+    with pytest.raises(mb.MonoError):
+        mb.mono_expire_slice(gpu.handle, cfg.steps, 3, 3)
+
+
+def test_interleaved_sweep_slices_evict_neither_early_nor_late():
+    """One slice per training step, with the time advancing: which step visits an ID's cell
+    depends on where the ID hashes, so the oracle cannot be swept the same way.  What is unique:
+    an ID whose occurrences are never more than ttl + 1 steps apart (and which is recent at the
+    end) cannot have been evicted, so its whole state equals that of an oracle that never
+    sweeps; an ID not seen for ttl + n_slices steps or more has met a visit of its cell that
+    evicts it, so it must be gone."""
+    n_slices, ttl = 5, 3
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=40, ttl=ttl, key_cells=1 << 16, capacity=1 << 15)
+    gpu = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, ttl, key_cells=cfg.key_cells, lr=cfg.lr,
+                       eps=cfg.eps, init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed)
+    cpu = mo.OracleTable(cfg.capacity, cfg.dim, cfg.filter_threshold, 0, lr=cfg.lr, eps=cfg.eps,
+                         init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed)
+    stream = wl.Stream(cfg)
+    seen_at = {}
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
+        mb.mono_expire_slice(gpu.handle, t, t % n_slices, n_slices)
+        for i in np.unique(s.ids[s.ids != np.uint64(wl.RESERVED_ID)]).tolist():
+            seen_at.setdefault(i, []).append(t)
+    end = cfg.steps - 1
+    g, o = gpu.export(), cpu.export()
+    g_at = {int(i): k for k, i in enumerate(g["ids"].tolist())}
+    o_at = {int(i): k for k, i in enumerate(o["ids"].tolist())}
+    n_safe = n_gone = 0
+    for i, times in seen_at.items():
+        gaps = np.diff(times)
+        if end - times[-1] >= ttl + n_slices:
+            assert i not in g_at, f"ID {i} last seen at {times[-1]} is still tracked at {end}"
+            n_gone += 1
+        elif end - times[-1] <= ttl and (gaps.size == 0 or gaps.max() <= ttl + 1):
+            assert i in g_at, f"ID {i} was evicted although it was never inactive for longer than ttl"
+            a, b = g_at[i], o_at[i]
+            assert g["count"][a] == o["count"][b] and g["last_seen"][a] == o["last_seen"][b]
+            assert g["resident"][a] == o["resident"][b]
+            if g["resident"][a]:
+                assert_vectors_close(g["w"][a][None], o["w"][b][None], f"row of ID {i}")
+                assert_vectors_close(g["acc"][a][None], o["acc"][b][None], f"accumulator of ID {i}")
+            n_safe += 1
+    assert n_safe > 100 and n_gone > 100, (n_safe, n_gone)
+    for i in g_at:                                     # nothing tracked that was never fed
+        assert i in seen_at
+    assert_audit_ok(gpu)
+
+
 def test_unswept_entries_survive_and_refresh():
     gpu = mb.MonoTable(64, 4, 1, 3, init_scale=0.1)
     cpu = mo.OracleTable(64, 4, 1, 3, init_scale=0.1)
