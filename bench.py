@@ -5,7 +5,9 @@ One "step" is one pass of the whole hot path over one fresh synthetic batch:
 mono_lookup_pool (probe, gather, sum pooling) + mono_apply_grads (dedup,
 count/stamp/admit, cuckoo insert, segmented gradient reduce, Adagrad), followed
 by one slice of the expiry sweep (mono_expire_slice: 1/`sweep_slices` of the key
-store per step, so every step carries the same share of the sweep).
+store per step, so every step carries the same share of the sweep).  Each batch is
+announced with mono_prepare_push before its lookup, so the ID-only part of the push
+runs beside the lookup; the per-kernel timing pass runs without it, each kernel alone.
 The table is pre-filled to the steady state of the configured stream, so the
 timed steps run at the load the stream would reach, not on an empty table.
 
@@ -216,7 +218,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0):
         "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
         "scatter_singletons": 4 * d * b + 16 * d * ur1,      # gradients once + rows of IDs seen once
         "reduce_adagrad": 16 * d * (ur - ur1),               # rows of repeated IDs (gradients counted above)
-        "expand_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
+        "expand_parts": 0, "order_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
         "expire": 16 * sweep_cells,                          # one streaming read of the swept cells
     }
     return per_kernel, sum(per_kernel.values())
@@ -225,7 +227,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0):
 KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
     "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
-    "table_update": "table", "table_insert": "table", "expand_parts": "table",
+    "table_update": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
     "scatter_singletons": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
     "combine_adagrad": "adagrad", "expire": "expire",
 }
@@ -307,9 +309,11 @@ def run_ours(args):
     torch.cuda.synchronize()
     setup_s = time.time() - t_setup
 
-    def step(i):
+    def step(i, prepare=True):
         """Step i of the stream (time now0 + 1 + i) on its own fresh batch."""
         ids, off, grad = dev_batches[i]
+        if prepare and args.prepare:
+            mb.mono_prepare_push(table.handle, ids, ids.numel(), off, cfg.n_bags)
         mb.mono_lookup_pool(table.handle, ids, ids.numel(), off, cfg.n_bags, out)
         mb.mono_apply_grads(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0 + 1 + i)
         if S > 0:
@@ -344,7 +348,7 @@ def run_ours(args):
     # ---- the same steps on fresh batches with every kernel bracketed by CUDA events
     mb.mono_timing_enable(table.handle, True)
     for t in range(KT):
-        step(W + K + t)
+        step(W + K + t, prepare=False)       # every kernel alone on the device
     torch.cuda.synchronize()
     tim = mb.mono_timing_read(table.handle, reset=True)
     mb.mono_timing_enable(table.handle, False)
@@ -422,6 +426,8 @@ def run_ours(args):
                 "sweep": (f"every step sweeps 1/{S} of the key store (a full sweep every {S} steps)" if S > 0
                           else "none"), "l2": "every step reads a fresh batch larger than L2",
                 "parallelism": f"{world} independent table(s), one per GPU",
+                "push_prepared": ("mono_prepare_push before each lookup: the grouping of the batch's IDs runs "
+                                  "beside the lookup" if args.prepare else "no"),
             },
             "bags_per_s": world * cfg.n_bags * K / (ms_max * 1e-3),
             "gpu_launches": launches,
@@ -604,6 +610,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS) + ["multi"])
+    ap.add_argument("--no-prepare", dest="prepare", action="store_false",
+                    help="do not announce each batch with mono_prepare_push before its lookup")
     ap.add_argument("--sweep-slices", type=int, default=32,
                     help="every step sweeps 1/S of the key store for expired IDs (0 = no sweep)")
     ap.add_argument("--e2e-steps", type=int, default=4)

@@ -224,6 +224,23 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids,
 int mono_expire(mono_table* t, int64_t now);
 
 /*
+ * Optional hint that overlaps the ID-only part of a push with the lookup of the same batch
+ * (the paper has no counterpart; it describes no batching below the level of Section 2.2's
+ * pull and push).  Announces the batch that the NEXT mono_apply_grads on this table will be
+ * given -- the same device pointers and sizes, contents unchanged until that call -- and
+ * starts grouping its occurrences by ID on a stream of the table's own, ordered after
+ * everything issued on the table's stream so far and running beside whatever is issued next
+ * (normally mono_lookup_pool of that batch).  mono_apply_grads called with exactly these
+ * `ids`, `n_ids`, `slot_offsets`, `n_bags` waits for the grouping and uses it; called with
+ * anything else it discards the preparation and groups its own batch, as does a second
+ * mono_prepare_push.  Results are the same with or without the hint.  The table is not
+ * changed by this call.  Errors: as mono_lookup_pool; malformed offsets raise
+ * MONO_DEV_BAD_OFFSETS in the status, as they would in mono_apply_grads.
+ */
+int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                      int64_t n_bags);
+
+/*
  * Incremental form of mono_expire: sweeps slice `slice` of `n_slices` equal parts of the key
  * store (the last slice also covers the overflow stash), so that the cost of a full sweep can
  * be spread over n_slices training steps.  Calling it for slice = 0 .. n_slices-1 with the

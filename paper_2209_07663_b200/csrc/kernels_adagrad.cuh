@@ -211,7 +211,7 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
         if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
       }
     } else {
-      const uint32_t p = item;
+      const uint32_t p = wk.part_order[item];
       const uint32_t li = wk.part_u[p];
       const uint32_t u = wk.long_u[li];
       const uint32_t k = p - wk.long_part0[li];

@@ -37,6 +37,7 @@ constexpr int kTileIds = 512;                  // occurrences per block of dedup
 constexpr int kTileSlots = 1024;               // shared-memory table of one tile
 constexpr int kTileThreads = 256;              // block size of dedup_tile_kernel
 constexpr int kPrimaryProbes = 16;             // positions tried in the primary tier of the per-call set
+constexpr uint32_t kWindows = 1024;            // the parts of long segments are scheduled by position in the batch, this finely
 
 // Scratch of one mono_apply_grads call.
 struct Work {
@@ -61,6 +62,8 @@ struct Work {
   uint32_t* long_u;          // [max_long] distinct IDs whose segment is reduced in parts
   uint32_t* long_part0;      // [max_long] first part of each
   uint32_t* part_u;          // [max_parts] owner (index into long_u) of each part
+  uint32_t* part_order;      // [max_parts] the parts in the order they are reduced in: by window of the batch
+  uint32_t* win_count;       // [2 * kWindows] parts per window, then a cursor per window; zero between calls
   double* partials;          // [max_parts][dim]
   uint32_t* fold_li;         // [max_folds] owner (index into long_u) of each fold
   uint32_t* fold_idx;        // [max_folds] which group of kFoldWidth parts of that owner

@@ -315,8 +315,15 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
   }
 }
 
+// Window of the batch that part k of a segment of `parts` parts falls into.  A segment lists
+// its occurrences roughly in batch order (tile by tile), so part k of n covers roughly the
+// k-th n-th of the bags.
+__device__ inline uint32_t part_window(uint32_t k, uint32_t parts) {
+  return (uint32_t)(((unsigned long long)k * kWindows) / parts);
+}
+
 // After phases 2 and 3: every part of a long segment learns which ID it belongs to
-// (one block per long ID, its threads share the parts).
+// (one block per long ID, its threads share the parts), and the parts are counted by window.
 __global__ void __launch_bounds__(128)
 expand_parts_kernel(TableView tv, Work wk) {
   uint32_t n_long = tv.st->n_long;
@@ -325,16 +332,61 @@ expand_parts_kernel(TableView tv, Work wk) {
     const uint32_t parts = (wk.ulen[wk.long_u[li]] + kSegChunk - 1) / kSegChunk;
     const uint32_t p0 = wk.long_part0[li];
     if (p0 + parts > wk.max_parts) continue;
-    for (uint32_t p = threadIdx.x; p < parts; p += blockDim.x) wk.part_u[p0 + p] = li;
+    for (uint32_t p = threadIdx.x; p < parts; p += blockDim.x) {
+      wk.part_u[p0 + p] = li;
+      atomicAdd(&wk.win_count[part_window(p, parts)], 1u);
+    }
   }
 }
 
-// End of a mono_apply_grads call: fold the per-call counters into the totals.
-__global__ void finish_apply_kernel(DevState* st) {
+// The order the parts are reduced in: window by window, so that the parts in flight at any
+// time -- of different IDs -- gather gradient rows of the same stretch of bags, and a row
+// that several hot IDs need is fetched from DRAM once and found in L2 by the others.
+// Every block scans the window counts for itself; positions inside a window are handed out
+// by a per-window cursor (their order does not matter: each part has its own partial sum).
+__global__ void __launch_bounds__(kWindows)
+order_parts_kernel(TableView tv, Work wk) {
+  __shared__ uint32_t s_start[kWindows];
+  __shared__ uint32_t s_warp[kWindows / 32];
+  uint32_t n_parts = tv.st->n_parts;
+  if (n_parts > wk.max_parts) n_parts = wk.max_parts;
+  if (n_parts == 0) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t c = wk.win_count[threadIdx.x];
+  uint32_t incl = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  uint32_t before = 0;
+  for (int w = 0; w < warp; ++w) before += s_warp[w];
+  s_start[threadIdx.x] = before + incl - c;
+  __syncthreads();
+  uint32_t* cursor = wk.win_count + kWindows;
+  for (uint32_t p = blockIdx.x * blockDim.x + threadIdx.x; p < n_parts; p += gridDim.x * blockDim.x) {
+    const uint32_t li = wk.part_u[p];
+    const uint32_t parts = (wk.ulen[wk.long_u[li]] + kSegChunk - 1) / kSegChunk;
+    const uint32_t w = part_window(p - wk.long_part0[li], parts);
+    wk.part_order[s_start[w] + atomicAdd(&cursor[w], 1u)] = p;
+  }
+}
+
+// End of a mono_apply_grads call: fold the per-call counters into the totals
+// (commit = 0: a grouping that was prepared but never applied is only forgotten).
+__global__ void finish_apply_kernel(DevState* st, uint32_t* win_count, int commit) {
+  const bool had_parts = st->n_parts != 0;
+  __syncthreads();                                   // everyone has read n_parts before it is reset
+  if (had_parts)
+    for (uint32_t i = threadIdx.x; i < 2 * kWindows; i += blockDim.x) win_count[i] = 0;
   if (threadIdx.x == 0 && blockIdx.x == 0) {
-    st->sum_ids += st->n_valid_ids;
-    st->sum_unique += st->n_unique;
-    st->sum_new += st->n_insert;
+    if (commit) {
+      st->sum_ids += st->n_valid_ids;
+      st->sum_unique += st->n_unique;
+      st->sum_new += st->n_insert;
+    }
     st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_folds = 0; st->n_valid_ids = 0;
     st->seg_cursor = 0; st->n_multi = 0;
   }

@@ -28,11 +28,11 @@ using namespace mono;
 static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
   K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
-  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "sketch_add", "table_insert", "expand_parts",
+  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "sketch_add", "table_insert", "expand_parts", "order_parts",
   "scatter_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
@@ -48,6 +48,14 @@ struct mono_table {
   TableView tv{};
   Work wk{};
   cudaStream_t stream = nullptr;
+  // Two internal streams, ordered against `stream` with events only: one runs the
+  // ID-only part of a push that mono_prepare_push announced, the other the sweep.
+  cudaStream_t prep_stream = nullptr, sweep_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_prepared = nullptr, ev_keys = nullptr, ev_swept = nullptr;
+  bool sweep_pending = false;     // the sweep stream has work `stream` has not waited for yet
+  bool keys_idle = false;         // nothing launched on `stream` after ev_keys touches the key store
+  struct { const void* ids; int64_t n_ids; const void* off; int64_t n_bags; bool valid; } prep = {nullptr, 0, nullptr, 0, false};
+  uint32_t* occ_row = nullptr;    // scratch of the lookup: row of every occurrence
   int sm_count = 148;
   uint64_t key_cells = 0;
   int64_t last_now = -1;
@@ -89,8 +97,8 @@ void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
   dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
-  dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
-  dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec);
+  dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.part_order); dev_free(w.win_count); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
+  dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec); dev_free(t->occ_row);
   t->max_ids = t->max_bags = 0;
 }
 
@@ -102,21 +110,29 @@ cudaEvent_t take_event(mono_table* t) {
   cudaEventCreate(&e);
   return e;
 }
-void launch_begin(mono_table* t, int kid) {
+void launch_begin(mono_table* t, int kid, cudaStream_t s) {
   ++t->launches[kid];
-  if (t->timing) { t->open_event = take_event(t); cudaEventRecord(t->open_event, t->stream); }
+  if (t->timing) { t->open_event = take_event(t); cudaEventRecord(t->open_event, s); }
 }
-void launch_end(mono_table* t, int kid) {
+void launch_end(mono_table* t, int kid, cudaStream_t s) {
   if (t->timing) {
     cudaEvent_t stop = take_event(t);
-    cudaEventRecord(stop, t->stream);
+    cudaEventRecord(stop, s);
     t->pending.push_back({kid, {t->open_event, stop}});
     t->open_event = nullptr;
   }
 }
 // Every kernel of the hot calls is launched through this, so that launches can
-// be counted and, on request, timed one by one on the table's stream.
-#define LAUNCH(t, kid, ...) do { launch_begin((t), (kid)); __VA_ARGS__; launch_end((t), (kid)); } while (0)
+// be counted and, on request, timed one by one on the stream it runs on.
+#define LAUNCH_ON(t, s, kid, ...) do { launch_begin((t), (kid), (s)); __VA_ARGS__; launch_end((t), (kid), (s)); } while (0)
+#define LAUNCH(t, kid, ...) LAUNCH_ON(t, (t)->stream, kid, __VA_ARGS__)
+
+// The table's stream waits for whatever the sweep stream still has in flight.
+// Called by every entry point before it launches on, or synchronises, `stream`.
+void join_sweep(mono_table* t) {
+  if (t->sweep_pending) { cudaStreamWaitEvent(t->stream, t->ev_swept, 0); t->sweep_pending = false; }
+  t->keys_idle = false;
+}
 
 int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   if (max_ids <= t->max_ids && max_bags <= t->max_bags) return MONO_OK;
@@ -125,6 +141,8 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   if (max_ids < 1024) max_ids = 1024;
   if (max_bags < 1024) max_bags = 1024;
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  CUDA_TRY(t, cudaStreamSynchronize(t->prep_stream));     // a prepared grouping is lost with the scratch it lives in
+  if (t->prep.valid) { t->prep.valid = false; finish_apply_kernel<<<1, 256, 0, t->stream>>>(t->tv.st, t->wk.win_count, 0); }
   free_scratch(t);
   Work& w = t->wk;
   const size_t n = (size_t)max_ids;
@@ -140,17 +158,19 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   ALLOC(w.multi_list, n / 2 + 1); ALLOC(w.ins_list, n);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
-  ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts);
+  ALLOC(w.long_u, w.max_long); ALLOC(w.long_part0, w.max_long); ALLOC(w.part_u, w.max_parts); ALLOC(w.part_order, w.max_parts); ALLOC(w.win_count, 2 * kWindows);
   ALLOC(w.partials, (size_t)w.max_parts * t->tv.dim);
   w.max_folds = w.max_parts / kFoldWidth + w.max_long + 1;
   ALLOC(w.fold_li, w.max_folds); ALLOC(w.fold_idx, w.max_folds);
   ALLOC(t->stage_ids, n); ALLOC(t->stage_off, (size_t)max_bags + 1);
   ALLOC(t->stage_vec, (size_t)max_bags * t->tv.dim);
+  ALLOC(t->occ_row, n);
 #undef ALLOC
   w.primary_mask = (uint32_t)(primary - 1);
   w.secondary_mask = (uint32_t)(secondary - 1);
   init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(w.bset, slots);
   CUDA_TRY(t, cudaGetLastError());
+  CUDA_TRY(t, cudaMemsetAsync(w.win_count, 0, 2 * kWindows * sizeof(uint32_t), t->stream));
   t->max_ids = max_ids;
   t->max_bags = max_bags;
   return MONO_OK;
@@ -179,7 +199,7 @@ int dispatch_dim(uint32_t dim, F&& f) {
 int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
                   int64_t n_bags, float* out) {
   if (n_bags == 0) return MONO_OK;
-  uint32_t* occ_row = t->wk.occ_rank;      // scratch shared with the backward call (calls never overlap)
+  uint32_t* occ_row = t->occ_row;
   if (n_ids > 0) {
     int64_t blocks = (n_ids + 255) / 256;
     const int64_t cap = (int64_t)grid_for(t, 8) * 4;
@@ -199,22 +219,56 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
   });
 }
 
+// The part of a push that depends on the IDs alone: bag of every occurrence, and the
+// occurrences grouped by ID in the per-call set.
+int launch_group(mono_table* t, cudaStream_t s, const unsigned long long* ids, int64_t n_ids, const long long* off,
+                 int64_t n_bags) {
+  const TableView& tv = t->tv;
+  const Work& wk = t->wk;
+  LAUNCH_ON(t, s, K_FILL_BAG, fill_occ_bag_kernel<<<grid_for(t, 8), 256, 0, s>>>(off, n_bags, n_ids, wk.occ_bag, tv.st));
+  const int tiles = (int)((n_ids + kTileIds - 1) / kTileIds);
+  LAUNCH_ON(t, s, K_DEDUP, dedup_tile_kernel<<<tiles, kTileThreads, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
+                                                                          tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
+  CUDA_TRY(t, cudaGetLastError());
+  return MONO_OK;
+}
+
+// Forget a prepared grouping: wait for it, then empty the per-call set and the per-call counters.
+int discard_prepared(mono_table* t) {
+  if (!t->prep.valid) return MONO_OK;
+  t->prep.valid = false;
+  CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_prepared, 0));
+  const uint64_t slots = (uint64_t)t->wk.primary_mask + 1 + (uint64_t)t->wk.secondary_mask + 1;
+  init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(t->wk.bset, slots);
+  finish_apply_kernel<<<1, 256, 0, t->stream>>>(t->tv.st, t->wk.win_count, 0);
+  CUDA_TRY(t, cudaGetLastError());
+  return MONO_OK;
+}
+
 int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
                  int64_t n_bags, const float* grad, uint32_t now) {
-  if (n_ids == 0 || n_bags == 0) return MONO_OK;
+  int rc0 = MONO_OK;
+  if (t->prep.valid && t->prep.ids == ids && t->prep.n_ids == n_ids && t->prep.off == off && t->prep.n_bags == n_bags) {
+    // the grouping of exactly this batch is ready, or in flight on the preparation stream
+    t->prep.valid = false;
+    CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_prepared, 0));
+  } else {
+    if ((rc0 = discard_prepared(t)) != MONO_OK) return rc0;
+    if (n_ids == 0 || n_bags == 0) return MONO_OK;
+    if ((rc0 = launch_group(t, t->stream, ids, n_ids, off, n_bags)) != MONO_OK) return rc0;
+  }
   cudaStream_t s = t->stream;
   const TableView& tv = t->tv;
   const Work& wk = t->wk;
   const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
-  LAUNCH(t, K_FILL_BAG, fill_occ_bag_kernel<<<g8, 256, 0, s>>>(off, n_bags, n_ids, wk.occ_bag, tv.st));
-  const int tiles = (int)((n_ids + kTileIds - 1) / kTileIds);
-  LAUNCH(t, K_DEDUP, dedup_tile_kernel<<<tiles, kTileThreads, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
-                                                            tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   LAUNCH(t, K_EXPAND, expand_parts_kernel<<<g4, 128, 0, s>>>(tv, wk));
+  LAUNCH(t, K_ORDER, order_parts_kernel<<<64, kWindows, 0, s>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
+  // the rest of the call touches rows and scratch only: a sweep may run beside it
+  CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     LAUNCH(t, K_SCATTER, scatter_singletons_kernel<G, NV><<<g8 * 2, 256, 0, s>>>(tv, wk, grad, n_ids, n_bags));
@@ -224,8 +278,9 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   if (rc != MONO_OK) return rc;
   LAUNCH(t, K_FOLD, fold_partials_kernel<<<g4, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g8, kCombineThreads, 0, s>>>(tv, wk));
-  LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 32, 0, s>>>(tv.st));
+  LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 256, 0, s>>>(tv.st, wk.win_count, 1));
   CUDA_TRY(t, cudaGetLastError());
+  t->keys_idle = true;
   return MONO_OK;
 }
 
@@ -263,6 +318,11 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   if (cudaGetDevice(&dev) != cudaSuccess) return fail(MONO_ERR_CUDA);
   if (cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || t->sm_count < 1)
     return fail(MONO_ERR_CUDA);
+  if (cudaStreamCreateWithFlags(&t->prep_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess)
+    return fail(MONO_ERR_CUDA);
+  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_prepared, &t->ev_keys, &t->ev_swept})
+    if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return fail(MONO_ERR_CUDA);
 
   TableView& tv = t->tv;
   tv.bucket_mask = key_cells / kCellsPerBucket - 1;
@@ -307,6 +367,9 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
 int mono_table_destroy(mono_table* t) {
   if (!t) return MONO_ERR_ARG;
   cudaStreamSynchronize(t->stream);
+  if (t->prep_stream) { cudaStreamSynchronize(t->prep_stream); cudaStreamDestroy(t->prep_stream); }
+  if (t->sweep_stream) { cudaStreamSynchronize(t->sweep_stream); cudaStreamDestroy(t->sweep_stream); }
+  for (cudaEvent_t e : {t->ev_fork, t->ev_prepared, t->ev_keys, t->ev_swept}) if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
   free_scratch(t);
@@ -316,12 +379,14 @@ int mono_table_destroy(mono_table* t) {
 }
 
 int mono_reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
+  if (t) join_sweep(t);
   if (!t || max_ids < 0 || max_bags < 0 || max_ids >= (1ll << 31) || max_bags >= (1ll << 31)) return MONO_ERR_ARG;
   return reserve(t, max_ids, max_bags);
 }
 
 int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                      int64_t n_bags, float* out) {
+  if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
@@ -332,6 +397,7 @@ int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
 
 int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                      int64_t n_bags, const float* grad_pooled, int64_t now) {
+  if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && (!grad_pooled || !aligned(grad_pooled, 16))) return MONO_ERR_ARG;
@@ -342,16 +408,43 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
                       reinterpret_cast<const long long*>(slot_offsets), n_bags, grad_pooled, (uint32_t)now);
 }
 
+int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets, int64_t n_bags) {
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  if ((rc = discard_prepared(t)) != MONO_OK) return rc;
+  if (n_ids == 0 || n_bags == 0) return MONO_OK;
+  // after everything already on the table's stream (the previous push still owns the scratch) ...
+  CUDA_TRY(t, cudaEventRecord(t->ev_fork, t->stream));
+  CUDA_TRY(t, cudaStreamWaitEvent(t->prep_stream, t->ev_fork, 0));
+  // ... and beside everything that comes next on it
+  if ((rc = launch_group(t, t->prep_stream, reinterpret_cast<const unsigned long long*>(ids), n_ids,
+                         reinterpret_cast<const long long*>(slot_offsets), n_bags)) != MONO_OK) return rc;
+  CUDA_TRY(t, cudaEventRecord(t->ev_prepared, t->prep_stream));
+  t->prep = {ids, n_ids, slot_offsets, n_bags, true};
+  return MONO_OK;
+}
+
 static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices) {
   if (!t || n_slices == 0 || slice >= n_slices) return MONO_ERR_ARG;
   int rc = check_now(t, now);
   if (rc != MONO_OK) return rc;
   t->last_now = now;
   if (t->tv.ttl == 0) return MONO_OK;
+  // The sweep runs on its own stream.  It has to follow everything launched so far that
+  // touches the key store, the free list or the sketch; the tail of a mono_apply_grads
+  // (gradient reduction and row updates) touches none of them, so a sweep that comes
+  // straight after one starts as soon as that call's key-store work is done and runs
+  // beside the rest.  The next call on the table's stream waits for the sweep.
+  cudaStream_t s = t->sweep_stream;
+  if (!t->sweep_pending) {
+    // (while kernels are being timed one by one, the sweep waits for the whole stream instead)
+    if (!t->keys_idle || t->timing) CUDA_TRY(t, cudaEventRecord(t->ev_keys, t->stream));
+    CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_keys, 0));
+  }                                               // else: it follows the previous sweep, which waited already
   if (slice == 0 && t->tv.sketch_depth && now - t->sketch_epoch > (int64_t)t->tv.ttl) {
     // the sketch forgets in whole windows: cleared when more than ttl has passed since the last clearing
-    CUDA_TRY(t, cudaMemsetAsync(t->tv.sketch, 0, (size_t)t->tv.sketch_depth * (t->tv.sketch_mask + 1) * sizeof(unsigned int),
-                                t->stream));
+    CUDA_TRY(t, cudaMemsetAsync(t->tv.sketch, 0, (size_t)t->tv.sketch_depth * (t->tv.sketch_mask + 1) * sizeof(unsigned int), s));
     t->sketch_epoch = now;
   }
   const unsigned long long total = t->key_cells + kStashCells;
@@ -360,10 +453,12 @@ static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_s
   if (last > first) {
     unsigned long long blocks = (last - first + 255) / 256;
     if (blocks > (unsigned long long)grid_for(t, 8)) blocks = grid_for(t, 8);
-    LAUNCH(t, K_EXPIRE, expire_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, t->key_cells, first, last, (long long)now));
+    LAUNCH_ON(t, s, K_EXPIRE, expire_kernel<<<(int)blocks, 256, 0, s>>>(t->tv, t->key_cells, first, last, (long long)now));
   }
-  if (slice + 1 == n_slices) LAUNCH(t, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, t->stream>>>(t->tv));
+  if (slice + 1 == n_slices) LAUNCH_ON(t, s, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, s>>>(t->tv));
   CUDA_TRY(t, cudaGetLastError());
+  CUDA_TRY(t, cudaEventRecord(t->ev_swept, s));
+  t->sweep_pending = true;
   return MONO_OK;
 }
 
@@ -394,6 +489,7 @@ static int noalloc_scratch(mono_table* t, uint32_t** out) {
 
 int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                              int64_t n_bags, float* out) {
+  if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
@@ -424,6 +520,7 @@ int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, 
 
 int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                           int64_t n_bags, float* out) {
+  if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && !out) return MONO_ERR_ARG;
@@ -440,6 +537,7 @@ int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, con
 
 int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                           int64_t n_bags, const float* grad_pooled, int64_t now) {
+  if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && !grad_pooled) return MONO_ERR_ARG;
@@ -455,6 +553,7 @@ int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids, con
 }
 
 int mono_status(mono_table* t, mono_status_t* host_out) {
+  if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   DevState d;
   CUDA_TRY(t, cudaMemcpyAsync(&d, t->tv.st, sizeof(d), cudaMemcpyDeviceToHost, t->stream));
@@ -483,6 +582,7 @@ int mono_status(mono_table* t, mono_status_t* host_out) {
 }
 
 int mono_clear_errors(mono_table* t) {
+  if (t) join_sweep(t);
   if (!t) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->error_bits, 0, sizeof(unsigned int), t->stream));
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
@@ -491,6 +591,7 @@ int mono_clear_errors(mono_table* t) {
 
 int mono_probe(mono_table* t, const uint64_t* ids, int64_t n, uint8_t* resident, uint32_t* count,
                int64_t* last_seen) {
+  if (t) join_sweep(t);
   if (!t || n < 0 || (n > 0 && (!ids || !aligned(ids, 8)))) return MONO_ERR_ARG;
   if (n > 0) {
     probe_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(t->tv, reinterpret_cast<const unsigned long long*>(ids), n,
@@ -502,6 +603,7 @@ int mono_probe(mono_table* t, const uint64_t* ids, int64_t n, uint8_t* resident,
 }
 
 int mono_read_rows(mono_table* t, const uint64_t* ids, int64_t n, float* w, float* acc) {
+  if (t) join_sweep(t);
   if (!t || n < 0 || (n > 0 && (!ids || !aligned(ids, 8)))) return MONO_ERR_ARG;
   if ((w && !aligned(w, 16)) || (acc && !aligned(acc, 16))) return MONO_ERR_ARG;
   if (n > 0) {
@@ -515,6 +617,7 @@ int mono_read_rows(mono_table* t, const uint64_t* ids, int64_t n, float* w, floa
 
 int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_seen, uint8_t* resident,
                 float* w, float* acc, int64_t max_n, int64_t* n_out) {
+  if (t) join_sweep(t);
   if (!t || !n_out || max_n < 0 || (max_n > 0 && !ids)) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->export_n, 0, sizeof(unsigned long long), t->stream));
   export_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells,
@@ -529,6 +632,7 @@ int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_see
 }
 
 int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
+  if (t) join_sweep(t);
   if (!t) return MONO_ERR_ARG;
   if (new_key_cells == 0) new_key_cells = t->key_cells;
   if (!is_pow2(new_key_cells) || new_key_cells < 64 || new_key_cells > (1ull << 34)) return MONO_ERR_ARG;
@@ -566,6 +670,7 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
 }
 
 int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, int64_t* n_out) {
+  if (t) join_sweep(t);
   if (!t || !n_out || max_n < 0 || (max_n > 0 && (!ids || !w || !aligned(w, 16) || !aligned(ids, 8)))) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->export_n, 0, sizeof(unsigned long long), t->stream));
   export_touched_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells,
@@ -580,6 +685,7 @@ int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, i
 
 int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const int64_t* last_seen,
                 const uint8_t* resident, const float* w, const float* acc, int64_t n) {
+  if (t) join_sweep(t);
   if (!t || n < 0) return MONO_ERR_ARG;
   if (n == 0) return MONO_OK;
   if (!ids || !count || !last_seen || !resident || !aligned(ids, 8)) return MONO_ERR_ARG;
@@ -606,6 +712,7 @@ int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const
 }
 
 int mono_audit(mono_table* t, mono_audit_t* host_out) {
+  if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   std::memset(host_out, 0, sizeof(*host_out));
   unsigned int* marks = nullptr;
@@ -658,8 +765,10 @@ int mono_timing_enable(mono_table* t, int on) {
 }
 
 int mono_timing_read(mono_table* t, mono_timing_t* host_out, int reset) {
+  if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  CUDA_TRY(t, cudaStreamSynchronize(t->prep_stream));
   for (auto& p : t->pending) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, p.second.first, p.second.second) == cudaSuccess) t->kernel_ms[p.first] += ms;

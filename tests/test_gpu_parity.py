@@ -186,6 +186,69 @@ def test_expiry_sets_and_row_recycling():
     assert a["resident_cells"] + a["free_rows"] == cfg.capacity
 
 
+def _dev_batch(s):
+    return (torch.from_numpy(s.ids.view(np.int64)).cuda(), torch.from_numpy(s.offsets).cuda(),
+            torch.from_numpy(s.grad_pooled).cuda())
+
+
+def test_prepared_push_gives_the_same_table_as_the_oracle():
+    """mono_prepare_push before the lookup of the same batch: the grouping runs beside the
+    lookup, and lookup outputs and table state stay those of the oracle, step by step.  Also
+    the ways a preparation is dropped: a different batch is pushed, a second preparation
+    replaces the first, the scratch grows in between, the prepared batch is never pushed."""
+    cfg = wl.scaled(wl.CONFIGS["medium"], n_examples=1024, steps=12, ttl=3)
+    gpu, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
+    h = gpu.handle
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        ids, off, grad = _dev_batch(s)
+        other = _dev_batch(stream.step(t + 100))
+        if t % 4 == 1:                                   # prepared for another batch, then replaced
+            mb.mono_prepare_push(h, other[0], other[0].numel(), other[1], cfg.n_bags)
+        if t % 4 != 3:
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+        else:                                            # the wrong batch stays prepared: the push must drop it
+            mb.mono_prepare_push(h, other[0], other[0].numel(), other[1], cfg.n_bags)
+        mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+        if t == 5:                                       # the scratch is reallocated under a prepared grouping
+            mb.mono_reserve(h, 4 * ids.numel(), 4 * cfg.n_bags)
+        mb.mono_apply_grads(h, ids, ids.numel(), off, cfg.n_bags, grad, t)
+        assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
+        if t % 2:
+            gpu.expire(t)
+            cpu.expire(t)
+        assert_state_equal(gpu, cpu, f"step {t}")
+    s = stream.step(50)
+    ids, off, grad = _dev_batch(s)
+    mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)       # never pushed
+    mb.mono_prepare_push(h, ids, 0, off[:1], 0)                      # an empty batch prepares nothing
+    st = gpu.status()
+    assert st["error_bits"] == 0 and st["sum_ids"] == cpu_sum_ids(stream, cfg.steps)
+    assert_state_equal(gpu, cpu, "after an abandoned preparation")
+    assert_audit_ok(gpu)
+    gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, cfg.steps)      # and the table still works
+    cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, cfg.steps)
+    assert_state_equal(gpu, cpu, "push after an abandoned preparation")
+
+
+def cpu_sum_ids(stream, steps):
+    return sum(int((stream.step(t).ids != np.uint64(wl.RESERVED_ID)).sum()) for t in range(steps))
+
+
+def test_prepared_push_with_malformed_offsets_is_flagged():
+    gpu = mb.MonoTable(1 << 10, 8, 1, 0)
+    ids = torch.arange(1, 9, dtype=torch.int64, device="cuda")
+    off = torch.tensor([0, 3, 2, 8], dtype=torch.int64, device="cuda")
+    grad = torch.ones((3, 8), dtype=torch.float32, device="cuda")
+    mb.mono_prepare_push(gpu.handle, ids, 8, off, 3)
+    mb.mono_apply_grads(gpu.handle, ids, 8, off, 3, grad, 0)
+    assert gpu.status()["error_bits"] & mb.MONO_DEV_BAD_OFFSETS
+    assert_audit_ok(gpu)
+
+
 @pytest.mark.parametrize("n_slices", [1, 3, 7, 64])
 def test_sliced_sweep_equals_one_full_sweep(n_slices):
     cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=8, ttl=2, key_cells=1 << 16)
