@@ -61,7 +61,8 @@ KERNEL_SOURCES = {
     "dedup_tile": ("kernels_dedup.cuh", "table_layout.cuh"),
     "table_update": ("kernels_table.cuh", "kernels_forward.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "table_insert": ("kernels_table.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
-    "scatter_singletons": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "update_singletons": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "file_segments": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "reduce_adagrad": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "combine_adagrad": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "fold_partials": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
@@ -216,8 +217,9 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0):
         "dedup_tile": 8 * n + 24 * n,                        # ids + (key, index) pairs written and read
         "table_update": 64 * u,                              # probe + count/stamp read-modify-write
         "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
-        "scatter_singletons": 4 * d * b + 16 * d * ur1,      # gradients once + rows of IDs seen once
-        "reduce_adagrad": 16 * d * (ur - ur1),               # rows of repeated IDs (gradients counted above)
+        "update_singletons": 20 * d * ur1,                   # IDs seen once: gradient row, row and accumulator in and out
+        "reduce_adagrad": 16 * d * (ur - ur1) + 4 * d * max(b - ur1, 0),   # rows of repeated IDs + the other gradient rows, once
+        "file_segments": 0,
         "expand_parts": 0, "order_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
         "expire": 16 * sweep_cells,                          # one streaming read of the swept cells
     }
@@ -228,7 +230,7 @@ KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
     "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
     "table_update": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
-    "scatter_singletons": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
+    "update_singletons": "adagrad", "file_segments": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
     "combine_adagrad": "adagrad", "expire": "expire",
 }
 

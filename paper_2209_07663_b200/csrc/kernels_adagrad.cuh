@@ -6,10 +6,9 @@
 //
 // Three cases, by how often the ID occurs in the batch:
 //  - once (most distinct IDs of a long-tailed batch): its gradient is the
-//    pooled gradient of its one bag, so scatter_singletons_kernel updates the
-//    row straight from the occurrence, in bag order, and the gradient rows
-//    stream through once;
-//  - 2 .. kSegChunk times: scatter_singletons_kernel drops each occurrence's
+//    pooled gradient of its one bag, so update_singletons_kernel updates the
+//    row straight from that bag's gradient row;
+//  - 2 .. kSegChunk times: file_segments_kernel drops each occurrence's
 //    bag into the ID's segment of bag_of_sorted[], and one lane group of
 //    reduce_adagrad_kernel gathers the segment's gradient rows;
 //  - more (the head of the Zipf distribution: one ID can own several percent of
@@ -105,39 +104,50 @@ __device__ inline void reduce_segment(const Work& wk, const float* __restrict__ 
   }
 }
 
-// One warp per 32 consecutive occurrences.  Each lane looks its occurrence up in
-// the per-call set: an occurrence of a repeated ID that has a row is filed
-// under its ID; the lanes whose ID occurs once and has a row are then served
-// in turn by lane groups of G, which read the bag's gradient row, the table
-// row and its accumulator, and write both back updated.
+// Every occurrence of a repeated ID that has a row is filed under its ID: its bag goes
+// into the ID's segment of bag_of_sorted[], at the occurrence's rank.  (The slot of an
+// ID that occurs once has been emptied by then, so its occurrence finds nothing.)
+__global__ void __launch_bounds__(256)
+file_segments_kernel(Work wk, long long n_ids, long long n_bags) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
+    const uint32_t s = wk.occ_slot[j];
+    if (s == kNoSlot) continue;
+    const BatchSlot bs = wk.bset[s];
+    if (bs.key == kEmptyKey || bs.b == kNoRow) continue;
+    const uint32_t bag = wk.occ_bag[j];
+    if (bag < n_bags) wk.bag_of_sorted[bs.a + wk.occ_rank[j]] = bag;
+  }
+}
+
+// The IDs that occur once in the batch (most distinct IDs of a long-tailed batch): the
+// gradient of such an ID is the pooled gradient of its one bag, so its row is updated
+// straight from there.  One warp per 32 consecutive distinct IDs, which are numbered in
+// the order the batch first shows them, so the gradient rows are read roughly in order;
+// the lanes whose ID occurs once and has a row are served in turn by lane groups of G,
+// which read the bag's gradient row, the table row and its accumulator, and write both
+// back updated.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-scatter_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_ids, long long n_bags) {
+update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
   constexpr int kGroups = 32 / G;
   const int lane = threadIdx.x & 31;
   const int gl = lane % G, grp = lane / G;
-  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const long long n_rounds = (n_ids + 31) / 32;
+  const uint32_t n = tv.st->n_unique;
+  const uint32_t n_warps = (gridDim.x * blockDim.x) >> 5;
+  const uint32_t n_rounds = (n + 31) / 32;
   unsigned int n_single = 0;
-  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rounds; r += n_warps) {
-    const long long j = r * 32 + lane;
+  for (uint32_t r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rounds; r += n_warps) {
+    const uint32_t u = r * 32 + lane;
     uint32_t row_word = kNoRow, bag = 0;
     unsigned long long id = 0;
     bool single = false;
-    if (j < n_ids) {
-      const uint32_t s = wk.occ_slot[j];
-      if (s != kNoSlot) {
-        const BatchSlot bs = wk.bset[s];
-        bag = wk.occ_bag[j];
-        if (bs.a == kSingleton) {
-          // the only occurrence of its ID: nobody else needs the slot, empty it for the next call
-          BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
-          wk.bset[s] = e;
-        }
-        if (bs.b != kNoRow && bag < n_bags) {
-          if (bs.a == kSingleton) { single = true; row_word = bs.b; id = bs.key; }
-          else wk.bag_of_sorted[bs.a + wk.occ_rank[j]] = bag;
-        }
+    if (u < n && wk.ulen[u] == 1u) {
+      row_word = wk.urow[u];
+      if (row_word != kNoRow) {
+        bag = wk.occ_bag[wk.uocc[u]];
+        single = bag < n_bags;
+        if (row_word & kFreshBit) id = wk.uid[u];
       }
     }
     unsigned todo = __ballot_sync(0xFFFFFFFFu, single);

@@ -21,8 +21,9 @@
 namespace mono {
 
 // One slot of the per-call set.  `a` is the ID's multiplicity while the batch
-// is being counted; once the table phases have run it is the start of the ID's
-// segment in bag_of_sorted[] (or kSingleton), and `b` is the ID's row word.
+// is being counted; once the table phases have run, the slot of an ID that
+// occurs once is empty again, and that of a repeated ID holds the start of its
+// segment in bag_of_sorted[] in `a` and its row word in `b`.
 struct __align__(16) BatchSlot {
   unsigned long long key;
   unsigned int a;
@@ -30,7 +31,6 @@ struct __align__(16) BatchSlot {
 };
 
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
-constexpr uint32_t kSingleton = 0xFFFFFFFFu;   // BatchSlot::a of an ID that occurs once in the batch
 constexpr uint32_t kSegChunk = 64;             // longest segment one lane group reduces alone
 constexpr uint32_t kFoldWidth = 64;           // parts added up by one block of fold_partials_kernel
 constexpr int kTileIds = 512;                  // occurrences per block of dedup_tile_kernel
@@ -54,6 +54,7 @@ struct Work {
   uint32_t* bag_of_sorted;   // [max_ids] bags of the occurrences of repeated IDs, grouped by ID
   unsigned long long* uid;   // [max_ids] distinct IDs
   uint32_t* uslot;           // [max_ids] slot of each distinct ID
+  uint32_t* uocc;            // [max_ids] one occurrence of each distinct ID (the occurrence, if there is only one)
   uint32_t* useg;            // [max_ids] start of the ID's segment in bag_of_sorted
   uint32_t* ulen;            // [max_ids] multiplicity of the ID in this batch
   uint32_t* urow;            // [max_ids] row word per distinct ID (kNoRow / row | kFreshBit)
@@ -116,6 +117,7 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   __shared__ unsigned long long s_key[kTileSlots];
   __shared__ unsigned int s_cnt[kTileSlots];     // multiplicity in the tile, then base rank
   __shared__ unsigned int s_gslot[kTileSlots];   // the ID's slot in the global set
+  __shared__ unsigned int s_occ[kTileSlots];     // one of the tile's occurrences of the ID
   __shared__ unsigned long long s_warp[kTileThreads / 32];
   __shared__ unsigned int s_ubase;
 
@@ -146,6 +148,7 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
       }
       my_slot[k] = s;
       my_rank[k] = atomicAdd(&s_cnt[s], 1u);
+      s_occ[s] = (unsigned int)j;                    // any of them will do
     }
   }
   __syncthreads();
@@ -223,6 +226,7 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
     if (is_new[k]) {
       wk.uid[my_u] = tid_[k];
       wk.uslot[my_u] = g[k];
+      wk.uocc[my_u] = s_occ[k * kTileThreads + threadIdx.x];
       ++my_u;
     }
   }

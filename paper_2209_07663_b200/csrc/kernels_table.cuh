@@ -164,7 +164,9 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
       where->meta = make_meta(now, low);
       wk.urow[u] = row_word;
       wk.useg[u] = rv.seg_start;
-      BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kSingleton; bs.b = row_word;
+      // a repeated ID leaves its segment and row in the slot for its occurrences to find; an ID that
+      // occurs once is updated from urow/uocc, and nobody needs its slot any more: empty it for the next call
+      BatchSlot bs; bs.key = m > 1 ? id : kEmptyKey; bs.a = m > 1 ? rv.seg_start : 0u; bs.b = m > 1 ? row_word : 0u;
       wk.bset[slot] = bs;
       if (m > 1) wk.multi_list[rv.multi_pos] = u;
       if (row_word != kNoRow) {
@@ -290,7 +292,7 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
     wk.urow[u] = row_word;
     wk.useg[u] = rv.seg_start;
-    BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kSingleton; bs.b = row_word;
+    BatchSlot bs; bs.key = m > 1 ? id : kEmptyKey; bs.a = m > 1 ? rv.seg_start : 0u; bs.b = m > 1 ? row_word : 0u;
     wk.bset[wk.uslot[u]] = bs;
     if (m > 1) wk.multi_list[rv.multi_pos] = u;
     if (row_word != kNoRow) {

@@ -28,12 +28,12 @@ using namespace mono;
 static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_SCATTER, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_FILE, K_SINGLES, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
   K_STASH_TRIM, K_COUNT
 };
 static const char* const kKernelNames[K_COUNT] = {
   "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "sketch_add", "table_insert", "expand_parts", "order_parts",
-  "scatter_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
+  "file_segments", "update_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
 
@@ -96,7 +96,7 @@ void dev_free(T*& p) { if (p) { cudaFree(p); p = nullptr; } }
 void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
-  dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
+  dev_free(w.uid); dev_free(w.uslot); dev_free(w.uocc); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
   dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.part_order); dev_free(w.win_count); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec); dev_free(t->occ_row);
   t->max_ids = t->max_bags = 0;
@@ -154,7 +154,7 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
 #define ALLOC(p, cnt) if ((rc = dev_alloc(t, &(p), (cnt))) != MONO_OK) { free_scratch(t); return rc; }
   ALLOC(w.bset, slots);
   ALLOC(w.occ_slot, n); ALLOC(w.occ_rank, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
-  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n);
+  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.uocc, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n);
   ALLOC(w.multi_list, n / 2 + 1); ALLOC(w.ins_list, n);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
@@ -271,7 +271,8 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
-    LAUNCH(t, K_SCATTER, scatter_singletons_kernel<G, NV><<<g8 * 2, 256, 0, s>>>(tv, wk, grad, n_ids, n_bags));
+    LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
+    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
     LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
