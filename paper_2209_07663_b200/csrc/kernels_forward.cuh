@@ -109,28 +109,55 @@ __device__ inline bool thread_lookup(const TableView& tv, unsigned long long id,
 }
 
 // Forward, step 1: one thread per ID occurrence resolves the ID to its row
-// index (kNoRow when the ID has none).  Every occurrence is independent, so
-// the random bucket reads of a whole batch are in flight together.  (Measured
-// against quad-cooperative variants: the shuffles those need cost more issue
-// slots than the extra L1 wavefronts of four 16-byte loads per thread.)
+// index; an ID without a row gets the index of the table's all-zero row (one
+// past the capacity), so that step 2 can add rows without asking.  Every
+// occurrence is independent, so the random bucket reads of a whole batch are in
+// flight together.  (Measured against quad-cooperative variants: the shuffles
+// those need cost more issue slots than the extra L1 wavefronts of four 16-byte
+// loads per thread.)
 __global__ void __launch_bounds__(256)
 probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
                   uint32_t* __restrict__ occ_row) {
   const unsigned stash_hw = tv.st->stash_hw;
+  const uint32_t zero_row = (uint32_t)tv.capacity;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
     const unsigned long long id = ids[j];
     unsigned long long meta = 0;
-    uint32_t row = kNoRow;
+    uint32_t row = zero_row;
     if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) row = meta_row(meta);
     occ_row[j] = row;
+  }
+}
+
+// sum += rows idx[0..K), in that order; all K loads are issued before the first add.
+template <int K, int G, int NV>
+__device__ inline void add_rows(const TableView& tv, const uint32_t* __restrict__ idx, int gl, float4 (&sum)[NV]) {
+  uint32_t row[K];
+#pragma unroll
+  for (int k = 0; k < K; ++k) row[k] = __ldg(idx + k);
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const uint32_t c4 = gl + v * G;
+    if (c4 * 4u < tv.dim) {
+      float4 x[K];
+#pragma unroll
+      for (int k = 0; k < K; ++k) x[k] = __ldg(reinterpret_cast<const float4*>(tv.w_row(row[k])) + c4);
+#pragma unroll
+      for (int k = 0; k < K; ++k) { sum[v].x += x[k].x; sum[v].y += x[k].y; sum[v].z += x[k].z; sum[v].w += x[k].w; }
+    }
   }
 }
 
 // Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
 // dim so that a lane owns NV 16-byte column vectors) adds up the rows of the
 // bag's IDs, in ID order, so the fp32 sum has one fixed order.  The row
-// indices are known, so the loads of up to four rows are issued together.
+// indices are known, so the loads of four rows are issued together; what is
+// left of the bag after the batches of four is added in one batch of its exact
+// size.  The kernel is bound by instruction issue, not by memory, so there are
+// no per-row validity tests (step 1 points an ID without a row at the zero row)
+// and no loads or adds for padding (measured: batches padded with the zero row
+// 0.31 ms on the largest configuration, exact tails 0.26 ms).
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long n_ids,
@@ -148,25 +175,15 @@ gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long
     float4 sum[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) sum[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (long long base = lo; base < hi; base += 4) {
-      uint32_t row[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) row[k] = base + k < hi ? __ldg(occ_row + base + k) : kNoRow;
-#pragma unroll
-      for (int v = 0; v < NV; ++v) {
-        const uint32_t c4 = gl + v * G;
-        if (c4 * 4u < dim) {
-          float4 x[4];
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            x[k] = row[k] != kNoRow ? __ldg(reinterpret_cast<const float4*>(tv.w_row(row[k])) + c4)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            if (row[k] != kNoRow) { sum[v].x += x[k].x; sum[v].y += x[k].y; sum[v].z += x[k].z; sum[v].w += x[k].w; }
-          }
-        }
-      }
+    const uint32_t* idx = occ_row + lo;
+    const uint32_t n = (uint32_t)(hi - lo);              // a call has fewer than 2^31 IDs
+    uint32_t i = 0;
+    for (; i + 4 <= n; i += 4) add_rows<4, G, NV>(tv, idx + i, gl, sum);
+    switch (n - i) {
+      case 3: add_rows<3, G, NV>(tv, idx + i, gl, sum); break;
+      case 2: add_rows<2, G, NV>(tv, idx + i, gl, sum); break;
+      case 1: add_rows<1, G, NV>(tv, idx + i, gl, sum); break;
+      default: break;
     }
     float4* dst = reinterpret_cast<float4*>(out + bag * (long long)dim);
 #pragma unroll

@@ -338,7 +338,11 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   tv.init_key1 = (uint32_t)(o.seed >> 32);
   if ((rc = dev_alloc(t, &tv.cells, key_cells)) != MONO_OK) return fail(rc);
   if ((rc = dev_alloc(t, &tv.stash, kStashCells)) != MONO_OK) return fail(rc);
-  if ((rc = dev_alloc(t, &tv.rows, (size_t)capacity * 2 * dim)) != MONO_OK) return fail(rc);
+  // one row more than the capacity: row index `capacity` is never handed out and stays all zero
+  // (the lookup adds it for an ID that has no row)
+  if ((rc = dev_alloc(t, &tv.rows, ((size_t)capacity + 1) * 2 * dim)) != MONO_OK) return fail(rc);
+  if (cudaMemsetAsync(tv.rows + (size_t)capacity * 2 * dim, 0, (size_t)2 * dim * sizeof(float), t->stream) != cudaSuccess)
+    return fail(MONO_ERR_CUDA);
   if ((rc = dev_alloc(t, &tv.free_rows, capacity)) != MONO_OK) return fail(rc);
   if ((rc = dev_alloc(t, &tv.st, 1)) != MONO_OK) return fail(rc);
   tv.sketch_depth = o.sketch_depth;

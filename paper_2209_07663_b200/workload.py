@@ -126,6 +126,11 @@ CONFIGS = {
     "large": Config("large", capacity=1 << 26, dim=64, filter_threshold=5, ttl=1000,
                     n_examples=16384, n_slots=100, bag_len=("geometric", 5.0, 1, 20),
                     zipf_s=1.05, n_distinct=1 << 30, steps=100, key_cells=1 << 30),
+    # the batch mix of `large` (half the examples) on a 3 GB table with the same row and key loads:
+    # the case profiler captures that replay every kernel many times are taken on
+    "large_profile": Config("large_profile", capacity=1 << 22, dim=64, filter_threshold=5, ttl=100,
+                            n_examples=8192, n_slots=100, bag_len=("geometric", 5.0, 1, 20),
+                            zipf_s=1.05, n_distinct=1 << 26, steps=100, key_cells=1 << 26),
     "drift": Config("drift", capacity=1 << 26, dim=32, filter_threshold=3, ttl=200,
                     n_examples=16384, n_slots=50, bag_len=("geometric", 5.0, 1, 20),
                     zipf_s=1.2, n_distinct=1 << 30, steps=400, key_cells=1 << 29,
