@@ -480,7 +480,7 @@ def run_ours(args):
 def run_multi(args):
     """The mixed-dim multi-table configuration: 8 independent tables, each on its own CUDA
     stream, so that the latency-bound kernels of one table overlap the bandwidth-bound kernels
-    of another.  A step = lookup_pool + apply_grads on every table."""
+    of another.  A step = lookup_pool + apply_grads + one slice of the expiry sweep on every table."""
     import torch
     from paper_2209_07663_b200 import binding as mb
     if not torch.cuda.is_available():
@@ -493,7 +493,7 @@ def run_multi(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
-    K, W = args.steps, args.warmup
+    K, W, S = args.steps, args.warmup, args.sweep_slices
     cfgs = [rank_config(c, rank) for c in wl.multi_table_configs()]
     streams = [torch.cuda.Stream(device=dev) for _ in cfgs]
     tables, now0 = [], []
@@ -534,8 +534,12 @@ def run_multi(args):
     def step(i, serial):
         for ti, (cfg, t) in enumerate(zip(cfgs, tables)):
             ids, off, grad = batches[ti][i]
+            if args.prepare:
+                mb.mono_prepare_push(t.handle, ids, ids.numel(), off, cfg.n_bags)
             mb.mono_lookup_pool(t.handle, ids, ids.numel(), off, cfg.n_bags, outs[ti])
             mb.mono_apply_grads(t.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0[ti] + 1 + i)
+            if S > 0:
+                mb.mono_expire_slice(t.handle, now0[ti] + 1 + i, i % S, S)
             if serial:
                 streams[ti].synchronize()
 
@@ -574,7 +578,7 @@ def run_multi(args):
         n = b["sum_ids"] - a["sum_ids"]
         u, ur = b["sum_unique"] - a["sum_unique"], b["sum_unique_resident"] - a["sum_unique_resident"]
         ur1, unew = b["sum_single_resident"] - a["sum_single_resident"], b["sum_new"] - a["sum_new"]
-        alg += algorithmic_bytes(n, cfg.n_bags * K, u, ur, ur1, unew, cfg.dim)[1]
+        alg += algorithmic_bytes(n, cfg.n_bags * K, u, ur, ur1, unew, cfg.dim, K * cfg.key_cells // S if S > 0 else 0)[1]
     if rank == 0:
         peak, peak_kind = measured_peaks()
         achieved = alg / (ms * 1e-3) / 1e9
@@ -588,7 +592,8 @@ def run_multi(args):
                                                          "key_load": s0["n_tracked"] / c.key_cells}
                                                         for c, s0 in zip(cfgs, before)],
                        "examples_per_step": cfgs[0].n_examples, "slots_total": sum(c.n_slots for c in cfgs),
-                       "ids_per_step": n_ids / K, "prefill": "steady state of each stream", "sweep": "none",
+                       "ids_per_step": n_ids / K, "prefill": "steady state of each stream",
+                       "sweep": f"every step sweeps 1/{S} of every key store" if S > 0 else "none",
                        "l2": "every step reads fresh batches larger than L2",
                        "parallelism": "8 tables on 8 CUDA streams of one GPU"},
             "serial": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,

@@ -142,7 +142,7 @@ CONFIGS = {
 MULTI_TABLE_DIMS = (8, 16, 16, 32, 32, 64, 64, 128)
 MULTI_TABLE_CAPACITY_LOG2 = (27, 26, 25, 24, 23, 22, 21, 20)
 MULTI_TABLE_ZIPF_S = (0.9, 0.95, 1.0, 1.05, 1.1, 1.2, 1.25, 1.3)
-MULTI_TABLE_SLOTS = (33, 23, 16, 12, 9, 11, 9, 7)
+MULTI_TABLE_SLOTS = (33, 22, 16, 12, 9, 12, 9, 7)
 MULTI_TABLE_UNIVERSE_LOG2_EXTRA = (2, 2, 2, 2, 2, 2, 1, 1)
 
 
