@@ -1,6 +1,6 @@
 """Parity at the full size of the `large` configuration, in the launch configuration the
 benchmark times: table pre-filled to the stream's steady state (hundreds of millions of
-tracked IDs, ~0.9 row load), whole batches of 1.6 M bags through mono_lookup_pool and
+tracked IDs, ~0.9 row load), whole batches of 1.6 M bags through mono_prepare_push, mono_lookup_pool and
 mono_apply_grads, then the sweep in the 32 slices the benchmark spreads over its steps
 (here all at one time, which makes them equal to one mono_expire).
 
@@ -85,6 +85,7 @@ def test_large_config_full_size_sampled_parity():
         grad = torch.from_numpy(s.grad_pooled).cuda()
         # the oracle's view: same bags, IDs outside the sample become padding
         masked = np.where(np.isin(s.ids, sample_ids), s.ids, np.uint64(mb.MONO_RESERVED_ID))
+        mb.mono_prepare_push(gpu.handle, ids, ids.numel(), off, cfg.n_bags)      # as the benchmark does
         mb.mono_lookup_pool(gpu.handle, ids, ids.numel(), off, cfg.n_bags, out)
         want = cpu.lookup_pool(masked, s.offsets)
         bags = bags_per_step[t]
