@@ -531,7 +531,25 @@ def run_multi(args):
         outs.append(torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device=dev))
     torch.cuda.synchronize()
 
+    handles = [t.handle for t in tables]
+
     def step(i, serial):
+        if not serial:
+            # the grouped calls: every table on its own stream, one C call for all eight
+            gs = torch.cuda.current_stream().cuda_stream
+            now = [n0 + 1 + i for n0 in now0]
+            assert len(set(now)) == 1
+            if args.prepare:
+                for ti, t in enumerate(tables):
+                    ids, off, _ = batches[ti][i]
+                    mb.mono_prepare_push(t.handle, ids, ids.numel(), off, cfgs[ti].n_bags)
+            mb.mono_group_lookup_pool(handles, [b[i][0] for b in batches], [b[i][1] for b in batches], outs, gs)
+            mb.mono_group_apply_grads(handles, [b[i][0] for b in batches], [b[i][1] for b in batches],
+                                      [b[i][2] for b in batches], now[0], gs)
+            if S > 0:
+                for ti, t in enumerate(tables):
+                    mb.mono_expire_slice(t.handle, now[0], i % S, S)
+            return
         for ti, (cfg, t) in enumerate(zip(cfgs, tables)):
             ids, off, grad = batches[ti][i]
             if args.prepare:
@@ -595,7 +613,7 @@ def run_multi(args):
                        "ids_per_step": n_ids / K, "prefill": "steady state of each stream",
                        "sweep": f"every step sweeps 1/{S} of every key store" if S > 0 else "none",
                        "l2": "every step reads fresh batches larger than L2",
-                       "parallelism": "8 tables on 8 CUDA streams of one GPU"},
+                       "parallelism": "8 tables on 8 CUDA streams of one GPU, one grouped call per step and direction"},
             "serial": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,
                        "what": "the same calls with each table's stream drained before the next table starts"},
             "gpu_launches": launches, "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],

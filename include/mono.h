@@ -241,6 +241,27 @@ int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const i
                       int64_t n_bags);
 
 /*
+ * Grouped calls: one call for several tables (Section 3.1: a production model holds many
+ * embedding tables of very uneven size).  Table i gets batch i: `tables`, `ids`, `n_ids`,
+ * `slot_offsets`, `n_bags`, `out` / `grad_pooled` are HOST arrays of `n_tables` entries whose
+ * elements are what the single-table call takes (device pointers, sizes).  Every table works
+ * on its own stream (the one it was created with), so the tables run beside one another --
+ * the short, latency-bound kernels of a small table fill the gaps of a large one -- if they
+ * were created with different streams; with one shared stream the calls are still correct
+ * and run one after the other.  `group_stream` orders the group as a whole: the tables start
+ * after everything issued on it so far, and it waits for all of them, so work issued on it
+ * afterwards sees every table's results.  The same table must not appear twice.
+ * Results are those of the n_tables single calls.  Returns the first error met (tables after
+ * it are not started); MONO_ERR_ARG for n_tables < 0 or a null array.
+ */
+int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
+                           const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
+                           float* const* out, void* group_stream);
+int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
+                           const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
+                           const float* const* grad_pooled, int64_t now, void* group_stream);
+
+/*
  * Incremental form of mono_expire: sweeps slice `slice` of `n_slices` equal parts of the key
  * store (the last slice also covers the overflow stash), so that the cost of a full sweep can
  * be spread over n_slices training steps.  Calling it for slice = 0 .. n_slices-1 with the

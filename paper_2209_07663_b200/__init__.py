@@ -6,7 +6,7 @@
 from . import workload  # noqa: F401
 from .binding import (  # noqa: F401
     MonoError, MonoTable, load_library, mono_apply_grads, mono_apply_grads_host, mono_audit,
-    mono_expire, mono_expire_slice, mono_export, mono_prepare_push, mono_export_touched, mono_import, mono_lookup_pool, mono_lookup_pool_host,
+    mono_expire, mono_expire_slice, mono_export, mono_prepare_push, mono_group_lookup_pool, mono_group_apply_grads, mono_export_touched, mono_import, mono_lookup_pool, mono_lookup_pool_host,
     mono_lookup_pool_noalloc, mono_probe, mono_rehash,
     mono_read_rows, mono_reserve, mono_status, mono_table_create, mono_table_destroy, mono_timing_enable,
     mono_timing_read,

@@ -26,6 +26,7 @@ EXPORTS = [
     "mono_expire", "mono_lookup_pool_host", "mono_apply_grads_host", "mono_status", "mono_clear_errors",
     "mono_probe", "mono_read_rows", "mono_export", "mono_import", "mono_audit", "mono_last_cuda_error",
     "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc", "mono_export_touched", "mono_rehash", "mono_expire_slice", "mono_prepare_push",
+    "mono_group_lookup_pool", "mono_group_apply_grads",
 ]
 
 
@@ -96,6 +97,8 @@ def load_library(path: Optional[str] = None):
         "mono_expire": (ci, [vp, i64]),
         "mono_prepare_push": (ci, [vp, vp, i64, vp, i64]),
         "mono_expire_slice": (ci, [vp, i64, u32, u32]),
+        "mono_group_lookup_pool": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp]),
+        "mono_group_apply_grads": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp, i64, vp]),
         "mono_lookup_pool_host": (ci, [vp, vp, i64, vp, i64, vp]),
         "mono_apply_grads_host": (ci, [vp, vp, i64, vp, i64, vp, i64]),
         "mono_status": (ci, [vp, ctypes.POINTER(mono_status_t)]),
@@ -201,6 +204,33 @@ def mono_expire(t: int, now: int) -> None:
 
 def mono_prepare_push(t: int, ids, n_ids: int, slot_offsets, n_bags: int) -> None:
     _check("mono_prepare_push", load_library().mono_prepare_push(t, _ptr(ids), n_ids, _ptr(slot_offsets), n_bags), t)
+
+
+def _group_args(handles, ids, slot_offsets, vectors):
+    """Host arrays of the grouped calls: one entry per table."""
+    n = len(handles)
+    if not (len(ids) == len(slot_offsets) == len(vectors) == n):
+        raise ValueError("grouped calls take one batch per table")
+    ptrs = ctypes.c_void_p * n
+    i64s = ctypes.c_int64 * n
+    return (n, ptrs(*handles), ptrs(*[_ptr(x) for x in ids]), i64s(*[x.numel() for x in ids]),
+            ptrs(*[_ptr(x) for x in slot_offsets]), i64s(*[x.numel() - 1 for x in slot_offsets]),
+            ptrs(*[_ptr(x) for x in vectors]))
+
+
+def mono_group_lookup_pool(handles, ids, slot_offsets, outs, group_stream: int = 0) -> None:
+    """ids / slot_offsets / outs: lists of device tensors, one per table."""
+    n, tp, ip, nip, op, nbp, vp_ = _group_args(handles, ids, slot_offsets, outs)
+    code = load_library().mono_group_lookup_pool(n, tp, ip, nip, op, nbp, vp_, group_stream or None)
+    if code != 0:
+        raise MonoError("mono_group_lookup_pool", code)
+
+
+def mono_group_apply_grads(handles, ids, slot_offsets, grads, now: int, group_stream: int = 0) -> None:
+    n, tp, ip, nip, op, nbp, vp_ = _group_args(handles, ids, slot_offsets, grads)
+    code = load_library().mono_group_apply_grads(n, tp, ip, nip, op, nbp, vp_, now, group_stream or None)
+    if code != 0:
+        raise MonoError("mono_group_apply_grads", code)
 
 
 def mono_expire_slice(t: int, now: int, slice_index: int, n_slices: int) -> None:

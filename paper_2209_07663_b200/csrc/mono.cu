@@ -52,6 +52,7 @@ struct mono_table {
   // ID-only part of a push that mono_prepare_push announced, the other the sweep.
   cudaStream_t prep_stream = nullptr, sweep_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_prepared = nullptr, ev_keys = nullptr, ev_swept = nullptr;
+  cudaEvent_t ev_group = nullptr;  // grouped calls: the group's start (first table's), this table's end
   bool sweep_pending = false;     // the sweep stream has work `stream` has not waited for yet
   bool keys_idle = false;         // nothing launched on `stream` after ev_keys touches the key store
   struct { const void* ids; int64_t n_ids; const void* off; int64_t n_bags; bool valid; } prep = {nullptr, 0, nullptr, 0, false};
@@ -290,6 +291,35 @@ int check_now(mono_table* t, int64_t now) {
   return MONO_OK;
 }
 
+// Fork/join of a grouped call around `one(i)`, the single-table call of table i.
+template <typename F>
+int group_call(int32_t n_tables, mono_table* const* tables, void* group_stream, F&& one) {
+  if (n_tables < 0 || (n_tables > 0 && !tables)) return MONO_ERR_ARG;
+  if (n_tables == 0) return MONO_OK;
+  for (int32_t i = 0; i < n_tables; ++i) {
+    if (!tables[i]) return MONO_ERR_ARG;
+    for (int32_t j = 0; j < i; ++j) if (tables[j] == tables[i]) return MONO_ERR_ARG;
+  }
+  cudaStream_t gs = static_cast<cudaStream_t>(group_stream);
+  mono_table* t0 = tables[0];
+  CUDA_TRY(t0, cudaEventRecord(t0->ev_fork, gs));              // (ev_fork is re-recorded by whoever uses it next)
+  int rc = MONO_OK;
+  int32_t started = 0;
+  for (; started < n_tables && rc == MONO_OK; ++started) {
+    mono_table* t = tables[started];
+    if (t->stream != gs) CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t0->ev_fork, 0));
+    rc = one(started);
+  }
+  // join what was started, also after an error
+  for (int32_t i = 0; i < started; ++i) {
+    mono_table* t = tables[i];
+    if (t->stream == gs) continue;
+    CUDA_TRY(t, cudaEventRecord(t->ev_group, t->stream));
+    CUDA_TRY(t, cudaStreamWaitEvent(gs, t->ev_group, 0));
+  }
+  return rc;
+}
+
 }  // namespace
 
 extern "C" {
@@ -322,7 +352,7 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   if (cudaStreamCreateWithFlags(&t->prep_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess)
     return fail(MONO_ERR_CUDA);
-  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_prepared, &t->ev_keys, &t->ev_swept})
+  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_prepared, &t->ev_keys, &t->ev_swept, &t->ev_group})
     if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return fail(MONO_ERR_CUDA);
 
   TableView& tv = t->tv;
@@ -374,7 +404,7 @@ int mono_table_destroy(mono_table* t) {
   cudaStreamSynchronize(t->stream);
   if (t->prep_stream) { cudaStreamSynchronize(t->prep_stream); cudaStreamDestroy(t->prep_stream); }
   if (t->sweep_stream) { cudaStreamSynchronize(t->sweep_stream); cudaStreamDestroy(t->sweep_stream); }
-  for (cudaEvent_t e : {t->ev_fork, t->ev_prepared, t->ev_keys, t->ev_swept}) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : {t->ev_fork, t->ev_prepared, t->ev_keys, t->ev_swept, t->ev_group}) if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
   free_scratch(t);
@@ -428,6 +458,24 @@ int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const i
   CUDA_TRY(t, cudaEventRecord(t->ev_prepared, t->prep_stream));
   t->prep = {ids, n_ids, slot_offsets, n_bags, true};
   return MONO_OK;
+}
+
+int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
+                           const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
+                           float* const* out, void* group_stream) {
+  if (n_tables > 0 && (!ids || !n_ids || !slot_offsets || !n_bags || !out)) return MONO_ERR_ARG;
+  return group_call(n_tables, tables, group_stream, [&](int32_t i) {
+    return mono_lookup_pool(tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], out[i]);
+  });
+}
+
+int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
+                           const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
+                           const float* const* grad_pooled, int64_t now, void* group_stream) {
+  if (n_tables > 0 && (!ids || !n_ids || !slot_offsets || !n_bags || !grad_pooled)) return MONO_ERR_ARG;
+  return group_call(n_tables, tables, group_stream, [&](int32_t i) {
+    return mono_apply_grads(tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], grad_pooled[i], now);
+  });
 }
 
 static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices) {

@@ -75,6 +75,47 @@ def test_multi_table_configs_scaled_down():
         run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5)
 
 
+def test_grouped_calls_on_eight_streams_match_eight_oracles():
+    """mono_group_lookup_pool / mono_group_apply_grads: the eight tables of the mixed-dim
+    configuration (scaled down), each on its own stream, one grouped call per step; every
+    table's outputs and state are those of its own oracle.  Also: a table named twice and a
+    null entry are refused, and an empty group is fine."""
+    cfgs = [wl.scaled(c, capacity=1 << 13, key_cells=1 << 15, n_distinct=1 << 14, steps=5, ttl=3)
+            for c in wl.multi_table_configs(n_examples=256, slots=3)]
+    streams = [torch.cuda.Stream() for _ in cfgs]
+    pairs = []
+    for c, st in zip(cfgs, streams):
+        kw = dict(lr=c.lr, eps=c.eps, init_acc=c.init_acc, init_scale=c.init_scale, seed=c.seed)
+        pairs.append((mb.MonoTable(c.capacity, c.dim, c.filter_threshold, c.ttl, key_cells=c.key_cells,
+                                   stream=st.cuda_stream, **kw),
+                      mo.OracleTable(c.capacity, c.dim, c.filter_threshold, c.ttl, **kw)))
+    gens = [wl.Stream(c) for c in cfgs]
+    handles = [g.handle for g, _ in pairs]
+    group_stream = torch.cuda.current_stream().cuda_stream
+    for t in range(5):
+        steps = [g.step(t) for g in gens]
+        dev = [_dev_batch(s) for s in steps]
+        outs = [torch.empty((c.n_bags, c.dim), dtype=torch.float32, device="cuda") for c in cfgs]
+        mb.mono_group_lookup_pool(handles, [d[0] for d in dev], [d[1] for d in dev], outs, group_stream)
+        for (gpu, cpu), s, out in zip(pairs, steps, outs):       # `out` is read on the group's stream
+            assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+        mb.mono_group_apply_grads(handles, [d[0] for d in dev], [d[1] for d in dev], [d[2] for d in dev], t, group_stream)
+        for (gpu, cpu), s in zip(pairs, steps):
+            assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
+            gpu.expire(t)
+            cpu.expire(t)
+            assert_state_equal(gpu, cpu, f"step {t}")
+    mb.mono_group_lookup_pool([], [], [], [], group_stream)
+    d0 = _dev_batch(gens[0].step(9))
+    out0 = torch.empty((cfgs[0].n_bags, cfgs[0].dim), dtype=torch.float32, device="cuda")
+    with pytest.raises(mb.MonoError):
+        mb.mono_group_lookup_pool([handles[0], handles[0]], [d0[0]] * 2, [d0[1]] * 2, [out0] * 2, group_stream)
+    with pytest.raises(mb.MonoError):
+        mb.mono_group_lookup_pool([handles[0], None], [d0[0]] * 2, [d0[1]] * 2, [out0] * 2, group_stream)
+    for gpu, _ in pairs:
+        assert_audit_ok(gpu)
+
+
 # ---------------------------------------------------------------- edge cases
 
 def test_empty_inputs_and_padding():
@@ -362,8 +403,13 @@ def test_probabilistic_filter_matches_the_sketch_oracle(depth, width):
         assert_vectors_close(got, cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
         gpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
         assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
-        if t % 3 == 2:
-            gpu.expire(t); cpu.expire(t)                  # clears the sketch every other sweep (ttl 4)
+        if t % 3 == 2:                                    # clears the sketch every other sweep (ttl 4)
+            if depth == 2:                                # once in slices: slice 0 is the one that clears
+                for k in range(5):
+                    mb.mono_expire_slice(gpu.handle, t, k, 5)
+            else:
+                gpu.expire(t)
+            cpu.expire(t)
         assert_state_equal(gpu, cpu, f"step {t}")         # only IDs with a row have entries
         ids = np.unique(np.concatenate(seen[-3:]))
         g, o = gpu.probe(ids, rows=False), cpu.probe(ids, rows=False)
