@@ -8,8 +8,8 @@ by one slice of the expiry sweep (mono_expire_slice: 1/`sweep_slices` of the key
 store per step, so every step carries the same share of the sweep).  Each batch is
 announced with mono_prepare_push before its lookup, so the ID-only part of the push
 runs beside the lookup; the per-kernel timing pass runs without it, each kernel alone.
-The table is pre-filled to the steady state of the configured stream, so the
-timed steps run at the load the stream would reach, not on an empty table.
+The table is pre-filled to the state the configured stream reaches after TTL steps
+from an empty table, so the timed steps run at that load, not on an empty table.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large]
     python bench.py --impl reference ...     # the CPU oracle, timed on the host
@@ -276,7 +276,7 @@ def run_ours(args):
     now0 = cfg.ttl - 1 if args.prefill else 0
     stream = wl.Stream(cfg)
 
-    # ---- table, pre-filled to the steady state of the stream
+    # ---- table, pre-filled to the state after ttl steps of the stream
     t_setup = time.time()
     table = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
                          init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed,
@@ -422,7 +422,7 @@ def run_ours(args):
                 "bags_per_step": cfg.n_bags, "ids_per_step": n, "unique_per_step": u,
                 "unique_resident_per_step": ur, "unique_resident_once_per_step": ur1, "new_per_step": unew, "zipf_s": cfg.zipf_s,
                 "id_universe": cfg.n_distinct, "filter_threshold": cfg.filter_threshold, "ttl": cfg.ttl,
-                "prefill": "steady state of the stream" if args.prefill else "empty table",
+                "prefill": "the state after ttl steps of the stream from an empty table (Poisson model)" if args.prefill else "empty table",
                 "rows_resident_at_start": st0["n_resident"], "ids_tracked_at_start": st0["n_tracked"],
                 "row_load": st0["n_resident"] / cfg.capacity, "key_load": st0["n_tracked"] / cfg.key_cells,
                 "sweep": (f"every step sweeps 1/{S} of the key store (a full sweep every {S} steps)" if S > 0
@@ -610,7 +610,7 @@ def run_multi(args):
                                                          "key_load": s0["n_tracked"] / c.key_cells}
                                                         for c, s0 in zip(cfgs, before)],
                        "examples_per_step": cfgs[0].n_examples, "slots_total": sum(c.n_slots for c in cfgs),
-                       "ids_per_step": n_ids / K, "prefill": "steady state of each stream",
+                       "ids_per_step": n_ids / K, "prefill": "the state after ttl steps of each stream from an empty table (Poisson model)",
                        "sweep": f"every step sweeps 1/{S} of every key store" if S > 0 else "none",
                        "l2": "every step reads fresh batches larger than L2",
                        "parallelism": "8 tables on 8 CUDA streams of one GPU, one grouped call per step and direction"},

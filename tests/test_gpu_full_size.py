@@ -1,5 +1,5 @@
 """Parity at the full size of the `large` configuration, in the launch configuration the
-benchmark times: table pre-filled to the stream's steady state (hundreds of millions of
+benchmark times: table pre-filled to the state after TTL steps of the stream (hundreds of millions of
 tracked IDs, ~0.9 row load), whole batches of 1.6 M bags through mono_prepare_push, mono_lookup_pool and
 mono_apply_grads, then the sweep in the 32 slices the benchmark spreads over its steps
 (here all at one time, which makes them equal to one mono_expire).
