@@ -203,7 +203,7 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
   uint32_t* occ_row = t->occ_row;
   if (n_ids > 0) {
     int64_t blocks = (n_ids + 255) / 256;
-    const int64_t cap = (int64_t)grid_for(t, 8) * 4;
+    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
     if (blocks > cap) blocks = cap;
     LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, occ_row));
   }
@@ -261,11 +261,13 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   cudaStream_t s = t->stream;
   const TableView& tv = t->tv;
   const Work& wk = t->wk;
+  // grids of the grid-stride kernels: several waves of blocks per SM where that measured faster
+  // (shorter tails), one wave elsewhere
   const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
-  LAUNCH(t, K_UPDATE, table_update_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
+  LAUNCH(t, K_UPDATE, table_update_kernel<<<g8 * 4, 256, 0, s>>>(tv, wk, now));
   if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
-  LAUNCH(t, K_EXPAND, expand_parts_kernel<<<g4, 128, 0, s>>>(tv, wk));
+  LAUNCH(t, K_EXPAND, expand_parts_kernel<<<g8 * 4, 128, 0, s>>>(tv, wk));
   LAUNCH(t, K_ORDER, order_parts_kernel<<<64, kWindows, 0, s>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
   // the rest of the call touches rows and scratch only: a sweep may run beside it
@@ -273,8 +275,8 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
-    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
-    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8, 256, 0, s>>>(tv, wk, grad, n_bags));
+    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 4, 256, 0, s>>>(tv, wk, grad, n_bags));
+    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 4, 256, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
