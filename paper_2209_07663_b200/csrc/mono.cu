@@ -275,8 +275,8 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
-    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 4, 256, 0, s>>>(tv, wk, grad, n_bags));
-    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 4, 256, 0, s>>>(tv, wk, grad, n_bags));
+    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
+    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
