@@ -28,6 +28,7 @@ import statistics
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 import numpy as np
@@ -100,28 +101,89 @@ def recorded_traffic(kernel: str, workload: str):
 
 
 class ClockSampler:
-    """nvidia-smi in the background while the timed region runs."""
+    """SM clock and clock-event reasons of one GPU, read through NVML every few milliseconds by a
+    thread while the timed region runs (the region lasts tens of milliseconds, too short for
+    nvidia-smi's own loop); nvidia-smi in the background when NVML cannot be loaded."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    PERIOD_S = 0.004
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, uuid: str = ""):
         self.gpu_index = gpu_index
+        self.uuid = uuid
         self.proc = None
         self.path = None
+        self.thread = None
+        self.halt = threading.Event()
+        self.sm, self.reason_bits, self.power_w = [], 0, []
+        self.sm_max = None
+        self.source = None
+
+    def _nvml_loop(self, nv, handle):
+        while not self.halt.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(handle))
+                self.power_w.append(nv.nvmlDeviceGetPowerUsage(handle) / 1000.0)
+            except Exception:
+                pass
+            self.halt.wait(self.PERIOD_S)
 
     def start(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            handle = None
+            if self.uuid:
+                try:
+                    handle = nv.nvmlDeviceGetHandleByUUID(("GPU-" + self.uuid).encode())
+                except Exception:
+                    handle = None
+            if handle is None:
+                handle = nv.nvmlDeviceGetHandleByIndex(self.gpu_index)
+            self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+            self.nv = nv
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, handle), daemon=True)
+            self.source = "nvml"
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
                  "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            self.source = "nvidia-smi"
         except Exception:
             self.proc = None
 
     def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": self.source}
+        if self.thread is not None:
+            self.halt.set()
+            self.thread.join(timeout=2)
+            nv = self.nv
+            names = (("hw_slowdown", "nvmlClocksEventReasonHwSlowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                     ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                     ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                     ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap", "nvmlClocksThrottleReasonSwPowerCap"))
+            reasons = []
+            for label, a, b in names:
+                bit = getattr(nv, a, None) or getattr(nv, b, 0)
+                if bit and (self.reason_bits & bit):
+                    reasons.append(label)
+            if self.sm:
+                out.update(sm_mhz=statistics.median(self.sm), sm_min_mhz=min(self.sm), sm_max_mhz=self.sm_max,
+                           reasons=sorted(reasons), samples=len(self.sm),
+                           power_w_max=max(self.power_w) if self.power_w else None)
+            try:
+                nv.nvmlShutdown()
+            except Exception:
+                pass
+            return out
         if self.proc is None:
             return out
         time.sleep(0.15)
@@ -151,6 +213,15 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
         return out
+
+
+def gpu_uuid(index: int) -> str:
+    """UUID of CUDA device `index` (what NVML knows it by, whatever CUDA_VISIBLE_DEVICES says)."""
+    try:
+        import torch
+        return str(torch.cuda.get_device_properties(index).uuid)
+    except Exception:
+        return ""
 
 
 def sample_of_step(step: wl.Step, n_bags: int) -> wl.Step:
@@ -332,7 +403,7 @@ def run_ours(args):
     barrier()
     st_a = table.status()
     mb.mono_timing_read(table.handle, reset=True)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, gpu_uuid(local_rank))
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -433,8 +504,7 @@ def run_ours(args):
             },
             "bags_per_s": world * cfg.n_bags * K / (ms_max * 1e-3),
             "gpu_launches": launches,
-            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
-                       "reasons": clocks["reasons"], "samples": clocks["samples"]},
+            "clocks": clocks,
             "roofline": {
                 "bound": "hbm", "kernel": dom + "_kernel",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -580,7 +650,7 @@ def run_multi(args):
     for i in range(W):
         step(i, False)
     before = [t.status() for t in tables]
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, gpu_uuid(local_rank))
     sampler.start()
     ms = timed(W, False)
     clocks = sampler.stop()
@@ -616,8 +686,7 @@ def run_multi(args):
                        "parallelism": "8 tables on 8 CUDA streams of one GPU, one grouped call per step and direction"},
             "serial": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,
                        "what": "the same calls with each table's stream drained before the next table starts"},
-            "gpu_launches": launches, "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
-                                                 "reasons": clocks["reasons"], "samples": clocks["samples"]},
+            "gpu_launches": launches, "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "all kernels of the 8 tables (whole step)", "achieved": achieved,
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": None},
