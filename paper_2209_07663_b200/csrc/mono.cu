@@ -51,6 +51,10 @@ struct mono_table {
   // Two internal streams, ordered against `stream` with events only: one runs the
   // ID-only part of a push that mono_prepare_push announced, the other the sweep.
   cudaStream_t prep_stream = nullptr, sweep_stream = nullptr;
+  // A third one runs the small kernels that serve only the few hottest IDs of a push beside
+  // the large ones (see launch_apply).
+  cudaStream_t aux_stream = nullptr;
+  cudaEvent_t ev_parts = nullptr, ev_reduced = nullptr, ev_aux = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_prepared = nullptr, ev_keys = nullptr, ev_swept = nullptr;
   cudaEvent_t ev_group = nullptr;  // grouped calls: the group's start (first table's), this table's end
   bool sweep_pending = false;     // the sweep stream has work `stream` has not waited for yet
@@ -267,21 +271,39 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   LAUNCH(t, K_UPDATE, table_update_kernel<<<g8 * 4, 256, 0, s>>>(tv, wk, now));
   if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
-  LAUNCH(t, K_EXPAND, expand_parts_kernel<<<g8 * 4, 128, 0, s>>>(tv, wk));
-  LAUNCH(t, K_ORDER, order_parts_kernel<<<64, kWindows, 0, s>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
   // the rest of the call touches rows and scratch only: a sweep may run beside it
   CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
+  // The kernels that prepare and finish the reduction of the long segments (the few hottest
+  // IDs) keep only a few blocks busy each, so they run on a stream of their own beside the
+  // kernels that work through the whole batch: expand/order beside file_segments, and
+  // fold/combine, which need only what reduce_adagrad left, beside update_singletons.  While
+  // kernels are being timed one by one, everything stays on the table's stream.
+  cudaStream_t a = t->timing ? s : t->aux_stream;
+  if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_keys, 0));
+  LAUNCH_ON(t, a, K_EXPAND, expand_parts_kernel<<<g8 * 4, 128, 0, a>>>(tv, wk));
+  LAUNCH_ON(t, a, K_ORDER, order_parts_kernel<<<64, kWindows, 0, a>>>(tv, wk));
+  CUDA_TRY(t, cudaGetLastError());
+  if (a != s) CUDA_TRY(t, cudaEventRecord(t->ev_parts, a));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
-    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
+    if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_parts, 0));
     LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
+    if (a != s) {
+      CUDA_TRY(t, cudaEventRecord(t->ev_reduced, s));
+      CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_reduced, 0));
+    }
+    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
-  LAUNCH(t, K_FOLD, fold_partials_kernel<<<g4, 256, 0, s>>>(tv, wk));
-  LAUNCH(t, K_COMBINE, combine_adagrad_kernel<<<g8, kCombineThreads, 0, s>>>(tv, wk));
+  LAUNCH_ON(t, a, K_FOLD, fold_partials_kernel<<<g4, 256, 0, a>>>(tv, wk));
+  LAUNCH_ON(t, a, K_COMBINE, combine_adagrad_kernel<<<g8, kCombineThreads, 0, a>>>(tv, wk));
+  if (a != s) {
+    CUDA_TRY(t, cudaEventRecord(t->ev_aux, a));
+    CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_aux, 0));
+  }
   LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 256, 0, s>>>(tv.st, wk.win_count, 1));
   CUDA_TRY(t, cudaGetLastError());
   t->keys_idle = true;
@@ -352,9 +374,11 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   if (cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || t->sm_count < 1)
     return fail(MONO_ERR_CUDA);
   if (cudaStreamCreateWithFlags(&t->prep_stream, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess)
+      cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&t->aux_stream, cudaStreamNonBlocking) != cudaSuccess)
     return fail(MONO_ERR_CUDA);
-  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_prepared, &t->ev_keys, &t->ev_swept, &t->ev_group})
+  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_prepared, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_parts,
+                         &t->ev_reduced, &t->ev_aux})
     if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return fail(MONO_ERR_CUDA);
 
   TableView& tv = t->tv;
@@ -406,7 +430,10 @@ int mono_table_destroy(mono_table* t) {
   cudaStreamSynchronize(t->stream);
   if (t->prep_stream) { cudaStreamSynchronize(t->prep_stream); cudaStreamDestroy(t->prep_stream); }
   if (t->sweep_stream) { cudaStreamSynchronize(t->sweep_stream); cudaStreamDestroy(t->sweep_stream); }
-  for (cudaEvent_t e : {t->ev_fork, t->ev_prepared, t->ev_keys, t->ev_swept, t->ev_group}) if (e) cudaEventDestroy(e);
+  if (t->aux_stream) { cudaStreamSynchronize(t->aux_stream); cudaStreamDestroy(t->aux_stream); }
+  for (cudaEvent_t e : {t->ev_fork, t->ev_prepared, t->ev_keys, t->ev_swept, t->ev_group, t->ev_parts, t->ev_reduced,
+                        t->ev_aux})
+    if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
   free_scratch(t);
