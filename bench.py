@@ -341,6 +341,16 @@ def run_ours(args):
 
     base = wl.CONFIGS[args.workload]
     cfg = rank_config(base, rank)
+    drift = cfg.drift_period > 0
+    if drift:
+        # The drift stream has no closed-form steady state to pre-fill: it starts from an empty
+        # table and warms up for more than ttl steps (past the first full expiry horizon and a
+        # re-keying), and the timed steps span at least one re-keying of the ID universe.
+        args.prefill = False
+        if args.warmup < cfg.ttl + cfg.drift_period + 10:
+            args.warmup = cfg.ttl + cfg.drift_period + 10
+        if args.steps < 2 * cfg.drift_period:
+            args.steps = 2 * cfg.drift_period
     K, W, E = args.steps, args.warmup, args.e2e_steps
     KT = min(K, args.kernel_steps)            # steps of the per-kernel timing pass
     S = args.sweep_slices
@@ -368,16 +378,21 @@ def run_ours(args):
     def make(i):
         return stream.step(now0 + 1 + i, with_grad=False)
 
-    with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
-        host_batches = list(pool.map(make, range(n_batches)))
     gg = torch.Generator(device=dev)
     gg.manual_seed(cfg.seed)
-    dev_batches = []
-    for t, s in enumerate(host_batches[:W + K + KT]):
-        ids = torch.from_numpy(s.ids.view(np.int64)).to(dev)
-        off = torch.from_numpy(s.offsets).to(dev)
-        grad = torch.randn((cfg.n_bags, cfg.dim), device=dev, generator=gg).mul_(cfg.grad_std)
-        dev_batches.append((ids, off, grad))
+    # every step has its own ids and offsets; its gradients too, except in a long drift run, where
+    # the steps take turns on a ring of gradient tensors that is still several times larger than L2
+    n_grads = min(W + K + KT, 16) if drift else W + K + KT
+    grads = [torch.randn((cfg.n_bags, cfg.dim), device=dev, generator=gg).mul_(cfg.grad_std) for _ in range(n_grads)]
+    dev_batches, host_batches = [], {}
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+        for t, s in enumerate(pool.map(make, range(n_batches))):
+            if t < W + K + KT:
+                ids = torch.from_numpy(s.ids.view(np.int64)).to(dev)
+                off = torch.from_numpy(s.offsets).to(dev)
+                dev_batches.append((ids, off, grads[t % n_grads]))
+            else:
+                host_batches[t] = s            # the end-to-end steps start from host memory
     out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device=dev)
     torch.cuda.synchronize()
     setup_s = time.time() - t_setup
@@ -431,7 +446,8 @@ def run_ours(args):
     e2e = None
     if E > 0:
         pinned = []
-        for s in host_batches[W + K + KT:]:
+        for t in sorted(host_batches):
+            s = host_batches[t]
             ids = torch.from_numpy(s.ids.view(np.int64)).pin_memory()
             off = torch.from_numpy(s.offsets).pin_memory()
             grad = torch.randn((cfg.n_bags, cfg.dim)).mul_(cfg.grad_std).pin_memory()
@@ -529,6 +545,19 @@ def run_ours(args):
                             "evictions": st_end["n_evictions_total"], "stash_used": st_end["stash_used"]},
             "setup_s": round(setup_s, 1),
         }
+        if drift:
+            sec = ms_max * 1e-3
+            line["drift"] = {
+                "re_keyed": f"{cfg.drift_new_frac:.0%} of a batch's occurrences get new identities every {cfg.drift_period} steps",
+                "inserts_per_s": (st_b["n_inserted_total"] - st_a["n_inserted_total"]) / sec,
+                "admissions_per_s": (st_b["n_admitted_total"] - st_a["n_admitted_total"]) / sec,
+                "expired_per_s": (st_b["n_expired_total"] - st_a["n_expired_total"]) / sec,
+                "displacements_per_s": (st_b["n_evictions_total"] - st_a["n_evictions_total"]) / sec,
+                "row_load_start": st_a["n_resident"] / cfg.capacity, "row_load_end": st_b["n_resident"] / cfg.capacity,
+                "key_load_start": st_a["n_tracked"] / cfg.key_cells, "key_load_end": st_b["n_tracked"] / cfg.key_cells,
+                "max_chain": st_b["max_chain"], "rows_refused": st_b["n_rows_refused"],
+                "keys_dropped": st_b["n_keys_dropped"],
+            }
         if e2e:
             line["e2e"] = {"value": e2e_ids_all / (e2e_ms_max * 1e-3), "unit": UNIT,
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
