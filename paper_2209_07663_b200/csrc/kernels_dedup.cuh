@@ -113,11 +113,9 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
                   const long long* __restrict__ offsets, long long n_bags, DevState* st,
                   unsigned long long seed) {
   constexpr int kPerThread = kTileIds / kTileThreads;
-  constexpr int kSlotsPerThread = kTileSlots / kTileThreads;
   __shared__ unsigned long long s_key[kTileSlots];
   __shared__ unsigned int s_cnt[kTileSlots];     // multiplicity in the tile, then base rank
   __shared__ unsigned int s_gslot[kTileSlots];   // the ID's slot in the global set
-  __shared__ unsigned int s_occ[kTileSlots];     // one of the tile's occurrences of the ID
   __shared__ unsigned long long s_warp[kTileThreads / 32];
   __shared__ unsigned int s_ubase;
 
@@ -127,50 +125,54 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   if (last > n_ids) last = n_ids;
   __syncthreads();
 
-  // 1. group the tile's occurrences in shared memory
+  // 1. group the tile's occurrences in shared memory.  The thread whose occurrence puts an ID
+  //    into the tile's table owns that ID for the rest of the kernel.
   const long long tile0 = (long long)blockIdx.x * kTileIds;
+  unsigned long long my_id[kPerThread];
   uint32_t my_slot[kPerThread], my_rank[kPerThread];
+  bool own[kPerThread];
   unsigned int n_valid = 0;
 #pragma unroll
   for (int k = 0; k < kPerThread; ++k) {
     const long long j = tile0 + k * kTileThreads + threadIdx.x;
     unsigned long long id = kEmptyKey;
     if (j >= first && j < last) id = ids[j];
+    my_id[k] = id;
     my_slot[k] = kNoSlot;
     my_rank[k] = 0;
+    own[k] = false;
     if (id != kEmptyKey) {
       ++n_valid;
       uint32_t s = (uint32_t)(mix_a(id ^ seed) >> 40) & (kTileSlots - 1);
       for (int probe = 0; probe < kTileSlots; ++probe) {      // at most kTileIds keys in kTileSlots slots
         const unsigned long long old = atomicCAS(&s_key[s], kEmptyKey, id);
-        if (old == kEmptyKey || old == id) break;
+        if (old == kEmptyKey) { own[k] = true; break; }
+        if (old == id) break;
         s = (s + 1) & (kTileSlots - 1);
       }
       my_slot[k] = s;
       my_rank[k] = atomicAdd(&s_cnt[s], 1u);
-      s_occ[s] = (unsigned int)j;                    // any of them will do
     }
   }
   __syncthreads();
 
-  // 2. one visit of the global set per distinct ID of the tile.  The first
-  //    probes of a thread's slots are issued together, then resolved, then the
-  //    counter updates are issued together, so their latencies overlap.
-  unsigned long long tid_[kSlotsPerThread], seen[kSlotsPerThread];
-  uint32_t g[kSlotsPerThread], base_rank[kSlotsPerThread];
-  bool is_new[kSlotsPerThread];
+  // 2. one visit of the global set per distinct ID of the tile, by the ID's owner.  The first
+  //    probes of a thread's IDs are issued together, then resolved, then the counter updates
+  //    are issued together, so their latencies overlap.
+  unsigned long long seen[kPerThread];
+  uint32_t g[kPerThread], base_rank[kPerThread];
+  bool is_new[kPerThread];
 #pragma unroll
-  for (int k = 0; k < kSlotsPerThread; ++k) {
-    tid_[k] = s_key[k * kTileThreads + threadIdx.x];
-    g[k] = (uint32_t)(mix_b(tid_[k] ^ seed) >> 20) & wk.primary_mask;
-    seen[k] = tid_[k] == kEmptyKey ? 0ull : *reinterpret_cast<volatile unsigned long long*>(&wk.bset[g[k]].key);
+  for (int k = 0; k < kPerThread; ++k) {
+    g[k] = (uint32_t)(mix_b(my_id[k] ^ seed) >> 20) & wk.primary_mask;
+    seen[k] = own[k] ? *reinterpret_cast<volatile unsigned long long*>(&wk.bset[g[k]].key) : 0ull;
   }
   unsigned int n_new = 0;
 #pragma unroll
-  for (int k = 0; k < kSlotsPerThread; ++k) {
+  for (int k = 0; k < kPerThread; ++k) {
     is_new[k] = false;
-    if (tid_[k] == kEmptyKey) continue;
-    const unsigned long long id = tid_[k];
+    if (!own[k]) continue;
+    const unsigned long long id = my_id[k];
     unsigned long long kk = seen[k];
     bool placed = false;
     // primary tier: a short window of consecutive positions
@@ -202,13 +204,13 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
     n_new += is_new[k];
   }
 #pragma unroll
-  for (int k = 0; k < kSlotsPerThread; ++k)
-    base_rank[k] = tid_[k] == kEmptyKey ? 0u : atomicAdd(&wk.bset[g[k]].a, s_cnt[k * kTileThreads + threadIdx.x]);
+  for (int k = 0; k < kPerThread; ++k)
+    base_rank[k] = own[k] ? atomicAdd(&wk.bset[g[k]].a, s_cnt[my_slot[k]]) : 0u;
 #pragma unroll
-  for (int k = 0; k < kSlotsPerThread; ++k) {
-    if (tid_[k] == kEmptyKey) continue;
-    s_cnt[k * kTileThreads + threadIdx.x] = base_rank[k];
-    s_gslot[k * kTileThreads + threadIdx.x] = g[k];
+  for (int k = 0; k < kPerThread; ++k) {
+    if (!own[k]) continue;
+    s_cnt[my_slot[k]] = base_rank[k];
+    s_gslot[my_slot[k]] = g[k];
   }
   // number the IDs this tile saw first: one counter update per tile
   // (new IDs in the low word, valid occurrences in the high word of one scan)
@@ -222,11 +224,11 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   __syncthreads();
   my_u += s_ubase;
 #pragma unroll
-  for (int k = 0; k < kSlotsPerThread; ++k) {
+  for (int k = 0; k < kPerThread; ++k) {
     if (is_new[k]) {
-      wk.uid[my_u] = tid_[k];
+      wk.uid[my_u] = my_id[k];
       wk.uslot[my_u] = g[k];
-      wk.uocc[my_u] = s_occ[k * kTileThreads + threadIdx.x];
+      wk.uocc[my_u] = (uint32_t)(tile0 + k * kTileThreads + threadIdx.x);     // the owner's own occurrence
       ++my_u;
     }
   }
