@@ -7,76 +7,6 @@
 
 namespace mono {
 
-// Look-up of four IDs by one quad.  Each lane brings its own ID (hashed once,
-// by its owner); the quad then resolves the four IDs in turn, every lane
-// reading one cell of the ID's bucket, so a bucket costs one coalesced 64-byte
-// request.  On return every lane knows, for its own ID, whether it is tracked,
-// its metadata and the index of its cell (in cells[], or n_cells + i for stash
-// cell i).  All four lanes must call; `active` false skips the lane's ID.
-struct Found {
-  bool hit;
-  unsigned long long meta;
-  unsigned long long cell;
-};
-
-__device__ inline Found quad4_find(const TableView& tv, unsigned long long id, bool active, int lane,
-                                   unsigned stash_hw) {
-  const int sub = lane & 3, q0 = lane - sub;
-  const unsigned quad_mask = 0xFu << q0;
-  const unsigned long long n_cells = (tv.bucket_mask + 1) * kCellsPerBucket;
-  const unsigned long long b0 = active ? tv.bucket0(id) : 0ull;
-  Found mine;
-  mine.hit = false; mine.meta = 0; mine.cell = 0;
-  // first buckets of the four IDs: all four reads are issued before any is examined
-  unsigned long long id_k[4], bkt[4];
-  Cell c[4];
-  unsigned act = __ballot_sync(quad_mask, active) >> q0;
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    id_k[k] = __shfl_sync(quad_mask, id, q0 + k);
-    bkt[k] = __shfl_sync(quad_mask, b0, q0 + k);
-    c[k] = (act >> k) & 1u ? load_cell_ro(tv.cells + bkt[k] * kCellsPerBucket + sub) : empty_cell();
-  }
-  unsigned bal[4];
-  unsigned miss = 0;
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    bal[k] = __ballot_sync(quad_mask, ((act >> k) & 1u) && c[k].key == id_k[k]) & quad_mask;
-    if (((act >> k) & 1u) && !bal[k]) miss |= 1u << k;
-  }
-  if (miss) {                                                    // quad-uniform
-    // second buckets of the IDs that missed, again read together
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if ((miss >> k) & 1u) {
-        bkt[k] = tv.bucket1(id_k[k]);
-        c[k] = load_cell_ro(tv.cells + bkt[k] * kCellsPerBucket + sub);
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if ((miss >> k) & 1u) bal[k] = __ballot_sync(quad_mask, c[k].key == id_k[k]) & quad_mask;
-  }
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    if (!((act >> k) & 1u)) continue;
-    unsigned long long cell = bkt[k] * kCellsPerBucket;
-    if (!bal[k] && stash_hw != 0) {
-      for (unsigned base = 0; base < stash_hw && !bal[k]; base += kCellsPerBucket) {
-        c[k] = base + sub < stash_hw ? load_cell_ro(tv.stash + base + sub) : empty_cell();
-        bal[k] = __ballot_sync(quad_mask, c[k].key == id_k[k]) & quad_mask;
-        cell = n_cells + base;
-      }
-    }
-    if (bal[k]) {
-      const int src = __ffs(bal[k]) - 1;                         // absolute lane that saw the key
-      const unsigned long long m = __shfl_sync(quad_mask, c[k].meta, src);
-      if (sub == k) { mine.hit = true; mine.meta = m; mine.cell = cell + (unsigned)(src - q0); }
-    }
-  }
-  return mine;
-}
-
 // Read-only look-up by one thread.  An insertion tries the cell named by the
 // top bits of the hash first, so that cell is read first and alone; the other
 // three cells of the bucket, the second bucket and the stash follow only on a
@@ -106,6 +36,35 @@ __device__ inline bool thread_lookup(const TableView& tv, unsigned long long id,
     if (s.key == id) { *meta = s.meta; return true; }
   }
   return false;
+}
+
+// The same look-up for a caller that goes on to modify the entry: it also returns where
+// the entry is (index into cells[], or n_cells + i for stash cell i; kNoCell if nowhere).
+constexpr unsigned long long kNoCell = 0xFFFFFFFFFFFFFFFFull;
+
+__device__ inline unsigned long long thread_locate(const TableView& tv, unsigned long long id, unsigned stash_hw,
+                                                   unsigned long long* meta) {
+  const unsigned long long h0 = tv.hash0(id);
+  const unsigned long long base0 = (h0 & tv.bucket_mask) * kCellsPerBucket;
+  const uint32_t first = (uint32_t)(h0 >> 62);
+  const Cell c0 = load_cell_ro(tv.cells + base0 + first);
+  if (c0.key == id) { *meta = c0.meta; return base0 + first; }
+#pragma unroll
+  for (uint32_t k = 1; k < kCellsPerBucket; ++k) {
+    const Cell c = load_cell_ro(tv.cells + base0 + ((first + k) & 3u));
+    if (c.key == id) { *meta = c.meta; return base0 + ((first + k) & 3u); }
+  }
+  const unsigned long long base1 = tv.bucket1(id) * kCellsPerBucket;
+#pragma unroll
+  for (uint32_t k = 0; k < kCellsPerBucket; ++k) {
+    const Cell c = load_cell_ro(tv.cells + base1 + k);
+    if (c.key == id) { *meta = c.meta; return base1 + k; }
+  }
+  for (unsigned i = 0; i < stash_hw; ++i) {
+    const Cell s = load_cell_ro(tv.stash + i);
+    if (s.key == id) { *meta = s.meta; return (tv.bucket_mask + 1) * kCellsPerBucket + i; }
+  }
+  return kNoCell;
 }
 
 // Forward, step 1: one thread per ID occurrence resolves the ID to its row

@@ -112,14 +112,15 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
   }
 }
 
-// Phase 2 of mono_apply_grads: one thread per distinct ID (look-ups shared
-// within quads: measured faster here than per-thread look-ups, because IDs new
-// to the table miss both buckets).  Tracked IDs get count += multiplicity (saturating at the
+// Phase 2 of mono_apply_grads: one thread per distinct ID (its own look-up, the cell an
+// insertion prefers first: measured 0.210 ms on the largest configuration at six blocks per
+// SM, against 0.222 ms for look-ups shared within quads, which need twice the registers).
+// Tracked IDs get count += multiplicity (saturating at the
 // threshold), last_seen = now, and a row if the count has reached the
 // threshold; the rest are queued for insertion.  No cell moves during this
 // kernel, so the thread whose ID sits in a cell owns it.  IDs that end up with a
 // row and occur more than once also get their segment of bag_of_sorted[] here.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 6)
 table_update_kernel(TableView tv, Work wk, uint32_t now) {
   __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_unique;
@@ -137,9 +138,10 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
       slot = wk.uslot[u];
       m = wk.bset[slot].a;
     }
-    const Found f = quad4_find(tv, id, active, lane, stash_hw);
-    const bool hit = f.hit;
-    uint32_t low = meta_low(f.meta);
+    unsigned long long meta = 0;
+    const unsigned long long cell = active ? thread_locate(tv, id, stash_hw, &meta) : kNoCell;
+    const bool hit = cell != kNoCell;
+    uint32_t low = meta_low(meta);
     bool resident = false, need_row = false;
     if (hit) {
       resident = (low & kResidentBit) != 0;
@@ -160,7 +162,7 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
       // every ID of the batch that has a row is trained in this call: mark it for the next sync
       if (resident) { row_word = low & kRowMask; low |= kTouchedBit; }
       else if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
-      Cell* where = f.cell < n_cells ? tv.cells + f.cell : tv.stash + (f.cell - n_cells);
+      Cell* where = cell < n_cells ? tv.cells + cell : tv.stash + (cell - n_cells);
       where->meta = make_meta(now, low);
       wk.urow[u] = row_word;
       wk.useg[u] = rv.seg_start;
