@@ -20,7 +20,10 @@
  *  - All work of a table is enqueued on the CUDA stream given at creation.  The
  *    hot calls (mono_lookup_pool, mono_apply_grads, mono_expire) return without
  *    synchronising.  Calls on one table must not overlap on the GPU: issue them
- *    from one thread, on that stream.
+ *    from one thread, on that stream.  (A call may run some of its kernels on
+ *    streams of the table's own; they start after everything issued on the
+ *    table's stream so far, and whatever is issued on it next waits for them,
+ *    so a caller sees the order of one stream.)
  *  - Conditions that only the device can see (no free row, key store full,
  *    malformed offsets) never trap or hang: every device loop is bounded, the
  *    condition sets a sticky bit and a counter, and mono_status reports them.
