@@ -6,8 +6,9 @@ mono_lookup_pool (probe, gather, sum pooling) + mono_apply_grads (dedup,
 count/stamp/admit, cuckoo insert, segmented gradient reduce, Adagrad), followed
 by one slice of the expiry sweep (mono_expire_slice: 1/`sweep_slices` of the key
 store per step, so every step carries the same share of the sweep).  Each batch is
-announced with mono_prepare_push before its lookup, so the ID-only part of the push
-runs beside the lookup; the per-kernel timing pass runs without it, each kernel alone.
+announced with mono_prepare_push before its lookup, so its IDs are grouped and looked up
+in the key store once, for the lookup and the push together.  The timed region is repeated
+--reps times from the same restored state (median and min reported).
 The table is pre-filled to the state the configured stream reaches after TTL steps
 from an empty table, so the timed steps run at that load, not on an empty table.
 
@@ -57,9 +58,10 @@ def measured_peaks():
 
 KERNEL_SOURCES = {
     "probe_rows": ("kernels_forward.cuh", "table_layout.cuh"),
-    "gather_pool": ("kernels_forward.cuh", "table_layout.cuh"),
+    "gather_pool": ("kernels_forward.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "fill_occ_bag": ("kernels_dedup.cuh", "table_layout.cuh"),
     "dedup_tile": ("kernels_dedup.cuh", "table_layout.cuh"),
+    "table_lookup": ("kernels_table.cuh", "kernels_forward.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "table_update": ("kernels_table.cuh", "kernels_forward.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "table_insert": ("kernels_table.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "update_singletons": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
@@ -277,16 +279,20 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- our arm
 
-def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0):
+def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
     """Bytes the method itself must move per step, per kernel (each distinct datum once per
     phase; 32-byte sector as the smallest random access).  n occurrences, b bags, u distinct
-    IDs, ur of them with a row, ur1 of those occurring once in the batch, unew new IDs."""
+    IDs, ur of them with a row, ur1 of those occurring once in the batch, unew new IDs.
+    prepared: the batch was announced, so the key store is read once per distinct ID ahead of
+    the lookup instead of once per occurrence inside it."""
     per_kernel = {
-        "probe_rows": 8 * n + 32 * n,                        # ids + one bucket sector per occurrence
-        "gather_pool": 8 * (b + 1) + 4 * d * ur + 4 * d * b,  # offsets, each distinct row once, out
+        "probe_rows": 0,
+        # offsets, one 8-byte record per occurrence (the ID, or its place in the grouping), each distinct row once, out
+        "gather_pool": 8 * (b + 1) + 8 * n + (0 if prepared else 32 * n) + 4 * d * ur + 4 * d * b,
         "fill_occ_bag": 8 * (b + 1),                         # offsets
         "dedup_tile": 8 * n + 24 * n,                        # ids + (key, index) pairs written and read
-        "table_update": 64 * u,                              # probe + count/stamp read-modify-write
+        "table_lookup": 32 * u if prepared else 0,           # one bucket sector per distinct ID
+        "table_update": 64 * u,                              # count/stamp read-modify-write of that sector
         "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
         "update_singletons": 20 * d * ur1,                   # IDs seen once: gradient row, row and accumulator in and out
         "reduce_adagrad": 16 * d * (ur - ur1) + 4 * d * max(b - ur1, 0),   # rows of repeated IDs + the other gradient rows, once
@@ -300,7 +306,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0):
 KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
     "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
-    "table_update": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
+    "table_lookup": "table", "table_update": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
     "update_singletons": "adagrad", "file_segments": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
     "combine_adagrad": "adagrad", "expire": "expire",
 }
@@ -412,31 +418,47 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- warm-up, then the timed region
+    # ---- warm-up, then the timed region: R repetitions of the same K steps, each from the state the
+    # warm-up left (a device-resident snapshot restored in between), so that the spread between
+    # repetitions is measurement noise and nothing else
+    R = max(args.reps, 1)
     for t in range(W):
         step(t)
     barrier()
-    st_a = table.status()
-    mb.mono_timing_read(table.handle, reset=True)
+    if R > 1:
+        mb.mono_snapshot_save(table.handle)
     sampler = ClockSampler(local_rank, gpu_uuid(local_rank))
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record()
-    for t in range(K):
-        step(W + t)
-    ev1.record()
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
+    rep_ms, launches, n_ids_timed = [], 0, 0
+    st_a = st_b = None
+    for r in range(R):
+        if r > 0:
+            mb.mono_snapshot_restore(table.handle)
+        barrier()
+        st_a = table.status()
+        mb.mono_timing_read(table.handle, reset=True)
+        if r == 0:
+            sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for t in range(K):
+            step(W + t)
+        mb.mono_fence(table.handle)            # the last step's sweep slice runs on a stream of the table's own
+        ev1.record()
+        barrier()
+        rep_ms.append(ev0.elapsed_time(ev1))
+        st_b = table.status()
+        launches = mb.mono_timing_read(table.handle, reset=True)["launches_total"]
+        n_ids_timed = st_b["sum_ids"] - st_a["sum_ids"]
     clocks = sampler.stop()
-    st_b = table.status()
-    launches = mb.mono_timing_read(table.handle, reset=True)["launches_total"]
-    n_ids_timed = st_b["sum_ids"] - st_a["sum_ids"]
+    if R > 1:
+        mb.mono_snapshot_drop(table.handle)
+    ms_total = statistics.median(rep_ms)
 
     # ---- the same steps on fresh batches with every kernel bracketed by CUDA events
     mb.mono_timing_enable(table.handle, True)
     for t in range(KT):
-        step(W + K + t, prepare=False)       # every kernel alone on the device
+        step(W + K + t)                      # the same calls; the events keep every kernel alone on the device
     torch.cuda.synchronize()
     tim = mb.mono_timing_read(table.handle, reset=True)
     mb.mono_timing_enable(table.handle, False)
@@ -485,7 +507,8 @@ def run_ours(args):
         ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / KT
         unew = (st_c["sum_new"] - st_b["sum_new"]) / KT
         ur1 = (st_c["sum_single_resident"] - st_b["sum_single_resident"]) / KT
-        alg_kernel, alg_total = algorithmic_bytes(n, cfg.n_bags, u, ur, ur1, unew, d, cfg.key_cells // S if S > 0 else 0)
+        alg_kernel, alg_total = algorithmic_bytes(n, cfg.n_bags, u, ur, ur1, unew, d, cfg.key_cells // S if S > 0 else 0,
+                                                  prepared=args.prepare)
         per_kernel = {}
         for name, v in tim["kernels"].items():
             if v["launches"] and name in KERNEL_GROUP:
@@ -503,6 +526,10 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": ids_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "reps": {"n": R, "what": f"the timed region ({K} steps) repeated from the same restored state; value and "
+                                     "ms_per_step are the median repetition (slowest rank)",
+                     "ms_per_step_median": statistics.median(rep_ms) / K, "ms_per_step_min": min(rep_ms) / K,
+                     "ms_per_step_max": max(rep_ms) / K, "ms_per_step_all_rank0": [round(x / K, 5) for x in rep_ms]},
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": args.workload, "capacity": cfg.capacity, "dim": d, "key_cells": cfg.key_cells,
@@ -515,8 +542,8 @@ def run_ours(args):
                 "sweep": (f"every step sweeps 1/{S} of the key store (a full sweep every {S} steps)" if S > 0
                           else "none"), "l2": "every step reads a fresh batch larger than L2",
                 "parallelism": f"{world} independent table(s), one per GPU",
-                "push_prepared": ("mono_prepare_push before each lookup: the grouping of the batch's IDs runs "
-                                  "beside the lookup" if args.prepare else "no"),
+                "push_prepared": ("mono_prepare_push before each lookup: the batch is grouped and every distinct ID "
+                                  "looked up once, for the lookup and the push together" if args.prepare else "no"),
             },
             "bags_per_s": world * cfg.n_bags * K / (ms_max * 1e-3),
             "gpu_launches": launches,
@@ -695,7 +722,8 @@ def run_multi(args):
         n = b["sum_ids"] - a["sum_ids"]
         u, ur = b["sum_unique"] - a["sum_unique"], b["sum_unique_resident"] - a["sum_unique_resident"]
         ur1, unew = b["sum_single_resident"] - a["sum_single_resident"], b["sum_new"] - a["sum_new"]
-        alg += algorithmic_bytes(n, cfg.n_bags * K, u, ur, ur1, unew, cfg.dim, K * cfg.key_cells // S if S > 0 else 0)[1]
+        alg += algorithmic_bytes(n, cfg.n_bags * K, u, ur, ur1, unew, cfg.dim, K * cfg.key_cells // S if S > 0 else 0,
+                                 prepared=args.prepare)[1]
     if rank == 0:
         peak, peak_kind = measured_peaks()
         achieved = alg / (ms * 1e-3) / 1e9
@@ -737,6 +765,8 @@ def main():
                     help="do not announce each batch with mono_prepare_push before its lookup")
     ap.add_argument("--sweep-slices", type=int, default=32,
                     help="every step sweeps 1/S of the key store for expired IDs (0 = no sweep)")
+    ap.add_argument("--reps", type=int, default=5,
+                    help="repetitions of the timed region, each from the same restored state (median reported)")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--kernel-steps", type=int, default=8, help="steps of the per-kernel CUDA-event pass")
     ap.add_argument("--no-prefill", dest="prefill", action="store_false")

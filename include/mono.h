@@ -65,8 +65,13 @@ enum {
                                  it stays tracked without a row and is retried later */
   MONO_DEV_KEYS_FULL = 2u,    /* an insertion found no cell after the bounded eviction
                                  chain and the stash was full: one tracked key was lost */
-  MONO_DEV_BAD_OFFSETS = 4u,  /* slot_offsets not monotone or out of [0, n_ids]; the
-                                 offending bag was treated as empty */
+  MONO_DEV_BAD_OFFSETS = 4u,  /* a bag with slot_offsets[b] < 0, slot_offsets[b+1] < slot_offsets[b]
+                                 or slot_offsets[b+1] > n_ids: that bag was treated as empty, by
+                                 the lookup (zeros) and by the push (its IDs are neither counted,
+                                 stamped nor trained).  After a decrease in the offsets two
+                                 well-formed bags can overlap; the lookup then pools the shared
+                                 IDs in both, the push counts each of them once, for one of the
+                                 two bags */
   MONO_DEV_IMPORT_DUP = 8u    /* mono_import met an ID that was already tracked; skipped */
 };
 
@@ -142,6 +147,8 @@ typedef struct {
   uint64_t sum_unique_resident; /* distinct IDs that had (or got) a row, summed */
   uint64_t sum_new;             /* distinct IDs that were new to the key store, summed */
   uint64_t sum_single_resident; /* distinct IDs with a row that occurred once in their batch, summed */
+  uint64_t scratch_reallocs;    /* times a call had to grow the scratch (cudaMalloc + synchronise inside
+                                   the call); stays 0 when max_ids / max_bags or mono_reserve were large enough */
 } mono_status_t;
 
 typedef struct {
@@ -210,7 +217,11 @@ int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids,
  *     rounded once to fp32):   acc += G*G;   w -= lr * G / (sqrt(acc) + eps).
  *     The whole batch's G applies even when the row was admitted in this call.
  *     Gradients of IDs without a row are dropped.
- * The outcome does not depend on the order of IDs or bags.
+ * Counts, times, admissions and the set of rows do not depend on the order of IDs or
+ * bags.  The fp64 sum G is taken in an order that can differ from run to run (it follows
+ * the order in which thread blocks reach an ID), so two runs on the same input can differ
+ * in the last bit of an updated element: the results are order-independent to within one
+ * fp32 rounding of G, not bitwise reproducible.
  *  grad_pooled   fp32 [n_bags, dim], 16-byte aligned
  *  now           time of this batch; MONO_ERR_TIME if it decreased
  */
@@ -227,16 +238,19 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids,
 int mono_expire(mono_table* t, int64_t now);
 
 /*
- * Optional hint that overlaps the ID-only part of a push with the lookup of the same batch
- * (the paper has no counterpart; it describes no batching below the level of Section 2.2's
- * pull and push).  Announces the batch that the NEXT mono_apply_grads on this table will be
- * given -- the same device pointers and sizes, contents unchanged until that call -- and
- * starts grouping its occurrences by ID on a stream of the table's own, ordered after
- * everything issued on the table's stream so far and running beside whatever is issued next
- * (normally mono_lookup_pool of that batch).  mono_apply_grads called with exactly these
- * `ids`, `n_ids`, `slot_offsets`, `n_bags` waits for the grouping and uses it; called with
- * anything else it discards the preparation and groups its own batch, as does a second
- * mono_prepare_push.  Results are the same with or without the hint.  The table is not
+ * Optional hint for a training loop that knows its batch before the pull (Section 2.2: a step
+ * pulls the parameters of a batch and later pushes updates for the same batch).  Announces
+ * the batch that the NEXT mono_lookup_pool and mono_apply_grads on this table will be given
+ * -- the same device pointers and sizes, contents unchanged until the push -- and does the
+ * work both calls share ahead of them: the occurrences are grouped by ID, and every distinct
+ * ID is looked up in the key store once.  mono_lookup_pool called with exactly these `ids`,
+ * `n_ids`, `slot_offsets`, `n_bags` then takes the rows from that look-up instead of probing
+ * the key store once per occurrence, and mono_apply_grads called with them goes straight to
+ * the cells the look-up found.  Called with anything else, either call works as if nothing
+ * had been announced (a push then forgets the announcement, as does a second
+ * mono_prepare_push).  Any call that changes the table between the announcement and the push
+ * -- mono_expire*, mono_import, mono_rehash, mono_export_touched, mono_snapshot_restore --
+ * forgets it too, so results are the same with or without the hint.  The table is not
  * changed by this call.  Errors: as mono_lookup_pool; malformed offsets raise
  * MONO_DEV_BAD_OFFSETS in the status, as they would in mono_apply_grads.
  */
@@ -244,19 +258,30 @@ int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const i
                       int64_t n_bags);
 
 /*
- * Grouped calls: one call for several tables (Section 3.1: a production model holds many
- * embedding tables of very uneven size).  Table i gets batch i: `tables`, `ids`, `n_ids`,
- * `slot_offsets`, `n_bags`, `out` / `grad_pooled` are HOST arrays of `n_tables` entries whose
- * elements are what the single-table call takes (device pointers, sizes).  Every table works
- * on its own stream (the one it was created with), so the tables run beside one another --
- * the short, latency-bound kernels of a small table fill the gaps of a large one -- if they
- * were created with different streams; with one shared stream the calls are still correct
- * and run one after the other.  `group_stream` orders the group as a whole: the tables start
- * after everything issued on it so far, and it waits for all of them, so work issued on it
- * afterwards sees every table's results.  The same table must not appear twice.
- * Results are those of the n_tables single calls.  Returns the first error met (tables after
- * it are not started); MONO_ERR_ARG for n_tables < 0 or a null array.
+ * Grouped calls: one call, and one kernel launch per step of the path, for several tables
+ * (Section 3.1: a production model holds many embedding tables of very uneven size, most of
+ * them far too small to fill a GPU on their own).  Table i gets batch i: `tables`, `ids`,
+ * `n_ids`, `slot_offsets`, `n_bags`, `out` / `grad_pooled` are HOST arrays of `n_tables`
+ * entries whose elements are what the single-table call takes (device pointers, sizes).  The
+ * grid of every kernel is the concatenation of the grids the tables would launch one by one;
+ * tables of different dims share a launch (rows wider than 128 columns get a second one).
+ * The group's work runs on `group_stream`: it starts after everything issued so far on
+ * `group_stream` and on the tables' own streams, and whatever is issued next on any of them
+ * waits for it.  Tables created on `group_stream` itself need no such ordering and are the
+ * cheapest to group.  All tables must live on the current device; the same table must not
+ * appear twice; successive grouped calls that share tables[0] must use the same
+ * `group_stream`.  Results are those of the n_tables single calls.  Errors: the first one met
+ * while checking the arguments, before anything is enqueued; MONO_ERR_ARG for n_tables < 0
+ * or a null array.
+ *
+ * mono_group_prepare_push announces every table's next batch, as mono_prepare_push does for
+ * one table.  mono_group_apply_grads uses the announcements if every table of the group (with
+ * a batch that is not empty) is given exactly the batch it was announced; otherwise it
+ * forgets them all and groups and looks up the batches itself.
  */
+int mono_group_prepare_push(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
+                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
+                            void* group_stream);
 int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
                            float* const* out, void* group_stream);
@@ -310,7 +335,13 @@ int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids,
  *    GPU that loads the library, from load until the process exits.
  *  - The first call on a device looks up the array's device address once
  *    (no allocation, but a runtime query): make that first call before any
- *    CUDA stream capture begins on that device.
+ *    CUDA stream capture begins on that device.  The address is remembered for
+ *    the life of the process; a cudaDeviceReset in between invalidates it.
+ *  - The table's device must be the current device (MONO_ERR_ARG otherwise:
+ *    another device's copy of the array would be the wrong memory).
+ *  - With mono_timing_enable switched on, the call creates CUDA events for its
+ *    two launches like every other hot call; leave timing off where even that
+ *    is unwelcome.
  *  - All tables and all calls on a device share the one array, and it keeps
  *    whatever the previous call left in it.  Nothing in it needs clearing --
  *    each call overwrites the entries it reads -- but two calls that are in
@@ -320,6 +351,32 @@ int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids,
 #define MONO_NOALLOC_MAX_IDS (1u << 20)
 int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids,
                              const int64_t* slot_offsets, int64_t n_bags, float* out);
+
+/*
+ * Order point for the table's internal streams (the paper has no counterpart).  A hot call may
+ * leave work running on streams of the table's own (the sweep of mono_expire*, most of all);
+ * the next call on the table waits for it by itself.  mono_fence makes the table's stream wait
+ * for all of it now, without synchronising the host, so that an event the caller records on
+ * the table's stream afterwards marks the end of everything issued so far.
+ */
+int mono_fence(mono_table* t);
+
+/*
+ * Device-resident snapshot (Section 2.3: the parameter servers snapshot their state so that
+ * training can go back to it; here the copy stays in device memory, for callers that want to
+ * return to a state quickly -- benchmarks that repeat a timed region from the same state,
+ * what-if runs).  mono_snapshot_save copies the key store, the rows and accumulators, the
+ * free-row list, the counters and the sketch into a second set of buffers owned by the table
+ * (allocated on the first save: as much memory again as the table itself; MONO_ERR_NOMEM if
+ * that does not fit) and remembers the table's clock.  mono_snapshot_restore copies them back
+ * and resets the clock, so calls may again use any `now` >= the saved one; a batch announced
+ * with mono_prepare_push is forgotten.  Both are asynchronous device-to-device copies on the
+ * table's stream.  A table that was rehashed since the save cannot be restored
+ * (MONO_ERR_ARG), nor one that has no snapshot.  mono_snapshot_drop frees the copy.
+ */
+int mono_snapshot_save(mono_table* t);
+int mono_snapshot_restore(mono_table* t);
+int mono_snapshot_drop(mono_table* t);
 
 /* ---- inspection and fixtures: not on the hot path, all synchronise ---- */
 
@@ -376,12 +433,14 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed);
 int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, int64_t* n_out);
 
 /*
- * Insert n entries given as (id, count, last_seen, resident[, w, acc]).  IDs
- * must be distinct; an ID that is already tracked is skipped and
- * MONO_DEV_IMPORT_DUP is set.  resident[i] != 0 claims a row; its values come
+ * Insert n entries given as (id, count, last_seen, resident[, w, acc]).  An ID
+ * that is already tracked is skipped and MONO_DEV_IMPORT_DUP is set.  The IDs of
+ * one call must be distinct: this is not checked, and a repeated ID ends up in
+ * two cells (mono_audit reports it as a duplicate key).  resident[i] != 0 claims a row; its values come
  * from w/acc, or from the initialisation rule (and init_acc) when w or acc is
- * NULL.  count is clamped to the threshold.  Restores a snapshot, or pre-fills
- * a table to a chosen load.
+ * NULL.  count is clamped to the threshold; an entry without a row whose count
+ * is at the threshold (an admission that was refused for lack of a row) is admitted
+ * at its next occurrence.  Restores a snapshot, or pre-fills a table to a chosen load.
  */
 int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count,
                 const int64_t* last_seen, const uint8_t* resident, const float* w,

@@ -26,7 +26,8 @@ EXPORTS = [
     "mono_expire", "mono_lookup_pool_host", "mono_apply_grads_host", "mono_status", "mono_clear_errors",
     "mono_probe", "mono_read_rows", "mono_export", "mono_import", "mono_audit", "mono_last_cuda_error",
     "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc", "mono_export_touched", "mono_rehash", "mono_expire_slice", "mono_prepare_push",
-    "mono_group_lookup_pool", "mono_group_apply_grads",
+    "mono_group_lookup_pool", "mono_group_apply_grads", "mono_group_prepare_push", "mono_fence", "mono_snapshot_save", "mono_snapshot_restore",
+    "mono_snapshot_drop",
 ]
 
 
@@ -51,7 +52,8 @@ class mono_status_t(ctypes.Structure):
                 ("n_keys_dropped", ctypes.c_uint64), ("n_evictions_total", ctypes.c_uint64),
                 ("max_chain", ctypes.c_uint32), ("stash_used", ctypes.c_uint32), ("sum_ids", ctypes.c_uint64),
                 ("sum_unique", ctypes.c_uint64), ("sum_unique_resident", ctypes.c_uint64),
-                ("sum_new", ctypes.c_uint64), ("sum_single_resident", ctypes.c_uint64)]
+                ("sum_new", ctypes.c_uint64), ("sum_single_resident", ctypes.c_uint64),
+                ("scratch_reallocs", ctypes.c_uint64)]
 
 
 class mono_audit_t(ctypes.Structure):
@@ -97,6 +99,7 @@ def load_library(path: Optional[str] = None):
         "mono_expire": (ci, [vp, i64]),
         "mono_prepare_push": (ci, [vp, vp, i64, vp, i64]),
         "mono_expire_slice": (ci, [vp, i64, u32, u32]),
+        "mono_group_prepare_push": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp]),
         "mono_group_lookup_pool": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp]),
         "mono_group_apply_grads": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp, i64, vp]),
         "mono_lookup_pool_host": (ci, [vp, vp, i64, vp, i64, vp]),
@@ -113,6 +116,10 @@ def load_library(path: Optional[str] = None):
         "mono_last_cuda_error": (ctypes.c_char_p, [vp]),
         "mono_error_string": (ctypes.c_char_p, [ci]),
         "mono_lookup_pool_noalloc": (ci, [vp, vp, i64, vp, i64, vp]),
+        "mono_fence": (ci, [vp]),
+        "mono_snapshot_save": (ci, [vp]),
+        "mono_snapshot_restore": (ci, [vp]),
+        "mono_snapshot_drop": (ci, [vp]),
         "mono_timing_enable": (ci, [vp, ci]),
         "mono_timing_read": (ci, [vp, ctypes.POINTER(mono_timing_t), ci]),
     }
@@ -218,6 +225,14 @@ def _group_args(handles, ids, slot_offsets, vectors):
             ptrs(*[_ptr(x) for x in vectors]))
 
 
+def mono_group_prepare_push(handles, ids, slot_offsets, group_stream: int = 0) -> None:
+    """Announce every table's next batch (lists of device tensors, one per table)."""
+    n, tp, ip, nip, op, nbp, _ = _group_args(handles, ids, slot_offsets, ids)
+    code = load_library().mono_group_prepare_push(n, tp, ip, nip, op, nbp, group_stream or None)
+    if code != 0:
+        raise MonoError("mono_group_prepare_push", code)
+
+
 def mono_group_lookup_pool(handles, ids, slot_offsets, outs, group_stream: int = 0) -> None:
     """ids / slot_offsets / outs: lists of device tensors, one per table."""
     n, tp, ip, nip, op, nbp, vp_ = _group_args(handles, ids, slot_offsets, outs)
@@ -235,6 +250,22 @@ def mono_group_apply_grads(handles, ids, slot_offsets, grads, now: int, group_st
 
 def mono_expire_slice(t: int, now: int, slice_index: int, n_slices: int) -> None:
     _check("mono_expire_slice", load_library().mono_expire_slice(t, now, slice_index, n_slices), t)
+
+
+def mono_fence(t: int) -> None:
+    _check("mono_fence", load_library().mono_fence(t), t)
+
+
+def mono_snapshot_save(t: int) -> None:
+    _check("mono_snapshot_save", load_library().mono_snapshot_save(t), t)
+
+
+def mono_snapshot_restore(t: int) -> None:
+    _check("mono_snapshot_restore", load_library().mono_snapshot_restore(t), t)
+
+
+def mono_snapshot_drop(t: int) -> None:
+    _check("mono_snapshot_drop", load_library().mono_snapshot_drop(t), t)
 
 
 def mono_lookup_pool_host(t: int, ids, n_ids: int, slot_offsets, n_bags: int, out) -> None:

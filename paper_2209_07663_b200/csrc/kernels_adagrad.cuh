@@ -5,12 +5,14 @@
 // paper.
 //
 // Three cases, by how often the ID occurs in the batch:
+// Every ID has a segment of bag_of_sorted[] that lists the bags of its
+// occurrences (filed by the lookup when the batch was announced, else by
+// file_segments_kernel).
 //  - once (most distinct IDs of a long-tailed batch): its gradient is the
 //    pooled gradient of its one bag, so update_singletons_kernel updates the
 //    row straight from that bag's gradient row;
-//  - 2 .. kSegChunk times: file_segments_kernel drops each occurrence's
-//    bag into the ID's segment of bag_of_sorted[], and one lane group of
-//    reduce_adagrad_kernel gathers the segment's gradient rows;
+//  - 2 .. kSegChunk times: one lane group of reduce_adagrad_kernel gathers
+//    the gradient rows of the segment's bags;
 //  - more (the head of the Zipf distribution: one ID can own several percent of
 //    a batch): the segment is cut into parts of kSegChunk that separate groups
 //    reduce into fp64 partial sums, combined by one block per ID in a fixed
@@ -104,20 +106,22 @@ __device__ inline void reduce_segment(const Work& wk, const float* __restrict__ 
   }
 }
 
-// Every occurrence of a repeated ID that has a row is filed under its ID: its bag goes
-// into the ID's segment of bag_of_sorted[], at the occurrence's rank.  (The slot of an
-// ID that occurs once has been emptied by then, so its occurrence finds nothing.)
+// Every occurrence is filed under its ID: its bag goes into the ID's segment of
+// bag_of_sorted[], at the occurrence's rank.  Only for a push whose batch did not pass
+// through the lookup after mono_prepare_push (the lookup files the bags while it pools).
+__device__ inline void file_segments_body(const Work& wk, long long n_ids, long long n_bags, uint32_t vblock, uint32_t vgrid) {
+  const long long stride = (long long)vgrid * blockDim.x;
+  for (long long j = (long long)vblock * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
+    const uint2 o = wk.occ[j];
+    if (o.x == kNoSlot) continue;
+    const uint32_t seg = wk.bset[o.x].a;
+    const uint32_t bag = wk.occ_bag[j];
+    if (bag < n_bags) wk.bag_of_sorted[seg + o.y] = bag;
+  }
+}
 __global__ void __launch_bounds__(256)
 file_segments_kernel(Work wk, long long n_ids, long long n_bags) {
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
-    const uint32_t s = wk.occ_slot[j];
-    if (s == kNoSlot) continue;
-    const BatchSlot bs = wk.bset[s];
-    if (bs.key == kEmptyKey || bs.b == kNoRow) continue;
-    const uint32_t bag = wk.occ_bag[j];
-    if (bag < n_bags) wk.bag_of_sorted[bs.a + wk.occ_rank[j]] = bag;
-  }
+  file_segments_body(wk, n_ids, n_bags, blockIdx.x, gridDim.x);
 }
 
 // The IDs that occur once in the batch (most distinct IDs of a long-tailed batch): the
@@ -126,26 +130,29 @@ file_segments_kernel(Work wk, long long n_ids, long long n_bags) {
 // the order the batch first shows them, so the gradient rows are read roughly in order;
 // the lanes whose ID occurs once and has a row are served in turn by lane groups of G,
 // which read the bag's gradient row, the table row and its accumulator, and write both
-// back updated.
+// back updated.  The ID's slot of the per-call set is emptied on the way (every
+// occurrence has been filed by now).
 template <int G, int NV>
-__global__ void __launch_bounds__(256)
-update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
+__device__ inline void update_singletons_body(const TableView& tv, const Work& wk, const float* __restrict__ grad,
+                                              long long n_bags, uint32_t vblock, uint32_t vgrid) {
   constexpr int kGroups = 32 / G;
   const int lane = threadIdx.x & 31;
   const int gl = lane % G, grp = lane / G;
   const uint32_t n = tv.st->n_unique;
-  const uint32_t n_warps = (gridDim.x * blockDim.x) >> 5;
+  const uint32_t n_warps = (vgrid * blockDim.x) >> 5;
   const uint32_t n_rounds = (n + 31) / 32;
   unsigned int n_single = 0;
-  for (uint32_t r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rounds; r += n_warps) {
+  for (uint32_t r = (vblock * blockDim.x + threadIdx.x) >> 5; r < n_rounds; r += n_warps) {
     const uint32_t u = r * 32 + lane;
     uint32_t row_word = kNoRow, bag = 0;
     unsigned long long id = 0;
     bool single = false;
     if (u < n && wk.ulen[u] == 1u) {
+      BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
+      wk.bset[wk.uslot[u]] = e;
       row_word = wk.urow[u];
       if (row_word != kNoRow) {
-        bag = wk.occ_bag[wk.uocc[u]];
+        bag = wk.bag_of_sorted[wk.useg[u]];
         single = bag < n_bags;
         if (row_word & kFreshBit) id = wk.uid[u];
       }
@@ -183,6 +190,11 @@ update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, 
   }
   if (lane == 0 && n_single) atomicAdd(&tv.st->sum_single_resident, (unsigned long long)n_single);
 }
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
+  update_singletons_body<G, NV>(tv, wk, grad, n_bags, blockIdx.x, gridDim.x);
+}
 
 // One lane group per work item.  Items [0, n_parts) are the parts of the long
 // segments (the heaviest items, so they are started first): a group reduces
@@ -190,16 +202,21 @@ update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, 
 // up afterwards.  Items [n_parts, n_parts + n_multi) are the repeated IDs: a
 // group empties the ID's slot of the per-call set (every occurrence has been
 // filed by now), and when the segment is short reduces it and updates the row.
+// `which` selects the items of one launch: kReduceParts, kReduceShort (the repeated IDs need
+// nothing from the kernels that order the parts, so they can run beside them), or both.
+enum : int { kReduceParts = 1, kReduceShort = 2 };
+
 template <int G, int NV>
-__global__ void __launch_bounds__(256)
-reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
+__device__ inline void reduce_adagrad_body(const TableView& tv, const Work& wk, const float* __restrict__ grad,
+                                           long long n_bags, int which, uint32_t vblock, uint32_t vgrid) {
   const uint32_t n = tv.st->n_multi;
   uint32_t n_parts = tv.st->n_parts;
   if (n_parts > wk.max_parts) n_parts = wk.max_parts;
-  const uint32_t n_items = n + n_parts;
+  const uint32_t first_item = (which & kReduceParts) ? 0u : n_parts;
+  const uint32_t n_items = (which & kReduceShort) ? n + n_parts : n_parts;
   const int gl = threadIdx.x % G;
-  const uint32_t groups = (gridDim.x * blockDim.x) / G;
-  for (uint32_t item = (blockIdx.x * blockDim.x + threadIdx.x) / G; item < n_items; item += groups) {
+  const uint32_t groups = (vgrid * blockDim.x) / G;
+  for (uint32_t item = first_item + (vblock * blockDim.x + threadIdx.x) / G; item < n_items; item += groups) {
     D4 s[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
@@ -242,16 +259,21 @@ reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, lon
   }
 }
 
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags, int which) {
+  reduce_adagrad_body<G, NV>(tv, wk, grad, n_bags, which, blockIdx.x, gridDim.x);
+}
+
 // First level of the combination for very long segments: one block adds up one
 // group of kFoldWidth consecutive parts of one ID, column by column, and leaves
 // the sum in the group's first part.  Fixed order within the block.
-__global__ void __launch_bounds__(256)
-fold_partials_kernel(TableView tv, Work wk) {
+__device__ inline void fold_partials_body(const TableView& tv, const Work& wk, uint32_t vblock, uint32_t vgrid) {
   __shared__ double s_sum[8][256];
   uint32_t n_folds = tv.st->n_folds;
   if (n_folds > wk.max_folds) n_folds = wk.max_folds;
   const uint32_t dim = tv.dim;
-  for (uint32_t fi = blockIdx.x; fi < n_folds; fi += gridDim.x) {
+  for (uint32_t fi = vblock; fi < n_folds; fi += vgrid) {
     const uint32_t li = wk.fold_li[fi], f = wk.fold_idx[fi];
     const uint32_t u = wk.long_u[li];
     if (wk.urow[u] == kNoRow) continue;               // block-uniform
@@ -285,19 +307,21 @@ fold_partials_kernel(TableView tv, Work wk) {
   }
 }
 
+__global__ void __launch_bounds__(256)
+fold_partials_kernel(TableView tv, Work wk) { fold_partials_body(tv, wk, blockIdx.x, gridDim.x); }
+
 // One block per long ID: the block's threads split into slices of the parts
 // (or, for a very long segment, of the group sums fold_partials_kernel left),
 // one column each; the slices' sums are added in increasing order, so the
 // combination order is fixed.
 constexpr int kCombineThreads = 256;
-__global__ void __launch_bounds__(kCombineThreads)
-combine_adagrad_kernel(TableView tv, Work wk) {
+__device__ inline void combine_adagrad_body(const TableView& tv, const Work& wk, uint32_t vblock, uint32_t vgrid) {
   constexpr int kMaxSlices = 8;
   __shared__ double s_sum[kMaxSlices][256];
   uint32_t n_long = tv.st->n_long;
   if (n_long > wk.max_long) n_long = wk.max_long;
   const uint32_t dim = tv.dim;
-  for (uint32_t li = blockIdx.x; li < n_long; li += gridDim.x) {
+  for (uint32_t li = vblock; li < n_long; li += vgrid) {
     const uint32_t u = wk.long_u[li];
     const uint32_t row_word = wk.urow[u];
     if (row_word == kNoRow) continue;                 // block-uniform
@@ -336,5 +360,8 @@ combine_adagrad_kernel(TableView tv, Work wk) {
     }
   }
 }
+
+__global__ void __launch_bounds__(kCombineThreads)
+combine_adagrad_kernel(TableView tv, Work wk) { combine_adagrad_body(tv, wk, blockIdx.x, gridDim.x); }
 
 }  // namespace mono

@@ -21,9 +21,11 @@
 namespace mono {
 
 // One slot of the per-call set.  `a` is the ID's multiplicity while the batch
-// is being counted; once the table phases have run, the slot of an ID that
-// occurs once is empty again, and that of a repeated ID holds the start of its
-// segment in bag_of_sorted[] in `a` and its row word in `b`.
+// is being counted.  Once the distinct IDs have been looked up in the key store
+// (table_update_kernel), `a` is the start of the ID's segment in bag_of_sorted[]
+// and `b` the row the ID owned before this push (kNoRow if none): what an
+// occurrence needs to pool the row and to file its bag.  The kernels that
+// update the rows empty the slots again for the next call.
 struct __align__(16) BatchSlot {
   unsigned long long key;
   unsigned int a;
@@ -48,16 +50,17 @@ struct Work {
   BatchSlot* bset;           // [primary_mask + 1 + secondary_mask + 1]
   uint32_t primary_mask;     // primary tier: slots [0, primary_mask]
   uint32_t secondary_mask;   // secondary tier: slots primary_mask + 1 + [0, secondary_mask]
-  uint32_t* occ_slot;        // [max_ids] slot of each occurrence, kNoSlot if padding / outside bags
-  uint32_t* occ_rank;        // [max_ids] rank of the occurrence among those of its ID
+  uint2* occ;                // [max_ids] per occurrence: x = slot of its ID (kNoSlot if padding / outside bags),
+                             //           y = rank of the occurrence among those of its ID
   uint32_t* occ_bag;         // [max_ids] bag of each occurrence
-  uint32_t* bag_of_sorted;   // [max_ids] bags of the occurrences of repeated IDs, grouped by ID
+  uint32_t* bag_of_sorted;   // [max_ids] bags of the occurrences, grouped by ID (an ID seen once has a segment of one)
   unsigned long long* uid;   // [max_ids] distinct IDs
   uint32_t* uslot;           // [max_ids] slot of each distinct ID
-  uint32_t* uocc;            // [max_ids] one occurrence of each distinct ID (the occurrence, if there is only one)
   uint32_t* useg;            // [max_ids] start of the ID's segment in bag_of_sorted
   uint32_t* ulen;            // [max_ids] multiplicity of the ID in this batch
   uint32_t* urow;            // [max_ids] row word per distinct ID (kNoRow / row | kFreshBit)
+  unsigned long long* ucell; // [max_ids] where the key store holds the ID (kNoCell: nowhere), from the look-up
+                             //           that mono_prepare_push does ahead of the push
   uint32_t* ins_list;        // [max_ids] distinct IDs that are not in the key store yet
   uint32_t* multi_list;      // [max_ids / 2 + 1] distinct IDs that occur more than once
   uint32_t* long_u;          // [max_long] distinct IDs whose segment is reduced in parts
@@ -71,16 +74,37 @@ struct Work {
   uint32_t max_long, max_parts, max_folds;
 };
 
-// bag -> occurrences: every occurrence learns which bag it belongs to.
+// A bag is well formed when 0 <= offsets[b] <= offsets[b+1] <= n_ids; any other bag is
+// treated as empty by every kernel.
+__device__ inline bool bag_ok(long long lo, long long hi, long long n_ids) { return lo >= 0 && hi >= lo && hi <= n_ids; }
+
+// bag -> occurrences: every occurrence learns which bag it belongs to.  A malformed bag
+// writes nothing, sets the sticky condition bit and marks the call, so that the grouping
+// pass checks every occurrence against the bag it claims (occurrence_covered).
+__device__ inline void fill_occ_bag_body(const long long* __restrict__ offsets, long long n_bags, long long n_ids,
+                                         uint32_t* __restrict__ occ_bag, DevState* st, uint32_t vblock, uint32_t vgrid) {
+  const long long stride = (long long)vgrid * blockDim.x;
+  for (long long b = (long long)vblock * blockDim.x + threadIdx.x; b < n_bags; b += stride) {
+    const long long lo = offsets[b], hi = offsets[b + 1];
+    if (!bag_ok(lo, hi, n_ids)) { atomicOr(&st->error_bits, 4u /* MONO_DEV_BAD_OFFSETS */); st->call_bad_offsets = 1u; continue; }
+    for (long long j = lo; j < hi; ++j) occ_bag[j] = (uint32_t)b;
+  }
+}
 __global__ void __launch_bounds__(256)
 fill_occ_bag_kernel(const long long* __restrict__ offsets, long long n_bags, long long n_ids,
                     uint32_t* __restrict__ occ_bag, DevState* st) {
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x; b < n_bags; b += stride) {
-    const long long lo = offsets[b], hi = offsets[b + 1];
-    if (lo < 0 || hi < lo || hi > n_ids) { atomicOr(&st->error_bits, 4u); continue; }
-    for (long long j = lo; j < hi; ++j) occ_bag[j] = (uint32_t)b;
-  }
+  fill_occ_bag_body(offsets, n_bags, n_ids, occ_bag, st, blockIdx.x, gridDim.x);
+}
+
+// Only used when the call's offsets are malformed: does a well-formed bag cover occurrence j,
+// and is it the one occ_bag[j] names?  (occ_bag[j] may be left over from an earlier call where
+// no bag of this call covers j; the test against this call's offsets settles it either way.)
+__device__ inline bool occurrence_covered(const uint32_t* __restrict__ occ_bag, const long long* __restrict__ offsets,
+                                          long long n_bags, long long n_ids, long long j) {
+  const uint32_t b = occ_bag[j];
+  if ((long long)b >= n_bags) return false;
+  const long long lo = offsets[b], hi = offsets[b + 1];
+  return bag_ok(lo, hi, n_ids) && j >= lo && j < hi;
 }
 
 // Sum of `v` over the block and this thread's exclusive prefix, with two
@@ -109,10 +133,9 @@ __device__ inline unsigned long long block_exclusive_scan(unsigned long long v, 
 
 // One block per tile of kTileIds consecutive occurrences.
 // (eight blocks per SM: measured 0.207 ms on the largest configuration against 0.234 ms with six)
-__global__ void __launch_bounds__(kTileThreads, 8)
-dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long n_ids,
-                  const long long* __restrict__ offsets, long long n_bags, DevState* st,
-                  unsigned long long seed) {
+__device__ inline void dedup_tile_body(const Work& wk, const unsigned long long* __restrict__ ids, long long n_ids,
+                                       const long long* __restrict__ offsets, long long n_bags, DevState* st,
+                                       unsigned long long seed, uint32_t vblock) {
   constexpr int kPerThread = kTileIds / kTileThreads;
   __shared__ unsigned long long s_key[kTileSlots];
   __shared__ unsigned int s_cnt[kTileSlots];     // multiplicity in the tile, then base rank
@@ -124,11 +147,13 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
   long long first = offsets[0], last = offsets[n_bags];
   if (first < 0) first = 0;
   if (last > n_ids) last = n_ids;
+  const bool check_each = st->call_bad_offsets != 0u;     // set by fill_occ_bag_kernel, earlier on this stream
+  if (check_each) { first = 0; last = n_ids; }
   __syncthreads();
 
   // 1. group the tile's occurrences in shared memory.  The thread whose occurrence puts an ID
   //    into the tile's table owns that ID for the rest of the kernel.
-  const long long tile0 = (long long)blockIdx.x * kTileIds;
+  const long long tile0 = (long long)vblock * kTileIds;
   unsigned long long my_id[kPerThread];
   uint32_t my_slot[kPerThread], my_rank[kPerThread];
   bool own[kPerThread];
@@ -138,6 +163,8 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
     const long long j = tile0 + k * kTileThreads + threadIdx.x;
     unsigned long long id = kEmptyKey;
     if (j >= first && j < last) id = ids[j];
+    // malformed offsets: an occurrence that no well-formed bag covers is padding, as in the lookup
+    if (check_each && id != kEmptyKey && !occurrence_covered(wk.occ_bag, offsets, n_bags, n_ids, j)) id = kEmptyKey;
     my_id[k] = id;
     my_slot[k] = kNoSlot;
     my_rank[k] = 0;
@@ -229,7 +256,6 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
     if (is_new[k]) {
       wk.uid[my_u] = my_id[k];
       wk.uslot[my_u] = g[k];
-      wk.uocc[my_u] = (uint32_t)(tile0 + k * kTileThreads + threadIdx.x);     // the owner's own occurrence
       ++my_u;
     }
   }
@@ -240,10 +266,16 @@ dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long
     const long long j = tile0 + k * kTileThreads + threadIdx.x;
     if (j < n_ids) {
       const uint32_t s = my_slot[k];
-      wk.occ_slot[j] = s == kNoSlot ? kNoSlot : s_gslot[s];
-      wk.occ_rank[j] = s == kNoSlot ? 0u : s_cnt[s] + my_rank[k];
+      wk.occ[j] = s == kNoSlot ? make_uint2(kNoSlot, 0u) : make_uint2(s_gslot[s], s_cnt[s] + my_rank[k]);
     }
   }
+}
+
+__global__ void __launch_bounds__(kTileThreads, 8)
+dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long n_ids,
+                  const long long* __restrict__ offsets, long long n_bags, DevState* st,
+                  unsigned long long seed) {
+  dedup_tile_body(wk, ids, n_ids, offsets, n_bags, st, seed, blockIdx.x);
 }
 
 }  // namespace mono

@@ -3,6 +3,7 @@
 // parameter pull of Section 2.2; sum pooling per bag).
 #pragma once
 
+#include "kernels_dedup.cuh"
 #include "table_layout.cuh"
 
 namespace mono {
@@ -16,21 +17,22 @@ __device__ inline bool thread_lookup(const TableView& tv, unsigned long long id,
   const unsigned long long h0 = tv.hash0(id);
   const Cell* b = tv.cells + (h0 & tv.bucket_mask) * kCellsPerBucket;
   const uint32_t first = (uint32_t)(h0 >> 62);
-  Cell c[kCellsPerBucket - 1];
   const Cell c0 = load_cell_ro(b + first);
   if (c0.key == id) { *meta = c0.meta; return true; }
-#pragma unroll
-  for (uint32_t k = 1; k < kCellsPerBucket; ++k) c[k - 1] = load_cell_ro(b + ((first + k) & 3u));
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket - 1; ++k)
-    if (c[k].key == id) { *meta = c[k].meta; return true; }
-  Cell d[kCellsPerBucket];
+  // the other three cells of the bucket, requested together (named values, not an array: an
+  // indexed array here ends up in local memory)
+  const Cell c1 = load_cell_ro(b + ((first + 1u) & 3u));
+  const Cell c2 = load_cell_ro(b + ((first + 2u) & 3u));
+  const Cell c3 = load_cell_ro(b + ((first + 3u) & 3u));
+  if (c1.key == id) { *meta = c1.meta; return true; }
+  if (c2.key == id) { *meta = c2.meta; return true; }
+  if (c3.key == id) { *meta = c3.meta; return true; }
   b = tv.cells + tv.bucket1(id) * kCellsPerBucket;
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k) d[k] = load_cell_ro(b + k);
-#pragma unroll
-  for (uint32_t k = 0; k < kCellsPerBucket; ++k)
-    if (d[k].key == id) { *meta = d[k].meta; return true; }
+  const Cell d0 = load_cell_ro(b), d1 = load_cell_ro(b + 1), d2 = load_cell_ro(b + 2), d3 = load_cell_ro(b + 3);
+  if (d0.key == id) { *meta = d0.meta; return true; }
+  if (d1.key == id) { *meta = d1.meta; return true; }
+  if (d2.key == id) { *meta = d2.meta; return true; }
+  if (d3.key == id) { *meta = d3.meta; return true; }
   for (unsigned i = 0; i < stash_hw; ++i) {
     const Cell s = load_cell_ro(tv.stash + i);
     if (s.key == id) { *meta = s.meta; return true; }
@@ -40,6 +42,8 @@ __device__ inline bool thread_lookup(const TableView& tv, unsigned long long id,
 
 // The same look-up for a caller that goes on to modify the entry: it also returns where
 // the entry is (index into cells[], or n_cells + i for stash cell i; kNoCell if nowhere).
+// Its kernel stores metadata into the cells it reads, so the loads are ordinary (coherent)
+// 16-byte loads, not the read-only path.
 constexpr unsigned long long kNoCell = 0xFFFFFFFFFFFFFFFFull;
 
 __device__ inline unsigned long long thread_locate(const TableView& tv, unsigned long long id, unsigned stash_hw,
@@ -47,21 +51,21 @@ __device__ inline unsigned long long thread_locate(const TableView& tv, unsigned
   const unsigned long long h0 = tv.hash0(id);
   const unsigned long long base0 = (h0 & tv.bucket_mask) * kCellsPerBucket;
   const uint32_t first = (uint32_t)(h0 >> 62);
-  const Cell c0 = load_cell_ro(tv.cells + base0 + first);
+  const Cell c0 = load_cell_whole(tv.cells + base0 + first);
   if (c0.key == id) { *meta = c0.meta; return base0 + first; }
 #pragma unroll
   for (uint32_t k = 1; k < kCellsPerBucket; ++k) {
-    const Cell c = load_cell_ro(tv.cells + base0 + ((first + k) & 3u));
+    const Cell c = load_cell_whole(tv.cells + base0 + ((first + k) & 3u));
     if (c.key == id) { *meta = c.meta; return base0 + ((first + k) & 3u); }
   }
   const unsigned long long base1 = tv.bucket1(id) * kCellsPerBucket;
 #pragma unroll
   for (uint32_t k = 0; k < kCellsPerBucket; ++k) {
-    const Cell c = load_cell_ro(tv.cells + base1 + k);
+    const Cell c = load_cell_whole(tv.cells + base1 + k);
     if (c.key == id) { *meta = c.meta; return base1 + k; }
   }
   for (unsigned i = 0; i < stash_hw; ++i) {
-    const Cell s = load_cell_ro(tv.stash + i);
+    const Cell s = load_cell_whole(tv.stash + i);
     if (s.key == id) { *meta = s.meta; return (tv.bucket_mask + 1) * kCellsPerBucket + i; }
   }
   return kNoCell;
@@ -89,12 +93,13 @@ probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long
   }
 }
 
-// sum += rows idx[0..K), in that order; all K loads are issued before the first add.
+// sum += the rows that lanes k .. k+K-1 of the group hold in `mine`, in that order; all K loads
+// are issued before the first add.
 template <int K, int G, int NV>
-__device__ inline void add_rows(const TableView& tv, const uint32_t* __restrict__ idx, int gl, float4 (&sum)[NV]) {
+__device__ inline void add_rows(const TableView& tv, unsigned gmask, uint32_t mine, uint32_t k, int gl, float4 (&sum)[NV]) {
   uint32_t row[K];
 #pragma unroll
-  for (int k = 0; k < K; ++k) row[k] = __ldg(idx + k);
+  for (int q = 0; q < K; ++q) row[q] = __shfl_sync(gmask, mine, k + q, G);
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     const uint32_t c4 = gl + v * G;
@@ -108,41 +113,82 @@ __device__ inline void add_rows(const TableView& tv, const uint32_t* __restrict_
   }
 }
 
+// Where the forward gets the row of an occurrence from:
+//  kFromRows  the array probe_rows_kernel filled (two kernels);
+//  kFromKeys  the key store, looked up here (one kernel: no row-index array in between);
+//  kFromSet   the per-call set of a batch that mono_prepare_push announced: every distinct ID was
+//             looked up once ahead of the call, its slot holds the row and the start of its segment,
+//             and the occurrence files its bag there for the push while it is at it.
+enum : int { kFromRows = 0, kFromKeys = 1, kFromSet = 2 };
+
+struct GatherSource {
+  const uint32_t* occ_row;                 // kFromRows
+  const unsigned long long* ids;           // kFromKeys
+  const uint2* occ;                        // kFromSet
+  const BatchSlot* bset;                    // kFromSet
+  uint32_t* bag_of_sorted;                 // kFromSet
+};
+
 // Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
 // dim so that a lane owns NV 16-byte column vectors) adds up the rows of the
-// bag's IDs, in ID order, so the fp32 sum has one fixed order.  The row
-// indices are known, so the loads of four rows are issued together; what is
-// left of the bag after the batches of four is added in one batch of its exact
-// size.  The kernel is bound by instruction issue, not by memory, so there are
-// no per-row validity tests (step 1 points an ID without a row at the zero row)
-// and no loads or adds for padding (measured: batches padded with the zero row
-// 0.31 ms on the largest configuration, exact tails 0.26 ms).
-template <int G, int NV>
-__global__ void __launch_bounds__(256)
-gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long n_ids,
-                   const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out) {
+// bag's IDs, in ID order, so the fp32 sum has one fixed order.  The lanes of the
+// group first resolve G occurrences of the bag at once, one each (row index read,
+// key store probed, or slot of the per-call set read, depending on SRC); the row
+// indices then go round the group by shuffle, so the loads of four rows are issued
+// together; what is left after the batches of four is added in one batch of its
+// exact size.  An ID without a row resolves to the table's all-zero row, so there
+// are no per-row validity tests and no loads or adds for padding.
+template <int G, int NV, int SRC>
+__device__ inline void gather_pool_body(const TableView& tv, const GatherSource& src, long long n_ids,
+                                        const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out,
+                                        uint32_t vblock, uint32_t vgrid) {
   const int gl = threadIdx.x % G;
+  const unsigned gmask = G == 32 ? 0xFFFFFFFFu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   const uint32_t dim = tv.dim;
+  const uint32_t zero_row = (uint32_t)tv.capacity;
+  unsigned stash_hw = 0;
+  if (SRC == kFromKeys) stash_hw = tv.st->stash_hw;
   const long long groups_per_block = blockDim.x / G;
-  const long long stride = (long long)gridDim.x * groups_per_block;
-  for (long long bag = (long long)blockIdx.x * groups_per_block + threadIdx.x / G; bag < n_bags; bag += stride) {
+  const long long stride = (long long)vgrid * groups_per_block;
+  for (long long bag = (long long)vblock * groups_per_block + threadIdx.x / G; bag < n_bags; bag += stride) {
     long long lo = offsets[bag], hi = offsets[bag + 1];
-    if (lo < 0 || hi < lo || hi > n_ids) {
+    if (lo < 0 || hi < lo || hi > n_ids) {                 // not a well-formed bag: flagged and treated as empty
       if (gl == 0) atomicOr(&tv.st->error_bits, 4u /* MONO_DEV_BAD_OFFSETS */);
       lo = hi = 0;
     }
     float4 sum[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) sum[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const uint32_t* idx = occ_row + lo;
     const uint32_t n = (uint32_t)(hi - lo);              // a call has fewer than 2^31 IDs
-    uint32_t i = 0;
-    for (; i + 4 <= n; i += 4) add_rows<4, G, NV>(tv, idx + i, gl, sum);
-    switch (n - i) {
-      case 3: add_rows<3, G, NV>(tv, idx + i, gl, sum); break;
-      case 2: add_rows<2, G, NV>(tv, idx + i, gl, sum); break;
-      case 1: add_rows<1, G, NV>(tv, idx + i, gl, sum); break;
-      default: break;
+    for (uint32_t base = 0; base < n; base += G) {
+      // this lane's occurrence of the round
+      uint32_t mine = zero_row;
+      if (base + gl < n) {
+        const long long j = lo + base + gl;
+        if (SRC == kFromRows) {
+          mine = __ldg(src.occ_row + j);
+        } else if (SRC == kFromKeys) {
+          const unsigned long long id = __ldg(src.ids + j);
+          unsigned long long meta = 0;
+          if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) mine = meta_row(meta);
+        } else {
+          const uint2 o = __ldg(src.occ + j);
+          if (o.x != kNoSlot) {
+            const uint4 bs = __ldg(reinterpret_cast<const uint4*>(src.bset + o.x));   // key (x, y), segment start, row
+            if (bs.w != kNoRow) mine = bs.w;
+            src.bag_of_sorted[bs.z + o.y] = (uint32_t)bag;
+          }
+        }
+      }
+      const uint32_t cnt = n - base < (uint32_t)G ? n - base : (uint32_t)G;
+      uint32_t k = 0;
+      for (; k + 4 <= cnt; k += 4) add_rows<4, G, NV>(tv, gmask, mine, k, gl, sum);
+      switch (cnt - k) {
+        case 3: add_rows<3, G, NV>(tv, gmask, mine, k, gl, sum); break;
+        case 2: add_rows<2, G, NV>(tv, gmask, mine, k, gl, sum); break;
+        case 1: add_rows<1, G, NV>(tv, gmask, mine, k, gl, sum); break;
+        default: break;
+      }
     }
     float4* dst = reinterpret_cast<float4*>(out + bag * (long long)dim);
 #pragma unroll
@@ -151,6 +197,13 @@ gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long
       if (c4 * 4u < dim) dst[c4] = sum[v];
     }
   }
+}
+
+template <int G, int NV, int SRC>
+__global__ void __launch_bounds__(256)
+gather_pool_kernel(TableView tv, GatherSource src, long long n_ids, const long long* __restrict__ offsets,
+                   long long n_bags, float* __restrict__ out) {
+  gather_pool_body<G, NV, SRC>(tv, src, n_ids, offsets, n_bags, out, blockIdx.x, gridDim.x);
 }
 
 }  // namespace mono

@@ -28,7 +28,7 @@ __device__ inline uint32_t alloc_row(const TableView& tv) {
 // ID needs a row, whether it must be inserted into the key store (it then gets
 // a place in ins_list[]), whether it occurs more than once in the batch (a
 // place in multi_list[]) and how many entries of bag_of_sorted[] its segment
-// takes; one thread does the counter updates for the whole block, so counters
+// takes (its multiplicity); one thread does the counter updates for the whole block, so counters
 // that every admission would otherwise hit are touched once per block and
 // round.  All threads of the block must call.
 struct BlockAlloc {
@@ -112,75 +112,106 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
   }
 }
 
-// Phase 2 of mono_apply_grads: one thread per distinct ID (its own look-up, the cell an
-// insertion prefers first: measured 0.210 ms on the largest configuration at six blocks per
-// SM, against 0.222 ms for look-ups shared within quads, which need twice the registers).
-// Tracked IDs get count += multiplicity (saturating at the
-// threshold), last_seen = now, and a row if the count has reached the
-// threshold; the rest are queued for insertion.  No cell moves during this
-// kernel, so the thread whose ID sits in a cell owns it.  IDs that end up with a
-// row and occur more than once also get their segment of bag_of_sorted[] here.
-__global__ void __launch_bounds__(256, 6)
-table_update_kernel(TableView tv, Work wk, uint32_t now) {
+// Phase 2 of a push: one thread per distinct ID, in up to two halves.
+//
+//  kLookUp  (can run ahead of the push, when mono_prepare_push announced the batch: it changes
+//           nothing in the table) -- the ID's multiplicity is read from the per-call set, the ID is
+//           looked up in the key store (the cell an insertion prefers first), every ID is given its
+//           segment of bag_of_sorted[] and, if it occurs more than once, its place in multi_list[];
+//           the ID's slot of the per-call set is rewritten to (segment start, row owned so far),
+//           which is what the occurrences need, and the cell is remembered in ucell[].
+//  kCommit  (the push itself) -- a tracked ID gets count += multiplicity (saturating at the
+//           threshold), last_seen = now, and a row if the count has reached the threshold; an ID
+//           the key store does not hold is queued for insertion.  With kLookUp in an earlier
+//           kernel, the remembered cell is read again (one line in, one out) and the search is
+//           repeated only if the key is no longer there.
+//
+// Both halves in one kernel is the push that was not announced.  No cell moves during either
+// half, so the thread whose ID sits in a cell owns it.
+enum : int { kLookUp = 1, kCommit = 2 };
+
+__device__ inline Cell* cell_address(const TableView& tv, unsigned long long cell, unsigned long long n_cells) {
+  return cell < n_cells ? tv.cells + cell : tv.stash + (cell - n_cells);
+}
+
+template <int MODE>
+__device__ inline void table_update_body(const TableView& tv, const Work& wk, uint32_t now, uint32_t vblock, uint32_t vgrid) {
   __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_unique;
   const unsigned stash_hw = tv.st->stash_hw;
   const unsigned long long n_cells = (tv.bucket_mask + 1) * kCellsPerBucket;
   const int lane = threadIdx.x & 31;
   unsigned int n_res = 0;
-  for (uint32_t base = blockIdx.x * blockDim.x; base < n; base += gridDim.x * blockDim.x) {   // block-uniform
+  for (uint32_t base = vblock * blockDim.x; base < n; base += vgrid * blockDim.x) {   // block-uniform
     const uint32_t u = base + threadIdx.x;
     const bool active = u < n;
-    unsigned long long id = kEmptyKey;
+    unsigned long long id = kEmptyKey, meta = 0, cell = kNoCell;
     uint32_t m = 0, slot = 0;
     if (active) {
       id = wk.uid[u];
-      slot = wk.uslot[u];
-      m = wk.bset[slot].a;
+      if (MODE & kLookUp) {
+        slot = wk.uslot[u];
+        m = wk.bset[slot].a;
+        cell = thread_locate(tv, id, stash_hw, &meta);
+      } else {
+        m = wk.ulen[u];
+        cell = wk.ucell[u];
+        if (cell != kNoCell) {
+          const Cell c = load_cell_whole(cell_address(tv, cell, n_cells));
+          if (c.key == id) meta = c.meta;
+          else cell = thread_locate(tv, id, stash_hw, &meta);          // moved since the look-up: search again
+        }
+      }
     }
-    unsigned long long meta = 0;
-    const unsigned long long cell = active ? thread_locate(tv, id, stash_hw, &meta) : kNoCell;
     const bool hit = cell != kNoCell;
     uint32_t low = meta_low(meta);
-    bool resident = false, need_row = false;
-    if (hit) {
-      resident = (low & kResidentBit) != 0;
-      if (!resident) {
-        const unsigned long long c = (unsigned long long)low + m;
-        low = c < tv.threshold ? (uint32_t)c : tv.threshold;
-        need_row = low >= tv.threshold;
-      }
+    const bool resident = hit && (low & kResidentBit) != 0;
+    bool need_row = false;
+    if ((MODE & kCommit) && hit && !resident) {
+      const unsigned long long c = (unsigned long long)low + m;
+      low = c < tv.threshold ? (uint32_t)c : tv.threshold;
+      need_row = low >= tv.threshold;
     }
-    // a segment is reserved for every repeated ID that may end up with a row
-    // (if the row is refused, the segment stays unused)
-    const uint32_t seg_len = (hit && (resident || need_row) && m > 1) ? m : 0u;
-    const Reservation rv = block_reserve(tv, &sh, need_row, hit && m > 1, active && !hit, seg_len);
+    const Reservation rv = block_reserve(tv, &sh, need_row, (MODE & kLookUp) && m > 1, (MODE & kCommit) && active && !hit,
+                                         (MODE & kLookUp) ? m : 0u);
     if (!active) continue;
-    wk.ulen[u] = m;
-    if (hit) {
-      uint32_t row_word = kNoRow;
-      // every ID of the batch that has a row is trained in this call: mark it for the next sync
-      if (resident) { row_word = low & kRowMask; low |= kTouchedBit; }
-      else if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
-      Cell* where = cell < n_cells ? tv.cells + cell : tv.stash + (cell - n_cells);
-      where->meta = make_meta(now, low);
-      wk.urow[u] = row_word;
+    if (MODE & kLookUp) {
+      wk.ulen[u] = m;
       wk.useg[u] = rv.seg_start;
-      // a repeated ID leaves its segment and row in the slot for its occurrences to find; an ID that
-      // occurs once is updated from urow/uocc, and nobody needs its slot any more: empty it for the next call
-      BatchSlot bs; bs.key = m > 1 ? id : kEmptyKey; bs.a = m > 1 ? rv.seg_start : 0u; bs.b = m > 1 ? row_word : 0u;
+      if (!(MODE & kCommit)) wk.ucell[u] = cell;
+      BatchSlot bs; bs.key = id; bs.a = rv.seg_start; bs.b = resident ? (low & kRowMask) : kNoRow;
       wk.bset[slot] = bs;
       if (m > 1) wk.multi_list[rv.multi_pos] = u;
-      if (row_word != kNoRow) {
-        ++n_res;
-        if (m > kSegChunk) register_long(tv, wk, u, m);
+    }
+    if (MODE & kCommit) {
+      if (hit) {
+        uint32_t row_word = kNoRow;
+        // every ID of the batch that has a row is trained in this call: mark it for the next sync
+        if (resident) { row_word = low & kRowMask; low |= kTouchedBit; }
+        else if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
+        cell_address(tv, cell, n_cells)->meta = make_meta(now, low);
+        wk.urow[u] = row_word;
+        if (row_word != kNoRow) {
+          ++n_res;
+          if (m > kSegChunk) register_long(tv, wk, u, m);
+        }
+      } else {
+        wk.ins_list[rv.ins_pos] = u;
       }
-    } else {
-      wk.ins_list[rv.ins_pos] = u;
     }
   }
-  for (int o = 16; o > 0; o >>= 1) n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
-  if (lane == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
+  if (MODE & kCommit) {
+    for (int o = 16; o > 0; o >>= 1) n_res += __shfl_down_sync(0xFFFFFFFFu, n_res, o);
+    if (lane == 0 && n_res) atomicAdd(&tv.st->sum_unique_resident, (unsigned long long)n_res);
+  }
+}
+
+// (six blocks per SM: measured 0.210 ms on the largest configuration for both halves in one kernel, against
+// 0.222 ms for look-ups shared within quads, which need twice the registers)
+template <int MODE>
+__global__ void __launch_bounds__(256, 6)
+table_update_kernel(TableView tv, Work wk, uint32_t now) {
+  table_update_body<MODE>(tv, wk, now, blockIdx.x, gridDim.x);
 }
 
 // Put `item` (a key that is in no cell) into the key store.  Lock-free against
@@ -253,30 +284,30 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
 // Probabilistic filter, between phases 2 and 3: every distinct ID that is not in the key
 // store adds its multiplicity to one counter per sketch row.  All additions of a batch are
 // done before any estimate is read (next kernel), so the outcome does not depend on order.
-__global__ void __launch_bounds__(256)
-sketch_add_kernel(TableView tv, Work wk) {
+__device__ inline void sketch_add_body(const TableView& tv, const Work& wk, uint32_t vblock, uint32_t vgrid) {
   const uint32_t n = tv.st->n_insert;
-  const uint32_t stride = gridDim.x * blockDim.x;
-  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+  const uint32_t stride = vgrid * blockDim.x;
+  for (uint32_t i = vblock * blockDim.x + threadIdx.x; i < n; i += stride) {
     const uint32_t u = wk.ins_list[i];
     const unsigned long long id = wk.uid[u];
     const uint32_t m = wk.ulen[u];
     for (uint32_t r = 0; r < tv.sketch_depth; ++r) atomicAdd(tv.sketch_counter(r, id), m);
   }
 }
+__global__ void __launch_bounds__(256)
+sketch_add_kernel(TableView tv, Work wk) { sketch_add_body(tv, wk, blockIdx.x, gridDim.x); }
 
-// Phase 3 of mono_apply_grads: one thread per ID that phase 2 found unknown to
+// Phase 3 of a push: one thread per ID that phase 2 found unknown to
 // the key store.  Exact filter: it is inserted (with a row straight away when
 // the batch alone reaches the threshold).  Probabilistic filter: it is inserted,
 // with a row, only if its sketch estimate has reached the threshold; otherwise
 // nothing is stored for it.
-__global__ void __launch_bounds__(256)
-table_insert_kernel(TableView tv, Work wk, uint32_t now) {
+__device__ inline void table_insert_body(const TableView& tv, const Work& wk, uint32_t now, uint32_t vblock, uint32_t vgrid) {
   __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_insert;
   const int lane = threadIdx.x & 31;
   unsigned int n_res = 0, n_done = 0;
-  for (uint32_t base = blockIdx.x * blockDim.x; base < n; base += gridDim.x * blockDim.x) {   // block-uniform
+  for (uint32_t base = vblock * blockDim.x; base < n; base += vgrid * blockDim.x) {   // block-uniform
     const bool todo = base + threadIdx.x < n;
     uint32_t u = 0, m = 0;
     if (todo) { u = wk.ins_list[base + threadIdx.x]; m = wk.ulen[u]; }
@@ -287,16 +318,12 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
       count = est < tv.threshold ? est : tv.threshold;
     }
     const bool need_row = todo && count >= tv.threshold;
-    const Reservation rv = block_reserve(tv, &sh, need_row, todo && m > 1, false, (need_row && m > 1) ? m : 0u);
+    const Reservation rv = block_reserve(tv, &sh, need_row, false, false, 0u);
     if (!todo) continue;
     const unsigned long long id = wk.uid[u];
     uint32_t low = count, row_word = kNoRow;
     if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
     wk.urow[u] = row_word;
-    wk.useg[u] = rv.seg_start;
-    BatchSlot bs; bs.key = m > 1 ? id : kEmptyKey; bs.a = m > 1 ? rv.seg_start : 0u; bs.b = m > 1 ? row_word : 0u;
-    wk.bset[wk.uslot[u]] = bs;
-    if (m > 1) wk.multi_list[rv.multi_pos] = u;
     if (row_word != kNoRow) {
       ++n_res;
       if (m > kSegChunk) register_long(tv, wk, u, m);
@@ -318,6 +345,10 @@ table_insert_kernel(TableView tv, Work wk, uint32_t now) {
     }
   }
 }
+__global__ void __launch_bounds__(256)
+table_insert_kernel(TableView tv, Work wk, uint32_t now) {
+  table_insert_body(tv, wk, now, blockIdx.x, gridDim.x);
+}
 
 // Window of the batch that part k of a segment of `parts` parts falls into.  A segment lists
 // its occurrences roughly in batch order (tile by tile), so part k of n covers roughly the
@@ -328,11 +359,10 @@ __device__ inline uint32_t part_window(uint32_t k, uint32_t parts) {
 
 // After phases 2 and 3: every part of a long segment learns which ID it belongs to
 // (one block per long ID, its threads share the parts), and the parts are counted by window.
-__global__ void __launch_bounds__(128)
-expand_parts_kernel(TableView tv, Work wk) {
+__device__ inline void expand_parts_body(const TableView& tv, const Work& wk, uint32_t vblock, uint32_t vgrid) {
   uint32_t n_long = tv.st->n_long;
   if (n_long > wk.max_long) n_long = wk.max_long;
-  for (uint32_t li = blockIdx.x; li < n_long; li += gridDim.x) {
+  for (uint32_t li = vblock; li < n_long; li += vgrid) {
     const uint32_t parts = (wk.ulen[wk.long_u[li]] + kSegChunk - 1) / kSegChunk;
     const uint32_t p0 = wk.long_part0[li];
     if (p0 + parts > wk.max_parts) continue;
@@ -342,14 +372,15 @@ expand_parts_kernel(TableView tv, Work wk) {
     }
   }
 }
+__global__ void __launch_bounds__(128)
+expand_parts_kernel(TableView tv, Work wk) { expand_parts_body(tv, wk, blockIdx.x, gridDim.x); }
 
 // The order the parts are reduced in: window by window, so that the parts in flight at any
 // time -- of different IDs -- gather gradient rows of the same stretch of bags, and a row
 // that several hot IDs need is fetched from DRAM once and found in L2 by the others.
 // Every block scans the window counts for itself; positions inside a window are handed out
 // by a per-window cursor (their order does not matter: each part has its own partial sum).
-__global__ void __launch_bounds__(kWindows)
-order_parts_kernel(TableView tv, Work wk) {
+__device__ inline void order_parts_body(const TableView& tv, const Work& wk, uint32_t vblock, uint32_t vgrid) {
   __shared__ uint32_t s_start[kWindows];
   __shared__ uint32_t s_warp[kWindows / 32];
   uint32_t n_parts = tv.st->n_parts;
@@ -370,47 +401,52 @@ order_parts_kernel(TableView tv, Work wk) {
   s_start[threadIdx.x] = before + incl - c;
   __syncthreads();
   uint32_t* cursor = wk.win_count + kWindows;
-  for (uint32_t p = blockIdx.x * blockDim.x + threadIdx.x; p < n_parts; p += gridDim.x * blockDim.x) {
+  for (uint32_t p = vblock * blockDim.x + threadIdx.x; p < n_parts; p += vgrid * blockDim.x) {
     const uint32_t li = wk.part_u[p];
     const uint32_t parts = (wk.ulen[wk.long_u[li]] + kSegChunk - 1) / kSegChunk;
     const uint32_t w = part_window(p - wk.long_part0[li], parts);
     wk.part_order[s_start[w] + atomicAdd(&cursor[w], 1u)] = p;
   }
 }
+__global__ void __launch_bounds__(kWindows)
+order_parts_kernel(TableView tv, Work wk) { order_parts_body(tv, wk, blockIdx.x, gridDim.x); }
 
 // End of a mono_apply_grads call: fold the per-call counters into the totals
 // (commit = 0: a grouping that was prepared but never applied is only forgotten).
-__global__ void finish_apply_kernel(DevState* st, uint32_t* win_count, int commit) {
+// (one block)
+__device__ inline void finish_apply_body(DevState* st, uint32_t* win_count, int commit) {
   const bool had_parts = st->n_parts != 0;
   __syncthreads();                                   // everyone has read n_parts before it is reset
   if (had_parts)
     for (uint32_t i = threadIdx.x; i < 2 * kWindows; i += blockDim.x) win_count[i] = 0;
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
+  if (threadIdx.x == 0) {
     if (commit) {
       st->sum_ids += st->n_valid_ids;
       st->sum_unique += st->n_unique;
       st->sum_new += st->n_insert;
     }
     st->n_unique = 0; st->n_insert = 0; st->n_long = 0; st->n_parts = 0; st->n_folds = 0; st->n_valid_ids = 0;
-    st->seg_cursor = 0; st->n_multi = 0;
+    st->seg_cursor = 0; st->n_multi = 0; st->call_bad_offsets = 0;
   }
+}
+__global__ void finish_apply_kernel(DevState* st, uint32_t* win_count, int commit) {
+  if (blockIdx.x == 0) finish_apply_body(st, win_count, commit);
 }
 
 // Expiry sweep (Section 2.1, heuristic 2): a streaming pass over the key
 // store; a cell whose ID has been inactive for longer than ttl is emptied and
 // its row, if it has one, goes back on the free list (one counter update per
 // warp and round).
-__global__ void __launch_bounds__(256)
-expire_kernel(TableView tv, unsigned long long n_cells, unsigned long long first, unsigned long long last,
-              long long now) {
+__device__ inline void expire_body(const TableView& tv, unsigned long long n_cells, unsigned long long first,
+                                   unsigned long long last, long long now, uint32_t vblock, uint32_t vgrid) {
   // sweeps cells [first, last) of the sequence "key store, then stash" (total n_cells + kStashCells)
   constexpr int kDepth = 4;                                                // independent loads per thread and round
-  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long stride = (unsigned long long)vgrid * blockDim.x;
   const unsigned long long rounds = (last - first + stride * kDepth - 1) / (stride * kDepth);  // same for every thread
   const int lane = threadIdx.x & 31;
   unsigned int n_gone = 0, n_rows = 0;
   for (unsigned long long r = 0; r < rounds; ++r) {
-    const unsigned long long i0 = first + r * kDepth * stride + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long i0 = first + r * kDepth * stride + (unsigned long long)vblock * blockDim.x + threadIdx.x;
     Cell* p[kDepth];
     ulonglong2 v[kDepth];
 #pragma unroll
@@ -450,6 +486,11 @@ expire_kernel(TableView tv, unsigned long long n_cells, unsigned long long first
     atomicAdd(&tv.st->n_expired_total, (unsigned long long)n_gone);
     if (n_rows) atomicAdd(&tv.st->n_resident, (unsigned long long)(-(long long)n_rows));
   }
+}
+__global__ void __launch_bounds__(256)
+expire_kernel(TableView tv, unsigned long long n_cells, unsigned long long first, unsigned long long last,
+              long long now) {
+  expire_body(tv, n_cells, first, last, now, blockIdx.x, gridDim.x);
 }
 
 // After a sweep: if the stash has become empty, probes may skip it again.
@@ -495,37 +536,48 @@ rehash_kernel(TableView fresh, const Cell* __restrict__ old_cells, unsigned long
 
 // ---- bulk import -----------------------------------------------------------
 
-// One thread per entry: skip IDs that are already tracked, claim a row for
-// resident entries, insert.  row_word[i] tells import_rows_kernel where the
-// entry's values go.
+// Import runs in two kernels, like the batch path: while an insertion is carrying a displaced
+// entry that key sits in no cell, so the test "is this ID tracked already?" is made for all
+// entries first, while nothing moves, and the insertions follow.
+constexpr uint32_t kImportSkip = 0xFFFFFFFEu;
+
+// One thread per entry: row_word[i] = kImportSkip for an ID that is already tracked (or is the
+// padding value), kNoRow otherwise.
+__global__ void __launch_bounds__(256)
+import_check_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n, uint32_t* __restrict__ row_word) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const unsigned stash_hw = tv.st->stash_hw;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const unsigned long long id = ids[i];
+    if (id == kEmptyKey) { row_word[i] = kImportSkip; continue; }
+    unsigned long long meta = 0;
+    const bool present = thread_lookup(tv, id, stash_hw, &meta);
+    if (present) atomicOr(&tv.st->error_bits, 8u /* MONO_DEV_IMPORT_DUP */);
+    row_word[i] = present ? kImportSkip : kNoRow;
+  }
+}
+
+// One thread per entry that passed the check: claim a row for resident entries, insert.
+// row_word[i] tells import_rows_kernel where the entry's values go.
 __global__ void __launch_bounds__(256)
 import_insert_kernel(TableView tv, const unsigned long long* __restrict__ ids, const uint32_t* __restrict__ count,
                      const long long* __restrict__ last_seen, const uint8_t* __restrict__ resident,
                      long long n, uint32_t* __restrict__ row_word) {
   const long long stride = (long long)gridDim.x * blockDim.x;
-  const unsigned stash_hw = tv.st->stash_hw;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
     const unsigned long long id = ids[i];
-    row_word[i] = kNoRow;
-    if (id == kEmptyKey) continue;
-    bool present = false;
-    const unsigned long long bk[2] = {tv.bucket0(id), tv.bucket1(id)};
-    for (int b = 0; b < 2 && !present; ++b)
-      for (uint32_t c = 0; c < kCellsPerBucket; ++c)
-        present |= load_cell(tv.cells + bk[b] * kCellsPerBucket + c).key == id;
-    for (unsigned s = 0; s < stash_hw && !present; ++s) present |= load_cell(tv.stash + s).key == id;
-    if (present) { atomicOr(&tv.st->error_bits, 8u /* MONO_DEV_IMPORT_DUP */); continue; }
+    if (row_word[i] == kImportSkip) { row_word[i] = kNoRow; continue; }
     if (tv.sketch_depth != 0 && !resident[i]) continue;     // probabilistic filter: IDs without a row have no entry
     long long seen = last_seen[i];
     if (seen < 0) seen = 0;
     if (seen > 0xFFFFFFFELL) seen = 0xFFFFFFFELL;
+    // an entry without a row keeps its count, up to the threshold: at the threshold it is an ID whose
+    // admission was refused for lack of a row, and the batch path retries it at its next occurrence
     uint32_t low = count[i] < tv.threshold ? count[i] : tv.threshold;
     if (resident[i]) {
       const uint32_t row = alloc_row(tv);
       if (row != kNoRow) { low = kResidentBit | row; row_word[i] = row; }
       else low = tv.threshold;
-    } else if (low >= tv.threshold) {
-      low = tv.threshold - 1;      // "not resident" entries stay below the threshold
     }
     Cell item; item.key = id; item.meta = make_meta((uint32_t)seen, low);
     atomicAdd(&tv.st->n_tracked, 1ull);

@@ -3,6 +3,7 @@
 // runs in the kernels included below; nothing here computes on the host.
 #include <cstdint>
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -16,6 +17,7 @@
 #include "kernels_adagrad.cuh"
 #include "kernels_dedup.cuh"
 #include "kernels_forward.cuh"
+#include "kernels_group.cuh"
 #include "kernels_inspect.cuh"
 #include "kernels_table.cuh"
 #include "table_layout.cuh"
@@ -28,14 +30,17 @@ using namespace mono;
 static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS];
 
 enum KernelId {
-  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_FILE, K_SINGLES, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
+  K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_LOOKUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_FILE, K_SINGLES, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
   K_STASH_TRIM, K_COUNT
 };
+// (table_lookup and table_update are the two halves of table_update_kernel; a push that was not
+// announced runs both in one launch, counted as table_update)
 static const char* const kKernelNames[K_COUNT] = {
-  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_update", "sketch_add", "table_insert", "expand_parts", "order_parts",
+  "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_lookup", "table_update", "sketch_add", "table_insert", "expand_parts", "order_parts",
   "file_segments", "update_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
   "finish_apply", "expire", "stash_trim"
 };
+static_assert(K_COUNT <= MONO_MAX_KERNELS, "mono_timing_t has room for MONO_MAX_KERNELS kernels");
 
 struct mono_table {
   // per-kernel launch counts, and (when timing is on) CUDA-event durations
@@ -48,19 +53,37 @@ struct mono_table {
   TableView tv{};
   Work wk{};
   cudaStream_t stream = nullptr;
-  // Two internal streams, ordered against `stream` with events only: one runs the
-  // ID-only part of a push that mono_prepare_push announced, the other the sweep.
-  cudaStream_t prep_stream = nullptr, sweep_stream = nullptr;
+  // An internal stream, ordered against `stream` with events only, runs the sweep.
+  cudaStream_t sweep_stream = nullptr;
   // A third one runs the small kernels that serve only the few hottest IDs of a push beside
   // the large ones (see launch_apply).
   cudaStream_t aux_stream = nullptr;
   cudaEvent_t ev_parts = nullptr, ev_reduced = nullptr, ev_aux = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_prepared = nullptr, ev_keys = nullptr, ev_swept = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_keys = nullptr, ev_swept = nullptr;
   cudaEvent_t ev_group = nullptr;  // grouped calls: the group's start (first table's), this table's end
   bool sweep_pending = false;     // the sweep stream has work `stream` has not waited for yet
   bool keys_idle = false;         // nothing launched on `stream` after ev_keys touches the key store
-  struct { const void* ids; int64_t n_ids; const void* off; int64_t n_bags; bool valid; } prep = {nullptr, 0, nullptr, 0, false};
-  uint32_t* occ_row = nullptr;    // scratch of the lookup: row of every occurrence
+  // The batch mono_prepare_push announced: grouped and looked up, waiting for its push.
+  // filed: its lookup has run too, so every occurrence's bag is in bag_of_sorted[] already.
+  struct { const void* ids; int64_t n_ids; const void* off; int64_t n_bags; bool valid; bool filed; } prep = {nullptr, 0, nullptr, 0, false, false};
+  uint32_t* occ_row = nullptr;    // scratch of the two-kernel lookup: row of every occurrence
+  int device = 0;                 // the device the table lives on
+  uint64_t scratch_reallocs = 0;  // times a hot call had to grow the scratch
+  // Grouped calls (one launch over several tables): the first table of a group keeps the
+  // descriptors of the group's tables and the block maps of its launches, on the device, and
+  // a small ring of pinned host copies they are uploaded from.
+  struct GroupScratch {
+    static constexpr int kRing = 4;
+    char* dev = nullptr; size_t dev_bytes = 0;
+    char* host[kRing] = {}; size_t host_bytes[kRing] = {}; cudaEvent_t used[kRing] = {};
+    int next = 0;
+  } grp;
+  // device-resident snapshot (mono_snapshot_save)
+  struct {
+    Cell* cells = nullptr; Cell* stash = nullptr; float* rows = nullptr; uint32_t* free_rows = nullptr;
+    DevState* st = nullptr; unsigned int* sketch = nullptr;
+    uint64_t key_cells = 0; int64_t last_now = -1, sketch_epoch = 0; bool valid = false;
+  } snap;
   int sm_count = 148;
   uint64_t key_cells = 0;
   int64_t last_now = -1;
@@ -100,11 +123,17 @@ void dev_free(T*& p) { if (p) { cudaFree(p); p = nullptr; } }
 
 void free_scratch(mono_table* t) {
   Work& w = t->wk;
-  dev_free(w.bset); dev_free(w.occ_slot); dev_free(w.occ_rank); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
-  dev_free(w.uid); dev_free(w.uslot); dev_free(w.uocc); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow);
+  dev_free(w.bset); dev_free(w.occ); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
+  dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow); dev_free(w.ucell);
   dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.part_order); dev_free(w.win_count); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec); dev_free(t->occ_row);
   t->max_ids = t->max_bags = 0;
+}
+
+void free_snapshot(mono_table* t) {
+  auto& sn = t->snap;
+  dev_free(sn.cells); dev_free(sn.stash); dev_free(sn.rows); dev_free(sn.free_rows); dev_free(sn.st); dev_free(sn.sketch);
+  sn.valid = false;
 }
 
 int grid_for(const mono_table* t, int per_sm) { return t->sm_count * per_sm; }
@@ -139,14 +168,26 @@ void join_sweep(mono_table* t) {
   t->keys_idle = false;
 }
 
+// Forget a prepared batch: empty the per-call set and the per-call counters.
+int discard_prepared(mono_table* t) {
+  if (!t->prep.valid) return MONO_OK;
+  t->prep.valid = false;
+  const uint64_t slots = (uint64_t)t->wk.primary_mask + 1 + (uint64_t)t->wk.secondary_mask + 1;
+  init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(t->wk.bset, slots);
+  finish_apply_kernel<<<1, 256, 0, t->stream>>>(t->tv.st, t->wk.win_count, 0);
+  CUDA_TRY(t, cudaGetLastError());
+  return MONO_OK;
+}
+
 int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   if (max_ids <= t->max_ids && max_bags <= t->max_bags) return MONO_OK;
   if (max_ids < t->max_ids) max_ids = t->max_ids;
   if (max_bags < t->max_bags) max_bags = t->max_bags;
   if (max_ids < 1024) max_ids = 1024;
   if (max_bags < 1024) max_bags = 1024;
+  if (t->max_ids > 0) ++t->scratch_reallocs;               // (the first sizing of a table created without one is not a regrowth)
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
-  CUDA_TRY(t, cudaStreamSynchronize(t->prep_stream));     // a prepared grouping is lost with the scratch it lives in
+  // a prepared batch is lost with the scratch it lives in
   if (t->prep.valid) { t->prep.valid = false; finish_apply_kernel<<<1, 256, 0, t->stream>>>(t->tv.st, t->wk.win_count, 0); }
   free_scratch(t);
   Work& w = t->wk;
@@ -158,8 +199,8 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   int rc;
 #define ALLOC(p, cnt) if ((rc = dev_alloc(t, &(p), (cnt))) != MONO_OK) { free_scratch(t); return rc; }
   ALLOC(w.bset, slots);
-  ALLOC(w.occ_slot, n); ALLOC(w.occ_rank, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
-  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.uocc, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n);
+  ALLOC(w.occ, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
+  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n); ALLOC(w.ucell, n);
   ALLOC(w.multi_list, n / 2 + 1); ALLOC(w.ins_list, n);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
@@ -189,6 +230,10 @@ int check_batch(const mono_table* t, const void* ids, int64_t n_ids, const void*
   return MONO_OK;
 }
 
+bool is_prepared_batch(const mono_table* t, const void* ids, int64_t n_ids, const void* off, int64_t n_bags) {
+  return t->prep.valid && t->prep.ids == ids && t->prep.n_ids == n_ids && t->prep.off == off && t->prep.n_bags == n_bags;
+}
+
 // lane-group width and column vectors per lane for a given dim
 template <typename F>
 int dispatch_dim(uint32_t dim, F&& f) {
@@ -201,27 +246,35 @@ int dispatch_dim(uint32_t dim, F&& f) {
   return f(std::integral_constant<int, 32>{}, std::integral_constant<int, 8>{});
 }
 
-int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
-                  int64_t n_bags, float* out) {
-  if (n_bags == 0) return MONO_OK;
-  uint32_t* occ_row = t->occ_row;
-  if (n_ids > 0) {
-    int64_t blocks = (n_ids + 255) / 256;
-    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
-    if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, occ_row));
-  }
+// The pooling kernel, with the rows of the occurrences taken from SRC.
+template <int SRC>
+int launch_gather(mono_table* t, const GatherSource& src, int64_t n_ids, const long long* off, int64_t n_bags, float* out) {
   return dispatch_dim(t->tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     const int64_t groups_per_block = 256 / G;
     int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
     const int64_t cap = (int64_t)grid_for(t, 8) * 8;
     if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, occ_row, n_ids, off,
-                                                                                    n_bags, out));
+    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV, SRC><<<(int)blocks, 256, 0, t->stream>>>(t->tv, src, n_ids, off, n_bags, out));
     CUDA_TRY(t, cudaGetLastError());
     return (int)MONO_OK;
   });
+}
+
+int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
+                  int64_t n_bags, float* out, bool prepared) {
+  if (n_bags == 0) return MONO_OK;
+  GatherSource src{};
+  if (prepared) {
+    // every distinct ID of this batch was looked up when it was announced: the rows come from the
+    // per-call set, and the occurrences file their bags for the push on the way
+    src.occ = t->wk.occ; src.bset = t->wk.bset; src.bag_of_sorted = t->wk.bag_of_sorted;
+    const int rc = launch_gather<kFromSet>(t, src, n_ids, off, n_bags, out);
+    if (rc == MONO_OK) t->prep.filed = true;
+    return rc;
+  }
+  src.ids = ids;
+  return launch_gather<kFromKeys>(t, src, n_ids, off, n_bags, out);
 }
 
 // The part of a push that depends on the IDs alone: bag of every occurrence, and the
@@ -238,37 +291,37 @@ int launch_group(mono_table* t, cudaStream_t s, const unsigned long long* ids, i
   return MONO_OK;
 }
 
-// Forget a prepared grouping: wait for it, then empty the per-call set and the per-call counters.
-int discard_prepared(mono_table* t) {
-  if (!t->prep.valid) return MONO_OK;
-  t->prep.valid = false;
-  CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_prepared, 0));
-  const uint64_t slots = (uint64_t)t->wk.primary_mask + 1 + (uint64_t)t->wk.secondary_mask + 1;
-  init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(t->wk.bset, slots);
-  finish_apply_kernel<<<1, 256, 0, t->stream>>>(t->tv.st, t->wk.win_count, 0);
+// mono_prepare_push: group the batch and look every distinct ID up once, for the lookup and the
+// push of this batch together.  Nothing in the table changes.
+int launch_prepare(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off, int64_t n_bags) {
+  int rc = launch_group(t, t->stream, ids, n_ids, off, n_bags);
+  if (rc != MONO_OK) return rc;
+  LAUNCH(t, K_LOOKUP, table_update_kernel<kLookUp><<<grid_for(t, 8) * 4, 256, 0, t->stream>>>(t->tv, t->wk, 0u));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
 }
 
 int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
                  int64_t n_bags, const float* grad, uint32_t now) {
-  int rc0 = MONO_OK;
-  if (t->prep.valid && t->prep.ids == ids && t->prep.n_ids == n_ids && t->prep.off == off && t->prep.n_bags == n_bags) {
-    // the grouping of exactly this batch is ready, or in flight on the preparation stream
-    t->prep.valid = false;
-    CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_prepared, 0));
-  } else {
-    if ((rc0 = discard_prepared(t)) != MONO_OK) return rc0;
-    if (n_ids == 0 || n_bags == 0) return MONO_OK;
-    if ((rc0 = launch_group(t, t->stream, ids, n_ids, off, n_bags)) != MONO_OK) return rc0;
-  }
   cudaStream_t s = t->stream;
   const TableView& tv = t->tv;
   const Work& wk = t->wk;
   // grids of the grid-stride kernels: several waves of blocks per SM where that measured faster
   // (shorter tails), one wave elsewhere
   const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
-  LAUNCH(t, K_UPDATE, table_update_kernel<<<g8 * 4, 256, 0, s>>>(tv, wk, now));
+  int rc0 = MONO_OK;
+  if (is_prepared_batch(t, ids, n_ids, off, n_bags)) {
+    // grouped and looked up already; filed too, if its lookup has run
+    t->prep.valid = false;
+    if (!t->prep.filed) LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
+    LAUNCH(t, K_UPDATE, table_update_kernel<kCommit><<<g8 * 4, 256, 0, s>>>(tv, wk, now));
+  } else {
+    if ((rc0 = discard_prepared(t)) != MONO_OK) return rc0;
+    if (n_ids == 0 || n_bags == 0) return MONO_OK;
+    if ((rc0 = launch_group(t, s, ids, n_ids, off, n_bags)) != MONO_OK) return rc0;
+    LAUNCH(t, K_UPDATE, table_update_kernel<kLookUp | kCommit><<<g8 * 4, 256, 0, s>>>(tv, wk, now));
+    LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
+  }
   if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
   CUDA_TRY(t, cudaGetLastError());
@@ -276,9 +329,10 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
   // The kernels that prepare and finish the reduction of the long segments (the few hottest
   // IDs) keep only a few blocks busy each, so they run on a stream of their own beside the
-  // kernels that work through the whole batch: expand/order beside file_segments, and
-  // fold/combine, which need only what reduce_adagrad left, beside update_singletons.  While
-  // kernels are being timed one by one, everything stays on the table's stream.
+  // kernels that work through the whole batch: expand/order beside the reduction of the short
+  // segments, and fold/combine, which need only what the parts left, beside update_singletons.
+  // While kernels are being timed one by one, everything stays on the table's stream and the
+  // segments are reduced in one launch.
   cudaStream_t a = t->timing ? s : t->aux_stream;
   if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_keys, 0));
   LAUNCH_ON(t, a, K_EXPAND, expand_parts_kernel<<<g8 * 4, 128, 0, a>>>(tv, wk));
@@ -287,12 +341,14 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   if (a != s) CUDA_TRY(t, cudaEventRecord(t->ev_parts, a));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
-    LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
-    if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_parts, 0));
-    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
     if (a != s) {
+      LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceShort));
+      CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_parts, 0));
+      LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceParts));
       CUDA_TRY(t, cudaEventRecord(t->ev_reduced, s));
       CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_reduced, 0));
+    } else {
+      LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceParts | kReduceShort));
     }
     LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
@@ -315,33 +371,185 @@ int check_now(mono_table* t, int64_t now) {
   return MONO_OK;
 }
 
-// Fork/join of a grouped call around `one(i)`, the single-table call of table i.
-template <typename F>
-int group_call(int32_t n_tables, mono_table* const* tables, void* group_stream, F&& one) {
+// ---- grouped calls: one launch over several tables -------------------------------------------
+
+enum GroupKernel {
+  GK_FILL, GK_DEDUP, GK_UPDATE, GK_INSERT, GK_FILE, GK_EXPAND, GK_ORDER, GK_GATHER, GK_GATHER_WIDE, GK_REDUCE, GK_REDUCE_WIDE,
+  GK_SINGLES, GK_SINGLES_WIDE, GK_FOLD, GK_COMBINE, GK_COUNT
+};
+
+uint32_t lane_class_of(uint32_t dim) {
+  return dim <= 16 ? 0u : dim <= 32 ? 1u : dim <= 64 ? 2u : dim <= 128 ? 3u : dim <= 256 ? 4u : dim <= 512 ? 5u : 6u;
+}
+int lanes_of_class(uint32_t c) { return c == 0 ? 4 : c == 1 ? 8 : c == 2 ? 16 : 32; }
+
+void free_group_scratch(mono_table* t) {
+  auto& g = t->grp;
+  if (g.dev) { cudaFree(g.dev); g.dev = nullptr; g.dev_bytes = 0; }
+  for (int i = 0; i < mono_table::GroupScratch::kRing; ++i) {
+    if (g.host[i]) { cudaFreeHost(g.host[i]); g.host[i] = nullptr; g.host_bytes[i] = 0; }
+    if (g.used[i]) { cudaEventDestroy(g.used[i]); g.used[i] = nullptr; }
+  }
+}
+
+int64_t clamp_blocks(int64_t work, int64_t per_block, int64_t cap) {
+  int64_t b = (work + per_block - 1) / per_block;
+  if (b < 1) b = 1;
+  return b > cap ? cap : b;
+}
+
+// Blocks that table `t` contributes to grouped kernel `k` (the grid it would launch alone, but no
+// larger than its batch needs: a group may hold hundreds of small tables).
+uint32_t group_blocks(const mono_table* t, int k, int64_t n_ids, int64_t n_bags) {
+  const int64_t g8 = grid_for(t, 8), g4 = grid_for(t, 4);
+  const uint32_t lc = lane_class_of(t->tv.dim);
+  const int G = lanes_of_class(lc);
+  const bool wide = lc >= 4;
+  switch (k) {
+    case GK_FILL: return (uint32_t)clamp_blocks(n_bags, 256, g8);
+    case GK_DEDUP: return (uint32_t)((n_ids + kTileIds - 1) / kTileIds);
+    case GK_UPDATE: return (uint32_t)clamp_blocks(n_ids, 256, g8 * 4);
+    case GK_INSERT: case GK_FILE: return (uint32_t)clamp_blocks(n_ids, 256, g8);
+    case GK_EXPAND: return (uint32_t)clamp_blocks(n_ids / kSegChunk + 1, 1, g8 * 4);
+    case GK_ORDER: return (uint32_t)clamp_blocks(n_ids / kSegChunk + 1, kWindows, 64);
+    case GK_GATHER: return wide ? 0u : (uint32_t)clamp_blocks(n_bags, 256 / G, g8 * 8);
+    case GK_GATHER_WIDE: return wide ? (uint32_t)clamp_blocks(n_bags, 256 / G, g8 * 8) : 0u;
+    case GK_REDUCE: return wide ? 0u : (uint32_t)clamp_blocks(n_ids / 2 + 1, 128 / G, g8 * 8);
+    case GK_REDUCE_WIDE: return wide ? (uint32_t)clamp_blocks(n_ids / 2 + 1, 128 / G, g8 * 8) : 0u;
+    case GK_SINGLES: return wide ? 0u : (uint32_t)clamp_blocks(n_ids, 128, g8 * 8);
+    case GK_SINGLES_WIDE: return wide ? (uint32_t)clamp_blocks(n_ids, 128, g8 * 8) : 0u;
+    case GK_FOLD: return (uint32_t)clamp_blocks(n_ids / (kSegChunk * kFoldWidth) + 1, 1, g4);
+    case GK_COMBINE: return (uint32_t)clamp_blocks(n_ids / kSegChunk + 1, 1, g8);
+    default: return 0u;
+  }
+}
+
+// A grouped call in the making: the tables' descriptors, the block map of every kernel, and where
+// both live on the device once uploaded.
+struct GroupPlan {
+  int32_t n = 0;
+  mono_table* owner = nullptr;               // tables[0]: holds the scratch and counts the launches
+  cudaStream_t gs = nullptr;
+  std::vector<GroupItem> items;
+  std::vector<uint32_t> starts;              // [GK_COUNT][n + 1]
+  const GroupItem* d_items = nullptr;
+  const uint32_t* d_starts = nullptr;
+  bool any_wide = false, any_narrow = false, any_sketch = false;
+  uint32_t grid(int k) const { return starts[(size_t)k * (n + 1) + n]; }
+  const uint32_t* map(int k) const { return d_starts + (size_t)k * (n + 1); }
+};
+
+int group_check(int32_t n_tables, mono_table* const* tables) {
   if (n_tables < 0 || (n_tables > 0 && !tables)) return MONO_ERR_ARG;
-  if (n_tables == 0) return MONO_OK;
   for (int32_t i = 0; i < n_tables; ++i) {
     if (!tables[i]) return MONO_ERR_ARG;
-    for (int32_t j = 0; j < i; ++j) if (tables[j] == tables[i]) return MONO_ERR_ARG;
+    if (tables[i]->device != tables[0]->device) return MONO_ERR_ARG;
   }
-  cudaStream_t gs = static_cast<cudaStream_t>(group_stream);
-  mono_table* t0 = tables[0];
-  CUDA_TRY(t0, cudaEventRecord(t0->ev_fork, gs));              // (ev_fork is re-recorded by whoever uses it next)
-  int rc = MONO_OK;
-  int32_t started = 0;
-  for (; started < n_tables && rc == MONO_OK; ++started) {
-    mono_table* t = tables[started];
-    if (t->stream != gs) CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t0->ev_fork, 0));
-    rc = one(started);
-  }
-  // join what was started, also after an error
-  for (int32_t i = 0; i < started; ++i) {
+  // the same table twice would run two batches through one scratch at the same time
+  std::vector<mono_table*> sorted(tables, tables + n_tables);
+  std::sort(sorted.begin(), sorted.end());
+  for (int32_t i = 1; i < n_tables; ++i) if (sorted[i] == sorted[i - 1]) return MONO_ERR_ARG;
+  return MONO_OK;
+}
+
+// Everything the tables have in flight on their own streams comes before the group's work on `gs`.
+int group_begin(GroupPlan& p, int32_t n_tables, mono_table* const* tables, void* group_stream) {
+  p.n = n_tables;
+  p.owner = tables[0];
+  p.gs = static_cast<cudaStream_t>(group_stream);
+  for (int32_t i = 0; i < n_tables; ++i) {
     mono_table* t = tables[i];
-    if (t->stream == gs) continue;
-    CUDA_TRY(t, cudaEventRecord(t->ev_group, t->stream));
-    CUDA_TRY(t, cudaStreamWaitEvent(gs, t->ev_group, 0));
+    join_sweep(t);
+    if (t->stream != p.gs) {
+      CUDA_TRY(t, cudaEventRecord(t->ev_group, t->stream));
+      CUDA_TRY(t, cudaStreamWaitEvent(p.gs, t->ev_group, 0));
+    }
   }
-  return rc;
+  p.items.assign(n_tables, GroupItem{});
+  p.starts.assign((size_t)GK_COUNT * (n_tables + 1), 0u);
+  return MONO_OK;
+}
+
+// ... and whatever the tables are given next on their own streams comes after it.
+int group_end(GroupPlan& p, mono_table* const* tables) {
+  bool other = false;
+  for (int32_t i = 0; i < p.n; ++i) other |= tables[i]->stream != p.gs;
+  if (!other) return MONO_OK;
+  CUDA_TRY(p.owner, cudaEventRecord(p.owner->ev_fork, p.gs));
+  for (int32_t i = 0; i < p.n; ++i)
+    if (tables[i]->stream != p.gs) CUDA_TRY(tables[i], cudaStreamWaitEvent(tables[i]->stream, p.owner->ev_fork, 0));
+  return MONO_OK;
+}
+
+void group_describe(GroupPlan& p, int32_t i, mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* off,
+                    int64_t n_bags, float* out, const float* grad, uint32_t now, bool prepared) {
+  GroupItem& it = p.items[i];
+  it.tv = t->tv; it.wk = t->wk;
+  it.ids = reinterpret_cast<const unsigned long long*>(ids);
+  it.off = reinterpret_cast<const long long*>(off);
+  it.n_ids = n_ids; it.n_bags = n_bags; it.out = out; it.grad = grad; it.now = now;
+  it.dedup_seed = t->tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull;
+  it.prepared = prepared ? 1u : 0u;
+  it.lane_class = lane_class_of(t->tv.dim);
+  it.active = (n_ids > 0 && n_bags > 0) ? 1u : 0u;
+  if (it.lane_class >= 4) p.any_wide = true; else p.any_narrow = true;
+  if (t->tv.sketch_depth) p.any_sketch = true;
+}
+
+// Block maps (a table whose batch is empty gets no blocks), then one upload of descriptors and maps.
+int group_upload(GroupPlan& p, mono_table* const* tables) {
+  for (int k = 0; k < GK_COUNT; ++k) {
+    uint32_t* st = p.starts.data() + (size_t)k * (p.n + 1);
+    uint64_t total = 0;
+    for (int32_t i = 0; i < p.n; ++i) {
+      st[i] = (uint32_t)total;
+      if (p.items[i].active) total += group_blocks(tables[i], k, p.items[i].n_ids, p.items[i].n_bags);
+      if (total >= (1ull << 31)) return MONO_ERR_ARG;
+    }
+    st[p.n] = (uint32_t)total;
+  }
+  auto& g = p.owner->grp;
+  const size_t items_bytes = ((p.items.size() * sizeof(GroupItem) + 255) / 256) * 256;
+  const size_t bytes = items_bytes + p.starts.size() * sizeof(uint32_t);
+  if (bytes > g.dev_bytes) {
+    CUDA_TRY(p.owner, cudaStreamSynchronize(p.gs));
+    if (g.dev) cudaFree(g.dev);
+    g.dev = nullptr; g.dev_bytes = 0;
+    CUDA_TRY(p.owner, cudaMalloc(reinterpret_cast<void**>(&g.dev), bytes * 2));
+    g.dev_bytes = bytes * 2;
+  }
+  const int slot = g.next;
+  g.next = (g.next + 1) % mono_table::GroupScratch::kRing;
+  if (!g.used[slot]) CUDA_TRY(p.owner, cudaEventCreateWithFlags(&g.used[slot], cudaEventDisableTiming));
+  else CUDA_TRY(p.owner, cudaEventSynchronize(g.used[slot]));          // the upload that last used this host copy is done
+  if (bytes > g.host_bytes[slot]) {
+    if (g.host[slot]) cudaFreeHost(g.host[slot]);
+    g.host[slot] = nullptr; g.host_bytes[slot] = 0;
+    CUDA_TRY(p.owner, cudaMallocHost(reinterpret_cast<void**>(&g.host[slot]), bytes * 2));
+    g.host_bytes[slot] = bytes * 2;
+  }
+  std::memcpy(g.host[slot], p.items.data(), p.items.size() * sizeof(GroupItem));
+  std::memcpy(g.host[slot] + items_bytes, p.starts.data(), p.starts.size() * sizeof(uint32_t));
+  CUDA_TRY(p.owner, cudaMemcpyAsync(g.dev, g.host[slot], bytes, cudaMemcpyHostToDevice, p.gs));
+  CUDA_TRY(p.owner, cudaEventRecord(g.used[slot], p.gs));
+  p.d_items = reinterpret_cast<const GroupItem*>(g.dev);
+  p.d_starts = reinterpret_cast<const uint32_t*>(g.dev + items_bytes);
+  return MONO_OK;
+}
+
+// launch grouped kernel `kernel` over block map `gk` with `threads` per block, counted under `kid`
+#define GROUP_LAUNCH(p, kid, gk, threads, kernel)                                                         \
+  do {                                                                                                    \
+    if ((p).grid(gk) > 0) {                                                                               \
+      ++(p).owner->launches[kid];                                                                         \
+      kernel<<<(p).grid(gk), (threads), 0, (p).gs>>>((p).d_items, (p).map(gk), (uint32_t)(p).n);           \
+    }                                                                                                     \
+  } while (0)
+
+int group_launch_ids_only(GroupPlan& p) {
+  GROUP_LAUNCH(p, K_FILL_BAG, GK_FILL, 256, group_fill_occ_bag_kernel);
+  GROUP_LAUNCH(p, K_DEDUP, GK_DEDUP, kTileThreads, group_dedup_tile_kernel);
+  return MONO_OK;
 }
 
 }  // namespace
@@ -373,11 +581,11 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   if (cudaGetDevice(&dev) != cudaSuccess) return fail(MONO_ERR_CUDA);
   if (cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || t->sm_count < 1)
     return fail(MONO_ERR_CUDA);
-  if (cudaStreamCreateWithFlags(&t->prep_stream, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess ||
+  t->device = dev;
+  if (cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaStreamCreateWithFlags(&t->aux_stream, cudaStreamNonBlocking) != cudaSuccess)
     return fail(MONO_ERR_CUDA);
-  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_prepared, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_parts,
+  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_parts,
                          &t->ev_reduced, &t->ev_aux})
     if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return fail(MONO_ERR_CUDA);
 
@@ -428,15 +636,15 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
 int mono_table_destroy(mono_table* t) {
   if (!t) return MONO_ERR_ARG;
   cudaStreamSynchronize(t->stream);
-  if (t->prep_stream) { cudaStreamSynchronize(t->prep_stream); cudaStreamDestroy(t->prep_stream); }
   if (t->sweep_stream) { cudaStreamSynchronize(t->sweep_stream); cudaStreamDestroy(t->sweep_stream); }
   if (t->aux_stream) { cudaStreamSynchronize(t->aux_stream); cudaStreamDestroy(t->aux_stream); }
-  for (cudaEvent_t e : {t->ev_fork, t->ev_prepared, t->ev_keys, t->ev_swept, t->ev_group, t->ev_parts, t->ev_reduced,
-                        t->ev_aux})
+  for (cudaEvent_t e : {t->ev_fork, t->ev_keys, t->ev_swept, t->ev_group, t->ev_parts, t->ev_reduced, t->ev_aux})
     if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
   free_scratch(t);
+  free_snapshot(t);
+  free_group_scratch(t);
   dev_free(t->tv.cells); dev_free(t->tv.stash); dev_free(t->tv.rows); dev_free(t->tv.free_rows); dev_free(t->tv.st); dev_free(t->tv.sketch);
   delete t;
   return MONO_OK;
@@ -456,7 +664,8 @@ int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
   if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
   if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
   return launch_lookup(t, reinterpret_cast<const unsigned long long*>(ids), n_ids,
-                       reinterpret_cast<const long long*>(slot_offsets), n_bags, out);
+                       reinterpret_cast<const long long*>(slot_offsets), n_bags, out,
+                       is_prepared_batch(t, ids, n_ids, slot_offsets, n_bags));
 }
 
 int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
@@ -473,46 +682,141 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
 }
 
 int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets, int64_t n_bags) {
+  if (t) join_sweep(t);                                    // the look-ups read the key store
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
   if ((rc = discard_prepared(t)) != MONO_OK) return rc;
   if (n_ids == 0 || n_bags == 0) return MONO_OK;
-  // after everything already on the table's stream (the previous push still owns the scratch) ...
-  CUDA_TRY(t, cudaEventRecord(t->ev_fork, t->stream));
-  CUDA_TRY(t, cudaStreamWaitEvent(t->prep_stream, t->ev_fork, 0));
-  // ... and beside everything that comes next on it
-  if ((rc = launch_group(t, t->prep_stream, reinterpret_cast<const unsigned long long*>(ids), n_ids,
-                         reinterpret_cast<const long long*>(slot_offsets), n_bags)) != MONO_OK) return rc;
-  CUDA_TRY(t, cudaEventRecord(t->ev_prepared, t->prep_stream));
-  t->prep = {ids, n_ids, slot_offsets, n_bags, true};
+  if ((rc = launch_prepare(t, reinterpret_cast<const unsigned long long*>(ids), n_ids,
+                           reinterpret_cast<const long long*>(slot_offsets), n_bags)) != MONO_OK) return rc;
+  t->prep = {ids, n_ids, slot_offsets, n_bags, true, false};
   return MONO_OK;
+}
+
+int mono_group_prepare_push(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
+                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
+                            void* group_stream) {
+  int rc = group_check(n_tables, tables);
+  if (rc != MONO_OK) return rc;
+  if (n_tables == 0) return MONO_OK;
+  if (!ids || !n_ids || !slot_offsets || !n_bags) return MONO_ERR_ARG;
+  for (int32_t i = 0; i < n_tables; ++i) {
+    mono_table* t = tables[i];
+    join_sweep(t);
+    if ((rc = check_batch(t, ids[i], n_ids[i], slot_offsets[i], n_bags[i])) != MONO_OK) return rc;
+    if ((rc = reserve(t, n_ids[i], n_bags[i])) != MONO_OK) return rc;
+    if ((rc = discard_prepared(t)) != MONO_OK) return rc;
+  }
+  GroupPlan p;
+  if ((rc = group_begin(p, n_tables, tables, group_stream)) != MONO_OK) return rc;
+  for (int32_t i = 0; i < n_tables; ++i)
+    group_describe(p, i, tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], nullptr, nullptr, 0u, false);
+  if ((rc = group_upload(p, tables)) != MONO_OK) return rc;
+  group_launch_ids_only(p);
+  GROUP_LAUNCH(p, K_LOOKUP, GK_UPDATE, 256, group_table_update_kernel<kLookUp>);
+  CUDA_TRY(p.owner, cudaGetLastError());
+  for (int32_t i = 0; i < n_tables; ++i)
+    if (p.items[i].active) tables[i]->prep = {ids[i], n_ids[i], slot_offsets[i], n_bags[i], true, false};
+  return group_end(p, tables);
 }
 
 int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
                            float* const* out, void* group_stream) {
-  if (n_tables > 0 && (!ids || !n_ids || !slot_offsets || !n_bags || !out)) return MONO_ERR_ARG;
-  return group_call(n_tables, tables, group_stream, [&](int32_t i) {
-    return mono_lookup_pool(tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], out[i]);
-  });
+  int rc = group_check(n_tables, tables);
+  if (rc != MONO_OK) return rc;
+  if (n_tables == 0) return MONO_OK;
+  if (!ids || !n_ids || !slot_offsets || !n_bags || !out) return MONO_ERR_ARG;
+  for (int32_t i = 0; i < n_tables; ++i) {
+    mono_table* t = tables[i];
+    join_sweep(t);
+    if ((rc = check_batch(t, ids[i], n_ids[i], slot_offsets[i], n_bags[i])) != MONO_OK) return rc;
+    if (n_bags[i] > 0 && (!out[i] || !aligned(out[i], 16))) return MONO_ERR_ARG;
+    if ((rc = reserve(t, n_ids[i], n_bags[i])) != MONO_OK) return rc;
+  }
+  GroupPlan p;
+  if ((rc = group_begin(p, n_tables, tables, group_stream)) != MONO_OK) return rc;
+  for (int32_t i = 0; i < n_tables; ++i) {
+    group_describe(p, i, tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], out[i], nullptr, 0u,
+                   is_prepared_batch(tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i]));
+    p.items[i].active = n_bags[i] > 0 ? 1u : 0u;           // a bag without IDs still pools to zeros
+  }
+  if ((rc = group_upload(p, tables)) != MONO_OK) return rc;
+  GROUP_LAUNCH(p, K_GATHER, GK_GATHER, 256, group_gather_pool_kernel<0>);
+  GROUP_LAUNCH(p, K_GATHER, GK_GATHER_WIDE, 256, group_gather_pool_kernel<1>);
+  CUDA_TRY(p.owner, cudaGetLastError());
+  for (int32_t i = 0; i < n_tables; ++i)
+    if (p.items[i].prepared) tables[i]->prep.filed = true;
+  return group_end(p, tables);
 }
 
 int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
                            const float* const* grad_pooled, int64_t now, void* group_stream) {
-  if (n_tables > 0 && (!ids || !n_ids || !slot_offsets || !n_bags || !grad_pooled)) return MONO_ERR_ARG;
-  return group_call(n_tables, tables, group_stream, [&](int32_t i) {
-    return mono_apply_grads(tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], grad_pooled[i], now);
-  });
+  int rc = group_check(n_tables, tables);
+  if (rc != MONO_OK) return rc;
+  if (n_tables == 0) return MONO_OK;
+  if (!ids || !n_ids || !slot_offsets || !n_bags || !grad_pooled) return MONO_ERR_ARG;
+  bool all_prepared = true, all_filed = true;
+  for (int32_t i = 0; i < n_tables; ++i) {
+    mono_table* t = tables[i];
+    join_sweep(t);
+    if ((rc = check_batch(t, ids[i], n_ids[i], slot_offsets[i], n_bags[i])) != MONO_OK) return rc;
+    if (n_bags[i] > 0 && (!grad_pooled[i] || !aligned(grad_pooled[i], 16))) return MONO_ERR_ARG;
+    if ((rc = check_now(t, now)) != MONO_OK) return rc;
+    if ((rc = reserve(t, n_ids[i], n_bags[i])) != MONO_OK) return rc;
+    if (n_ids[i] == 0 || n_bags[i] == 0) continue;
+    const bool prepared = is_prepared_batch(t, ids[i], n_ids[i], slot_offsets[i], n_bags[i]);
+    all_prepared &= prepared;
+    all_filed &= prepared && t->prep.filed;
+  }
+  // either every table's batch was announced, or the group is pushed as if none had been
+  for (int32_t i = 0; i < n_tables; ++i) {
+    mono_table* t = tables[i];
+    const bool empty = n_ids[i] == 0 || n_bags[i] == 0;
+    if ((!all_prepared || empty) && (rc = discard_prepared(t)) != MONO_OK) return rc;
+    t->last_now = now;
+  }
+  GroupPlan p;
+  if ((rc = group_begin(p, n_tables, tables, group_stream)) != MONO_OK) return rc;
+  for (int32_t i = 0; i < n_tables; ++i)
+    group_describe(p, i, tables[i], ids[i], n_ids[i], slot_offsets[i], n_bags[i], nullptr, grad_pooled[i], (uint32_t)now, all_prepared);
+  if ((rc = group_upload(p, tables)) != MONO_OK) return rc;
+  if (all_prepared) {
+    if (!all_filed) GROUP_LAUNCH(p, K_FILE, GK_FILE, 256, group_file_segments_kernel);
+    GROUP_LAUNCH(p, K_UPDATE, GK_UPDATE, 256, group_table_update_kernel<kCommit>);
+  } else {
+    group_launch_ids_only(p);
+    GROUP_LAUNCH(p, K_UPDATE, GK_UPDATE, 256, group_table_update_kernel<kLookUp | kCommit>);
+    GROUP_LAUNCH(p, K_FILE, GK_FILE, 256, group_file_segments_kernel);
+  }
+  if (p.any_sketch) GROUP_LAUNCH(p, K_SKETCH, GK_INSERT, 256, group_sketch_add_kernel);
+  GROUP_LAUNCH(p, K_INSERT, GK_INSERT, 256, group_table_insert_kernel);
+  GROUP_LAUNCH(p, K_EXPAND, GK_EXPAND, 128, group_expand_parts_kernel);
+  GROUP_LAUNCH(p, K_ORDER, GK_ORDER, kWindows, group_order_parts_kernel);
+  GROUP_LAUNCH(p, K_REDUCE, GK_REDUCE, 128, group_reduce_adagrad_kernel<0>);
+  GROUP_LAUNCH(p, K_REDUCE, GK_REDUCE_WIDE, 128, group_reduce_adagrad_kernel<1>);
+  GROUP_LAUNCH(p, K_SINGLES, GK_SINGLES, 128, group_update_singletons_kernel<0>);
+  GROUP_LAUNCH(p, K_SINGLES, GK_SINGLES_WIDE, 128, group_update_singletons_kernel<1>);
+  GROUP_LAUNCH(p, K_FOLD, GK_FOLD, 256, group_fold_partials_kernel);
+  GROUP_LAUNCH(p, K_COMBINE, GK_COMBINE, kCombineThreads, group_combine_adagrad_kernel);
+  ++p.owner->launches[K_FINISH];
+  group_finish_apply_kernel<<<(unsigned)n_tables, 256, 0, p.gs>>>(p.d_items, (uint32_t)n_tables, 1);
+  CUDA_TRY(p.owner, cudaGetLastError());
+  for (int32_t i = 0; i < n_tables; ++i) tables[i]->prep.valid = false;
+  return group_end(p, tables);
 }
 
 static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices) {
   if (!t || n_slices == 0 || slice >= n_slices) return MONO_ERR_ARG;
+  if (t->prep.valid) join_sweep(t);                        // (forgetting the announced batch works on the table's stream)
   int rc = check_now(t, now);
   if (rc != MONO_OK) return rc;
   t->last_now = now;
   if (t->tv.ttl == 0) return MONO_OK;
+  // a batch that was announced but not pushed yet was looked up in the table as it was: forget it
+  if ((rc = discard_prepared(t)) != MONO_OK) return rc;
   // The sweep runs on its own stream.  It has to follow everything launched so far that
   // touches the key store, the free list or the sketch; the tail of a mono_apply_grads
   // (gradient reduction and row updates) touches none of them, so a sweep that comes
@@ -577,6 +881,9 @@ int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, 
   if (n_bags > 0 && (!out || !aligned(out, 16))) return MONO_ERR_ARG;
   if (n_ids > (int64_t)MONO_NOALLOC_MAX_IDS) return MONO_ERR_LIMIT;
   if (n_bags == 0) return MONO_OK;
+  int dev = -1;
+  CUDA_TRY(t, cudaGetDevice(&dev));
+  if (dev != t->device) return MONO_ERR_ARG;               // the array of another device would be the wrong memory
   uint32_t* occ_row = nullptr;
   if ((rc = noalloc_scratch(t, &occ_row)) != MONO_OK) return rc;
   const unsigned long long* d_ids = reinterpret_cast<const unsigned long long*>(ids);
@@ -587,17 +894,9 @@ int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, 
     if (blocks > cap) blocks = cap;
     LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, d_ids, n_ids, occ_row));
   }
-  return dispatch_dim(t->tv.dim, [&](auto g, auto nv) -> int {
-    constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
-    const int64_t groups_per_block = 256 / G;
-    int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
-    const int64_t cap = (int64_t)grid_for(t, 8) * 8;
-    if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, occ_row, n_ids, d_off,
-                                                                                    n_bags, out));
-    CUDA_TRY(t, cudaGetLastError());
-    return (int)MONO_OK;
-  });
+  GatherSource src{};
+  src.occ_row = occ_row;
+  return launch_gather<kFromRows>(t, src, n_ids, d_off, n_bags, out);
 }
 
 int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
@@ -610,7 +909,7 @@ int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, con
   cudaStream_t s = t->stream;
   if (n_ids) CUDA_TRY(t, cudaMemcpyAsync(t->stage_ids, ids, (size_t)n_ids * 8, cudaMemcpyHostToDevice, s));
   CUDA_TRY(t, cudaMemcpyAsync(t->stage_off, slot_offsets, (size_t)(n_bags + 1) * 8, cudaMemcpyHostToDevice, s));
-  if ((rc = launch_lookup(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec)) != MONO_OK) return rc;
+  if ((rc = launch_lookup(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec, false)) != MONO_OK) return rc;
   if (n_bags)
     CUDA_TRY(t, cudaMemcpyAsync(out, t->stage_vec, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyDeviceToHost, s));
   CUDA_TRY(t, cudaStreamSynchronize(s));
@@ -632,6 +931,76 @@ int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids, con
     CUDA_TRY(t, cudaMemcpyAsync(t->stage_vec, grad_pooled, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyHostToDevice, s));
   t->last_now = now;
   return launch_apply(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec, (uint32_t)now);
+}
+
+int mono_fence(mono_table* t) {
+  if (!t) return MONO_ERR_ARG;
+  join_sweep(t);
+  return MONO_OK;
+}
+
+int mono_snapshot_save(mono_table* t) {
+  if (!t) return MONO_ERR_ARG;
+  join_sweep(t);
+  auto& sn = t->snap;
+  { const int rc0 = discard_prepared(t); if (rc0 != MONO_OK) return rc0; }   // the per-call counters must be at rest
+  const TableView& tv = t->tv;
+  const size_t row_floats = ((size_t)tv.capacity + 1) * 2 * tv.dim;
+  const size_t counters = tv.sketch_depth ? (size_t)tv.sketch_depth * (tv.sketch_mask + 1) : 0;
+  if (sn.cells && sn.key_cells != t->key_cells) free_snapshot(t);            // the key store was resized since
+  if (!sn.cells) {
+    int rc = dev_alloc(t, &sn.cells, t->key_cells);
+    if (rc == MONO_OK) rc = dev_alloc(t, &sn.stash, kStashCells);
+    if (rc == MONO_OK) rc = dev_alloc(t, &sn.rows, row_floats);
+    if (rc == MONO_OK) rc = dev_alloc(t, &sn.free_rows, tv.capacity);
+    if (rc == MONO_OK) rc = dev_alloc(t, &sn.st, 1);
+    if (rc == MONO_OK && counters) rc = dev_alloc(t, &sn.sketch, counters);
+    if (rc != MONO_OK) { free_snapshot(t); return rc; }
+    sn.key_cells = t->key_cells;
+  }
+  cudaStream_t s = t->stream;
+  const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
+  CUDA_TRY(t, cudaMemcpyAsync(sn.cells, tv.cells, t->key_cells * sizeof(Cell), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(sn.stash, tv.stash, kStashCells * sizeof(Cell), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(sn.rows, tv.rows, row_floats * sizeof(float), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(sn.free_rows, tv.free_rows, tv.capacity * sizeof(uint32_t), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(sn.st, tv.st, sizeof(DevState), dd, s));
+  if (counters) CUDA_TRY(t, cudaMemcpyAsync(sn.sketch, tv.sketch, counters * sizeof(unsigned int), dd, s));
+  sn.last_now = t->last_now;
+  sn.sketch_epoch = t->sketch_epoch;
+  sn.valid = true;
+  return MONO_OK;
+}
+
+int mono_snapshot_restore(mono_table* t) {
+  if (!t) return MONO_ERR_ARG;
+  join_sweep(t);
+  auto& sn = t->snap;
+  if (!sn.valid || sn.key_cells != t->key_cells) return MONO_ERR_ARG;
+  int rc = discard_prepared(t);
+  if (rc != MONO_OK) return rc;
+  const TableView& tv = t->tv;
+  const size_t row_floats = ((size_t)tv.capacity + 1) * 2 * tv.dim;
+  const size_t counters = tv.sketch_depth ? (size_t)tv.sketch_depth * (tv.sketch_mask + 1) : 0;
+  cudaStream_t s = t->stream;
+  const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
+  CUDA_TRY(t, cudaMemcpyAsync(tv.cells, sn.cells, t->key_cells * sizeof(Cell), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(tv.stash, sn.stash, kStashCells * sizeof(Cell), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(tv.rows, sn.rows, row_floats * sizeof(float), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(tv.free_rows, sn.free_rows, tv.capacity * sizeof(uint32_t), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(tv.st, sn.st, sizeof(DevState), dd, s));
+  if (counters) CUDA_TRY(t, cudaMemcpyAsync(tv.sketch, sn.sketch, counters * sizeof(unsigned int), dd, s));
+  t->last_now = sn.last_now;
+  t->sketch_epoch = sn.sketch_epoch;
+  return MONO_OK;
+}
+
+int mono_snapshot_drop(mono_table* t) {
+  if (!t) return MONO_ERR_ARG;
+  join_sweep(t);
+  CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  free_snapshot(t);
+  return MONO_OK;
 }
 
 int mono_status(mono_table* t, mono_status_t* host_out) {
@@ -660,6 +1029,7 @@ int mono_status(mono_table* t, mono_status_t* host_out) {
   host_out->sum_unique_resident = d.sum_unique_resident;
   host_out->sum_new = d.sum_new;
   host_out->sum_single_resident = d.sum_single_resident;
+  host_out->scratch_reallocs = t->scratch_reallocs;
   return MONO_OK;
 }
 
@@ -718,6 +1088,7 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
   if (!t) return MONO_ERR_ARG;
   if (new_key_cells == 0) new_key_cells = t->key_cells;
   if (!is_pow2(new_key_cells) || new_key_cells < 64 || new_key_cells > (1ull << 34)) return MONO_ERR_ARG;
+  { const int rc0 = discard_prepared(t); if (rc0 != MONO_OK) return rc0; }     // its remembered cells are about to move
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
   TableView fresh = t->tv;
   fresh.cells = nullptr;
@@ -754,6 +1125,7 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
 int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, int64_t* n_out) {
   if (t) join_sweep(t);
   if (!t || !n_out || max_n < 0 || (max_n > 0 && (!ids || !w || !aligned(w, 16) || !aligned(ids, 8)))) return MONO_ERR_ARG;
+  { const int rc0 = discard_prepared(t); if (rc0 != MONO_OK) return rc0; }
   CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->export_n, 0, sizeof(unsigned long long), t->stream));
   export_touched_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->tv, t->key_cells,
                                                                reinterpret_cast<unsigned long long*>(ids), w, max_n);
@@ -772,13 +1144,17 @@ int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const
   if (n == 0) return MONO_OK;
   if (!ids || !count || !last_seen || !resident || !aligned(ids, 8)) return MONO_ERR_ARG;
   if ((w && !aligned(w, 16)) || (acc && !aligned(acc, 16))) return MONO_ERR_ARG;
+  int rc = discard_prepared(t);
+  if (rc != MONO_OK) return rc;
   uint32_t* row_word = nullptr;
   const int64_t chunk = n < (1ll << 24) ? n : (1ll << 24);
-  int rc = dev_alloc(t, &row_word, (size_t)chunk);
+  rc = dev_alloc(t, &row_word, (size_t)chunk);
   if (rc != MONO_OK) return rc;
   for (int64_t lo = 0; lo < n; lo += chunk) {
     const int64_t m = n - lo < chunk ? n - lo : chunk;
     const size_t ro = (size_t)lo * t->tv.dim;
+    import_check_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(
+        t->tv, reinterpret_cast<const unsigned long long*>(ids) + lo, m, row_word);
     import_insert_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(
         t->tv, reinterpret_cast<const unsigned long long*>(ids) + lo, count + lo,
         reinterpret_cast<const long long*>(last_seen) + lo, resident + lo, m, row_word);
@@ -850,7 +1226,6 @@ int mono_timing_read(mono_table* t, mono_timing_t* host_out, int reset) {
   if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
-  CUDA_TRY(t, cudaStreamSynchronize(t->prep_stream));
   for (auto& p : t->pending) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, p.second.first, p.second.second) == cudaSuccess) t->kernel_ms[p.first] += ms;

@@ -101,7 +101,7 @@ struct DevState {
   unsigned int n_long;                   // distinct IDs whose segment is split into parts
   unsigned int n_parts;
   unsigned int n_folds;                  // groups of kFoldWidth parts that are added up before the final combine
-  unsigned int pad2;
+  unsigned int call_bad_offsets;         // this call's offsets were malformed: occurrences are checked one by one
   unsigned int n_valid_ids;
   unsigned int seg_cursor;               // entries of bag_of_sorted[] handed out so far
   unsigned int n_multi;                  // distinct IDs that occur more than once in the batch
@@ -194,6 +194,12 @@ __device__ inline Cell load_cell(const Cell* p) {
   c.meta = *reinterpret_cast<const volatile unsigned long long*>(&p->meta);
   return c;
 }
+// One ordinary 16-byte load: for kernels that also write cells (no key moves while they run).
+__device__ inline Cell load_cell_whole(const Cell* p) {
+  const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
+  Cell c; c.key = v.x; c.meta = v.y; return c;
+}
+// The same through the read-only data path: only for kernels that write no cell.
 __device__ inline Cell load_cell_ro(const Cell* p) {
   const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2*>(p));
   Cell c; c.key = v.x; c.meta = v.y; return c;

@@ -50,15 +50,31 @@ def assert_audit_ok(gpu_table, what: str = "audit"):
 
 
 def run_stream(gpu_table, oracle, stream, steps, *, sweep_every: int = 1, check_every: int = 1,
-               time_scale: int = 1, check_forward: bool = True):
-    """Feed steps [0, steps) of `stream` to both sides; compare as it goes."""
+               time_scale: int = 1, check_forward: bool = True, prepare: bool = False):
+    """Feed steps [0, steps) of `stream` to both sides; compare as it goes.  With `prepare`
+    every batch is announced with mono_prepare_push before its lookup, as a training loop
+    that knows its batch ahead of the pull would do."""
+    import torch
+    from paper_2209_07663_b200 import binding as mb
     for t in range(steps):
         s = stream.step(t)
         now = t * time_scale
-        if check_forward:
-            got = gpu_table.lookup_pool(s.ids, s.offsets).cpu().numpy()
-            assert_vectors_close(got, oracle.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
-        gpu_table.apply_grads(s.ids, s.offsets, s.grad_pooled, now)
+        if prepare:
+            ids = torch.from_numpy(s.ids.view(np.int64)).cuda()
+            off = torch.from_numpy(s.offsets).cuda()
+            grad = torch.from_numpy(s.grad_pooled).cuda()
+            n_bags = off.numel() - 1
+            mb.mono_prepare_push(gpu_table.handle, ids, ids.numel(), off, n_bags)
+            if check_forward:
+                out = torch.empty((n_bags, gpu_table.dim), dtype=torch.float32, device="cuda")
+                mb.mono_lookup_pool(gpu_table.handle, ids, ids.numel(), off, n_bags, out)
+                assert_vectors_close(out.cpu().numpy(), oracle.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+            mb.mono_apply_grads(gpu_table.handle, ids, ids.numel(), off, n_bags, grad, now)
+        else:
+            if check_forward:
+                got = gpu_table.lookup_pool(s.ids, s.offsets).cpu().numpy()
+                assert_vectors_close(got, oracle.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+            gpu_table.apply_grads(s.ids, s.offsets, s.grad_pooled, now)
         assert oracle.apply_grads(s.ids, s.offsets, s.grad_pooled, now) == 0, "stream overflowed the oracle"
         if sweep_every and t % sweep_every == sweep_every - 1:
             gpu_table.expire(now)

@@ -58,8 +58,12 @@ def test_algorithmic_bytes_adds_up():
     n, b, u, ur, ur1, unew, d = 1000, 600, 400, 300, 250, 50, 64
     per, total = bench.algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=1 << 10)
     assert total == sum(per.values())
-    assert per["probe_rows"] == 40 * n and per["dedup_tile"] == 32 * n and per["table_update"] == 64 * u
-    assert per["gather_pool"] == 8 * (b + 1) + 4 * d * ur + 4 * d * b
+    assert per["dedup_tile"] == 32 * n and per["table_lookup"] == 32 * u and per["table_update"] == 64 * u
+    assert per["gather_pool"] == 8 * (b + 1) + 8 * n + 4 * d * ur + 4 * d * b
+    # a batch that was not announced pays one key-store sector per occurrence inside the lookup instead
+    per_u, total_u = bench.algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=1 << 10, prepared=False)
+    assert per_u["table_lookup"] == 0 and per_u["gather_pool"] == per["gather_pool"] + 32 * n
+    assert total_u - total == 32 * n - 32 * u
     # the Adagrad phase reads every gradient row once and reads and writes row + accumulator of every ID with a row
     assert per["update_singletons"] + per["reduce_adagrad"] == 16 * d * ur + 4 * d * b
     assert per["expire"] == 16 << 10

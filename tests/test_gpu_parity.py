@@ -31,10 +31,11 @@ def bags(lists):
 
 # ---------------------------------------------------------------- configured streams
 
-def test_tiny_config_full_stream():
+@pytest.mark.parametrize("prepare", [False, True])
+def test_tiny_config_full_stream(prepare):
     cfg = wl.CONFIGS["tiny"]
     gpu, cpu = make_pair(cfg)
-    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=1)
+    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=1, prepare=prepare)
     assert st["n_expired_total"] > 0 and st["n_admitted_total"] > 0
     assert st["n_tracked"] > st["n_resident"] > 0
 
@@ -45,27 +46,31 @@ def test_medium_config_prefix():
     run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=4, check_every=4)
 
 
-def test_medium_config_short_ttl_churn():
+@pytest.mark.parametrize("prepare", [False, True])
+def test_medium_config_short_ttl_churn(prepare):
     # the medium shape with a TTL short enough that rows are recycled many times
     cfg = wl.scaled(wl.CONFIGS["medium"], steps=10, ttl=2, n_examples=2048, capacity=1 << 18, key_cells=1 << 20)
     gpu, cpu = make_pair(cfg)
-    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5)
+    st = run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5, prepare=prepare)
     assert st["n_expired_total"] > 10000
 
 
-def test_drift_config_scaled_down():
+@pytest.mark.parametrize("prepare", [False, True])
+def test_drift_config_scaled_down(prepare):
     cfg = wl.scaled(wl.CONFIGS["drift"], n_examples=512, n_slots=10, n_distinct=1 << 18, capacity=1 << 16,
                     key_cells=1 << 18, ttl=6, drift_period=4, steps=16)
     gpu, cpu = make_pair(cfg)
-    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=4)
+    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=4, prepare=prepare)
 
 
+@pytest.mark.parametrize("prepare", [False, True])
 @pytest.mark.parametrize("dim", [4, 8, 12, 16, 32, 48, 64, 128, 200, 256, 512, 1024])
-def test_every_dim_variant(dim):
+def test_every_dim_variant(dim, prepare):
+    # bags of 0 to 40 IDs: longer than the widest lane group, so a bag takes several rounds
     cfg = wl.scaled(wl.CONFIGS["tiny"], dim=dim, n_examples=160, n_slots=5, n_distinct=1 << 12, steps=6,
-                    capacity=1 << 12, key_cells=1 << 13, bag_len=("uniform", 0, 9))
+                    capacity=1 << 12, key_cells=1 << 13, bag_len=("uniform", 0, 40))
     gpu, cpu = make_pair(cfg)
-    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=3)
+    run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=3, prepare=prepare)
 
 
 def test_multi_table_configs_scaled_down():
@@ -75,14 +80,19 @@ def test_multi_table_configs_scaled_down():
         run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=5)
 
 
-def test_grouped_calls_on_eight_streams_match_eight_oracles():
-    """mono_group_lookup_pool / mono_group_apply_grads: the eight tables of the mixed-dim
-    configuration (scaled down), each on its own stream, one grouped call per step; every
-    table's outputs and state are those of its own oracle.  Also: a table named twice and a
-    null entry are refused, and an empty group is fine."""
+@pytest.mark.parametrize("announce", [False, True])
+@pytest.mark.parametrize("own_streams", [False, True])
+def test_grouped_calls_match_one_oracle_per_table(own_streams, announce):
+    """mono_group_prepare_push / _lookup_pool / _apply_grads: the eight tables of the mixed-dim
+    configuration (scaled down) and a ninth with rows of 256 columns, one launch per kernel
+    for all of them; every table's outputs and state are those of its own oracle.  With the
+    tables on the group's stream or each on a stream of its own; with the batches announced
+    or not, and once with one table's announcement missing.  Also: a table whose batch is
+    empty, a table named twice and a null entry are refused, an empty group is fine."""
     cfgs = [wl.scaled(c, capacity=1 << 13, key_cells=1 << 15, n_distinct=1 << 14, steps=5, ttl=3)
             for c in wl.multi_table_configs(n_examples=256, slots=3)]
-    streams = [torch.cuda.Stream() for _ in cfgs]
+    cfgs.append(wl.scaled(cfgs[2], dim=256, seed=cfgs[2].seed + 1, name="wide"))
+    streams = [torch.cuda.Stream() if own_streams else torch.cuda.current_stream() for _ in cfgs]
     pairs = []
     for c, st in zip(cfgs, streams):
         kw = dict(lr=c.lr, eps=c.eps, init_acc=c.init_acc, init_scale=c.init_scale, seed=c.seed)
@@ -92,10 +102,18 @@ def test_grouped_calls_on_eight_streams_match_eight_oracles():
     gens = [wl.Stream(c) for c in cfgs]
     handles = [g.handle for g, _ in pairs]
     group_stream = torch.cuda.current_stream().cuda_stream
-    for t in range(5):
+    for t in range(6):
         steps = [g.step(t) for g in gens]
+        if t == 3:                                               # table 1 sits this step out
+            steps[1] = wl.Step(ids=steps[1].ids[:0], offsets=np.zeros(1, np.int64),
+                               grad_pooled=steps[1].grad_pooled[:0], now=t)
         dev = [_dev_batch(s) for s in steps]
-        outs = [torch.empty((c.n_bags, c.dim), dtype=torch.float32, device="cuda") for c in cfgs]
+        outs = [torch.empty((s.offsets.size - 1, c.dim), dtype=torch.float32, device="cuda") for c, s in zip(cfgs, steps)]
+        if announce:
+            mb.mono_group_prepare_push(handles, [d[0] for d in dev], [d[1] for d in dev], group_stream)
+            if t == 4:                                           # one announcement is replaced by another batch's
+                o = _dev_batch(gens[5].step(77))
+                mb.mono_prepare_push(handles[5], o[0], o[0].numel(), o[1], cfgs[5].n_bags)
         mb.mono_group_lookup_pool(handles, [d[0] for d in dev], [d[1] for d in dev], outs, group_stream)
         for (gpu, cpu), s, out in zip(pairs, steps, outs):       # `out` is read on the group's stream
             assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
@@ -112,8 +130,13 @@ def test_grouped_calls_on_eight_streams_match_eight_oracles():
         mb.mono_group_lookup_pool([handles[0], handles[0]], [d0[0]] * 2, [d0[1]] * 2, [out0] * 2, group_stream)
     with pytest.raises(mb.MonoError):
         mb.mono_group_lookup_pool([handles[0], None], [d0[0]] * 2, [d0[1]] * 2, [out0] * 2, group_stream)
+    # the whole step of nine tables is a handful of launches, not nine times the single-table count
+    n_launches = mb.mono_timing_read(handles[0], reset=True)["launches_total"]
     for gpu, _ in pairs:
         assert_audit_ok(gpu)
+        assert gpu.status()["error_bits"] == 0
+    per_step = 3 + 2 + 15
+    assert n_launches <= 6 * per_step + 6 * 2 + 4              # grouped kernels + table 0's own sweeps (gpu.expire)
 
 
 # ---------------------------------------------------------------- edge cases
@@ -154,8 +177,9 @@ def test_offsets_that_skip_ids():
     assert_vectors_close(gpu.lookup_pool(ids, off).cpu().numpy(), cpu.lookup_pool(ids, off), "pooled")
 
 
+@pytest.mark.parametrize("prepare", [False, True])
 @pytest.mark.parametrize("n_occ", [63, 64, 65, 255, 257, 1000, 4096, 4097, 4200, 70000])
-def test_one_hot_id_long_segment(n_occ):
+def test_one_hot_id_long_segment(n_occ, prepare):
     # a single ID owning a whole batch: the segment is split into parts and recombined
     dim = 64
     rng = np.random.default_rng(n_occ)
@@ -168,9 +192,15 @@ def test_one_hot_id_long_segment(n_occ):
     off[1:] = np.cumsum(lens)
     ids = np.full(n_occ, 0xABCDEF0123456789, np.uint64)
     ids[::97] = 77          # a second, cooler ID mixed in
+    d_ids, d_off = torch.from_numpy(ids.view(np.int64)).cuda(), torch.from_numpy(off).cuda()
     for t in range(2):
         grad = (rng.standard_normal((n_bags, dim)) * 0.01).astype(f32)
-        gpu.apply_grads(ids, off, grad, t)
+        if prepare:
+            # announced and pushed without a lookup in between: the push files the bags itself
+            mb.mono_prepare_push(gpu.handle, d_ids, n_occ, d_off, n_bags)
+            mb.mono_apply_grads(gpu.handle, d_ids, n_occ, d_off, n_bags, torch.from_numpy(grad).cuda(), t)
+        else:
+            gpu.apply_grads(ids, off, grad, t)
         cpu.apply_grads(ids, off, grad, t)
     assert_state_equal(gpu, cpu)
     assert_vectors_close(gpu.lookup_pool(ids[:7], np.array([0, 7], np.int64)).cpu().numpy(),
@@ -495,6 +525,107 @@ def test_touched_key_export_matches_the_oracle():
 
 # ---------------------------------------------------------------- cuckoo structure under load
 
+def test_announced_batch_survives_reads_and_is_dropped_by_anything_that_changes_the_table():
+    """Between mono_prepare_push and the push of that batch: a second lookup of the batch, a lookup
+    of another batch and the read-only fixtures leave the announcement in force; a sweep, an import,
+    a rehash or an incremental export make the push look everything up again.  Either way the
+    table ends up as the oracle's."""
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=14, ttl=2, key_cells=1 << 16)
+    gpu, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    h = gpu.handle
+    out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
+    for t in range(cfg.steps):
+        s = stream.step(t)
+        ids, off, grad = _dev_batch(s)
+        mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+        kind = t % 7
+        if kind == 0:                       # two lookups of the announced batch
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        elif kind == 1:                     # a lookup of another batch in between, then the announced one
+            o = _dev_batch(stream.step(t + 50))
+            got = gpu.lookup_pool(o[0], o[1]).cpu().numpy()
+            assert_vectors_close(got, cpu.lookup_pool(stream.step(t + 50).ids, stream.step(t + 50).offsets), "other batch")
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        elif kind == 2:                     # read-only fixtures
+            gpu.status(); gpu.probe(s.ids[:50]); gpu.audit()
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        elif kind == 3:                     # a sweep between the announcement and the lookup
+            gpu.expire(t - 1); cpu.expire(t - 1)
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        elif kind == 4:                     # ... and between the lookup and the push
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+            want = cpu.lookup_pool(s.ids, s.offsets)
+            assert_vectors_close(out.cpu().numpy(), want, f"step {t}: pooled before the sweep")
+            for k in range(3):
+                mb.mono_expire_slice(h, t - 1, k, 3)
+            cpu.expire(t - 1)
+        elif kind == 5:                     # a rehash moves every key
+            gpu.rehash(0, 1000 + t)
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        else:                               # an incremental export rewrites metadata
+            g, o = gpu.export_touched(), cpu.export_touched()
+            assert (g["ids"] == o["ids"]).all()
+            mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        if kind != 4:
+            assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+        mb.mono_apply_grads(h, ids, ids.numel(), off, cfg.n_bags, grad, t)
+        assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
+        assert_state_equal(gpu, cpu, f"step {t}")
+        assert_audit_ok(gpu, f"step {t}")
+    st = gpu.status()
+    assert st["error_bits"] == 0 and st["n_expired_total"] > 0 and st["scratch_reallocs"] == 0
+
+
+def test_snapshot_restore_returns_to_the_saved_state():
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=9, ttl=3, key_cells=1 << 16)
+    gpu, cpu = make_pair(cfg)
+    stream = wl.Stream(cfg)
+    with pytest.raises(mb.MonoError):
+        mb.mono_snapshot_restore(gpu.handle)              # nothing saved yet
+    run_stream(gpu, cpu, stream, 4, sweep_every=2, check_every=4)
+    mb.mono_snapshot_save(gpu.handle)
+    saved = gpu.export()
+    for rep in range(2):                                  # the same five steps twice, from the same state
+        twin = mo.OracleTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
+                              init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed)
+        assert twin.import_entries(saved["ids"], saved["count"], saved["last_seen"], saved["resident"],
+                                   saved["w"], saved["acc"]) == 0
+        for t in range(4, 9):
+            s = stream.step(t)
+            ids, off, grad = _dev_batch(s)
+            mb.mono_prepare_push(gpu.handle, ids, ids.numel(), off, cfg.n_bags)
+            gpu_out = torch.empty((cfg.n_bags, cfg.dim), device="cuda")
+            mb.mono_lookup_pool(gpu.handle, ids, ids.numel(), off, cfg.n_bags, gpu_out)
+            assert_vectors_close(gpu_out.cpu().numpy(), twin.lookup_pool(s.ids, s.offsets), f"rep {rep} step {t}")
+            mb.mono_apply_grads(gpu.handle, ids, ids.numel(), off, cfg.n_bags, grad, t)
+            twin.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+            gpu.expire(t); twin.expire(t)
+        assert_state_equal(gpu, twin, f"rep {rep}")
+        assert_audit_ok(gpu)
+        mb.mono_snapshot_restore(gpu.handle)              # time goes back with the state
+        g = gpu.export()
+        assert (g["ids"] == saved["ids"]).all() and (g["last_seen"] == saved["last_seen"]).all()
+        assert np.array_equal(g["w"], saved["w"]) and np.array_equal(g["acc"], saved["acc"])
+    mb.mono_snapshot_drop(gpu.handle)
+    with pytest.raises(mb.MonoError):
+        mb.mono_snapshot_restore(gpu.handle)
+
+
+def test_growing_scratch_inside_a_hot_call_is_counted():
+    gpu = mb.MonoTable(1 << 10, 8, 1, 0, max_ids=2048, max_bags=2048)
+    ids = np.arange(1, 5001, dtype=np.uint64)
+    off = np.arange(0, 5001, dtype=np.int64)
+    assert gpu.status()["scratch_reallocs"] == 0
+    gpu.lookup_pool(ids[:2000], off[:2001])
+    assert gpu.status()["scratch_reallocs"] == 0
+    gpu.lookup_pool(ids, off)                             # 5000 IDs: larger than the scratch
+    assert gpu.status()["scratch_reallocs"] == 1
+    gpu.apply_grads(ids, off, np.zeros((5000, 8), f32), 0)
+    assert gpu.status()["scratch_reallocs"] == 1
+
+
 @pytest.mark.parametrize("load", [0.5, 0.8, 0.9])
 @pytest.mark.parametrize("kind", ["random", "sequential", "high_bits", "stride_4096"])
 def test_cuckoo_membership_at_load(load, kind):
@@ -578,15 +709,52 @@ def test_key_store_full_is_flagged_without_duplicates():
     assert (gpu.probe(sub, rows=False)["count"] == 2).all()
 
 
-def test_malformed_offsets_are_flagged_not_followed():
-    gpu = mb.MonoTable(64, 4, 1, 0)
+def _well_formed_only(ids, off):
+    """The batch an oracle sees when every malformed bag is emptied."""
+    lists = []
+    for b in range(len(off) - 1):
+        lo, hi = int(off[b]), int(off[b + 1])
+        lists.append(list(ids[lo:hi]) if 0 <= lo <= hi <= len(ids) else [])
+    return bags(lists)
+
+
+@pytest.mark.parametrize("prepared", [False, True])
+def test_malformed_offsets_empty_the_offending_bags_in_both_directions(prepared):
+    kw = dict(init_scale=0.1, seed=5)
+    gpu, cpu = mb.MonoTable(64, 4, 1, 0, **kw), mo.OracleTable(64, 4, 1, 0, **kw)
     ids = np.arange(1, 9, dtype=np.uint64)
-    off = np.array([0, 4, 2, 100], np.int64)           # decreasing, then past the end
-    out = gpu.lookup_pool(ids, off).cpu().numpy()
-    assert out.shape == (3, 4)
-    gpu.apply_grads(ids, off, np.ones((3, 4), f32), 0)
-    assert gpu.status()["error_bits"] & mb.MONO_DEV_BAD_OFFSETS
-    assert_audit_ok(gpu)
+    rng = np.random.default_rng(3)
+    # a well-formed call first, so that the per-occurrence scratch holds plausible left-overs
+    good = np.array([0, 2, 4, 6, 8], np.int64)
+    g0 = rng.standard_normal((4, 4)).astype(f32)
+    gpu.apply_grads(ids, good, g0, 0)
+    cpu.apply_grads(ids, good, g0, 0)
+    fresh = np.arange(101, 109, dtype=np.uint64)           # IDs 103..105 occur only in malformed bags
+    for t, off in enumerate([np.array([0, 2, -1, 5, 8], np.int64),      # bags 1 and 2 malformed
+                             np.array([0, 4, 2, 100, 100], np.int64)], 1):   # decreasing, then past the end
+        grad = rng.standard_normal((4, 4)).astype(f32)
+        ids_t = torch.from_numpy(fresh.view(np.int64)).cuda()
+        off_t = torch.from_numpy(off).cuda()
+        grad_t = torch.from_numpy(grad).cuda()
+        o_ids, o_off = _well_formed_only(fresh, off)
+        out = torch.empty((4, 4), device="cuda")
+        if prepared:
+            mb.mono_prepare_push(gpu.handle, ids_t, 8, off_t, 4)
+        mb.mono_lookup_pool(gpu.handle, ids_t, 8, off_t, 4, out)
+        assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(o_ids, o_off), f"call {t}: pooled")
+        mb.mono_apply_grads(gpu.handle, ids_t, 8, off_t, 4, grad_t, t)
+        assert cpu.apply_grads(o_ids, o_off, grad, t) == 0
+        assert gpu.status()["error_bits"] & mb.MONO_DEV_BAD_OFFSETS
+        assert_state_equal(gpu, cpu, f"call {t}")
+        assert_audit_ok(gpu)
+        mb.mono_clear_errors(gpu.handle)
+    tracked = set(gpu.export(rows=False)["ids"].tolist())
+    assert tracked & set(range(101, 109)) == {101, 102, 103, 104, 106, 107, 108}   # 105: only ever in malformed bags
+    # a well-formed call afterwards is not affected by the earlier flag
+    gpu.apply_grads(ids, good, g0, 3)
+    cpu.apply_grads(ids, good, g0, 3)
+    assert_state_equal(gpu, cpu, "well-formed call after malformed ones")
+    assert gpu.status()["error_bits"] == 0
 
 
 def test_host_detected_errors():
