@@ -294,6 +294,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
         "table_lookup": 32 * u if prepared else 0,           # one bucket sector per distinct ID
         "table_update": 64 * u,                              # count/stamp read-modify-write of that sector
         "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
+        "sketch_add": 0,                                     # (probabilistic filter: counted with table_insert's new IDs)
         "update_singletons": 20 * d * ur1,                   # IDs seen once: gradient row, row and accumulator in and out
         "reduce_adagrad": 16 * d * (ur - ur1) + 4 * d * max(b - ur1, 0),   # rows of repeated IDs + the other gradient rows, once
         "file_segments": 0,
@@ -306,7 +307,7 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
 KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
     "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
-    "table_lookup": "table", "table_update": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
+    "table_lookup": "table", "table_update": "table", "sketch_add": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
     "update_singletons": "adagrad", "file_segments": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
     "combine_adagrad": "adagrad", "expire": "expire",
 }
@@ -347,6 +348,11 @@ def run_ours(args):
 
     base = wl.CONFIGS[args.workload]
     cfg = rank_config(base, rank)
+    sketch = args.filter == "sketch"
+    if sketch:
+        # probabilistic admission filter: IDs without a row live in a count-min sketch, not in the key
+        # store, which is therefore sized for the IDs that own rows only
+        cfg = wl.scaled(cfg, key_cells=max(cfg.key_cells >> args.sketch_key_shrink_log2, 1 << 10))
     drift = cfg.drift_period > 0
     if drift:
         # The drift stream has no closed-form steady state to pre-fill: it starts from an empty
@@ -368,9 +374,13 @@ def run_ours(args):
     table = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
                          init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed,
                          key_cells=cfg.key_cells, max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1),
-                         max_bags=cfg.n_bags)
+                         max_bags=cfg.n_bags, sketch_depth=args.sketch_depth if sketch else 0,
+                         sketch_width=(1 << args.sketch_width_log2) if sketch else 0)
     if args.prefill:
         for ids, cnt, seen in wl.steady_state_population_torch(cfg, now0, dev):
+            if sketch:      # only IDs with a row have an entry; the sketch starts empty, as after one of its clearings
+                keep = cnt >= cfg.filter_threshold
+                ids, cnt, seen = ids[keep], cnt[keep], seen[keep]
             res = (cnt >= cfg.filter_threshold).to(torch.uint8)
             mb.mono_import(table.handle, ids, cnt, seen, res, None, None, ids.numel())
             del ids, cnt, seen, res
@@ -486,8 +496,9 @@ def run_ours(args):
             if S > 0:
                 mb.mono_expire_slice(table.handle, now, (W + K + KT + t) % S, S)
             n_e2e_ids += ids.numel()
-            h2d += 2 * (ids.numel() * 8 + off.numel() * 8) + grad.numel() * 4
+            h2d += ids.numel() * 8 + off.numel() * 8 + grad.numel() * 4    # the push reuses the IDs its lookup staged
             d2h += out_h.numel() * 4
+        mb.mono_fence(table.handle)              # the copies run on streams of the table's own
         e1.record()
         barrier()
         e2e_ms = e0.elapsed_time(e1)
@@ -542,6 +553,16 @@ def run_ours(args):
                 "sweep": (f"every step sweeps 1/{S} of the key store (a full sweep every {S} steps)" if S > 0
                           else "none"), "l2": "every step reads a fresh batch larger than L2",
                 "parallelism": f"{world} independent table(s), one per GPU",
+                "filter": ({"kind": "count-min sketch", "depth": args.sketch_depth, "width": 1 << args.sketch_width_log2,
+                            "sketch_bytes": 4 * args.sketch_depth << args.sketch_width_log2,
+                            "key_store_bytes": 16 * cfg.key_cells, "key_store_bytes_exact_filter": 16 * base.key_cells,
+                            "state": "sketch empty at the start (as after one of its clearings), rows pre-filled",
+                            "admitted_per_step": (st_b["n_admitted_total"] - st_a["n_admitted_total"]) / K,
+                            "entered_key_store_per_step": (st_b["n_inserted_total"] - st_a["n_inserted_total"]) / K}
+                           if sketch else
+                           {"kind": "exact per-ID counters in the key store", "key_store_bytes": 16 * cfg.key_cells,
+                            "admitted_per_step": (st_b["n_admitted_total"] - st_a["n_admitted_total"]) / K,
+                            "entered_key_store_per_step": (st_b["n_inserted_total"] - st_a["n_inserted_total"]) / K}),
                 "push_prepared": ("mono_prepare_push before each lookup: the batch is grouped and every distinct ID "
                                   "looked up once, for the lookup and the push together" if args.prepare else "no"),
             },
@@ -604,9 +625,11 @@ def run_ours(args):
 
 
 def run_multi(args):
-    """The mixed-dim multi-table configuration: 8 independent tables, each on its own CUDA
-    stream, so that the latency-bound kernels of one table overlap the bandwidth-bound kernels
-    of another.  A step = lookup_pool + apply_grads + one slice of the expiry sweep on every table."""
+    """The mixed-dim multi-table configuration: 8 tables of one process on one stream, every
+    step through the grouped calls (one kernel launch per step of the path for all eight
+    tables).  A step = prepare + lookup_pool + apply_grads on every table, and one slice of the
+    expiry sweep per table.  The same steps through the single-table calls, table after
+    table, are timed beside it."""
     import torch
     from paper_2209_07663_b200 import binding as mb
     if not torch.cuda.is_available():
@@ -621,13 +644,11 @@ def run_multi(args):
     dev = torch.device("cuda", local_rank)
     K, W, S = args.steps, args.warmup, args.sweep_slices
     cfgs = [rank_config(c, rank) for c in wl.multi_table_configs()]
-    streams = [torch.cuda.Stream(device=dev) for _ in cfgs]
     tables, now0 = [], []
-    for cfg, st in zip(cfgs, streams):
+    for cfg in cfgs:
         t = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
                          init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed, key_cells=cfg.key_cells,
-                         max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1), max_bags=cfg.n_bags,
-                         stream=st.cuda_stream)
+                         max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1), max_bags=cfg.n_bags)
         n0 = cfg.ttl - 1
         for ids, cnt, seen in wl.steady_state_population_torch(cfg, n0, dev):
             res = (cnt >= cfg.filter_threshold).to(torch.uint8)
@@ -658,64 +679,58 @@ def run_multi(args):
     torch.cuda.synchronize()
 
     handles = [t.handle for t in tables]
+    gs = torch.cuda.current_stream().cuda_stream
+    assert len(set(now0)) == 1
 
-    def step(i, serial):
-        if not serial:
-            # the grouped calls: every table on its own stream, one C call for all eight
-            gs = torch.cuda.current_stream().cuda_stream
-            now = [n0 + 1 + i for n0 in now0]
-            assert len(set(now)) == 1
+    def step(i, grouped):
+        now = now0[0] + 1 + i
+        if grouped:
+            ids, off, grad = [b[i][0] for b in batches], [b[i][1] for b in batches], [b[i][2] for b in batches]
             if args.prepare:
-                for ti, t in enumerate(tables):
-                    ids, off, _ = batches[ti][i]
-                    mb.mono_prepare_push(t.handle, ids, ids.numel(), off, cfgs[ti].n_bags)
-            mb.mono_group_lookup_pool(handles, [b[i][0] for b in batches], [b[i][1] for b in batches], outs, gs)
-            mb.mono_group_apply_grads(handles, [b[i][0] for b in batches], [b[i][1] for b in batches],
-                                      [b[i][2] for b in batches], now[0], gs)
-            if S > 0:
-                for ti, t in enumerate(tables):
-                    mb.mono_expire_slice(t.handle, now[0], i % S, S)
-            return
-        for ti, (cfg, t) in enumerate(zip(cfgs, tables)):
-            ids, off, grad = batches[ti][i]
-            if args.prepare:
-                mb.mono_prepare_push(t.handle, ids, ids.numel(), off, cfg.n_bags)
-            mb.mono_lookup_pool(t.handle, ids, ids.numel(), off, cfg.n_bags, outs[ti])
-            mb.mono_apply_grads(t.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0[ti] + 1 + i)
-            if S > 0:
-                mb.mono_expire_slice(t.handle, now0[ti] + 1 + i, i % S, S)
-            if serial:
-                streams[ti].synchronize()
+                mb.mono_group_prepare_push(handles, ids, off, gs)
+            mb.mono_group_lookup_pool(handles, ids, off, outs, gs)
+            mb.mono_group_apply_grads(handles, ids, off, grad, now, gs)
+        else:
+            for ti, (cfg, t) in enumerate(zip(cfgs, tables)):
+                ids, off, grad = batches[ti][i]
+                if args.prepare:
+                    mb.mono_prepare_push(t.handle, ids, ids.numel(), off, cfg.n_bags)
+                mb.mono_lookup_pool(t.handle, ids, ids.numel(), off, cfg.n_bags, outs[ti])
+                mb.mono_apply_grads(t.handle, ids, ids.numel(), off, cfg.n_bags, grad, now)
+        if S > 0:
+            for t in tables:
+                mb.mono_expire_slice(t.handle, now, i % S, S)
 
-    def timed(first, serial):
+    def timed(first, grouped):
         torch.cuda.synchronize()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
-        for st in streams:
-            st.wait_event(ev0)
         for i in range(first, first + K):
-            step(i, serial)
-        for st in streams:
-            done = torch.cuda.Event()
-            done.record(st)
-            torch.cuda.current_stream().wait_event(done)
+            step(i, grouped)
+        for t in tables:
+            mb.mono_fence(t.handle)
         ev1.record()
         torch.cuda.synchronize()
         return ev0.elapsed_time(ev1)
 
+    def launches_now():
+        return sum(mb.mono_timing_read(t.handle, reset=True)["launches_total"] for t in tables)
+
     for i in range(W):
-        step(i, False)
+        step(i, True)
     before = [t.status() for t in tables]
+    launches_now()
     sampler = ClockSampler(local_rank, gpu_uuid(local_rank))
     sampler.start()
-    ms = timed(W, False)
+    ms = timed(W, True)
     clocks = sampler.stop()
+    launches = launches_now()
     mid = [t.status() for t in tables]
-    ms_serial = timed(W + K, True)
+    ms_serial = timed(W + K, False)
+    launches_serial = launches_now()
     after = [t.status() for t in tables]
     n_ids = sum(b["sum_ids"] - a["sum_ids"] for a, b in zip(before, mid))
     n_ids_serial = sum(b["sum_ids"] - a["sum_ids"] for a, b in zip(mid, after))
-    launches = sum(mb.mono_timing_read(t.handle)["launches_total"] for t in tables)
     (ms_max,), (ids_all,) = aggregate_over_ranks([ms], [float(n_ids)], dev)
     alg = 0
     for cfg, a, b in zip(cfgs, before, mid):
@@ -740,9 +755,11 @@ def run_multi(args):
                        "ids_per_step": n_ids / K, "prefill": "the state after ttl steps of each stream from an empty table (Poisson model)",
                        "sweep": f"every step sweeps 1/{S} of every key store" if S > 0 else "none",
                        "l2": "every step reads fresh batches larger than L2",
-                       "parallelism": "8 tables on 8 CUDA streams of one GPU, one grouped call per step and direction"},
-            "serial": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,
-                       "what": "the same calls with each table's stream drained before the next table starts"},
+                       "parallelism": "8 tables on one CUDA stream of one GPU; grouped calls: one launch per kernel for all tables"},
+            "launches_per_step": launches / K,
+            "one_table_at_a_time": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,
+                                    "launches_per_step": launches_serial / K,
+                                    "what": "the same steps through the single-table calls, table after table"},
             "gpu_launches": launches, "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "all kernels of the 8 tables (whole step)", "achieved": achieved,
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
@@ -765,6 +782,12 @@ def main():
                     help="do not announce each batch with mono_prepare_push before its lookup")
     ap.add_argument("--sweep-slices", type=int, default=32,
                     help="every step sweeps 1/S of the key store for expired IDs (0 = no sweep)")
+    ap.add_argument("--filter", default="exact", choices=["exact", "sketch"],
+                    help="admission filter: exact per-ID counters (default) or the count-min sketch")
+    ap.add_argument("--sketch-depth", type=int, default=4)
+    ap.add_argument("--sketch-width-log2", type=int, default=28, help="counters per sketch row = 2^this")
+    ap.add_argument("--sketch-key-shrink-log2", type=int, default=3,
+                    help="with --filter sketch the key store has 2^-this of the configured cells")
     ap.add_argument("--reps", type=int, default=5,
                     help="repetitions of the timed region, each from the same restored state (median reported)")
     ap.add_argument("--e2e-steps", type=int, default=4)

@@ -72,7 +72,9 @@ enum {
                                  well-formed bags can overlap; the lookup then pools the shared
                                  IDs in both, the push counts each of them once, for one of the
                                  two bags */
-  MONO_DEV_IMPORT_DUP = 8u    /* mono_import met an ID that was already tracked; skipped */
+  MONO_DEV_IMPORT_DUP = 8u,   /* mono_import met an ID that was already tracked; skipped */
+  MONO_DEV_INTERNAL = 16u     /* only in the checked build (-DMONO_DEBUG): an index the library computed
+                                 for itself fell outside its array; the access was skipped */
 };
 
 enum { MONO_OPT_ADAGRAD = 1 };
@@ -300,13 +302,20 @@ int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const ui
 int mono_expire_slice(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices);
 
 /*
- * Host-buffer forms of the two hot calls, for callers whose batches live in
- * host memory (pinned memory makes the copies asynchronous).  They copy the
- * inputs to library-owned device staging on the table's stream, run the same
- * kernels as the device-pointer forms, and (lookup) copy the result back.
- * mono_lookup_pool_host synchronises the stream before returning so that
- * `out` is readable; mono_apply_grads_host does not synchronise, so the host
- * buffers must stay valid until the stream has passed the copies.
+ * Host-buffer forms of the two hot calls, for callers whose batches live in host memory
+ * (pinned memory makes the copies asynchronous).  Same kernels as the device-pointer forms;
+ * the library copies the inputs into staging buffers of its own and the pooled rows back out,
+ * on two copy streams of the table's own (one per direction), so that the gradients of a step
+ * come in while its pooled rows still go out and both run beside the kernels.
+ *  - Neither call synchronises.  `out` holds the result, and the host input buffers may be
+ *    reused, once the table's stream has passed a mono_fence issued after the calls
+ *    (mono_fence, then synchronise the stream or wait for an event recorded on it).
+ *  - mono_lookup_pool_host stages `ids` and `slot_offsets` on the device and treats the staged
+ *    batch as announced (see mono_prepare_push).  mono_apply_grads_host given the same host
+ *    pointers and sizes as the mono_lookup_pool_host call directly before it reuses that copy
+ *    and that announcement -- the contents must not have changed in between; given anything
+ *    else it copies its own.
+ *  - The two bag-by-dim staging matrices are allocated by the first host-buffer call.
  * All pointers HOST.
  */
 int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids,

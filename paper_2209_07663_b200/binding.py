@@ -12,12 +12,13 @@ import os
 from typing import Optional
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmono.so")
+# MONO_LIBRARY=checked selects the build with device-side index checks (libmono_checked.so, see build.py)
+LIB_PATH = os.path.join(_PKG, "libmono_checked.so" if os.environ.get("MONO_LIBRARY") == "checked" else "libmono.so")
 
 MONO_OK, MONO_ERR_ARG, MONO_ERR_TIME, MONO_ERR_CUDA, MONO_ERR_NOMEM, MONO_ERR_SIZE = 0, -1, -2, -3, -4, -5
 MONO_ERR_LIMIT = -6
 MONO_NOALLOC_MAX_IDS = 1 << 20
-MONO_DEV_ROWS_FULL, MONO_DEV_KEYS_FULL, MONO_DEV_BAD_OFFSETS, MONO_DEV_IMPORT_DUP = 1, 2, 4, 8
+MONO_DEV_ROWS_FULL, MONO_DEV_KEYS_FULL, MONO_DEV_BAD_OFFSETS, MONO_DEV_IMPORT_DUP, MONO_DEV_INTERNAL = 1, 2, 4, 8, 16
 MONO_RESERVED_ID = 0xFFFFFFFFFFFFFFFF
 MONO_MAX_NOW = 0xFFFFFFFE
 

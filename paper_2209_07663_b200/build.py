@@ -9,9 +9,12 @@ import subprocess
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmono.so")
+# the same sources with -DMONO_DEBUG: every index the library computes for itself is range-checked
+# on the device and a bad one reported through the status bits (binding: MONO_LIBRARY=checked)
+LIB_CHECKED = os.path.join(PKG, "libmono_checked.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC", "--cudart", "static"]
+              "-shared", "-Xcompiler", "-fPIC", "--cudart", "static", "-ldl"]
 
 
 def _sources():
@@ -30,19 +33,22 @@ def find_nvcc() -> str:
     return nvcc
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile csrc/*.cu into libmono.so unless it is already up to date."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_input():
-        return LIB
-    tmp = f"{LIB}.{os.getpid()}.tmp"
-    cmd = [find_nvcc(), *NVCC_FLAGS, "-o", tmp, *_sources()]
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile csrc/*.cu into libmono.so (or, with `checked`, into libmono_checked.so) unless it is
+    already up to date."""
+    lib = LIB_CHECKED if checked else LIB
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_input():
+        return lib
+    tmp = f"{lib}.{os.getpid()}.tmp"
+    cmd = [find_nvcc(), *NVCC_FLAGS, *(["-DMONO_DEBUG"] if checked else []), "-o", tmp, *_sources()]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
     print(build(force=True, verbose=True))
+    print(build(force=True, checked=True))

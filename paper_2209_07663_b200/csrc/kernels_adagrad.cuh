@@ -114,9 +114,10 @@ __device__ inline void file_segments_body(const Work& wk, long long n_ids, long 
   for (long long j = (long long)vblock * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
     const uint2 o = wk.occ[j];
     if (o.x == kNoSlot) continue;
+    if (!MONO_INDEX_OK(wk.error_bits, o.x, wk.n_slots)) continue;
     const uint32_t seg = wk.bset[o.x].a;
     const uint32_t bag = wk.occ_bag[j];
-    if (bag < n_bags) wk.bag_of_sorted[seg + o.y] = bag;
+    if (bag < n_bags && MONO_INDEX_OK(wk.error_bits, (unsigned long long)seg + o.y, wk.max_ids)) wk.bag_of_sorted[seg + o.y] = bag;
   }
 }
 __global__ void __launch_bounds__(256)
@@ -151,7 +152,7 @@ __device__ inline void update_singletons_body(const TableView& tv, const Work& w
       BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
       wk.bset[wk.uslot[u]] = e;
       row_word = wk.urow[u];
-      if (row_word != kNoRow) {
+      if (row_word != kNoRow && MONO_INDEX_OK(wk.error_bits, wk.useg[u], wk.max_ids)) {
         bag = wk.bag_of_sorted[wk.useg[u]];
         single = bag < n_bags;
         if (row_word & kFreshBit) id = wk.uid[u];
@@ -230,6 +231,7 @@ __device__ inline void reduce_adagrad_body(const TableView& tv, const Work& wk, 
       const uint32_t row_word = wk.urow[u];
       if (row_word == kNoRow || m > kSegChunk) continue;      // no row: gradient dropped; long: in parts
       const uint32_t begin = wk.useg[u];
+      if (!MONO_INDEX_OK(wk.error_bits, (unsigned long long)begin + m - 1, wk.max_ids)) continue;
       reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, begin + m, s);
       const unsigned long long id = wk.uid[u];
 #pragma unroll
@@ -239,12 +241,15 @@ __device__ inline void reduce_adagrad_body(const TableView& tv, const Work& wk, 
       }
     } else {
       const uint32_t p = wk.part_order[item];
+      if (!MONO_INDEX_OK(wk.error_bits, p, wk.max_parts)) continue;
       const uint32_t li = wk.part_u[p];
+      if (!MONO_INDEX_OK(wk.error_bits, li, wk.max_long)) continue;
       const uint32_t u = wk.long_u[li];
       const uint32_t k = p - wk.long_part0[li];
       const uint32_t seg_end = wk.useg[u] + wk.ulen[u];
       const uint32_t begin = wk.useg[u] + k * kSegChunk;
       const uint32_t end = begin + kSegChunk < seg_end ? begin + kSegChunk : seg_end;
+      if (!MONO_INDEX_OK(wk.error_bits, (unsigned long long)end - 1, wk.max_ids)) continue;
       reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, end, s);
       double* dst = wk.partials + (size_t)p * tv.dim;
 #pragma unroll

@@ -72,6 +72,9 @@ struct Work {
   uint32_t* fold_li;         // [max_folds] owner (index into long_u) of each fold
   uint32_t* fold_idx;        // [max_folds] which group of kFoldWidth parts of that owner
   uint32_t max_long, max_parts, max_folds;
+  uint32_t max_ids;          // entries of the per-occurrence and per-distinct-ID arrays
+  uint32_t n_slots;          // slots of bset, both tiers
+  unsigned int* error_bits;  // the table's sticky condition bits (the checked build reports through them)
 };
 
 // A bag is well formed when 0 <= offsets[b] <= offsets[b+1] <= n_ids; any other bag is
@@ -254,8 +257,10 @@ __device__ inline void dedup_tile_body(const Work& wk, const unsigned long long*
 #pragma unroll
   for (int k = 0; k < kPerThread; ++k) {
     if (is_new[k]) {
-      wk.uid[my_u] = my_id[k];
-      wk.uslot[my_u] = g[k];
+      if (MONO_INDEX_OK(wk.error_bits, my_u, wk.max_ids)) {
+        wk.uid[my_u] = my_id[k];
+        wk.uslot[my_u] = g[k];
+      }
       ++my_u;
     }
   }

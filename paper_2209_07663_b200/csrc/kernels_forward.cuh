@@ -125,8 +125,9 @@ struct GatherSource {
   const uint32_t* occ_row;                 // kFromRows
   const unsigned long long* ids;           // kFromKeys
   const uint2* occ;                        // kFromSet
-  const BatchSlot* bset;                    // kFromSet
+  const BatchSlot* bset;                   // kFromSet
   uint32_t* bag_of_sorted;                 // kFromSet
+  uint32_t n_slots, max_ids;               // kFromSet: sizes of bset and bag_of_sorted (for the checked build)
 };
 
 // Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
@@ -173,10 +174,10 @@ __device__ inline void gather_pool_body(const TableView& tv, const GatherSource&
           if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) mine = meta_row(meta);
         } else {
           const uint2 o = __ldg(src.occ + j);
-          if (o.x != kNoSlot) {
+          if (o.x != kNoSlot && MONO_INDEX_OK(&tv.st->error_bits, o.x, src.n_slots)) {
             const uint4 bs = __ldg(reinterpret_cast<const uint4*>(src.bset + o.x));   // key (x, y), segment start, row
             if (bs.w != kNoRow) mine = bs.w;
-            src.bag_of_sorted[bs.z + o.y] = (uint32_t)bag;
+            if (MONO_INDEX_OK(&tv.st->error_bits, (unsigned long long)bs.z + o.y, src.max_ids)) src.bag_of_sorted[bs.z + o.y] = (uint32_t)bag;
           }
         }
       }

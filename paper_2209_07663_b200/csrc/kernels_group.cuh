@@ -146,6 +146,7 @@ group_gather_pool_kernel(const GroupItem* __restrict__ items, const uint32_t* __
   MONO_GROUP_PROLOGUE;
   GatherSource src{};
   src.ids = it.ids; src.occ = it.wk.occ; src.bset = it.wk.bset; src.bag_of_sorted = it.wk.bag_of_sorted;
+  src.n_slots = it.wk.n_slots; src.max_ids = it.wk.max_ids;
   by_lane_class<WIDE>(it.lane_class, [&](auto g, auto nv) {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     if (it.prepared) gather_pool_body<G, NV, kFromSet>(it.tv, src, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);

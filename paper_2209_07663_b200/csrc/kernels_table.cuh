@@ -88,7 +88,9 @@ __device__ inline Reservation block_reserve(const TableView& tv, BlockAlloc* sh,
   r.ins_pos = sh->ins_base + ((unsigned int)(before >> 42) & 0x3FFu);
   const unsigned int my_row_index = (unsigned int)(before >> 52) & 0x3FFu;
   r.row = kNoRow;
-  if (need_row && my_row_index < sh->rows_granted) r.row = tv.free_rows[sh->row_base - 1 - my_row_index];
+  if (need_row && my_row_index < sh->rows_granted &&
+      MONO_INDEX_OK(&tv.st->error_bits, sh->row_base - 1 - (long long)my_row_index, tv.capacity))
+    r.row = tv.free_rows[sh->row_base - 1 - my_row_index];
   return r;
 }
 
@@ -151,6 +153,7 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
       id = wk.uid[u];
       if (MODE & kLookUp) {
         slot = wk.uslot[u];
+        if (!MONO_INDEX_OK(wk.error_bits, slot, wk.n_slots)) slot = 0;
         m = wk.bset[slot].a;
         cell = thread_locate(tv, id, stash_hw, &meta);
       } else {
@@ -181,7 +184,8 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
       if (!(MODE & kCommit)) wk.ucell[u] = cell;
       BatchSlot bs; bs.key = id; bs.a = rv.seg_start; bs.b = resident ? (low & kRowMask) : kNoRow;
       wk.bset[slot] = bs;
-      if (m > 1) wk.multi_list[rv.multi_pos] = u;
+      (void)MONO_INDEX_OK(wk.error_bits, (unsigned long long)rv.seg_start + m - 1, wk.max_ids);
+      if (m > 1 && MONO_INDEX_OK(wk.error_bits, rv.multi_pos, wk.max_ids / 2 + 1)) wk.multi_list[rv.multi_pos] = u;
     }
     if (MODE & kCommit) {
       if (hit) {
@@ -195,7 +199,7 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
           ++n_res;
           if (m > kSegChunk) register_long(tv, wk, u, m);
         }
-      } else {
+      } else if (MONO_INDEX_OK(wk.error_bits, rv.ins_pos, wk.max_ids)) {
         wk.ins_list[rv.ins_pos] = u;
       }
     }
@@ -405,7 +409,8 @@ __device__ inline void order_parts_body(const TableView& tv, const Work& wk, uin
     const uint32_t li = wk.part_u[p];
     const uint32_t parts = (wk.ulen[wk.long_u[li]] + kSegChunk - 1) / kSegChunk;
     const uint32_t w = part_window(p - wk.long_part0[li], parts);
-    wk.part_order[s_start[w] + atomicAdd(&cursor[w], 1u)] = p;
+    const uint32_t at = s_start[w] + atomicAdd(&cursor[w], 1u);
+    if (MONO_INDEX_OK(wk.error_bits, at, wk.max_parts)) wk.part_order[at] = p;
   }
 }
 __global__ void __launch_bounds__(kWindows)
@@ -473,7 +478,8 @@ __device__ inline void expire_body(const TableView& tv, unsigned long long n_cel
         if (lane == leader)
           pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)__popc(mask));
         pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
-        if (frees_row) tv.free_rows[pos + __popc(mask & ((1u << lane) - 1u))] = row;
+        const unsigned long long at = pos + __popc(mask & ((1u << lane) - 1u));
+        if (frees_row && MONO_INDEX_OK(&tv.st->error_bits, at, tv.capacity)) tv.free_rows[at] = row;
       }
     }
   }

@@ -12,6 +12,7 @@
 #include <vector>
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include "../../include/mono.h"
 #include "kernels_adagrad.cuh"
@@ -92,11 +93,31 @@ struct mono_table {
   // device staging for the host-buffer calls
   unsigned long long* stage_ids = nullptr;
   long long* stage_off = nullptr;
-  float* stage_vec = nullptr;
+  float* stage_out = nullptr;     // pooled rows on their way to the host
+  float* stage_grad = nullptr;    // gradients on their way in
+  // The host-buffer calls copy on two streams of their own, one per direction, so that a step's
+  // gradients come in while its pooled rows still go out (the link is full duplex) and both
+  // run beside the kernels.  ev_staged: the IDs or gradients have arrived; ev_out: the pooled
+  // rows are ready to leave; ev_d2h: they have left; ev_stage_free: the kernels are done with
+  // the staged inputs.
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_staged = nullptr, ev_grad_in = nullptr, ev_out = nullptr, ev_d2h = nullptr, ev_stage_free = nullptr;
+  bool d2h_pending = false;       // a copy to the host is in flight that `stream` has not waited for
+  bool stage_used = false;        // ev_stage_free has been recorded
+  // the host batch whose IDs and offsets are on the device, staged by mono_lookup_pool_host
+  struct { const void* ids; int64_t n_ids; const void* off; int64_t n_bags; bool valid; } staged = {nullptr, 0, nullptr, 0, false};
   std::string last_err;
 };
 
 namespace {
+
+// A named range around every call of the ABI, for timelines taken with a profiler that reads
+// NVTX (a pointer test when none is attached).
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+};
+#define MONO_API_RANGE() ApiRange api_range__(__func__)
 
 #define CUDA_TRY(t, expr)                                                         \
   do {                                                                            \
@@ -126,7 +147,8 @@ void free_scratch(mono_table* t) {
   dev_free(w.bset); dev_free(w.occ); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
   dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow); dev_free(w.ucell);
   dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.part_order); dev_free(w.win_count); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
-  dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_vec); dev_free(t->occ_row);
+  dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_out); dev_free(t->stage_grad); dev_free(t->occ_row);
+  t->staged.valid = false;
   t->max_ids = t->max_bags = 0;
 }
 
@@ -187,6 +209,9 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   if (max_bags < 1024) max_bags = 1024;
   if (t->max_ids > 0) ++t->scratch_reallocs;               // (the first sizing of a table created without one is not a regrowth)
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  if (t->h2d_stream) CUDA_TRY(t, cudaStreamSynchronize(t->h2d_stream));      // copies in flight use the staging buffers
+  if (t->d2h_stream) CUDA_TRY(t, cudaStreamSynchronize(t->d2h_stream));
+  t->d2h_pending = false;
   // a prepared batch is lost with the scratch it lives in
   if (t->prep.valid) { t->prep.valid = false; finish_apply_kernel<<<1, 256, 0, t->stream>>>(t->tv.st, t->wk.win_count, 0); }
   free_scratch(t);
@@ -209,11 +234,15 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   w.max_folds = w.max_parts / kFoldWidth + w.max_long + 1;
   ALLOC(w.fold_li, w.max_folds); ALLOC(w.fold_idx, w.max_folds);
   ALLOC(t->stage_ids, n); ALLOC(t->stage_off, (size_t)max_bags + 1);
-  ALLOC(t->stage_vec, (size_t)max_bags * t->tv.dim);
+  // (the two staging buffers of the host-buffer calls, one bag-by-dim matrix each, are allocated by the
+  // first such call: callers that keep their batches on the device never pay for them)
   ALLOC(t->occ_row, n);
 #undef ALLOC
   w.primary_mask = (uint32_t)(primary - 1);
   w.secondary_mask = (uint32_t)(secondary - 1);
+  w.max_ids = (uint32_t)max_ids;
+  w.n_slots = (uint32_t)slots;
+  w.error_bits = &t->tv.st->error_bits;
   init_bset_kernel<<<grid_for(t, 4), 256, 0, t->stream>>>(w.bset, slots);
   CUDA_TRY(t, cudaGetLastError());
   CUDA_TRY(t, cudaMemsetAsync(w.win_count, 0, 2 * kWindows * sizeof(uint32_t), t->stream));
@@ -269,6 +298,7 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
     // every distinct ID of this batch was looked up when it was announced: the rows come from the
     // per-call set, and the occurrences file their bags for the push on the way
     src.occ = t->wk.occ; src.bset = t->wk.bset; src.bag_of_sorted = t->wk.bag_of_sorted;
+    src.n_slots = t->wk.n_slots; src.max_ids = t->wk.max_ids;
     const int rc = launch_gather<kFromSet>(t, src, n_ids, off, n_bags, out);
     if (rc == MONO_OK) t->prep.filed = true;
     return rc;
@@ -301,8 +331,9 @@ int launch_prepare(mono_table* t, const unsigned long long* ids, int64_t n_ids, 
   return MONO_OK;
 }
 
+// grad_ready: if not null, the gradients are still being copied in; the kernels that read them wait for it
 int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
-                 int64_t n_bags, const float* grad, uint32_t now) {
+                 int64_t n_bags, const float* grad, uint32_t now, cudaEvent_t grad_ready = nullptr) {
   cudaStream_t s = t->stream;
   const TableView& tv = t->tv;
   const Work& wk = t->wk;
@@ -339,6 +370,7 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   LAUNCH_ON(t, a, K_ORDER, order_parts_kernel<<<64, kWindows, 0, a>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
   if (a != s) CUDA_TRY(t, cudaEventRecord(t->ev_parts, a));
+  if (grad_ready) CUDA_TRY(t, cudaStreamWaitEvent(s, grad_ready, 0));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     if (a != s) {
@@ -558,6 +590,7 @@ extern "C" {
 
 int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_t filter_threshold,
                       uint32_t ttl, const mono_opt* opt, void* cuda_stream) {
+  MONO_API_RANGE();
   if (!out) return MONO_ERR_ARG;
   *out = nullptr;
   if (capacity == 0 || capacity > MONO_MAX_CAPACITY) return MONO_ERR_ARG;
@@ -634,10 +667,14 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
 }
 
 int mono_table_destroy(mono_table* t) {
+  MONO_API_RANGE();
   if (!t) return MONO_ERR_ARG;
   cudaStreamSynchronize(t->stream);
   if (t->sweep_stream) { cudaStreamSynchronize(t->sweep_stream); cudaStreamDestroy(t->sweep_stream); }
   if (t->aux_stream) { cudaStreamSynchronize(t->aux_stream); cudaStreamDestroy(t->aux_stream); }
+  if (t->h2d_stream) { cudaStreamSynchronize(t->h2d_stream); cudaStreamDestroy(t->h2d_stream); }
+  if (t->d2h_stream) { cudaStreamSynchronize(t->d2h_stream); cudaStreamDestroy(t->d2h_stream); }
+  for (cudaEvent_t e : {t->ev_staged, t->ev_grad_in, t->ev_out, t->ev_d2h, t->ev_stage_free}) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : {t->ev_fork, t->ev_keys, t->ev_swept, t->ev_group, t->ev_parts, t->ev_reduced, t->ev_aux})
     if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
@@ -651,6 +688,7 @@ int mono_table_destroy(mono_table* t) {
 }
 
 int mono_reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || max_ids < 0 || max_bags < 0 || max_ids >= (1ll << 31) || max_bags >= (1ll << 31)) return MONO_ERR_ARG;
   return reserve(t, max_ids, max_bags);
@@ -658,6 +696,7 @@ int mono_reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
 
 int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                      int64_t n_bags, float* out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
@@ -670,6 +709,7 @@ int mono_lookup_pool(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
 
 int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                      int64_t n_bags, const float* grad_pooled, int64_t now) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
@@ -682,6 +722,7 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
 }
 
 int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets, int64_t n_bags) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);                                    // the look-ups read the key store
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
@@ -697,6 +738,7 @@ int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const i
 int mono_group_prepare_push(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
                             const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
                             void* group_stream) {
+  MONO_API_RANGE();
   int rc = group_check(n_tables, tables);
   if (rc != MONO_OK) return rc;
   if (n_tables == 0) return MONO_OK;
@@ -724,6 +766,7 @@ int mono_group_prepare_push(int32_t n_tables, mono_table* const* tables, const u
 int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
                            float* const* out, void* group_stream) {
+  MONO_API_RANGE();
   int rc = group_check(n_tables, tables);
   if (rc != MONO_OK) return rc;
   if (n_tables == 0) return MONO_OK;
@@ -754,6 +797,7 @@ int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const ui
 int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const uint64_t* const* ids,
                            const int64_t* n_ids, const int64_t* const* slot_offsets, const int64_t* n_bags,
                            const float* const* grad_pooled, int64_t now, void* group_stream) {
+  MONO_API_RANGE();
   int rc = group_check(n_tables, tables);
   if (rc != MONO_OK) return rc;
   if (n_tables == 0) return MONO_OK;
@@ -848,9 +892,13 @@ static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_s
   return MONO_OK;
 }
 
-int mono_expire(mono_table* t, int64_t now) { return expire_range(t, now, 0, 1); }
+int mono_expire(mono_table* t, int64_t now) {
+  MONO_API_RANGE();
+  return expire_range(t, now, 0, 1);
+}
 
 int mono_expire_slice(mono_table* t, int64_t now, uint32_t slice, uint32_t n_slices) {
+  MONO_API_RANGE();
   if (n_slices > 65536) return MONO_ERR_ARG;
   return expire_range(t, now, slice, n_slices);
 }
@@ -875,6 +923,7 @@ static int noalloc_scratch(mono_table* t, uint32_t** out) {
 
 int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                              int64_t n_bags, float* out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
@@ -899,47 +948,121 @@ int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, 
   return launch_gather<kFromRows>(t, src, n_ids, d_off, n_bags, out);
 }
 
+// Streams, events and staging of the host-buffer calls, made by the first of them.
+static int host_path_ready(mono_table* t, int64_t n_bags) {
+  if (!t->h2d_stream) {
+    CUDA_TRY(t, cudaStreamCreateWithFlags(&t->h2d_stream, cudaStreamNonBlocking));
+    CUDA_TRY(t, cudaStreamCreateWithFlags(&t->d2h_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t* e : {&t->ev_staged, &t->ev_grad_in, &t->ev_out, &t->ev_d2h, &t->ev_stage_free})
+      CUDA_TRY(t, cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+  }
+  if (!t->stage_out) {                                     // sized with the rest of the scratch: max_bags rows
+    (void)n_bags;
+    int rc = dev_alloc(t, &t->stage_out, (size_t)t->max_bags * t->tv.dim);
+    if (rc == MONO_OK) rc = dev_alloc(t, &t->stage_grad, (size_t)t->max_bags * t->tv.dim);
+    if (rc != MONO_OK) { dev_free(t->stage_out); dev_free(t->stage_grad); return rc; }
+  }
+  return MONO_OK;
+}
+
+// IDs and offsets of a host batch to the staging buffers, on the inbound copy stream, once the
+// kernels of the previous step are done with what is there.
+static int stage_batch(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* off, int64_t n_bags) {
+  cudaStream_t c = t->h2d_stream;
+  if (t->stage_used) CUDA_TRY(t, cudaStreamWaitEvent(c, t->ev_stage_free, 0));
+  if (n_ids) CUDA_TRY(t, cudaMemcpyAsync(t->stage_ids, ids, (size_t)n_ids * 8, cudaMemcpyHostToDevice, c));
+  CUDA_TRY(t, cudaMemcpyAsync(t->stage_off, off, (size_t)(n_bags + 1) * 8, cudaMemcpyHostToDevice, c));
+  CUDA_TRY(t, cudaEventRecord(t->ev_staged, c));
+  CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_staged, 0));
+  return MONO_OK;
+}
+
 int mono_lookup_pool_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                           int64_t n_bags, float* out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && !out) return MONO_ERR_ARG;
   if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  if ((rc = host_path_ready(t, n_bags)) != MONO_OK) return rc;
+  if ((rc = discard_prepared(t)) != MONO_OK) return rc;
+  t->staged.valid = false;
   cudaStream_t s = t->stream;
-  if (n_ids) CUDA_TRY(t, cudaMemcpyAsync(t->stage_ids, ids, (size_t)n_ids * 8, cudaMemcpyHostToDevice, s));
-  CUDA_TRY(t, cudaMemcpyAsync(t->stage_off, slot_offsets, (size_t)(n_bags + 1) * 8, cudaMemcpyHostToDevice, s));
-  if ((rc = launch_lookup(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec, false)) != MONO_OK) return rc;
-  if (n_bags)
-    CUDA_TRY(t, cudaMemcpyAsync(out, t->stage_vec, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyDeviceToHost, s));
-  CUDA_TRY(t, cudaStreamSynchronize(s));
+  // the staging buffers must be free: the kernels that read the last staged batch have been issued on `s`
+  CUDA_TRY(t, cudaEventRecord(t->ev_stage_free, s));
+  t->stage_used = true;
+  if ((rc = stage_batch(t, ids, n_ids, slot_offsets, n_bags)) != MONO_OK) return rc;
+  if (n_bags == 0) return MONO_OK;
+  // the staged batch is the one the push that follows will be given: group it and look its IDs up once for both
+  bool prepared = false;
+  if (n_ids > 0) {
+    if ((rc = launch_prepare(t, t->stage_ids, n_ids, t->stage_off, n_bags)) != MONO_OK) return rc;
+    t->prep = {t->stage_ids, n_ids, t->stage_off, n_bags, true, false};
+    t->staged = {ids, n_ids, slot_offsets, n_bags, true};
+    prepared = true;
+  }
+  // the previous result must have left stage_out before this one is written there
+  if (t->d2h_pending) { CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_d2h, 0)); t->d2h_pending = false; }
+  if ((rc = launch_lookup(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_out, prepared)) != MONO_OK) return rc;
+  CUDA_TRY(t, cudaEventRecord(t->ev_out, s));
+  CUDA_TRY(t, cudaStreamWaitEvent(t->d2h_stream, t->ev_out, 0));
+  CUDA_TRY(t, cudaMemcpyAsync(out, t->stage_out, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyDeviceToHost, t->d2h_stream));
+  CUDA_TRY(t, cudaEventRecord(t->ev_d2h, t->d2h_stream));
+  t->d2h_pending = true;
   return MONO_OK;
 }
 
 int mono_apply_grads_host(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
                           int64_t n_bags, const float* grad_pooled, int64_t now) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
   if (rc != MONO_OK) return rc;
   if (n_bags > 0 && !grad_pooled) return MONO_ERR_ARG;
   if ((rc = check_now(t, now)) != MONO_OK) return rc;
   if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  if ((rc = host_path_ready(t, n_bags)) != MONO_OK) return rc;
   cudaStream_t s = t->stream;
-  if (n_ids) CUDA_TRY(t, cudaMemcpyAsync(t->stage_ids, ids, (size_t)n_ids * 8, cudaMemcpyHostToDevice, s));
-  CUDA_TRY(t, cudaMemcpyAsync(t->stage_off, slot_offsets, (size_t)(n_bags + 1) * 8, cudaMemcpyHostToDevice, s));
-  if (n_bags)
-    CUDA_TRY(t, cudaMemcpyAsync(t->stage_vec, grad_pooled, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyHostToDevice, s));
+  const bool reuse = t->staged.valid && t->staged.ids == ids && t->staged.n_ids == n_ids && t->staged.off == slot_offsets &&
+                     t->staged.n_bags == n_bags;
+  t->staged.valid = false;
+  if (!reuse) {
+    // not the batch the lookup staged: bring its IDs and offsets in now (what was announced from the
+    // staging buffers is about to be overwritten)
+    if ((rc = discard_prepared(t)) != MONO_OK) return rc;
+    CUDA_TRY(t, cudaEventRecord(t->ev_stage_free, s));
+    t->stage_used = true;
+    if ((rc = stage_batch(t, ids, n_ids, slot_offsets, n_bags)) != MONO_OK) return rc;
+  }
+  // the gradients come in on the copy stream while the ID-only kernels of the push run (the previous
+  // push, the last reader of stage_grad, was issued before ev_stage_free was last recorded)
+  cudaEvent_t grad_ready = nullptr;
+  if (n_bags) {
+    cudaStream_t c = t->h2d_stream;
+    if (t->stage_used) CUDA_TRY(t, cudaStreamWaitEvent(c, t->ev_stage_free, 0));
+    CUDA_TRY(t, cudaMemcpyAsync(t->stage_grad, grad_pooled, (size_t)n_bags * t->tv.dim * 4, cudaMemcpyHostToDevice, c));
+    CUDA_TRY(t, cudaEventRecord(t->ev_grad_in, c));
+    grad_ready = t->ev_grad_in;
+  }
   t->last_now = now;
-  return launch_apply(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_vec, (uint32_t)now);
+  rc = launch_apply(t, t->stage_ids, n_ids, t->stage_off, n_bags, t->stage_grad, (uint32_t)now, grad_ready);
+  if (rc != MONO_OK) return rc;
+  // (an empty batch launches nothing, so nothing has waited for the gradient copy yet)
+  if (grad_ready && (n_ids == 0 || n_bags == 0)) CUDA_TRY(t, cudaStreamWaitEvent(s, grad_ready, 0));
+  return MONO_OK;
 }
 
 int mono_fence(mono_table* t) {
+  MONO_API_RANGE();
   if (!t) return MONO_ERR_ARG;
   join_sweep(t);
+  if (t->d2h_pending) { CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_d2h, 0)); t->d2h_pending = false; }
   return MONO_OK;
 }
 
 int mono_snapshot_save(mono_table* t) {
+  MONO_API_RANGE();
   if (!t) return MONO_ERR_ARG;
   join_sweep(t);
   auto& sn = t->snap;
@@ -973,6 +1096,7 @@ int mono_snapshot_save(mono_table* t) {
 }
 
 int mono_snapshot_restore(mono_table* t) {
+  MONO_API_RANGE();
   if (!t) return MONO_ERR_ARG;
   join_sweep(t);
   auto& sn = t->snap;
@@ -996,6 +1120,7 @@ int mono_snapshot_restore(mono_table* t) {
 }
 
 int mono_snapshot_drop(mono_table* t) {
+  MONO_API_RANGE();
   if (!t) return MONO_ERR_ARG;
   join_sweep(t);
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
@@ -1004,6 +1129,7 @@ int mono_snapshot_drop(mono_table* t) {
 }
 
 int mono_status(mono_table* t, mono_status_t* host_out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   DevState d;
@@ -1034,6 +1160,7 @@ int mono_status(mono_table* t, mono_status_t* host_out) {
 }
 
 int mono_clear_errors(mono_table* t) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->error_bits, 0, sizeof(unsigned int), t->stream));
@@ -1043,6 +1170,7 @@ int mono_clear_errors(mono_table* t) {
 
 int mono_probe(mono_table* t, const uint64_t* ids, int64_t n, uint8_t* resident, uint32_t* count,
                int64_t* last_seen) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || n < 0 || (n > 0 && (!ids || !aligned(ids, 8)))) return MONO_ERR_ARG;
   if (n > 0) {
@@ -1055,6 +1183,7 @@ int mono_probe(mono_table* t, const uint64_t* ids, int64_t n, uint8_t* resident,
 }
 
 int mono_read_rows(mono_table* t, const uint64_t* ids, int64_t n, float* w, float* acc) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || n < 0 || (n > 0 && (!ids || !aligned(ids, 8)))) return MONO_ERR_ARG;
   if ((w && !aligned(w, 16)) || (acc && !aligned(acc, 16))) return MONO_ERR_ARG;
@@ -1069,6 +1198,7 @@ int mono_read_rows(mono_table* t, const uint64_t* ids, int64_t n, float* w, floa
 
 int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_seen, uint8_t* resident,
                 float* w, float* acc, int64_t max_n, int64_t* n_out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || !n_out || max_n < 0 || (max_n > 0 && !ids)) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaMemsetAsync(&t->tv.st->export_n, 0, sizeof(unsigned long long), t->stream));
@@ -1084,6 +1214,7 @@ int mono_export(mono_table* t, uint64_t* ids, uint32_t* count, int64_t* last_see
 }
 
 int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t) return MONO_ERR_ARG;
   if (new_key_cells == 0) new_key_cells = t->key_cells;
@@ -1123,6 +1254,7 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
 }
 
 int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, int64_t* n_out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || !n_out || max_n < 0 || (max_n > 0 && (!ids || !w || !aligned(w, 16) || !aligned(ids, 8)))) return MONO_ERR_ARG;
   { const int rc0 = discard_prepared(t); if (rc0 != MONO_OK) return rc0; }
@@ -1139,6 +1271,7 @@ int mono_export_touched(mono_table* t, uint64_t* ids, float* w, int64_t max_n, i
 
 int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const int64_t* last_seen,
                 const uint8_t* resident, const float* w, const float* acc, int64_t n) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || n < 0) return MONO_ERR_ARG;
   if (n == 0) return MONO_OK;
@@ -1170,6 +1303,7 @@ int mono_import(mono_table* t, const uint64_t* ids, const uint32_t* count, const
 }
 
 int mono_audit(mono_table* t, mono_audit_t* host_out) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   std::memset(host_out, 0, sizeof(*host_out));
@@ -1223,6 +1357,7 @@ int mono_timing_enable(mono_table* t, int on) {
 }
 
 int mono_timing_read(mono_table* t, mono_timing_t* host_out, int reset) {
+  MONO_API_RANGE();
   if (t) join_sweep(t);
   if (!t || !host_out) return MONO_ERR_ARG;
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));

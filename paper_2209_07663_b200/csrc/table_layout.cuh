@@ -110,6 +110,19 @@ struct DevState {
   unsigned long long export_n;
 };
 
+// Checked build (-DMONO_DEBUG): every index the library computes for itself -- a segment
+// position, a place in one of the per-call lists, a slot of the per-call set, a position of
+// the free-row stack -- is tested against the size of its array before it is used; one that
+// falls outside sets the sticky MONO_DEV_INTERNAL bit and the access is skipped.  The release
+// build compiles the tests away.  (Indices that come from the caller, the bag offsets, are
+// checked in every build.)
+#ifdef MONO_DEBUG
+#define MONO_INDEX_OK(error_bits, i, n) \
+  ((unsigned long long)(i) < (unsigned long long)(n) ? true : (atomicOr((error_bits), 16u /* MONO_DEV_INTERNAL */), false))
+#else
+#define MONO_INDEX_OK(error_bits, i, n) true
+#endif
+
 // Everything a kernel needs to know about a table; passed by value.
 struct TableView {
   Cell* cells;                 // [n_buckets * 4]

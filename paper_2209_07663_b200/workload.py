@@ -135,6 +135,13 @@ CONFIGS = {
                     n_examples=16384, n_slots=50, bag_len=("geometric", 5.0, 1, 20),
                     zipf_s=1.2, n_distinct=1 << 30, steps=400, key_cells=1 << 29,
                     drift_period=50, drift_new_frac=0.30),
+    # the same stream on a table sized for it: the drift stream keeps about 5.4e6 rows and 2.9e7 tracked IDs
+    # alive within its TTL, so this row store and key store run at load 0.85-0.9, where cuckoo
+    # insertions displace other keys (on the 2^26-row table above they never have to)
+    "drift_dense": Config("drift_dense", capacity=6_200_000, dim=32, filter_threshold=3, ttl=200,
+                          n_examples=16384, n_slots=50, bag_len=("geometric", 5.0, 1, 20),
+                          zipf_s=1.2, n_distinct=1 << 30, steps=400, key_cells=1 << 25,
+                          drift_period=50, drift_new_frac=0.30),
 }
 
 # Mixed-dim multi-table configuration: 8 tables, 120 feature slots spread over them so that

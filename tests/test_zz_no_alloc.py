@@ -59,3 +59,28 @@ def test_noalloc_lookup_refuses_batches_beyond_its_fixed_scratch():
     mb.mono_lookup_pool_noalloc(t.handle, ids, n - 1, torch.tensor([0, n - 1], dtype=torch.int64, device="cuda"), 1, out)
     torch.cuda.synchronize()
     assert out.abs().sum().item() == 0          # ID 0 has no row
+
+
+def test_noalloc_lookup_on_a_table_that_never_sized_its_own_scratch():
+    """A table filled through mono_import only, created without max_ids: no call has sized the
+    table's own scratch yet, and the no-alloc lookup, called first, must not need it."""
+    dim, n = 16, 3000
+    rng = np.random.default_rng(4)
+    ids = wl.splitmix64(np.arange(1, n + 1, dtype=np.uint64))
+    w = rng.standard_normal((n, dim)).astype(np.float32)
+    t = mb.MonoTable(1 << 12, dim, 1, 0, key_cells=1 << 14)
+    t.import_entries(ids, np.ones(n, np.uint32), np.zeros(n, np.int64), np.ones(n, np.uint8), w, np.zeros_like(w))
+    assert t.status()["scratch_reallocs"] == 0
+    lists = [rng.choice(n, rng.integers(0, 7), replace=False) for _ in range(500)]
+    off = np.zeros(len(lists) + 1, np.int64)
+    off[1:] = np.cumsum([len(x) for x in lists])
+    flat = np.concatenate(lists).astype(np.int64)
+    want = np.stack([w[x].astype(np.float64).sum(axis=0) if len(x) else np.zeros(dim) for x in lists]).astype(np.float32)
+    d_ids = torch.from_numpy(ids[flat].view(np.int64)).cuda()
+    d_off = torch.from_numpy(off).cuda()
+    got = torch.full((len(lists), dim), float("nan"), device="cuda")
+    mb.mono_lookup_pool_noalloc(t.handle, d_ids, d_ids.numel(), d_off, len(lists), got)
+    torch.cuda.synchronize()
+    assert_vectors_close(got.cpu().numpy(), want, "no-alloc lookup on an imported table")
+    st = t.status()
+    assert st["error_bits"] == 0 and st["scratch_reallocs"] == 0
