@@ -67,6 +67,7 @@ KERNEL_SOURCES = {
     "update_singletons": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "file_segments": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "reduce_adagrad": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
+    "reduce_parts": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "combine_adagrad": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
     "fold_partials": ("kernels_adagrad.cuh", "kernels_dedup.cuh", "table_layout.cuh"),
 }
@@ -296,8 +297,10 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
         "table_insert": (16 + 8 * d) * unew,                 # key write + row/accumulator initialisation
         "sketch_add": 0,                                     # (probabilistic filter: counted with table_insert's new IDs)
         "update_singletons": 20 * d * ur1,                   # IDs seen once: gradient row, row and accumulator in and out
-        "reduce_adagrad": 16 * d * (ur - ur1) + 4 * d * max(b - ur1, 0),   # rows of repeated IDs + the other gradient rows, once
-        "file_segments": 0,
+        # rows of repeated IDs + the gradient rows the singletons did not read, once (the two launches of
+        # reduce_adagrad_kernel, short segments and the parts of long ones, share them; counted on the first)
+        "reduce_adagrad": 16 * d * (ur - ur1) + 4 * d * max(b - ur1, 0), "reduce_parts": 0,
+        "file_segments": 0, "clear_set": 0,
         "expand_parts": 0, "order_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
         "expire": 16 * sweep_cells,                          # one streaming read of the swept cells
     }
@@ -306,9 +309,9 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
 
 KERNEL_GROUP = {
     "probe_rows": "lookup_pool", "gather_pool": "lookup_pool",
-    "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup",
+    "fill_occ_bag": "dedup", "dedup_tile": "dedup", "finish_apply": "dedup", "clear_set": "dedup",
     "table_lookup": "table", "table_update": "table", "sketch_add": "table", "table_insert": "table", "expand_parts": "table", "order_parts": "table",
-    "update_singletons": "adagrad", "file_segments": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
+    "update_singletons": "adagrad", "file_segments": "lookup_pool", "reduce_parts": "adagrad", "reduce_adagrad": "adagrad", "fold_partials": "adagrad",
     "combine_adagrad": "adagrad", "expire": "expire",
 }
 
@@ -529,7 +532,12 @@ def run_ours(args):
             g = KERNEL_GROUP[name]
             group_ms[g] = group_ms.get(g, 0.0) + v["ms_per_launch"]
             group_bytes[g] = group_bytes.get(g, 0) + alg_kernel[name]
-        # the kernel that takes the most device time
+        # the kernel that takes the most device time (reduce_adagrad_kernel is launched twice per step, for the
+        # short segments and for the parts of the long ones: its time is the two launches together)
+        if "reduce_parts" in per_kernel and "reduce_adagrad" in per_kernel:
+            per_kernel["reduce_adagrad"]["ms_short_segments"] = per_kernel["reduce_adagrad"]["ms_per_launch"]
+            per_kernel["reduce_adagrad"]["ms_parts"] = per_kernel["reduce_parts"]["ms_per_launch"]
+            per_kernel["reduce_adagrad"]["ms_per_launch"] += per_kernel.pop("reduce_parts")["ms_per_launch"]
         dom = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_launch"])
         dom_bytes, dom_ms = alg_kernel[dom], per_kernel[dom]["ms_per_launch"]
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
@@ -585,6 +593,8 @@ def run_ours(args):
                                    for k, v in per_kernel.items()},
                 "frac_by_phase": {g: round(group_bytes[g] / (group_ms[g] * 1e-3) / 1e9 / peak, 3) for g in group_ms},
                 "ms_by_kernel": {k: round(v["ms_per_launch"], 4) for k, v in per_kernel.items()},
+                "reduce_adagrad_ms": {"short_segments": per_kernel.get("reduce_adagrad", {}).get("ms_short_segments"),
+                                      "parts": per_kernel.get("reduce_adagrad", {}).get("ms_parts")},
                 "expire_ms_per_launch": (tim["kernels"]["expire"]["ms"] / tim["kernels"]["expire"]["launches"]
                                          if tim["kernels"]["expire"]["launches"] else None),
             },

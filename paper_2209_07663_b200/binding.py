@@ -12,8 +12,11 @@ import os
 from typing import Optional
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-# MONO_LIBRARY=checked selects the build with device-side index checks (libmono_checked.so, see build.py)
-LIB_PATH = os.path.join(_PKG, "libmono_checked.so" if os.environ.get("MONO_LIBRARY") == "checked" else "libmono.so")
+# MONO_LIBRARY=checked selects the build with device-side index checks (libmono_checked.so, see build.py);
+# any other value is taken as the path of a build of the library
+_WHICH = os.environ.get("MONO_LIBRARY", "")
+LIB_PATH = (os.path.join(_PKG, "libmono_checked.so") if _WHICH == "checked" else
+            os.path.abspath(_WHICH) if _WHICH else os.path.join(_PKG, "libmono.so"))
 
 MONO_OK, MONO_ERR_ARG, MONO_ERR_TIME, MONO_ERR_CUDA, MONO_ERR_NOMEM, MONO_ERR_SIZE = 0, -1, -2, -3, -4, -5
 MONO_ERR_LIMIT = -6

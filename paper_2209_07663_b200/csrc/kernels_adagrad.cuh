@@ -5,9 +5,9 @@
 // paper.
 //
 // Three cases, by how often the ID occurs in the batch:
-// Every ID has a segment of bag_of_sorted[] that lists the bags of its
-// occurrences (filed by the lookup when the batch was announced, else by
-// file_segments_kernel).
+// Every repeated ID has a segment of bag_of_sorted[] that lists the bags of its
+// occurrences (filed by file_segments_kernel: inside the lookup when the batch was
+// announced, else inside the push).
 //  - once (most distinct IDs of a long-tailed batch): its gradient is the
 //    pooled gradient of its one bag, so update_singletons_kernel updates the
 //    row straight from that bag's gradient row;
@@ -60,6 +60,26 @@ __device__ inline void update_row(const TableView& tv, uint32_t row_word, unsign
   *pa = a;
 }
 
+// The per-call set must be empty again when the push ends.  Its primary tier is wiped as a whole
+// (clear_primary_kernel: a streaming write costs less than one scattered store per ID); an ID
+// that overflowed into the secondary tier, which is far larger and almost empty, has its slot
+// emptied by the kernel that updates its row.
+__device__ inline void clear_overflow_slot(const Work& wk, uint32_t slot) {
+  if (slot > wk.primary_mask) {
+    BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
+    wk.bset[slot] = e;
+  }
+}
+
+__device__ inline void clear_primary_body(const Work& wk, uint32_t vblock, uint32_t vgrid) {
+  const uint32_t n = wk.primary_mask + 1u;
+  ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+  for (uint32_t i = vblock * blockDim.x + threadIdx.x; i < n; i += vgrid * blockDim.x)
+    *reinterpret_cast<ulonglong2*>(wk.bset + i) = e;
+}
+__global__ void __launch_bounds__(256)
+clear_primary_kernel(Work wk) { clear_primary_body(wk, blockIdx.x, gridDim.x); }
+
 // Sum of grad rows of bags bag_of_sorted[begin .. end) for the NV column
 // vectors this lane owns.  Eight independent row loads in flight per step.
 template <int G, int NV>
@@ -106,23 +126,31 @@ __device__ inline void reduce_segment(const Work& wk, const float* __restrict__ 
   }
 }
 
-// Every occurrence is filed under its ID: its bag goes into the ID's segment of
-// bag_of_sorted[], at the occurrence's rank.  Only for a push whose batch did not pass
-// through the lookup after mono_prepare_push (the lookup files the bags while it pools).
-__device__ inline void file_segments_body(const Work& wk, long long n_ids, long long n_bags, uint32_t vblock, uint32_t vgrid) {
+// One pass over the occurrences once the distinct IDs have been looked up: every
+// occurrence of a repeated ID reads its ID's slot of the per-call set and is filed under
+// its ID -- its bag goes into the ID's segment of bag_of_sorted[], at the occurrence's rank -- and, when
+// occ_row is given (the lookup of a batch that was announced), leaves there the row its ID
+// owns, or the table's all-zero row, for the pooling kernel.
+__device__ inline void file_segments_body(const Work& wk, long long n_ids, long long n_bags, uint32_t* __restrict__ occ_row,
+                                          uint32_t zero_row, uint32_t vblock, uint32_t vgrid) {
   const long long stride = (long long)vgrid * blockDim.x;
   for (long long j = (long long)vblock * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
     const uint2 o = wk.occ[j];
-    if (o.x == kNoSlot) continue;
-    if (!MONO_INDEX_OK(wk.error_bits, o.x, wk.n_slots)) continue;
-    const uint32_t seg = wk.bset[o.x].a;
-    const uint32_t bag = wk.occ_bag[j];
-    if (bag < n_bags && MONO_INDEX_OK(wk.error_bits, (unsigned long long)seg + o.y, wk.max_ids)) wk.bag_of_sorted[seg + o.y] = bag;
+    uint32_t row = zero_row;
+    if (o.x != kNoSlot && MONO_INDEX_OK(wk.error_bits, o.x, wk.n_slots)) {
+      const uint4 bs = __ldg(reinterpret_cast<const uint4*>(wk.bset + o.x));     // key (x, y), segment start, row
+      if (bs.w != kNoRow) row = bs.w;
+      if (bs.z != kNoSegment) {                                                   // (an ID that occurs once has no segment)
+        const uint32_t bag = wk.occ_bag[j];
+        if (bag < n_bags && MONO_INDEX_OK(wk.error_bits, (unsigned long long)bs.z + o.y, wk.max_ids)) wk.bag_of_sorted[bs.z + o.y] = bag;
+      }
+    }
+    if (occ_row) occ_row[j] = row;
   }
 }
 __global__ void __launch_bounds__(256)
-file_segments_kernel(Work wk, long long n_ids, long long n_bags) {
-  file_segments_body(wk, n_ids, n_bags, blockIdx.x, gridDim.x);
+file_segments_kernel(Work wk, long long n_ids, long long n_bags, uint32_t* __restrict__ occ_row, uint32_t zero_row) {
+  file_segments_body(wk, n_ids, n_bags, occ_row, zero_row, blockIdx.x, gridDim.x);
 }
 
 // The IDs that occur once in the batch (most distinct IDs of a long-tailed batch): the
@@ -131,8 +159,7 @@ file_segments_kernel(Work wk, long long n_ids, long long n_bags) {
 // the order the batch first shows them, so the gradient rows are read roughly in order;
 // the lanes whose ID occurs once and has a row are served in turn by lane groups of G,
 // which read the bag's gradient row, the table row and its accumulator, and write both
-// back updated.  The ID's slot of the per-call set is emptied on the way (every
-// occurrence has been filed by now).
+// back updated.
 template <int G, int NV>
 __device__ inline void update_singletons_body(const TableView& tv, const Work& wk, const float* __restrict__ grad,
                                               long long n_bags, uint32_t vblock, uint32_t vgrid) {
@@ -149,14 +176,14 @@ __device__ inline void update_singletons_body(const TableView& tv, const Work& w
     unsigned long long id = 0;
     bool single = false;
     if (u < n && wk.ulen[u] == 1u) {
-      BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
-      wk.bset[wk.uslot[u]] = e;
+      const uint32_t slot = wk.uslot[u];
       row_word = wk.urow[u];
-      if (row_word != kNoRow && MONO_INDEX_OK(wk.error_bits, wk.useg[u], wk.max_ids)) {
-        bag = wk.bag_of_sorted[wk.useg[u]];
+      if (row_word != kNoRow && MONO_INDEX_OK(wk.error_bits, wk.uocc[u], wk.max_ids)) {
+        bag = wk.occ_bag[wk.uocc[u]];
         single = bag < n_bags;
         if (row_word & kFreshBit) id = wk.uid[u];
       }
+      clear_overflow_slot(wk, slot);                     // (after the loads: a store in between would hold them back)
     }
     unsigned todo = __ballot_sync(0xFFFFFFFFu, single);
     n_single += __popc(todo);
@@ -217,28 +244,31 @@ __device__ inline void reduce_adagrad_body(const TableView& tv, const Work& wk, 
   const uint32_t n_items = (which & kReduceShort) ? n + n_parts : n_parts;
   const int gl = threadIdx.x % G;
   const uint32_t groups = (vgrid * blockDim.x) / G;
+  uint4 next_rec = make_uint4(0u, 0u, 0u, 0u);
+  bool have_next = false;
   for (uint32_t item = first_item + (vblock * blockDim.x + threadIdx.x) / G; item < n_items; item += groups) {
     D4 s[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) s[v] = D4{0.0, 0.0, 0.0, 0.0};
     if (item >= n_parts) {
-      const uint32_t u = wk.multi_list[item - n_parts];
-      if (gl == 0) {
-        BatchSlot e; e.key = kEmptyKey; e.a = 0; e.b = 0;
-        wk.bset[wk.uslot[u]] = e;
-      }
-      const uint32_t m = wk.ulen[u];
+      // everything the reduction needs to know about the ID comes in one record; the record of the
+      // group's next item is requested now, so that it is there when this item is done
+      const uint4 rec = have_next ? next_rec : __ldg(wk.multi_list + (item - n_parts));
+      have_next = item + groups < n_items;
+      if (have_next) next_rec = __ldg(wk.multi_list + (item + groups - n_parts));
+      const uint32_t u = rec.x, m = rec.y, begin = rec.z;
       const uint32_t row_word = wk.urow[u];
-      if (row_word == kNoRow || m > kSegChunk) continue;      // no row: gradient dropped; long: in parts
-      const uint32_t begin = wk.useg[u];
-      if (!MONO_INDEX_OK(wk.error_bits, (unsigned long long)begin + m - 1, wk.max_ids)) continue;
-      reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, begin + m, s);
-      const unsigned long long id = wk.uid[u];
+      if (row_word != kNoRow && m <= kSegChunk &&                  // no row: gradient dropped; long: in parts
+          MONO_INDEX_OK(wk.error_bits, (unsigned long long)begin + m - 1, wk.max_ids)) {
+        reduce_segment<G, NV>(wk, grad, n_bags, tv.dim, gl, begin, begin + m, s);
+        const unsigned long long id = (row_word & kFreshBit) ? wk.uid[u] : 0ull;
 #pragma unroll
-      for (int v = 0; v < NV; ++v) {
-        const uint32_t c4 = gl + v * G;
-        if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
+        for (int v = 0; v < NV; ++v) {
+          const uint32_t c4 = gl + v * G;
+          if (c4 * 4u < tv.dim) update_row(tv, row_word, id, c4, s[v]);
+        }
       }
+      if (gl == 0) clear_overflow_slot(wk, rec.w);
     } else {
       const uint32_t p = wk.part_order[item];
       if (!MONO_INDEX_OK(wk.error_bits, p, wk.max_parts)) continue;

@@ -23,7 +23,8 @@ namespace mono {
 // One slot of the per-call set.  `a` is the ID's multiplicity while the batch
 // is being counted.  Once the distinct IDs have been looked up in the key store
 // (table_update_kernel), `a` is the start of the ID's segment in bag_of_sorted[]
-// and `b` the row the ID owned before this push (kNoRow if none): what an
+// (kNoSegment for an ID that occurs once: its bag is found through uocc[]) and
+// `b` the row the ID owned before this push (kNoRow if none): what an
 // occurrence needs to pool the row and to file its bag.  The kernels that
 // update the rows empty the slots again for the next call.
 struct __align__(16) BatchSlot {
@@ -33,6 +34,7 @@ struct __align__(16) BatchSlot {
 };
 
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
+constexpr uint32_t kNoSegment = 0xFFFFFFFFu;
 constexpr uint32_t kSegChunk = 64;             // longest segment one lane group reduces alone
 constexpr uint32_t kFoldWidth = 64;           // parts added up by one block of fold_partials_kernel
 constexpr int kTileIds = 512;                  // occurrences per block of dedup_tile_kernel
@@ -53,16 +55,19 @@ struct Work {
   uint2* occ;                // [max_ids] per occurrence: x = slot of its ID (kNoSlot if padding / outside bags),
                              //           y = rank of the occurrence among those of its ID
   uint32_t* occ_bag;         // [max_ids] bag of each occurrence
-  uint32_t* bag_of_sorted;   // [max_ids] bags of the occurrences, grouped by ID (an ID seen once has a segment of one)
+  uint32_t* bag_of_sorted;   // [max_ids] bags of the occurrences of repeated IDs, grouped by ID
   unsigned long long* uid;   // [max_ids] distinct IDs
   uint32_t* uslot;           // [max_ids] slot of each distinct ID
+  uint32_t* uocc;            // [max_ids] one occurrence of each distinct ID (the occurrence, if there is only one)
   uint32_t* useg;            // [max_ids] start of the ID's segment in bag_of_sorted
   uint32_t* ulen;            // [max_ids] multiplicity of the ID in this batch
   uint32_t* urow;            // [max_ids] row word per distinct ID (kNoRow / row | kFreshBit)
-  unsigned long long* ucell; // [max_ids] where the key store holds the ID (kNoCell: nowhere), from the look-up
-                             //           that mono_prepare_push does ahead of the push
+  unsigned long long* ucell; // [max_ids] where the key store holds the ID (kNoCell: nowhere) and
+  unsigned long long* umeta; // [max_ids] the metadata found there, from the look-up that mono_prepare_push does
+                             //           ahead of the push
   uint32_t* ins_list;        // [max_ids] distinct IDs that are not in the key store yet
-  uint32_t* multi_list;      // [max_ids / 2 + 1] distinct IDs that occur more than once
+  uint4* multi_list;         // [max_ids / 2 + 1] the distinct IDs that occur more than once, in one record each:
+                             //           x = its number u, y = multiplicity, z = segment start, w = slot
   uint32_t* long_u;          // [max_long] distinct IDs whose segment is reduced in parts
   uint32_t* long_part0;      // [max_long] first part of each
   uint32_t* part_u;          // [max_parts] owner (index into long_u) of each part
@@ -260,6 +265,7 @@ __device__ inline void dedup_tile_body(const Work& wk, const unsigned long long*
       if (MONO_INDEX_OK(wk.error_bits, my_u, wk.max_ids)) {
         wk.uid[my_u] = my_id[k];
         wk.uslot[my_u] = g[k];
+        wk.uocc[my_u] = (uint32_t)(tile0 + k * kTileThreads + threadIdx.x);     // the owner's own occurrence
       }
       ++my_u;
     }

@@ -114,27 +114,21 @@ __device__ inline void add_rows(const TableView& tv, unsigned gmask, uint32_t mi
 }
 
 // Where the forward gets the row of an occurrence from:
-//  kFromRows  the array probe_rows_kernel filled (two kernels);
-//  kFromKeys  the key store, looked up here (one kernel: no row-index array in between);
-//  kFromSet   the per-call set of a batch that mono_prepare_push announced: every distinct ID was
-//             looked up once ahead of the call, its slot holds the row and the start of its segment,
-//             and the occurrence files its bag there for the push while it is at it.
-enum : int { kFromRows = 0, kFromKeys = 1, kFromSet = 2 };
+//  kFromRows  an array of row indices, one per occurrence, filled by an earlier kernel
+//             (probe_rows_kernel, or resolve_rows_kernel for a batch that was announced);
+//  kFromKeys  the key store, looked up here (one kernel: no row-index array in between).
+enum : int { kFromRows = 0, kFromKeys = 1 };
 
 struct GatherSource {
   const uint32_t* occ_row;                 // kFromRows
   const unsigned long long* ids;           // kFromKeys
-  const uint2* occ;                        // kFromSet
-  const BatchSlot* bset;                   // kFromSet
-  uint32_t* bag_of_sorted;                 // kFromSet
-  uint32_t n_slots, max_ids;               // kFromSet: sizes of bset and bag_of_sorted (for the checked build)
 };
 
 // Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
 // dim so that a lane owns NV 16-byte column vectors) adds up the rows of the
 // bag's IDs, in ID order, so the fp32 sum has one fixed order.  The lanes of the
-// group first resolve G occurrences of the bag at once, one each (row index read,
-// key store probed, or slot of the per-call set read, depending on SRC); the row
+// group first resolve G occurrences of the bag at once, one each (row index read
+// or key store probed, depending on SRC); the row
 // indices then go round the group by shuffle, so the loads of four rows are issued
 // together; what is left after the batches of four is added in one batch of its
 // exact size.  An ID without a row resolves to the table's all-zero row, so there
@@ -168,17 +162,10 @@ __device__ inline void gather_pool_body(const TableView& tv, const GatherSource&
         const long long j = lo + base + gl;
         if (SRC == kFromRows) {
           mine = __ldg(src.occ_row + j);
-        } else if (SRC == kFromKeys) {
+        } else {
           const unsigned long long id = __ldg(src.ids + j);
           unsigned long long meta = 0;
           if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) mine = meta_row(meta);
-        } else {
-          const uint2 o = __ldg(src.occ + j);
-          if (o.x != kNoSlot && MONO_INDEX_OK(&tv.st->error_bits, o.x, src.n_slots)) {
-            const uint4 bs = __ldg(reinterpret_cast<const uint4*>(src.bset + o.x));   // key (x, y), segment start, row
-            if (bs.w != kNoRow) mine = bs.w;
-            if (MONO_INDEX_OK(&tv.st->error_bits, (unsigned long long)bs.z + o.y, src.max_ids)) src.bag_of_sorted[bs.z + o.y] = (uint32_t)bag;
-          }
         }
       }
       const uint32_t cnt = n - base < (uint32_t)G ? n - base : (uint32_t)G;
@@ -200,11 +187,78 @@ __device__ inline void gather_pool_body(const TableView& tv, const GatherSource&
   }
 }
 
+// The pooling for SRC = kFromRows: every lane of the group reads the row indices itself (the
+// loads of a group hit one cache line, and the kernel is bound by instruction issue: measured
+// against passing them round by shuffle, 0.26 ms against 0.33 ms on the largest configuration,
+// and against a software pipeline over three bags, 0.41 ms, and a walk over runs of occurrences
+// that is uniform across bags, 0.33 ms -- both need half as many registers again).
+template <int K, int G, int NV>
+__device__ inline void add_indexed_rows(const TableView& tv, const uint32_t* __restrict__ idx, int gl, float4 (&sum)[NV]) {
+  uint32_t row[K];
+#pragma unroll
+  for (int k = 0; k < K; ++k) row[k] = __ldg(idx + k);
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const uint32_t c4 = gl + v * G;
+    if (c4 * 4u < tv.dim) {
+      float4 x[K];
+#pragma unroll
+      for (int k = 0; k < K; ++k) x[k] = __ldg(reinterpret_cast<const float4*>(tv.w_row(row[k])) + c4);
+#pragma unroll
+      for (int k = 0; k < K; ++k) { sum[v].x += x[k].x; sum[v].y += x[k].y; sum[v].z += x[k].z; sum[v].w += x[k].w; }
+    }
+  }
+}
+
+template <int G, int NV>
+__device__ inline void gather_rows_body(const TableView& tv, const uint32_t* __restrict__ occ_row, long long n_ids,
+                                        const long long* __restrict__ offsets, long long n_bags,
+                                        float* __restrict__ out, uint32_t vblock, uint32_t vgrid) {
+  const int gl = threadIdx.x % G;
+  const uint32_t dim = tv.dim;
+  const long long groups_per_block = blockDim.x / G;
+  const long long stride = (long long)vgrid * groups_per_block;
+  for (long long bag = (long long)vblock * groups_per_block + threadIdx.x / G; bag < n_bags; bag += stride) {
+    long long lo = offsets[bag], hi = offsets[bag + 1];
+    if (lo < 0 || hi < lo || hi > n_ids) {                 // not a well-formed bag: flagged and treated as empty
+      if (gl == 0) atomicOr(&tv.st->error_bits, 4u /* MONO_DEV_BAD_OFFSETS */);
+      lo = hi = 0;
+    }
+    float4 sum[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) sum[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint32_t* idx = occ_row + lo;
+    const uint32_t n = (uint32_t)(hi - lo);              // a call has fewer than 2^31 IDs
+    uint32_t i = 0;
+    for (; i + 4 <= n; i += 4) add_indexed_rows<4, G, NV>(tv, idx + i, gl, sum);
+    switch (n - i) {
+      case 3: add_indexed_rows<3, G, NV>(tv, idx + i, gl, sum); break;
+      case 2: add_indexed_rows<2, G, NV>(tv, idx + i, gl, sum); break;
+      case 1: add_indexed_rows<1, G, NV>(tv, idx + i, gl, sum); break;
+      default: break;
+    }
+    float4* dst = reinterpret_cast<float4*>(out + bag * (long long)dim);
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const uint32_t c4 = gl + v * G;
+      if (c4 * 4u < dim) dst[c4] = sum[v];
+    }
+  }
+}
+
+template <int G, int NV, int SRC>
+__device__ inline void gather_pool_dispatch(const TableView& tv, const GatherSource& src, long long n_ids,
+                                            const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out,
+                                            uint32_t vblock, uint32_t vgrid) {
+  if (SRC == kFromRows) gather_rows_body<G, NV>(tv, src.occ_row, n_ids, offsets, n_bags, out, vblock, vgrid);
+  else gather_pool_body<G, NV, SRC>(tv, src, n_ids, offsets, n_bags, out, vblock, vgrid);
+}
+
 template <int G, int NV, int SRC>
 __global__ void __launch_bounds__(256)
 gather_pool_kernel(TableView tv, GatherSource src, long long n_ids, const long long* __restrict__ offsets,
                    long long n_bags, float* __restrict__ out) {
-  gather_pool_body<G, NV, SRC>(tv, src, n_ids, offsets, n_bags, out, blockIdx.x, gridDim.x);
+  gather_pool_dispatch<G, NV, SRC>(tv, src, n_ids, offsets, n_bags, out, blockIdx.x, gridDim.x);
 }
 
 }  // namespace mono

@@ -21,6 +21,7 @@ struct GroupItem {
   const long long* off;
   long long n_ids, n_bags;
   float* out;                    // lookup
+  uint32_t* occ_row;             // lookup of an announced batch: row of every occurrence
   const float* grad;             // push
   unsigned long long dedup_seed;
   uint32_t now;
@@ -80,10 +81,24 @@ group_table_insert_kernel(const GroupItem* __restrict__ items, const uint32_t* _
   table_insert_body(it.tv, it.wk, it.now, vblock, vgrid);
 }
 
+// the filing pass inside a push ...
 __global__ void __launch_bounds__(256)
 group_file_segments_kernel(const GroupItem* __restrict__ items, const uint32_t* __restrict__ start, uint32_t n_tables) {
   MONO_GROUP_PROLOGUE;
-  file_segments_body(it.wk, it.n_ids, it.n_bags, vblock, vgrid);
+  file_segments_body(it.wk, it.n_ids, it.n_bags, nullptr, 0u, vblock, vgrid);
+}
+
+// ... and inside the lookup of announced batches, where it also leaves every occurrence's row
+__global__ void __launch_bounds__(256)
+group_file_rows_kernel(const GroupItem* __restrict__ items, const uint32_t* __restrict__ start, uint32_t n_tables) {
+  MONO_GROUP_PROLOGUE;
+  if (it.prepared) file_segments_body(it.wk, it.n_ids, it.n_bags, it.occ_row, (uint32_t)it.tv.capacity, vblock, vgrid);
+}
+
+__global__ void __launch_bounds__(256)
+group_clear_primary_kernel(const GroupItem* __restrict__ items, const uint32_t* __restrict__ start, uint32_t n_tables) {
+  MONO_GROUP_PROLOGUE;
+  clear_primary_body(it.wk, vblock, vgrid);
 }
 
 __global__ void __launch_bounds__(128)
@@ -145,11 +160,10 @@ __global__ void __launch_bounds__(256)
 group_gather_pool_kernel(const GroupItem* __restrict__ items, const uint32_t* __restrict__ start, uint32_t n_tables) {
   MONO_GROUP_PROLOGUE;
   GatherSource src{};
-  src.ids = it.ids; src.occ = it.wk.occ; src.bset = it.wk.bset; src.bag_of_sorted = it.wk.bag_of_sorted;
-  src.n_slots = it.wk.n_slots; src.max_ids = it.wk.max_ids;
+  src.ids = it.ids; src.occ_row = it.occ_row;
   by_lane_class<WIDE>(it.lane_class, [&](auto g, auto nv) {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
-    if (it.prepared) gather_pool_body<G, NV, kFromSet>(it.tv, src, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);
+    if (it.prepared) gather_pool_dispatch<G, NV, kFromRows>(it.tv, src, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);
     else gather_pool_body<G, NV, kFromKeys>(it.tv, src, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);
   });
 }

@@ -118,15 +118,15 @@ __device__ inline void register_long(const TableView& tv, const Work& wk, uint32
 //
 //  kLookUp  (can run ahead of the push, when mono_prepare_push announced the batch: it changes
 //           nothing in the table) -- the ID's multiplicity is read from the per-call set, the ID is
-//           looked up in the key store (the cell an insertion prefers first), every ID is given its
-//           segment of bag_of_sorted[] and, if it occurs more than once, its place in multi_list[];
+//           looked up in the key store (the cell an insertion prefers first), an ID that occurs more
+//           than once is given its segment of bag_of_sorted[] and its place in multi_list[];
 //           the ID's slot of the per-call set is rewritten to (segment start, row owned so far),
 //           which is what the occurrences need, and the cell is remembered in ucell[].
 //  kCommit  (the push itself) -- a tracked ID gets count += multiplicity (saturating at the
 //           threshold), last_seen = now, and a row if the count has reached the threshold; an ID
 //           the key store does not hold is queued for insertion.  With kLookUp in an earlier
-//           kernel, the remembered cell is read again (one line in, one out) and the search is
-//           repeated only if the key is no longer there.
+//           kernel, the cell and its metadata are the remembered ones: the kernel reads its
+//           inputs in order and only scatters the new metadata words.
 //
 // Both halves in one kernel is the push that was not announced.  No cell moves during either
 // half, so the thread whose ID sits in a cell owns it.
@@ -157,13 +157,17 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
         m = wk.bset[slot].a;
         cell = thread_locate(tv, id, stash_hw, &meta);
       } else {
+        // nothing has changed the table since the look-up (every call that could forgets the
+        // announcement), so the cell and its metadata are as remembered
         m = wk.ulen[u];
         cell = wk.ucell[u];
+        meta = wk.umeta[u];
+#ifdef MONO_DEBUG
         if (cell != kNoCell) {
           const Cell c = load_cell_whole(cell_address(tv, cell, n_cells));
-          if (c.key == id) meta = c.meta;
-          else cell = thread_locate(tv, id, stash_hw, &meta);          // moved since the look-up: search again
+          if (c.key != id || c.meta != meta) { atomicOr(&tv.st->error_bits, 16u /* MONO_DEV_INTERNAL */); cell = thread_locate(tv, id, stash_hw, &meta); }
         }
+#endif
       }
     }
     const bool hit = cell != kNoCell;
@@ -176,16 +180,16 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
       need_row = low >= tv.threshold;
     }
     const Reservation rv = block_reserve(tv, &sh, need_row, (MODE & kLookUp) && m > 1, (MODE & kCommit) && active && !hit,
-                                         (MODE & kLookUp) ? m : 0u);
+                                         ((MODE & kLookUp) && m > 1) ? m : 0u);
     if (!active) continue;
     if (MODE & kLookUp) {
       wk.ulen[u] = m;
       wk.useg[u] = rv.seg_start;
-      if (!(MODE & kCommit)) wk.ucell[u] = cell;
-      BatchSlot bs; bs.key = id; bs.a = rv.seg_start; bs.b = resident ? (low & kRowMask) : kNoRow;
+      if (!(MODE & kCommit)) { wk.ucell[u] = cell; wk.umeta[u] = meta; }
+      BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kNoSegment; bs.b = resident ? (low & kRowMask) : kNoRow;
       wk.bset[slot] = bs;
       (void)MONO_INDEX_OK(wk.error_bits, (unsigned long long)rv.seg_start + m - 1, wk.max_ids);
-      if (m > 1 && MONO_INDEX_OK(wk.error_bits, rv.multi_pos, wk.max_ids / 2 + 1)) wk.multi_list[rv.multi_pos] = u;
+      if (m > 1 && MONO_INDEX_OK(wk.error_bits, rv.multi_pos, wk.max_ids / 2 + 1)) wk.multi_list[rv.multi_pos] = make_uint4(u, m, rv.seg_start, slot);
     }
     if (MODE & kCommit) {
       if (hit) {

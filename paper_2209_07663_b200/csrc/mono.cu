@@ -32,14 +32,14 @@ static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS
 
 enum KernelId {
   K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_LOOKUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_FILE, K_SINGLES, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
-  K_STASH_TRIM, K_COUNT
+  K_STASH_TRIM, K_CLEAR, K_REDUCE_PARTS, K_COUNT
 };
 // (table_lookup and table_update are the two halves of table_update_kernel; a push that was not
 // announced runs both in one launch, counted as table_update)
 static const char* const kKernelNames[K_COUNT] = {
   "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_lookup", "table_update", "sketch_add", "table_insert", "expand_parts", "order_parts",
   "file_segments", "update_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
-  "finish_apply", "expire", "stash_trim"
+  "finish_apply", "expire", "stash_trim", "clear_set", "reduce_parts"
 };
 static_assert(K_COUNT <= MONO_MAX_KERNELS, "mono_timing_t has room for MONO_MAX_KERNELS kernels");
 
@@ -145,7 +145,7 @@ void dev_free(T*& p) { if (p) { cudaFree(p); p = nullptr; } }
 void free_scratch(mono_table* t) {
   Work& w = t->wk;
   dev_free(w.bset); dev_free(w.occ); dev_free(w.occ_bag); dev_free(w.bag_of_sorted);
-  dev_free(w.uid); dev_free(w.uslot); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow); dev_free(w.ucell);
+  dev_free(w.uid); dev_free(w.uslot); dev_free(w.uocc); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow); dev_free(w.ucell); dev_free(w.umeta);
   dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.part_order); dev_free(w.win_count); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_out); dev_free(t->stage_grad); dev_free(t->occ_row);
   t->staged.valid = false;
@@ -225,7 +225,7 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
 #define ALLOC(p, cnt) if ((rc = dev_alloc(t, &(p), (cnt))) != MONO_OK) { free_scratch(t); return rc; }
   ALLOC(w.bset, slots);
   ALLOC(w.occ, n); ALLOC(w.occ_bag, n); ALLOC(w.bag_of_sorted, n);
-  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n); ALLOC(w.ucell, n);
+  ALLOC(w.uid, n); ALLOC(w.uslot, n); ALLOC(w.uocc, n); ALLOC(w.useg, n); ALLOC(w.ulen, n); ALLOC(w.urow, n); ALLOC(w.ucell, n); ALLOC(w.umeta, n);
   ALLOC(w.multi_list, n / 2 + 1); ALLOC(w.ins_list, n);
   w.max_long = (uint32_t)(n / kSegChunk + 1);
   w.max_parts = (uint32_t)(2 * (n / kSegChunk) + 2);
@@ -295,13 +295,15 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
   if (n_bags == 0) return MONO_OK;
   GatherSource src{};
   if (prepared) {
-    // every distinct ID of this batch was looked up when it was announced: the rows come from the
-    // per-call set, and the occurrences file their bags for the push on the way
-    src.occ = t->wk.occ; src.bset = t->wk.bset; src.bag_of_sorted = t->wk.bag_of_sorted;
-    src.n_slots = t->wk.n_slots; src.max_ids = t->wk.max_ids;
-    const int rc = launch_gather<kFromSet>(t, src, n_ids, off, n_bags, out);
-    if (rc == MONO_OK) t->prep.filed = true;
-    return rc;
+    // every distinct ID of this batch was looked up when it was announced: one pass over the
+    // occurrences takes the rows from the per-call set and files the bags for the push
+    if (n_ids > 0) {
+      LAUNCH(t, K_FILE, file_segments_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->wk, n_ids, n_bags, t->occ_row,
+                                                                                    (uint32_t)t->tv.capacity));
+      t->prep.filed = true;
+    }
+    src.occ_row = t->occ_row;
+    return launch_gather<kFromRows>(t, src, n_ids, off, n_bags, out);
   }
   src.ids = ids;
   return launch_gather<kFromKeys>(t, src, n_ids, off, n_bags, out);
@@ -344,14 +346,14 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   if (is_prepared_batch(t, ids, n_ids, off, n_bags)) {
     // grouped and looked up already; filed too, if its lookup has run
     t->prep.valid = false;
-    if (!t->prep.filed) LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
+    if (!t->prep.filed) LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags, nullptr, 0u));
     LAUNCH(t, K_UPDATE, table_update_kernel<kCommit><<<g8 * 4, 256, 0, s>>>(tv, wk, now));
   } else {
     if ((rc0 = discard_prepared(t)) != MONO_OK) return rc0;
     if (n_ids == 0 || n_bags == 0) return MONO_OK;
     if ((rc0 = launch_group(t, s, ids, n_ids, off, n_bags)) != MONO_OK) return rc0;
     LAUNCH(t, K_UPDATE, table_update_kernel<kLookUp | kCommit><<<g8 * 4, 256, 0, s>>>(tv, wk, now));
-    LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags));
+    LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags, nullptr, 0u));
   }
   if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
   LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
@@ -362,10 +364,11 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   // IDs) keep only a few blocks busy each, so they run on a stream of their own beside the
   // kernels that work through the whole batch: expand/order beside the reduction of the short
   // segments, and fold/combine, which need only what the parts left, beside update_singletons.
-  // While kernels are being timed one by one, everything stays on the table's stream and the
-  // segments are reduced in one launch.
+  // While kernels are being timed one by one, everything stays on the table's stream.
   cudaStream_t a = t->timing ? s : t->aux_stream;
   if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_keys, 0));
+  // (nobody reads the per-call set after the key-store work: its primary tier is wiped beside the rest)
+  LAUNCH_ON(t, a, K_CLEAR, clear_primary_kernel<<<g8, 256, 0, a>>>(wk));
   LAUNCH_ON(t, a, K_EXPAND, expand_parts_kernel<<<g8 * 4, 128, 0, a>>>(tv, wk));
   LAUNCH_ON(t, a, K_ORDER, order_parts_kernel<<<64, kWindows, 0, a>>>(tv, wk));
   CUDA_TRY(t, cudaGetLastError());
@@ -373,14 +376,12 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   if (grad_ready) CUDA_TRY(t, cudaStreamWaitEvent(s, grad_ready, 0));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
+    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceShort));
+    if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_parts, 0));
+    LAUNCH(t, K_REDUCE_PARTS, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceParts));
     if (a != s) {
-      LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceShort));
-      CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_parts, 0));
-      LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceParts));
       CUDA_TRY(t, cudaEventRecord(t->ev_reduced, s));
       CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_reduced, 0));
-    } else {
-      LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceParts | kReduceShort));
     }
     LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
     return (int)MONO_OK;
@@ -407,7 +408,7 @@ int check_now(mono_table* t, int64_t now) {
 
 enum GroupKernel {
   GK_FILL, GK_DEDUP, GK_UPDATE, GK_INSERT, GK_FILE, GK_EXPAND, GK_ORDER, GK_GATHER, GK_GATHER_WIDE, GK_REDUCE, GK_REDUCE_WIDE,
-  GK_SINGLES, GK_SINGLES_WIDE, GK_FOLD, GK_COMBINE, GK_COUNT
+  GK_SINGLES, GK_SINGLES_WIDE, GK_FOLD, GK_COMBINE, GK_CLEAR, GK_COUNT
 };
 
 uint32_t lane_class_of(uint32_t dim) {
@@ -452,6 +453,7 @@ uint32_t group_blocks(const mono_table* t, int k, int64_t n_ids, int64_t n_bags)
     case GK_SINGLES_WIDE: return wide ? (uint32_t)clamp_blocks(n_ids, 128, g8 * 8) : 0u;
     case GK_FOLD: return (uint32_t)clamp_blocks(n_ids / (kSegChunk * kFoldWidth) + 1, 1, g4);
     case GK_COMBINE: return (uint32_t)clamp_blocks(n_ids / kSegChunk + 1, 1, g8);
+    case GK_CLEAR: return (uint32_t)clamp_blocks((int64_t)t->wk.primary_mask + 1, 2048, g8);
     default: return 0u;
   }
 }
@@ -520,6 +522,7 @@ void group_describe(GroupPlan& p, int32_t i, mono_table* t, const uint64_t* ids,
   it.ids = reinterpret_cast<const unsigned long long*>(ids);
   it.off = reinterpret_cast<const long long*>(off);
   it.n_ids = n_ids; it.n_bags = n_bags; it.out = out; it.grad = grad; it.now = now;
+  it.occ_row = t->occ_row;
   it.dedup_seed = t->tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull;
   it.prepared = prepared ? 1u : 0u;
   it.lane_class = lane_class_of(t->tv.dim);
@@ -786,11 +789,15 @@ int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const ui
     p.items[i].active = n_bags[i] > 0 ? 1u : 0u;           // a bag without IDs still pools to zeros
   }
   if ((rc = group_upload(p, tables)) != MONO_OK) return rc;
+  bool any_prepared = false;
+  for (int32_t i = 0; i < n_tables; ++i) any_prepared |= p.items[i].prepared && p.items[i].n_ids > 0;
+  // (the filing pass skips the tables that were not announced: their lookup probes the key store itself)
+  if (any_prepared) GROUP_LAUNCH(p, K_FILE, GK_FILE, 256, group_file_rows_kernel);
   GROUP_LAUNCH(p, K_GATHER, GK_GATHER, 256, group_gather_pool_kernel<0>);
   GROUP_LAUNCH(p, K_GATHER, GK_GATHER_WIDE, 256, group_gather_pool_kernel<1>);
   CUDA_TRY(p.owner, cudaGetLastError());
   for (int32_t i = 0; i < n_tables; ++i)
-    if (p.items[i].prepared) tables[i]->prep.filed = true;
+    if (p.items[i].prepared && p.items[i].n_ids > 0) tables[i]->prep.filed = true;
   return group_end(p, tables);
 }
 
@@ -837,6 +844,7 @@ int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const ui
   }
   if (p.any_sketch) GROUP_LAUNCH(p, K_SKETCH, GK_INSERT, 256, group_sketch_add_kernel);
   GROUP_LAUNCH(p, K_INSERT, GK_INSERT, 256, group_table_insert_kernel);
+  GROUP_LAUNCH(p, K_CLEAR, GK_CLEAR, 256, group_clear_primary_kernel);
   GROUP_LAUNCH(p, K_EXPAND, GK_EXPAND, 128, group_expand_parts_kernel);
   GROUP_LAUNCH(p, K_ORDER, GK_ORDER, kWindows, group_order_parts_kernel);
   GROUP_LAUNCH(p, K_REDUCE, GK_REDUCE, 128, group_reduce_adagrad_kernel<0>);
