@@ -392,7 +392,8 @@ def run_ours(args):
         raise SystemExit(f"pre-fill overflowed the table: {st0}")
 
     # ---- batches: ids/offsets from the seeded host generator, gradients drawn on the device
-    n_batches = W + K + KT + E
+    EW = 1 if E > 0 else 0                     # one untimed end-to-end step first: it allocates the staging buffers
+    n_batches = W + K + KT + EW + E
 
     def make(i):
         return stream.step(now0 + 1 + i, with_grad=False)
@@ -488,16 +489,20 @@ def run_ours(args):
             grad = torch.randn((cfg.n_bags, cfg.dim)).mul_(cfg.grad_std).pin_memory()
             pinned.append((ids, off, grad))
         out_h = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32).pin_memory()
-        barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n_e2e_ids, h2d, d2h = 0, 0, 0
-        e0.record()
         for t, (ids, off, grad) in enumerate(pinned):
+            if t == EW:
+                mb.mono_fence(table.handle)
+                barrier()
+                e0.record()
             now = now0 + 1 + W + K + KT + t
             mb.mono_lookup_pool_host(table.handle, ids, ids.numel(), off, cfg.n_bags, out_h)
             mb.mono_apply_grads_host(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now)
             if S > 0:
                 mb.mono_expire_slice(table.handle, now, (W + K + KT + t) % S, S)
+            if t < EW:
+                continue
             n_e2e_ids += ids.numel()
             h2d += ids.numel() * 8 + off.numel() * 8 + grad.numel() * 4    # the push reuses the IDs its lookup staged
             d2h += out_h.numel() * 4
@@ -653,12 +658,16 @@ def run_multi(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
     K, W, S = args.steps, args.warmup, args.sweep_slices
-    cfgs = [rank_config(c, rank) for c in wl.multi_table_configs()]
+    base_cfgs = wl.many_small_table_configs() if args.workload == "multi_small" else wl.multi_table_configs()
+    cfgs = [rank_config(c, rank) for c in base_cfgs]
+    own_streams = args.multi_mode == "streams"
+    streams = [torch.cuda.Stream(device=dev) for _ in cfgs] if own_streams else []
     tables, now0 = [], []
-    for cfg in cfgs:
+    for ti, cfg in enumerate(cfgs):
         t = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, lr=cfg.lr, eps=cfg.eps,
                          init_acc=cfg.init_acc, init_scale=cfg.init_scale, seed=cfg.seed, key_cells=cfg.key_cells,
-                         max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1), max_bags=cfg.n_bags)
+                         max_ids=int(cfg.n_bags * wl._mean_bag_len(cfg.bag_len) * 1.1), max_bags=cfg.n_bags,
+                         **({"stream": streams[ti].cuda_stream} if own_streams else {}))
         n0 = cfg.ttl - 1
         for ids, cnt, seen in wl.steady_state_population_torch(cfg, n0, dev):
             res = (cnt >= cfg.filter_threshold).to(torch.uint8)
@@ -715,10 +724,16 @@ def run_multi(args):
         torch.cuda.synchronize()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
+        for st in streams:
+            st.wait_event(ev0)
         for i in range(first, first + K):
             step(i, grouped)
         for t in tables:
             mb.mono_fence(t.handle)
+        for st in streams:                       # tables on streams of their own: the stop event waits for all of them
+            done = torch.cuda.Event()
+            done.record(st)
+            torch.cuda.current_stream().wait_event(done)
         ev1.record()
         torch.cuda.synchronize()
         return ev0.elapsed_time(ev1)
@@ -726,13 +741,14 @@ def run_multi(args):
     def launches_now():
         return sum(mb.mono_timing_read(t.handle, reset=True)["launches_total"] for t in tables)
 
+    first_mode = not own_streams                 # grouped calls first, unless the tables sit on streams of their own
     for i in range(W):
-        step(i, True)
+        step(i, first_mode)
     before = [t.status() for t in tables]
     launches_now()
     sampler = ClockSampler(local_rank, gpu_uuid(local_rank))
     sampler.start()
-    ms = timed(W, True)
+    ms = timed(W, first_mode)
     clocks = sampler.stop()
     launches = launches_now()
     mid = [t.status() for t in tables]
@@ -756,7 +772,9 @@ def run_multi(args):
             "metric": METRIC, "value": ids_all / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "multi", "tables": [{"name": c.name, "capacity": c.capacity, "dim": c.dim,
+            "config": {"workload": args.workload, "calls": ("single-table calls, every table on a CUDA stream of its own"
+                                                            if own_streams else "grouped calls, all tables on one stream"),
+                       "tables": [{"name": c.name, "capacity": c.capacity, "dim": c.dim,
                                                          "slots": c.n_slots, "zipf_s": c.zipf_s,
                                                          "row_load": s0["n_resident"] / c.capacity,
                                                          "key_load": s0["n_tracked"] / c.key_cells}
@@ -765,7 +783,9 @@ def run_multi(args):
                        "ids_per_step": n_ids / K, "prefill": "the state after ttl steps of each stream from an empty table (Poisson model)",
                        "sweep": f"every step sweeps 1/{S} of every key store" if S > 0 else "none",
                        "l2": "every step reads fresh batches larger than L2",
-                       "parallelism": "8 tables on one CUDA stream of one GPU; grouped calls: one launch per kernel for all tables"},
+                       "parallelism": (f"{len(cfgs)} tables of one process on one GPU; " +
+                                       ("single-table calls on one stream per table" if own_streams else
+                                        "grouped calls: one launch per kernel for all tables"))},
             "launches_per_step": launches / K,
             "one_table_at_a_time": {"value": n_ids_serial / (ms_serial * 1e-3), "ms_per_step": ms_serial / K,
                                     "launches_per_step": launches_serial / K,
@@ -787,7 +807,10 @@ def main():
     ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS) + ["multi"])
+    ap.add_argument("--workload", default="large", choices=sorted(wl.CONFIGS) + ["multi", "multi_small"])
+    ap.add_argument("--multi-mode", default="grouped", choices=["grouped", "streams"],
+                    help="multi-table workloads: grouped calls on one stream (then, for comparison, the single-table "
+                         "calls table after table), or single-table calls with every table on a stream of its own")
     ap.add_argument("--no-prepare", dest="prepare", action="store_false",
                     help="do not announce each batch with mono_prepare_push before its lookup")
     ap.add_argument("--sweep-slices", type=int, default=32,
@@ -800,7 +823,7 @@ def main():
                     help="with --filter sketch the key store has 2^-this of the configured cells")
     ap.add_argument("--reps", type=int, default=5,
                     help="repetitions of the timed region, each from the same restored state (median reported)")
-    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--kernel-steps", type=int, default=8, help="steps of the per-kernel CUDA-event pass")
     ap.add_argument("--no-prefill", dest="prefill", action="store_false")
     ap.add_argument("--oracle-steps", type=int, default=4)
@@ -809,10 +832,10 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
-        if args.workload == "multi":
+        if args.workload in ("multi", "multi_small"):
             args.workload = "large"
         run_reference(args)
-    elif args.workload == "multi":
+    elif args.workload in ("multi", "multi_small"):
         run_multi(args)
     else:
         run_ours(args)

@@ -66,7 +66,7 @@ struct Work {
   unsigned long long* umeta; // [max_ids] the metadata found there, from the look-up that mono_prepare_push does
                              //           ahead of the push
   uint32_t* ins_list;        // [max_ids] distinct IDs that are not in the key store yet
-  uint4* multi_list;         // [max_ids / 2 + 1] the distinct IDs that occur more than once, in one record each:
+  uint32_t* multi_list;         // [max_ids / 2 + 1] the distinct IDs that occur more than once, in one record each:
                              //           x = its number u, y = multiplicity, z = segment start, w = slot
   uint32_t* long_u;          // [max_long] distinct IDs whose segment is reduced in parts
   uint32_t* long_part0;      // [max_long] first part of each

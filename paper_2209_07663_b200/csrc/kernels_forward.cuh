@@ -71,20 +71,21 @@ __device__ inline unsigned long long thread_locate(const TableView& tv, unsigned
   return kNoCell;
 }
 
-// Forward, step 1: one thread per ID occurrence resolves the ID to its row
-// index; an ID without a row gets the index of the table's all-zero row (one
-// past the capacity), so that step 2 can add rows without asking.  Every
-// occurrence is independent, so the random bucket reads of a whole batch are in
-// flight together.  (Measured against quad-cooperative variants: the shuffles
-// those need cost more issue slots than the extra L1 wavefronts of four 16-byte
-// loads per thread.)
-__global__ void __launch_bounds__(256)
-probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
-                  uint32_t* __restrict__ occ_row) {
+// Forward, step 1, for a batch that was not announced: one thread per ID occurrence resolves
+// the ID to its row index; an ID without a row gets the index of the table's all-zero row (one
+// past the capacity), so that step 2 can add rows without asking.  Every occurrence is
+// independent, so the random bucket reads of a whole batch are in flight together.  (Measured
+// against quad-cooperative variants: the shuffles those need cost more issue slots than the
+// extra L1 wavefronts of four 16-byte loads per thread.  Measured against doing the look-ups
+// inside step 2, one per lane of the bag's group: 0.50 ms against 0.15 + 0.27 ms for the two
+// kernels on the largest configuration.)  For a batch that was announced, file_segments_kernel
+// writes the same array from the look-up that was done once per distinct ID.
+__device__ inline void probe_rows_body(const TableView& tv, const unsigned long long* __restrict__ ids, long long n_ids,
+                                       uint32_t* __restrict__ occ_row, uint32_t vblock, uint32_t vgrid) {
   const unsigned stash_hw = tv.st->stash_hw;
   const uint32_t zero_row = (uint32_t)tv.capacity;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
+  const long long stride = (long long)vgrid * blockDim.x;
+  for (long long j = (long long)vblock * blockDim.x + threadIdx.x; j < n_ids; j += stride) {
     const unsigned long long id = ids[j];
     unsigned long long meta = 0;
     uint32_t row = zero_row;
@@ -92,108 +93,15 @@ probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long
     occ_row[j] = row;
   }
 }
-
-// sum += the rows that lanes k .. k+K-1 of the group hold in `mine`, in that order; all K loads
-// are issued before the first add.
-template <int K, int G, int NV>
-__device__ inline void add_rows(const TableView& tv, unsigned gmask, uint32_t mine, uint32_t k, int gl, float4 (&sum)[NV]) {
-  uint32_t row[K];
-#pragma unroll
-  for (int q = 0; q < K; ++q) row[q] = __shfl_sync(gmask, mine, k + q, G);
-#pragma unroll
-  for (int v = 0; v < NV; ++v) {
-    const uint32_t c4 = gl + v * G;
-    if (c4 * 4u < tv.dim) {
-      float4 x[K];
-#pragma unroll
-      for (int k = 0; k < K; ++k) x[k] = __ldg(reinterpret_cast<const float4*>(tv.w_row(row[k])) + c4);
-#pragma unroll
-      for (int k = 0; k < K; ++k) { sum[v].x += x[k].x; sum[v].y += x[k].y; sum[v].z += x[k].z; sum[v].w += x[k].w; }
-    }
-  }
+__global__ void __launch_bounds__(256)
+probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
+                  uint32_t* __restrict__ occ_row) {
+  probe_rows_body(tv, ids, n_ids, occ_row, blockIdx.x, gridDim.x);
 }
 
-// Where the forward gets the row of an occurrence from:
-//  kFromRows  an array of row indices, one per occurrence, filled by an earlier kernel
-//             (probe_rows_kernel, or resolve_rows_kernel for a batch that was announced);
-//  kFromKeys  the key store, looked up here (one kernel: no row-index array in between).
-enum : int { kFromRows = 0, kFromKeys = 1 };
-
-struct GatherSource {
-  const uint32_t* occ_row;                 // kFromRows
-  const unsigned long long* ids;           // kFromKeys
-};
-
-// Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
-// dim so that a lane owns NV 16-byte column vectors) adds up the rows of the
-// bag's IDs, in ID order, so the fp32 sum has one fixed order.  The lanes of the
-// group first resolve G occurrences of the bag at once, one each (row index read
-// or key store probed, depending on SRC); the row
-// indices then go round the group by shuffle, so the loads of four rows are issued
-// together; what is left after the batches of four is added in one batch of its
-// exact size.  An ID without a row resolves to the table's all-zero row, so there
-// are no per-row validity tests and no loads or adds for padding.
-template <int G, int NV, int SRC>
-__device__ inline void gather_pool_body(const TableView& tv, const GatherSource& src, long long n_ids,
-                                        const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out,
-                                        uint32_t vblock, uint32_t vgrid) {
-  const int gl = threadIdx.x % G;
-  const unsigned gmask = G == 32 ? 0xFFFFFFFFu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
-  const uint32_t dim = tv.dim;
-  const uint32_t zero_row = (uint32_t)tv.capacity;
-  unsigned stash_hw = 0;
-  if (SRC == kFromKeys) stash_hw = tv.st->stash_hw;
-  const long long groups_per_block = blockDim.x / G;
-  const long long stride = (long long)vgrid * groups_per_block;
-  for (long long bag = (long long)vblock * groups_per_block + threadIdx.x / G; bag < n_bags; bag += stride) {
-    long long lo = offsets[bag], hi = offsets[bag + 1];
-    if (lo < 0 || hi < lo || hi > n_ids) {                 // not a well-formed bag: flagged and treated as empty
-      if (gl == 0) atomicOr(&tv.st->error_bits, 4u /* MONO_DEV_BAD_OFFSETS */);
-      lo = hi = 0;
-    }
-    float4 sum[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) sum[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const uint32_t n = (uint32_t)(hi - lo);              // a call has fewer than 2^31 IDs
-    for (uint32_t base = 0; base < n; base += G) {
-      // this lane's occurrence of the round
-      uint32_t mine = zero_row;
-      if (base + gl < n) {
-        const long long j = lo + base + gl;
-        if (SRC == kFromRows) {
-          mine = __ldg(src.occ_row + j);
-        } else {
-          const unsigned long long id = __ldg(src.ids + j);
-          unsigned long long meta = 0;
-          if (id != kEmptyKey && thread_lookup(tv, id, stash_hw, &meta) && meta_resident(meta)) mine = meta_row(meta);
-        }
-      }
-      const uint32_t cnt = n - base < (uint32_t)G ? n - base : (uint32_t)G;
-      uint32_t k = 0;
-      for (; k + 4 <= cnt; k += 4) add_rows<4, G, NV>(tv, gmask, mine, k, gl, sum);
-      switch (cnt - k) {
-        case 3: add_rows<3, G, NV>(tv, gmask, mine, k, gl, sum); break;
-        case 2: add_rows<2, G, NV>(tv, gmask, mine, k, gl, sum); break;
-        case 1: add_rows<1, G, NV>(tv, gmask, mine, k, gl, sum); break;
-        default: break;
-      }
-    }
-    float4* dst = reinterpret_cast<float4*>(out + bag * (long long)dim);
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-      const uint32_t c4 = gl + v * G;
-      if (c4 * 4u < dim) dst[c4] = sum[v];
-    }
-  }
-}
-
-// The pooling for SRC = kFromRows: every lane of the group reads the row indices itself (the
-// loads of a group hit one cache line, and the kernel is bound by instruction issue: measured
-// against passing them round by shuffle, 0.26 ms against 0.33 ms on the largest configuration,
-// and against a software pipeline over three bags, 0.41 ms, and a walk over runs of occurrences
-// that is uniform across bags, 0.33 ms -- both need half as many registers again).
+// sum += rows idx[0..K), in that order; all K loads are issued before the first add.
 template <int K, int G, int NV>
-__device__ inline void add_indexed_rows(const TableView& tv, const uint32_t* __restrict__ idx, int gl, float4 (&sum)[NV]) {
+__device__ inline void add_rows(const TableView& tv, const uint32_t* __restrict__ idx, int gl, float4 (&sum)[NV]) {
   uint32_t row[K];
 #pragma unroll
   for (int k = 0; k < K; ++k) row[k] = __ldg(idx + k);
@@ -210,10 +118,26 @@ __device__ inline void add_indexed_rows(const TableView& tv, const uint32_t* __r
   }
 }
 
+// Forward, step 2: one group of G lanes per bag (G = 4, 8, 16 or 32 chosen from
+// dim so that a lane owns NV 16-byte column vectors) adds up the rows of the
+// bag's IDs, in ID order, so the fp32 sum has one fixed order.  The row
+// indices are known, so the loads of four rows are issued together; what is
+// left of the bag after the batches of four is added in one batch of its exact
+// size.  The kernel is bound by instruction issue, not by memory, so there are
+// no per-row validity tests (step 1 points an ID without a row at the zero row)
+// and no loads or adds for padding (measured: batches padded with the zero row
+// 0.31 ms on the largest configuration, exact tails 0.26 ms).  Every lane of the
+// group reads the row indices itself: the loads of a group hit one cache line.
+// Three other shapes of this loop were measured slower on the largest configuration
+// (0.26 - 0.28 ms as it stands): the indices read once per group and passed round by
+// shuffle, 0.33 ms; a software pipeline over three bags (offsets, indices and rows of
+// successive bags in flight together), 0.41 ms; and a walk over each group's run of
+// occurrences in uniform batches of four with only the end of a bag depending on the
+// offsets, 0.33 ms -- the last two need half as many registers again.
 template <int G, int NV>
-__device__ inline void gather_rows_body(const TableView& tv, const uint32_t* __restrict__ occ_row, long long n_ids,
-                                        const long long* __restrict__ offsets, long long n_bags,
-                                        float* __restrict__ out, uint32_t vblock, uint32_t vgrid) {
+__device__ inline void gather_pool_body(const TableView& tv, const uint32_t* __restrict__ occ_row, long long n_ids,
+                                        const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out,
+                                        uint32_t vblock, uint32_t vgrid) {
   const int gl = threadIdx.x % G;
   const uint32_t dim = tv.dim;
   const long long groups_per_block = blockDim.x / G;
@@ -230,11 +154,11 @@ __device__ inline void gather_rows_body(const TableView& tv, const uint32_t* __r
     const uint32_t* idx = occ_row + lo;
     const uint32_t n = (uint32_t)(hi - lo);              // a call has fewer than 2^31 IDs
     uint32_t i = 0;
-    for (; i + 4 <= n; i += 4) add_indexed_rows<4, G, NV>(tv, idx + i, gl, sum);
+    for (; i + 4 <= n; i += 4) add_rows<4, G, NV>(tv, idx + i, gl, sum);
     switch (n - i) {
-      case 3: add_indexed_rows<3, G, NV>(tv, idx + i, gl, sum); break;
-      case 2: add_indexed_rows<2, G, NV>(tv, idx + i, gl, sum); break;
-      case 1: add_indexed_rows<1, G, NV>(tv, idx + i, gl, sum); break;
+      case 3: add_rows<3, G, NV>(tv, idx + i, gl, sum); break;
+      case 2: add_rows<2, G, NV>(tv, idx + i, gl, sum); break;
+      case 1: add_rows<1, G, NV>(tv, idx + i, gl, sum); break;
       default: break;
     }
     float4* dst = reinterpret_cast<float4*>(out + bag * (long long)dim);
@@ -246,19 +170,11 @@ __device__ inline void gather_rows_body(const TableView& tv, const uint32_t* __r
   }
 }
 
-template <int G, int NV, int SRC>
-__device__ inline void gather_pool_dispatch(const TableView& tv, const GatherSource& src, long long n_ids,
-                                            const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out,
-                                            uint32_t vblock, uint32_t vgrid) {
-  if (SRC == kFromRows) gather_rows_body<G, NV>(tv, src.occ_row, n_ids, offsets, n_bags, out, vblock, vgrid);
-  else gather_pool_body<G, NV, SRC>(tv, src, n_ids, offsets, n_bags, out, vblock, vgrid);
-}
-
-template <int G, int NV, int SRC>
+template <int G, int NV>
 __global__ void __launch_bounds__(256)
-gather_pool_kernel(TableView tv, GatherSource src, long long n_ids, const long long* __restrict__ offsets,
-                   long long n_bags, float* __restrict__ out) {
-  gather_pool_dispatch<G, NV, SRC>(tv, src, n_ids, offsets, n_bags, out, blockIdx.x, gridDim.x);
+gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long n_ids,
+                   const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out) {
+  gather_pool_body<G, NV>(tv, occ_row, n_ids, offsets, n_bags, out, blockIdx.x, gridDim.x);
 }
 
 }  // namespace mono

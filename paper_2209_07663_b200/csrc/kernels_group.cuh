@@ -21,7 +21,7 @@ struct GroupItem {
   const long long* off;
   long long n_ids, n_bags;
   float* out;                    // lookup
-  uint32_t* occ_row;             // lookup of an announced batch: row of every occurrence
+  uint32_t* occ_row;             // lookup: row of every occurrence
   const float* grad;             // push
   unsigned long long dedup_seed;
   uint32_t now;
@@ -155,16 +155,19 @@ __device__ inline void by_lane_class(uint32_t lane_class, F&& f) {
   }
 }
 
+// (lookup of the tables whose batches were not announced: their occurrences probe the key store)
+__global__ void __launch_bounds__(256)
+group_probe_rows_kernel(const GroupItem* __restrict__ items, const uint32_t* __restrict__ start, uint32_t n_tables) {
+  MONO_GROUP_PROLOGUE;
+  if (!it.prepared) probe_rows_body(it.tv, it.ids, it.n_ids, it.occ_row, vblock, vgrid);
+}
+
 template <int WIDE>
 __global__ void __launch_bounds__(256)
 group_gather_pool_kernel(const GroupItem* __restrict__ items, const uint32_t* __restrict__ start, uint32_t n_tables) {
   MONO_GROUP_PROLOGUE;
-  GatherSource src{};
-  src.ids = it.ids; src.occ_row = it.occ_row;
   by_lane_class<WIDE>(it.lane_class, [&](auto g, auto nv) {
-    constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
-    if (it.prepared) gather_pool_dispatch<G, NV, kFromRows>(it.tv, src, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);
-    else gather_pool_body<G, NV, kFromKeys>(it.tv, src, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);
+    gather_pool_body<decltype(g)::value, decltype(nv)::value>(it.tv, it.occ_row, it.n_ids, it.off, it.n_bags, it.out, vblock, vgrid);
   });
 }
 

@@ -189,7 +189,7 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
       BatchSlot bs; bs.key = id; bs.a = m > 1 ? rv.seg_start : kNoSegment; bs.b = resident ? (low & kRowMask) : kNoRow;
       wk.bset[slot] = bs;
       (void)MONO_INDEX_OK(wk.error_bits, (unsigned long long)rv.seg_start + m - 1, wk.max_ids);
-      if (m > 1 && MONO_INDEX_OK(wk.error_bits, rv.multi_pos, wk.max_ids / 2 + 1)) wk.multi_list[rv.multi_pos] = make_uint4(u, m, rv.seg_start, slot);
+      if (m > 1 && MONO_INDEX_OK(wk.error_bits, rv.multi_pos, wk.max_ids / 2 + 1)) wk.multi_list[rv.multi_pos] = u;
     }
     if (MODE & kCommit) {
       if (hit) {

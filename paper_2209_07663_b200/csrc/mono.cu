@@ -275,38 +275,44 @@ int dispatch_dim(uint32_t dim, F&& f) {
   return f(std::integral_constant<int, 32>{}, std::integral_constant<int, 8>{});
 }
 
-// The pooling kernel, with the rows of the occurrences taken from SRC.
-template <int SRC>
-int launch_gather(mono_table* t, const GatherSource& src, int64_t n_ids, const long long* off, int64_t n_bags, float* out) {
+// The pooling kernel over the row indices in `occ_row`.
+int launch_gather(mono_table* t, const uint32_t* occ_row, int64_t n_ids, const long long* off, int64_t n_bags, float* out) {
   return dispatch_dim(t->tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     const int64_t groups_per_block = 256 / G;
     int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
     const int64_t cap = (int64_t)grid_for(t, 8) * 8;
     if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV, SRC><<<(int)blocks, 256, 0, t->stream>>>(t->tv, src, n_ids, off, n_bags, out));
+    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, occ_row, n_ids, off, n_bags, out));
     CUDA_TRY(t, cudaGetLastError());
     return (int)MONO_OK;
   });
 }
 
+int launch_probe(mono_table* t, const unsigned long long* ids, int64_t n_ids, uint32_t* occ_row) {
+  if (n_ids <= 0) return MONO_OK;
+  int64_t blocks = (n_ids + 255) / 256;
+  const int64_t cap = (int64_t)grid_for(t, 8) * 8;
+  if (blocks > cap) blocks = cap;
+  LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, occ_row));
+  CUDA_TRY(t, cudaGetLastError());
+  return MONO_OK;
+}
+
 int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off,
                   int64_t n_bags, float* out, bool prepared) {
   if (n_bags == 0) return MONO_OK;
-  GatherSource src{};
-  if (prepared) {
+  if (prepared && n_ids > 0) {
     // every distinct ID of this batch was looked up when it was announced: one pass over the
     // occurrences takes the rows from the per-call set and files the bags for the push
-    if (n_ids > 0) {
-      LAUNCH(t, K_FILE, file_segments_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->wk, n_ids, n_bags, t->occ_row,
-                                                                                    (uint32_t)t->tv.capacity));
-      t->prep.filed = true;
-    }
-    src.occ_row = t->occ_row;
-    return launch_gather<kFromRows>(t, src, n_ids, off, n_bags, out);
+    LAUNCH(t, K_FILE, file_segments_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->wk, n_ids, n_bags, t->occ_row,
+                                                                                  (uint32_t)t->tv.capacity));
+    t->prep.filed = true;
+  } else {
+    const int rc = launch_probe(t, ids, n_ids, t->occ_row);
+    if (rc != MONO_OK) return rc;
   }
-  src.ids = ids;
-  return launch_gather<kFromKeys>(t, src, n_ids, off, n_bags, out);
+  return launch_gather(t, t->occ_row, n_ids, off, n_bags, out);
 }
 
 // The part of a push that depends on the IDs alone: bag of every occurrence, and the
@@ -791,8 +797,11 @@ int mono_group_lookup_pool(int32_t n_tables, mono_table* const* tables, const ui
   if ((rc = group_upload(p, tables)) != MONO_OK) return rc;
   bool any_prepared = false;
   for (int32_t i = 0; i < n_tables; ++i) any_prepared |= p.items[i].prepared && p.items[i].n_ids > 0;
-  // (the filing pass skips the tables that were not announced: their lookup probes the key store itself)
+  bool any_unprepared = false;
+  for (int32_t i = 0; i < n_tables; ++i) any_unprepared |= !p.items[i].prepared && p.items[i].n_ids > 0;
+  // (each of the two passes skips the other kind of table)
   if (any_prepared) GROUP_LAUNCH(p, K_FILE, GK_FILE, 256, group_file_rows_kernel);
+  if (any_unprepared) GROUP_LAUNCH(p, K_PROBE, GK_FILE, 256, group_probe_rows_kernel);
   GROUP_LAUNCH(p, K_GATHER, GK_GATHER, 256, group_gather_pool_kernel<0>);
   GROUP_LAUNCH(p, K_GATHER, GK_GATHER_WIDE, 256, group_gather_pool_kernel<1>);
   CUDA_TRY(p.owner, cudaGetLastError());
@@ -945,15 +954,8 @@ int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids, 
   if ((rc = noalloc_scratch(t, &occ_row)) != MONO_OK) return rc;
   const unsigned long long* d_ids = reinterpret_cast<const unsigned long long*>(ids);
   const long long* d_off = reinterpret_cast<const long long*>(slot_offsets);
-  if (n_ids > 0) {
-    int64_t blocks = (n_ids + 255) / 256;
-    const int64_t cap = (int64_t)grid_for(t, 8) * 4;
-    if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, d_ids, n_ids, occ_row));
-  }
-  GatherSource src{};
-  src.occ_row = occ_row;
-  return launch_gather<kFromRows>(t, src, n_ids, d_off, n_bags, out);
+  if ((rc = launch_probe(t, d_ids, n_ids, occ_row)) != MONO_OK) return rc;
+  return launch_gather(t, occ_row, n_ids, d_off, n_bags, out);
 }
 
 // Streams, events and staging of the host-buffer calls, made by the first of them.

@@ -138,7 +138,7 @@ CONFIGS = {
     # the same stream on a table sized for it: the drift stream keeps about 5.4e6 rows and 2.9e7 tracked IDs
     # alive within its TTL, so this row store and key store run at load 0.85-0.9, where cuckoo
     # insertions displace other keys (on the 2^26-row table above they never have to)
-    "drift_dense": Config("drift_dense", capacity=6_200_000, dim=32, filter_threshold=3, ttl=200,
+    "drift_dense": Config("drift_dense", capacity=5_900_000, dim=32, filter_threshold=3, ttl=200,
                           n_examples=16384, n_slots=50, bag_len=("geometric", 5.0, 1, 20),
                           zipf_s=1.2, n_distinct=1 << 30, steps=400, key_cells=1 << 25,
                           drift_period=50, drift_new_frac=0.30),
@@ -166,6 +166,17 @@ def multi_table_configs(n_examples: int = 32768, slots=MULTI_TABLE_SLOTS) -> lis
                           bag_len=("uniform", 1, 8), zipf_s=s, n_distinct=1 << min(cl + ex, 30),
                           steps=50, key_cells=1 << min(cl + 2, 30), seed=20220923 + 101 * t))
     return out
+
+
+def many_small_table_configs(n_tables: int = 64, n_examples: int = 4096) -> list:
+    """The other end of Section 3.1's "many tables of very uneven size": `n_tables` small tables
+    (2^17 rows, two feature slots each, dims cycling through 8, 16, 32, 64), each far too small to
+    fill a GPU on its own -- the case grouped launches are for."""
+    dims = (8, 16, 32, 64)
+    return [Config(f"small{t}", capacity=1 << 17, dim=dims[t % 4], filter_threshold=2, ttl=50,
+                   n_examples=n_examples, n_slots=2, bag_len=("uniform", 1, 4), zipf_s=1.0 + 0.05 * (t % 5),
+                   n_distinct=1 << 18, steps=50, key_cells=1 << 19, seed=20220923 + 977 * t)
+            for t in range(n_tables)]
 
 
 def expected_steady_state(cfg: Config, window: Optional[int] = None):
