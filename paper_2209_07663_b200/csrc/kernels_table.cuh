@@ -55,31 +55,39 @@ __device__ inline Reservation block_reserve(const TableView& tv, BlockAlloc* sh,
                                   ((unsigned long long)(need_insert ? 1u : 0u) << 42) |
                                   ((unsigned long long)(is_multi ? 1u : 0u) << 32) | seg_len;
   const unsigned long long before = block_exclusive_scan(mine, sh->warp_sums, &total);
-  if (threadIdx.x == 0) {
-    const unsigned int rows_wanted = (unsigned int)(total >> 52) & 0x3FFu, ins_total = (unsigned int)(total >> 42) & 0x3FFu,
-                       multi_total = (unsigned int)(total >> 32) & 0x3FFu, seg_total = (unsigned int)total;
-    unsigned int granted = 0;
-    long long old = 0;
-    if (rows_wanted) {
-      old = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top),
-                                 (unsigned long long)(-(long long)rows_wanted));
-      const long long avail = old > 0 ? old : 0;
-      granted = avail >= (long long)rows_wanted ? rows_wanted : (unsigned int)avail;
-      if (granted < rows_wanted) {
-        atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)(rows_wanted - granted));
-        atomicOr(&tv.st->error_bits, 1u /* MONO_DEV_ROWS_FULL */);
-        atomicAdd(&tv.st->n_rows_refused, (unsigned long long)(rows_wanted - granted));
+  // the four counters are updated by the first lanes of four different warps, so that their round
+  // trips to memory overlap instead of following one another (blocks have at least four warps)
+  const unsigned int rows_wanted = (unsigned int)(total >> 52) & 0x3FFu, ins_total = (unsigned int)(total >> 42) & 0x3FFu,
+                     multi_total = (unsigned int)(total >> 32) & 0x3FFu, seg_total = (unsigned int)total;
+  const unsigned int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31u) == 0u && warp < 4u) {
+    if (warp == 0u) {
+      unsigned int granted = 0;
+      long long old = 0;
+      if (rows_wanted) {
+        old = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top),
+                                   (unsigned long long)(-(long long)rows_wanted));
+        const long long avail = old > 0 ? old : 0;
+        granted = avail >= (long long)rows_wanted ? rows_wanted : (unsigned int)avail;
+        if (granted < rows_wanted) {
+          atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)(rows_wanted - granted));
+          atomicOr(&tv.st->error_bits, 1u /* MONO_DEV_ROWS_FULL */);
+          atomicAdd(&tv.st->n_rows_refused, (unsigned long long)(rows_wanted - granted));
+        }
+        if (granted) {
+          atomicAdd(&tv.st->n_resident, (unsigned long long)granted);
+          atomicAdd(&tv.st->n_admitted_total, (unsigned long long)granted);
+        }
       }
-      if (granted) {
-        atomicAdd(&tv.st->n_resident, (unsigned long long)granted);
-        atomicAdd(&tv.st->n_admitted_total, (unsigned long long)granted);
-      }
+      sh->row_base = old;
+      sh->rows_granted = granted;
+    } else if (warp == 1u) {
+      sh->seg_base = seg_total ? atomicAdd(&tv.st->seg_cursor, seg_total) : 0u;
+    } else if (warp == 2u) {
+      sh->multi_base = multi_total ? atomicAdd(&tv.st->n_multi, multi_total) : 0u;
+    } else {
+      sh->ins_base = ins_total ? atomicAdd(&tv.st->n_insert, ins_total) : 0u;
     }
-    sh->row_base = old;
-    sh->rows_granted = granted;
-    sh->seg_base = seg_total ? atomicAdd(&tv.st->seg_cursor, seg_total) : 0u;
-    sh->multi_base = multi_total ? atomicAdd(&tv.st->n_multi, multi_total) : 0u;
-    sh->ins_base = ins_total ? atomicAdd(&tv.st->n_insert, ins_total) : 0u;
   }
   __syncthreads();
   Reservation r;
