@@ -439,8 +439,20 @@ def run_ours(args):
     for t in range(W):
         step(t)
     barrier()
+    reps_note = None
     if R > 1:
-        mb.mono_snapshot_save(table.handle)
+        try:
+            mb.mono_snapshot_save(table.handle)
+        except mb.MonoError as e:          # no room for a second copy of the table: one repetition, and say so
+            if e.code != mb.MONO_ERR_NOMEM:
+                raise
+            R, reps_note = 1, "no device memory for the snapshot the repetitions return to: one repetition only"
+        if world > 1:                      # every rank repeats as often as the rank with the least room
+            r_all = torch.tensor([R], dtype=torch.int64, device=dev)
+            dist.all_reduce(r_all, op=dist.ReduceOp.MIN)
+            if int(r_all.item()) < R:
+                R, reps_note = 1, "another rank had no device memory for the snapshot: one repetition only"
+                mb.mono_snapshot_drop(table.handle)
     sampler = ClockSampler(local_rank, gpu_uuid(local_rank))
     rep_ms, launches, n_ids_timed = [], 0, 0
     st_a = st_b = None
@@ -553,7 +565,8 @@ def run_ours(args):
             "reps": {"n": R, "what": f"the timed region ({K} steps) repeated from the same restored state; value and "
                                      "ms_per_step are the median repetition (slowest rank)",
                      "ms_per_step_median": statistics.median(rep_ms) / K, "ms_per_step_min": min(rep_ms) / K,
-                     "ms_per_step_max": max(rep_ms) / K, "ms_per_step_all_rank0": [round(x / K, 5) for x in rep_ms]},
+                     "ms_per_step_max": max(rep_ms) / K, "ms_per_step_all_rank0": [round(x / K, 5) for x in rep_ms],
+                     **({"note": reps_note} if reps_note else {})},
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": args.workload, "capacity": cfg.capacity, "dim": d, "key_cells": cfg.key_cells,
