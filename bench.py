@@ -601,6 +601,10 @@ def run_ours(args):
                 "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": dom_bytes,
                 "ms_per_launch": dom_ms,
                 "traffic": recorded_traffic(dom, args.workload),
+                **({"launches_per_step": 2,
+                    "note": "this kernel runs twice per step (short segments, then the parts of long ones); bytes, "
+                            "time and traffic are those of the two launches together"}
+                   if dom == "reduce_adagrad" and "ms_parts" in per_kernel[dom] else {}),
             },
             "whole_step": {
                 "algorithmic_bytes": alg_total, "achieved_gbs": alg_total / (step_ms * 1e-3) / 1e9,
