@@ -229,7 +229,7 @@ def test_forward_equals_torch_embedding_bag():
 def test_host_buffer_calls_match_device_calls():
     """mono_lookup_pool_host / mono_apply_grads_host: pinned host buffers in, pooled rows back out, no
     synchronisation inside the calls.  Steps are issued back to back (the result of each is read after
-    a fence); one push is given a batch other than the one its lookup staged."""
+    a fence); one push is given a batch other than the one its lookup staged, one follows a sweep."""
     cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=256, steps=6)
     a, cpu = make_pair(cfg)
     stream = wl.Stream(cfg)
@@ -241,14 +241,15 @@ def test_host_buffer_calls_match_device_calls():
         outs.append(torch.full((cfg.n_bags, cfg.dim), float("nan"), dtype=torch.float32).pin_memory())
     for t, (ids, off, grad, s) in enumerate(host):
         mb.mono_lookup_pool_host(a.handle, ids, ids.numel(), off, cfg.n_bags, outs[t])
+        want = cpu.lookup_pool(s.ids, s.offsets)
+        if t == 4:       # a sweep between the lookup and the push: the push groups and looks up its batch again
+            a.expire(t - 1); cpu.expire(t - 1)
         if t == 3:       # the push of another batch than the one just looked up: it brings its own IDs in
             o_ids, o_off, o_grad, o = host[5]
             mb.mono_apply_grads_host(a.handle, o_ids, o_ids.numel(), o_off, cfg.n_bags, o_grad, t)
-            want = cpu.lookup_pool(s.ids, s.offsets)
             cpu.apply_grads(o.ids, o.offsets, o.grad_pooled, t)
         else:
             mb.mono_apply_grads_host(a.handle, ids, ids.numel(), off, cfg.n_bags, grad, t)
-            want = cpu.lookup_pool(s.ids, s.offsets)
             cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t)
         if t % 2:        # every other step the host reads the result before it goes on
             mb.mono_fence(a.handle)
