@@ -402,7 +402,9 @@ def run_ours(args):
     gg.manual_seed(cfg.seed)
     # every step has its own ids and offsets; its gradients too, except in a long drift run, where
     # the steps take turns on a ring of gradient tensors that is still several times larger than L2
-    n_grads = min(W + K + KT, 16) if drift else W + K + KT
+    # (and in any run of more than 48 steps: a ring of 48 gradient tensors, 20 GB on `large`, keeps long runs within
+    # device memory; consecutive steps still never share one)
+    n_grads = min(W + K + KT, 16) if drift else min(W + K + KT, 48)
     grads = [torch.randn((cfg.n_bags, cfg.dim), device=dev, generator=gg).mul_(cfg.grad_std) for _ in range(n_grads)]
     dev_batches, host_batches = [], {}
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
