@@ -110,11 +110,15 @@ def _sampled_view(s, sample_ids, dim):
 
 def test_drift_config_full_size_sampled_parity():
     """The concept-drift configuration at its full size, from an empty table, across five re-keyings of
-    the ID universe and past one TTL, so that insertions, admissions and expiries all occur."""
+    the ID universe and past one TTL, so that insertions, admissions and expiries all occur.  Two tables
+    take the same stream: the configured one (2^26 rows, which this stream fills to a tenth) and the one
+    sized for the stream (`drift_dense`: both stores near load 0.9, where insertions displace other
+    keys).  What a table holds does not depend on its size, so one oracle checks both."""
     free, _ = torch.cuda.mem_get_info()
     if free < 40 * (1 << 30):
         pytest.skip("needs ~30 GB of free device memory")
-    cfg = wl.CONFIGS["drift"]
+    cfg, dense = wl.CONFIGS["drift"], wl.CONFIGS["drift_dense"]
+    assert wl.scaled(dense, name=cfg.name, capacity=cfg.capacity, key_cells=cfg.key_cells) == cfg    # same stream
     n_steps, sweep_every = cfg.ttl + cfg.drift_period + 12, 20
     stream = wl.Stream(cfg)
     rng = np.random.default_rng(17)
@@ -128,43 +132,57 @@ def test_drift_config_full_size_sampled_parity():
             picks.append(s.ids[s.offsets[b]:s.offsets[b + 1]])
     sample_ids = np.unique(np.concatenate(picks))
 
-    gpu = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, key_cells=cfg.key_cells,
-                       max_ids=int(cfg.n_bags * 5.6), max_bags=cfg.n_bags, **_kw(cfg))
+    gpus = [mb.MonoTable(c.capacity, c.dim, c.filter_threshold, c.ttl, key_cells=c.key_cells,
+                         max_ids=int(c.n_bags * 5.6), max_bags=c.n_bags, **_kw(c)) for c in (cfg, dense)]
     cpu = mo.OracleTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, **_kw(cfg))
-    out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
-    h = gpu.handle
+    outs = [torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda") for _ in gpus]
     n_pure = 0
     for t, (s, view) in enumerate(_steps_ahead(stream, 0, n_steps, lambda s: _sampled_view(s, sample_ids, cfg.dim))):
         ids, off, grad = _dev(s)
         o_ids, o_off, o_grad, bags, pure = view
-        mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
-        mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        for gpu, out in zip(gpus, outs):
+            mb.mono_prepare_push(gpu.handle, ids, ids.numel(), off, cfg.n_bags)
+            mb.mono_lookup_pool(gpu.handle, ids, ids.numel(), off, cfg.n_bags, out)
         if t % 10 == 0 or t >= n_steps - 3:
             want = cpu.lookup_pool(o_ids, o_off)[pure]
-            got = out[torch.from_numpy(bags[pure]).cuda()].cpu().numpy()
-            assert_vectors_close(got, want, f"step {t}: pooled output of sampled bags")
+            for k, out in enumerate(outs):
+                got = out[torch.from_numpy(bags[pure]).cuda()].cpu().numpy()
+                assert_vectors_close(got, want, f"table {k} step {t}: pooled output of sampled bags")
             n_pure += int(pure.sum())
-        mb.mono_apply_grads(h, ids, ids.numel(), off, cfg.n_bags, grad, t)
+        for gpu in gpus:
+            mb.mono_apply_grads(gpu.handle, ids, ids.numel(), off, cfg.n_bags, grad, t)
         assert cpu.apply_grads(o_ids, o_off, o_grad, t) == 0
         if t % sweep_every == sweep_every - 1:
-            gpu.expire(t)
+            for gpu in gpus:
+                gpu.expire(t)
             cpu.expire(t)
         if t % 60 == 59 or t == n_steps - 1:
-            g, o = gpu.probe(sample_ids), cpu.probe(sample_ids)
-            assert (g["resident"] == o["resident"]).all() and (g["count"] == o["count"]).all(), f"step {t}"
-            assert (g["last_seen"] == o["last_seen"]).all(), f"step {t}"
-            assert_vectors_close(g["w"], o["w"], f"step {t}: rows of sampled IDs")
-            assert_vectors_close(g["acc"], o["acc"], f"step {t}: accumulators of sampled IDs")
+            o = cpu.probe(sample_ids)
+            for k, gpu in enumerate(gpus):
+                g = gpu.probe(sample_ids)
+                assert (g["resident"] == o["resident"]).all() and (g["count"] == o["count"]).all(), f"table {k} step {t}"
+                assert (g["last_seen"] == o["last_seen"]).all(), f"table {k} step {t}"
+                assert_vectors_close(g["w"], o["w"], f"table {k} step {t}: rows of sampled IDs")
+                assert_vectors_close(g["acc"], o["acc"], f"table {k} step {t}: accumulators of sampled IDs")
         del ids, off, grad
-    st = gpu.status()
-    assert st["error_bits"] == 0 and st["scratch_reallocs"] == 0
     assert n_pure > 500
-    # insertions, admissions and expiries all took place, on the GPU and among the sampled IDs
-    assert st["n_inserted_total"] > st["n_tracked"] > 1000000 and st["n_expired_total"] > 1000000
-    assert st["n_admitted_total"] > st["n_resident"] > 0
     o = cpu.probe(sample_ids, rows=False)
     assert (o["count"] == 0).sum() > 50 and o["resident"].sum() > 50        # some sampled IDs expired, some own a row
-    assert_audit_ok(gpu)
+    stats = [gpu.status() for gpu in gpus]
+    for k, (gpu, st) in enumerate(zip(gpus, stats)):
+        assert st["error_bits"] == 0 and st["scratch_reallocs"] == 0, f"table {k}: {st}"
+        # insertions, admissions and expiries all took place
+        assert st["n_inserted_total"] > st["n_tracked"] > 1000000 and st["n_expired_total"] > 1000000
+        assert st["n_admitted_total"] > st["n_resident"] > 0
+        assert_audit_ok(gpu, f"table {k}")
+    # the two tables hold the same IDs and rows ...
+    for key in ("n_tracked", "n_resident", "n_inserted_total", "n_expired_total", "n_admitted_total"):
+        assert stats[0][key] == stats[1][key], key
+    # ... the small one under displacement: loads near 0.9, chains, no key lost
+    st = stats[1]
+    assert st["n_resident"] > 0.7 * dense.capacity and st["n_tracked"] > 0.8 * dense.key_cells
+    assert st["max_chain"] > 0 and st["n_evictions_total"] > 1000000 and st["n_keys_dropped"] == 0
+    assert stats[0]["n_evictions_total"] < st["n_evictions_total"]
 
 
 def test_eight_tables_full_size_grouped_calls_sampled_parity():
