@@ -280,12 +280,13 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- our arm
 
-def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
+def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True, expired=0):
     """Bytes the method itself must move per step, per kernel (each distinct datum once per
     phase; 32-byte sector as the smallest random access).  n occurrences, b bags, u distinct
     IDs, ur of them with a row, ur1 of those occurring once in the batch, unew new IDs.
     prepared: the batch was announced, so the key store is read once per distinct ID ahead of
-    the lookup instead of once per occurrence inside it."""
+    the lookup instead of once per occurrence inside it.  sweep_cells: key cells the step's slice
+    of the expiry sweep covers, expired: entries it removes."""
     per_kernel = {
         "probe_rows": 0,
         # offsets, one 8-byte record per occurrence (the ID, or its place in the grouping), each distinct row once, out
@@ -302,7 +303,8 @@ def algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=0, prepared=True):
         "reduce_adagrad": 16 * d * (ur - ur1) + 4 * d * max(b - ur1, 0), "reduce_parts": 0,
         "file_segments": 0, "clear_set": 0,
         "expand_parts": 0, "order_parts": 0, "fold_partials": 0, "combine_adagrad": 0, "finish_apply": 0,
-        "expire": 16 * sweep_cells,                          # one streaming read of the swept cells
+        # the sweep's 4-byte record per 4-cell bucket in order; a removed entry's bucket read (64) and its cell cleared (32)
+        "expire": sweep_cells + 96 * expired,
     }
     return per_kernel, sum(per_kernel.values())
 
@@ -540,8 +542,9 @@ def run_ours(args):
         ur = (st_c["sum_unique_resident"] - st_b["sum_unique_resident"]) / KT
         unew = (st_c["sum_new"] - st_b["sum_new"]) / KT
         ur1 = (st_c["sum_single_resident"] - st_b["sum_single_resident"]) / KT
+        gone = (st_c["n_expired_total"] - st_b["n_expired_total"]) / KT
         alg_kernel, alg_total = algorithmic_bytes(n, cfg.n_bags, u, ur, ur1, unew, d, cfg.key_cells // S if S > 0 else 0,
-                                                  prepared=args.prepare)
+                                                  prepared=args.prepare, expired=gone)
         per_kernel = {}
         for name, v in tim["kernels"].items():
             if v["launches"] and name in KERNEL_GROUP:
@@ -783,7 +786,7 @@ def run_multi(args):
         u, ur = b["sum_unique"] - a["sum_unique"], b["sum_unique_resident"] - a["sum_unique_resident"]
         ur1, unew = b["sum_single_resident"] - a["sum_single_resident"], b["sum_new"] - a["sum_new"]
         alg += algorithmic_bytes(n, cfg.n_bags * K, u, ur, ur1, unew, cfg.dim, K * cfg.key_cells // S if S > 0 else 0,
-                                 prepared=args.prepare)[1]
+                                 prepared=args.prepare, expired=b["n_expired_total"] - a["n_expired_total"])[1]
     if rank == 0:
         peak, peak_kind = measured_peaks()
         achieved = alg / (ms * 1e-3) / 1e9

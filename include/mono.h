@@ -163,7 +163,8 @@ typedef struct {
   uint64_t free_rows;
   uint64_t unaccounted_rows;    /* rows neither owned nor free */
   uint32_t ok;                  /* 1 iff all of the above are consistent with the counters */
-  uint32_t pad_;
+  uint32_t behind_records;      /* entries last seen before the time their bucket's sweep record holds
+                                   (saturating); the expiry sweep would not find them */
 } mono_audit_t;
 
 /*
@@ -178,7 +179,8 @@ typedef struct {
  *  opt               HOST, may be NULL for defaults (lr 0.05, eps 1e-8, zeros)
  *  cuda_stream       a cudaStream_t (NULL = the default stream) on the current device
  * Allocates capacity * dim * 8 bytes of rows+accumulators, key_cells * 16 bytes
- * of keys, capacity * 4 bytes of free-row bookkeeping and the scratch.
+ * of keys, key_cells bytes of sweep records (below, mono_expire), capacity * 4
+ * bytes of free-row bookkeeping and the scratch.
  */
 int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim,
                       uint32_t filter_threshold, uint32_t ttl, const mono_opt* opt,
@@ -236,6 +238,10 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids,
  * without a row, for which  now - last_seen > ttl; free its row and forget its
  * count.  Expiry takes effect only here; a stale ID that re-occurs before a
  * sweep is refreshed.  No-op when ttl == 0.
+ * The sweep does not read every cell: beside each 4-cell bucket the table keeps a
+ * time that is not later than the last_seen of any entry in it, reads those (4
+ * bytes per bucket) and opens only the buckets where that time is past the ttl.
+ * The set of IDs removed is that of a sweep over all cells.
  */
 int mono_expire(mono_table* t, int64_t now);
 
@@ -293,7 +299,7 @@ int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const ui
 
 /*
  * Incremental form of mono_expire: sweeps slice `slice` of `n_slices` equal parts of the key
- * store (the last slice also covers the overflow stash), so that the cost of a full sweep can
+ * store (multiples of 16 cells; the last slice also covers the remainder and the overflow stash), so that the cost of a full sweep can
  * be spread over n_slices training steps.  Calling it for slice = 0 .. n_slices-1 with the
  * same `now` (and no other call in between) has exactly the effect of mono_expire(now).
  * 1 <= n_slices <= 65536, slice < n_slices.  With the probabilistic filter, slice 0 is the

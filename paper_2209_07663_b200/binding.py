@@ -64,7 +64,7 @@ class mono_audit_t(ctypes.Structure):
     _fields_ = [("occupied_cells", ctypes.c_uint64), ("misplaced", ctypes.c_uint64),
                 ("duplicate_keys", ctypes.c_uint64), ("resident_cells", ctypes.c_uint64),
                 ("bad_rows", ctypes.c_uint64), ("shared_rows", ctypes.c_uint64), ("free_rows", ctypes.c_uint64),
-                ("unaccounted_rows", ctypes.c_uint64), ("ok", ctypes.c_uint32), ("pad_", ctypes.c_uint32)]
+                ("unaccounted_rows", ctypes.c_uint64), ("ok", ctypes.c_uint32), ("behind_records", ctypes.c_uint32)]
 
 
 class mono_kernel_time_t(ctypes.Structure):

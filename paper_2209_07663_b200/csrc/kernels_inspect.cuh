@@ -121,7 +121,7 @@ export_touched_kernel(TableView tv, unsigned long long n_cells, unsigned long lo
 
 struct AuditCounters {
   unsigned long long occupied, misplaced, duplicate_keys, resident_cells, bad_rows, shared_rows, free_rows,
-      unaccounted_rows;
+      unaccounted_rows, behind_records;
 };
 
 // row_marks: one bit per row, zeroed by the caller.
@@ -141,6 +141,7 @@ audit_cells_kernel(TableView tv, unsigned long long n_cells, unsigned int* row_m
     } else {
       const unsigned long long b = i / kCellsPerBucket;
       if (b != tv.bucket0(c.key) && b != tv.bucket1(c.key)) atomicAdd(&out->misplaced, 1ull);
+      if (meta_time(c.meta) < tv.oldest[b]) atomicAdd(&out->behind_records, 1ull);   // the sweep could pass this entry by
     }
     // the key must occur exactly once among its two buckets and the stash
     unsigned copies = 0;

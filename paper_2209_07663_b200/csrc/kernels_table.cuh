@@ -230,6 +230,16 @@ table_update_kernel(TableView tv, Work wk, uint32_t now) {
   table_update_body<MODE>(tv, wk, now, blockIdx.x, gridDim.x);
 }
 
+// An entry whose metadata is `meta` has just been written into a cell of bucket `bkt`: the
+// bucket's record of its oldest stamp may not stay above that entry's.  (Entries that leave a
+// bucket, and stamps that are renewed, leave the record as it is: it only has to be a lower
+// bound, and the sweep makes it exact again whenever it visits the bucket.)  `rec` is the
+// record as read before the write; records only fall while entries are being inserted, so a
+// value read earlier is at or above the present one and the test errs on the safe side.
+__device__ inline void note_stamp(const TableView& tv, unsigned long long bkt, unsigned long long meta, uint32_t rec) {
+  if (rec > meta_time(meta)) atomicMin(tv.oldest + bkt, meta_time(meta));
+}
+
 // Put `item` (a key that is in no cell) into the key store.  Lock-free against
 // other inserters: an empty cell is claimed, and an occupant displaced, with a
 // single 16-byte atomic, so every entry is at all times either in exactly one
@@ -246,6 +256,7 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
   bool placed = false;
   for (;;) {
     Cell* base = tv.cells + bkt * kCellsPerBucket;
+    const uint32_t rec = __ldcg(tv.oldest + bkt);
     for (uint32_t c = 0; c < kCellsPerBucket && !placed; ++c) {
       Cell* p = base + ((c + first) & 3u);
       if (*reinterpret_cast<volatile unsigned long long*>(&p->key) == kEmptyKey) {
@@ -253,7 +264,7 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
         placed = old.key == kEmptyKey;
       }
     }
-    if (placed) break;
+    if (placed) { note_stamp(tv, bkt, item.meta, rec); break; }
     if (chain == 0) {
       // a new ID may take an empty cell of its second bucket before displacing anyone
       const unsigned long long alt = h1 & tv.bucket_mask;
@@ -265,12 +276,13 @@ __device__ inline void cuckoo_insert(const TableView& tv, Cell item) {
           placed = old.key == kEmptyKey;
         }
       }
-      if (placed) break;
+      if (placed) { note_stamp(tv, alt, item.meta, __ldcg(tv.oldest + alt)); break; }
     }
     if (chain >= kMaxChain) break;
     ++chain;
     rnd = rnd * 1664525u + 1013904223u;
     const Cell old = atomicExch(base + (rnd >> 30), item);
+    note_stamp(tv, bkt, item.meta, rec);
     if (old.key == kEmptyKey) { placed = true; break; }
     item = old;
     h0 = tv.hash0(item.key);
@@ -454,45 +466,102 @@ __global__ void finish_apply_kernel(DevState* st, uint32_t* win_count, int commi
 // store; a cell whose ID has been inactive for longer than ttl is emptied and
 // its row, if it has one, goes back on the free list (one counter update per
 // warp and round).
-__device__ inline void expire_body(const TableView& tv, unsigned long long n_cells, unsigned long long first,
-                                   unsigned long long last, long long now, uint32_t vblock, uint32_t vgrid) {
-  // sweeps cells [first, last) of the sequence "key store, then stash" (total n_cells + kStashCells)
-  constexpr int kDepth = 4;                                                // independent loads per thread and round
-  const unsigned long long stride = (unsigned long long)vgrid * blockDim.x;
-  const unsigned long long rounds = (last - first + stride * kDepth - 1) / (stride * kDepth);  // same for every thread
+// Rows of expired entries go back on the free stack: one counter update per warp.  Every lane
+// of the warp calls this.
+__device__ inline void warp_free_row(const TableView& tv, bool frees_row, uint32_t row, int lane) {
+  const unsigned mask = __ballot_sync(0xFFFFFFFFu, frees_row);
+  if (mask == 0) return;
+  unsigned long long pos = 0;
+  const int leader = __ffs(mask) - 1;
+  if (lane == leader)
+    pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)__popc(mask));
+  pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
+  const unsigned long long at = pos + __popc(mask & ((1u << lane) - 1u));
+  if (frees_row && MONO_INDEX_OK(&tv.st->error_bits, at, tv.capacity)) tv.free_rows[at] = row;
+}
+
+// Sweep of buckets [first_bkt, last_bkt) of the key store, and of the stash if `with_stash`.
+// The sweep reads, per bucket, the record of its oldest stamp (4 bytes, in order) and opens only
+// the buckets in which that stamp is past the expire time: an entry that has to go has a stamp at
+// or above its bucket's record, so its bucket is always opened, and the outcome is that of a sweep
+// over every cell.  A bucket that is opened gets an exact record again.  Nothing else touches the
+// key store while this runs.
+// A block lists the buckets to open in shared memory, then takes them one cell per thread, so that
+// all their loads are in flight together and the four lanes of a bucket read its 64 bytes as one.
+constexpr int kSweepDepth = 2;                                             // 16-byte loads of four records per thread and round
+__device__ inline void expire_body(const TableView& tv, unsigned long long first_bkt, unsigned long long last_bkt,
+                                   bool with_stash, long long now, uint32_t vblock, uint32_t vgrid) {
+  // first_bkt and last_bkt are multiples of four
+  __shared__ unsigned long long open_list[256 * kSweepDepth * 4];
+  __shared__ unsigned int n_open;
+  const unsigned long long stride = (unsigned long long)vgrid * blockDim.x * 4u;
+  const unsigned long long rounds = (last_bkt - first_bkt + stride * kSweepDepth - 1) / (stride * kSweepDepth);  // same for every thread
   const int lane = threadIdx.x & 31;
+  const long long ttl = (long long)tv.ttl;
   unsigned int n_gone = 0, n_rows = 0;
   for (unsigned long long r = 0; r < rounds; ++r) {
-    const unsigned long long i0 = first + r * kDepth * stride + (unsigned long long)vblock * blockDim.x + threadIdx.x;
-    Cell* p[kDepth];
-    ulonglong2 v[kDepth];
+    if (threadIdx.x == 0) n_open = 0;
+    __syncthreads();
+    const unsigned long long b0 = first_bkt + r * kSweepDepth * stride + ((unsigned long long)vblock * blockDim.x + threadIdx.x) * 4u;
+    uint4 rec[kSweepDepth];
 #pragma unroll
-    for (int k = 0; k < kDepth; ++k) {
-      const unsigned long long i = i0 + k * stride;
-      p[k] = i < last ? (i < n_cells ? tv.cells + i : tv.stash + (i - n_cells)) : nullptr;
-      v[k].x = kEmptyKey; v[k].y = 0ull;
-      if (p[k]) v[k] = *reinterpret_cast<const ulonglong2*>(p[k]);
+    for (int k = 0; k < kSweepDepth; ++k) {
+      const unsigned long long b = b0 + k * stride;
+      rec[k] = make_uint4(kNoStamp, kNoStamp, kNoStamp, kNoStamp);
+      if (b < last_bkt) rec[k] = *reinterpret_cast<const uint4*>(tv.oldest + b);
     }
 #pragma unroll
-    for (int k = 0; k < kDepth; ++k) {
+    for (int k = 0; k < kSweepDepth; ++k) {
+      const uint32_t four[4] = {rec[k].x, rec[k].y, rec[k].z, rec[k].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (four[q] != kNoStamp && now - (long long)four[q] > ttl) open_list[atomicAdd(&n_open, 1u)] = b0 + k * stride + q;
+    }
+    __syncthreads();
+    const unsigned int n_cells_open = n_open * kCellsPerBucket;
+    for (unsigned int base = 0; base < n_cells_open; base += blockDim.x) {      // block-uniform
+      const unsigned int idx = base + threadIdx.x;
+      const bool valid = idx < n_cells_open;
+      const unsigned long long b = valid ? open_list[idx / kCellsPerBucket] : 0ull;
+      ulonglong2* cell = reinterpret_cast<ulonglong2*>(tv.cells + b * kCellsPerBucket + (idx % kCellsPerBucket));
+      ulonglong2 v; v.x = kEmptyKey; v.y = 0ull;
+      if (valid) v = *cell;
+      bool frees_row = false;
+      uint32_t row = 0, kept = kNoStamp;
+      if (v.x != kEmptyKey) {
+        const uint32_t seen = meta_time(v.y);
+        if (now - (long long)seen > ttl) {
+          ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+          *cell = e;
+          ++n_gone;
+          if (meta_resident(v.y)) { frees_row = true; row = meta_row(v.y); ++n_rows; }
+        } else {
+          kept = seen;
+        }
+      }
+      // the oldest stamp that stays in the bucket: its four cells sit in four adjacent lanes
+      kept = min(kept, __shfl_xor_sync(0xFFFFFFFFu, kept, 1));
+      kept = min(kept, __shfl_xor_sync(0xFFFFFFFFu, kept, 2));
+      if (valid && (idx % kCellsPerBucket) == 0) tv.oldest[b] = kept;
+      warp_free_row(tv, frees_row, row, lane);
+    }
+    __syncthreads();                                       // everyone has read n_open before the next round resets it
+  }
+  if (with_stash) {
+    for (uint32_t base = vblock * blockDim.x; base < kStashCells; base += vgrid * blockDim.x) {   // block-uniform
+      const uint32_t i = base + threadIdx.x;
       bool frees_row = false;
       uint32_t row = 0;
-      if (v[k].x != kEmptyKey && now - (long long)meta_time(v[k].y) > (long long)tv.ttl) {
-        ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
-        *reinterpret_cast<ulonglong2*>(p[k]) = e;
-        ++n_gone;
-        if (meta_resident(v[k].y)) { frees_row = true; row = meta_row(v[k].y); ++n_rows; }
+      if (i < kStashCells) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(tv.stash + i);
+        if (v.x != kEmptyKey && now - (long long)meta_time(v.y) > ttl) {
+          ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
+          *reinterpret_cast<ulonglong2*>(tv.stash + i) = e;
+          ++n_gone;
+          if (meta_resident(v.y)) { frees_row = true; row = meta_row(v.y); ++n_rows; }
+        }
       }
-      const unsigned mask = __ballot_sync(0xFFFFFFFFu, frees_row);
-      if (mask) {
-        unsigned long long pos = 0;
-        const int leader = __ffs(mask) - 1;
-        if (lane == leader)
-          pos = atomicAdd(reinterpret_cast<unsigned long long*>(&tv.st->free_top), (unsigned long long)__popc(mask));
-        pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
-        const unsigned long long at = pos + __popc(mask & ((1u << lane) - 1u));
-        if (frees_row && MONO_INDEX_OK(&tv.st->error_bits, at, tv.capacity)) tv.free_rows[at] = row;
-      }
+      warp_free_row(tv, frees_row, row, lane);
     }
   }
   for (int o = 16; o > 0; o >>= 1) {
@@ -506,9 +575,8 @@ __device__ inline void expire_body(const TableView& tv, unsigned long long n_cel
   }
 }
 __global__ void __launch_bounds__(256)
-expire_kernel(TableView tv, unsigned long long n_cells, unsigned long long first, unsigned long long last,
-              long long now) {
-  expire_body(tv, n_cells, first, last, now, blockIdx.x, gridDim.x);
+expire_kernel(TableView tv, unsigned long long first_bkt, unsigned long long last_bkt, int with_stash, long long now) {
+  expire_body(tv, first_bkt, last_bkt, with_stash != 0, now, blockIdx.x, gridDim.x);
 }
 
 // After a sweep: if the stash has become empty, probes may skip it again.
@@ -527,6 +595,7 @@ init_table_kernel(TableView tv, unsigned long long n_cells) {
   ulonglong2 e; e.x = kEmptyKey; e.y = 0ull;
   for (unsigned long long i = tid; i < n_cells; i += stride) *reinterpret_cast<ulonglong2*>(tv.cells + i) = e;
   for (unsigned long long i = tid; i < kStashCells; i += stride) *reinterpret_cast<ulonglong2*>(tv.stash + i) = e;
+  for (unsigned long long i = tid; i < n_cells / kCellsPerBucket; i += stride) tv.oldest[i] = kNoStamp;
   // rows are handed out in increasing order from a fresh table
   for (unsigned long long i = tid; i < tv.capacity; i += stride) tv.free_rows[i] = (uint32_t)(tv.capacity - 1 - i);
 }

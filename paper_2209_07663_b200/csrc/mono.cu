@@ -82,7 +82,7 @@ struct mono_table {
   // device-resident snapshot (mono_snapshot_save)
   struct {
     Cell* cells = nullptr; Cell* stash = nullptr; float* rows = nullptr; uint32_t* free_rows = nullptr;
-    DevState* st = nullptr; unsigned int* sketch = nullptr;
+    uint32_t* oldest = nullptr; DevState* st = nullptr; unsigned int* sketch = nullptr;
     uint64_t key_cells = 0; int64_t last_now = -1, sketch_epoch = 0; bool valid = false;
   } snap;
   int sm_count = 148;
@@ -154,7 +154,7 @@ void free_scratch(mono_table* t) {
 
 void free_snapshot(mono_table* t) {
   auto& sn = t->snap;
-  dev_free(sn.cells); dev_free(sn.stash); dev_free(sn.rows); dev_free(sn.free_rows); dev_free(sn.st); dev_free(sn.sketch);
+  dev_free(sn.cells); dev_free(sn.stash); dev_free(sn.oldest); dev_free(sn.rows); dev_free(sn.free_rows); dev_free(sn.st); dev_free(sn.sketch);
   sn.valid = false;
 }
 
@@ -644,6 +644,7 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   tv.init_key1 = (uint32_t)(o.seed >> 32);
   if ((rc = dev_alloc(t, &tv.cells, key_cells)) != MONO_OK) return fail(rc);
   if ((rc = dev_alloc(t, &tv.stash, kStashCells)) != MONO_OK) return fail(rc);
+  if ((rc = dev_alloc(t, &tv.oldest, key_cells / kCellsPerBucket)) != MONO_OK) return fail(rc);
   // one row more than the capacity: row index `capacity` is never handed out and stays all zero
   // (the lookup adds it for an ID that has no row)
   if ((rc = dev_alloc(t, &tv.rows, ((size_t)capacity + 1) * 2 * dim)) != MONO_OK) return fail(rc);
@@ -691,7 +692,7 @@ int mono_table_destroy(mono_table* t) {
   free_scratch(t);
   free_snapshot(t);
   free_group_scratch(t);
-  dev_free(t->tv.cells); dev_free(t->tv.stash); dev_free(t->tv.rows); dev_free(t->tv.free_rows); dev_free(t->tv.st); dev_free(t->tv.sketch);
+  dev_free(t->tv.cells); dev_free(t->tv.stash); dev_free(t->tv.oldest); dev_free(t->tv.rows); dev_free(t->tv.free_rows); dev_free(t->tv.st); dev_free(t->tv.sketch);
   delete t;
   return MONO_OK;
 }
@@ -894,13 +895,18 @@ static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_s
     CUDA_TRY(t, cudaMemsetAsync(t->tv.sketch, 0, (size_t)t->tv.sketch_depth * (t->tv.sketch_mask + 1) * sizeof(unsigned int), s));
     t->sketch_epoch = now;
   }
-  const unsigned long long total = t->key_cells + kStashCells;
-  const unsigned long long first = t->key_cells / n_slices * slice;             // key_cells is a power of two >= 64
-  const unsigned long long last = slice + 1 == n_slices ? total : t->key_cells / n_slices * (slice + 1);
-  if (last > first) {
-    unsigned long long blocks = (last - first + 255) / 256;
+  // slices are multiples of four buckets; the last one takes the remainder and the stash
+  const unsigned long long n_buckets = t->key_cells / kCellsPerBucket;           // a power of two >= 16
+  const unsigned long long per_slice = n_buckets / n_slices & ~3ull;
+  const bool is_last = slice + 1 == n_slices;
+  const unsigned long long first = per_slice * slice;
+  const unsigned long long last = is_last ? n_buckets : per_slice * (slice + 1);
+  if (last > first || is_last) {
+    const unsigned long long per_block = 256ull * 4 * kSweepDepth;               // buckets a block reads per round
+    unsigned long long blocks = (last - first + per_block - 1) / per_block;
+    if (blocks < 1) blocks = 1;
     if (blocks > (unsigned long long)grid_for(t, 8)) blocks = grid_for(t, 8);
-    LAUNCH_ON(t, s, K_EXPIRE, expire_kernel<<<(int)blocks, 256, 0, s>>>(t->tv, t->key_cells, first, last, (long long)now));
+    LAUNCH_ON(t, s, K_EXPIRE, expire_kernel<<<(int)blocks, 256, 0, s>>>(t->tv, first, last, is_last ? 1 : 0, (long long)now));
   }
   if (slice + 1 == n_slices) LAUNCH_ON(t, s, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, s>>>(t->tv));
   CUDA_TRY(t, cudaGetLastError());
@@ -1084,6 +1090,7 @@ int mono_snapshot_save(mono_table* t) {
   if (!sn.cells) {
     int rc = dev_alloc(t, &sn.cells, t->key_cells);
     if (rc == MONO_OK) rc = dev_alloc(t, &sn.stash, kStashCells);
+    if (rc == MONO_OK) rc = dev_alloc(t, &sn.oldest, t->key_cells / kCellsPerBucket);
     if (rc == MONO_OK) rc = dev_alloc(t, &sn.rows, row_floats);
     if (rc == MONO_OK) rc = dev_alloc(t, &sn.free_rows, tv.capacity);
     if (rc == MONO_OK) rc = dev_alloc(t, &sn.st, 1);
@@ -1095,6 +1102,7 @@ int mono_snapshot_save(mono_table* t) {
   const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
   CUDA_TRY(t, cudaMemcpyAsync(sn.cells, tv.cells, t->key_cells * sizeof(Cell), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(sn.stash, tv.stash, kStashCells * sizeof(Cell), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(sn.oldest, tv.oldest, t->key_cells / kCellsPerBucket * sizeof(uint32_t), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(sn.rows, tv.rows, row_floats * sizeof(float), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(sn.free_rows, tv.free_rows, tv.capacity * sizeof(uint32_t), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(sn.st, tv.st, sizeof(DevState), dd, s));
@@ -1120,6 +1128,7 @@ int mono_snapshot_restore(mono_table* t) {
   const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
   CUDA_TRY(t, cudaMemcpyAsync(tv.cells, sn.cells, t->key_cells * sizeof(Cell), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(tv.stash, sn.stash, kStashCells * sizeof(Cell), dd, s));
+  CUDA_TRY(t, cudaMemcpyAsync(tv.oldest, sn.oldest, t->key_cells / kCellsPerBucket * sizeof(uint32_t), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(tv.rows, sn.rows, row_floats * sizeof(float), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(tv.free_rows, sn.free_rows, tv.capacity * sizeof(uint32_t), dd, s));
   CUDA_TRY(t, cudaMemcpyAsync(tv.st, sn.st, sizeof(DevState), dd, s));
@@ -1234,9 +1243,11 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
   TableView fresh = t->tv;
   fresh.cells = nullptr;
   fresh.stash = nullptr;
+  fresh.oldest = nullptr;
   int rc = dev_alloc(t, &fresh.cells, new_key_cells);
   if (rc == MONO_OK) rc = dev_alloc(t, &fresh.stash, kStashCells);
-  if (rc != MONO_OK) { dev_free(fresh.cells); dev_free(fresh.stash); return rc; }
+  if (rc == MONO_OK) rc = dev_alloc(t, &fresh.oldest, new_key_cells / kCellsPerBucket);
+  if (rc != MONO_OK) { dev_free(fresh.cells); dev_free(fresh.stash); dev_free(fresh.oldest); return rc; }
   fresh.bucket_mask = new_key_cells / kCellsPerBucket - 1;
   fresh.seed0 = mix_a(new_seed + 0x1234567ull);
   fresh.seed1 = mix_b(new_seed + 0x89ABCDEFull);
@@ -1253,11 +1264,12 @@ int mono_rehash(mono_table* t, uint64_t new_key_cells, uint64_t new_seed) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(t->stream);
   if (e != cudaSuccess) {
     t->last_err = cudaGetErrorString(e);
-    dev_free(fresh.cells); dev_free(fresh.stash);
+    dev_free(fresh.cells); dev_free(fresh.stash); dev_free(fresh.oldest);
     return MONO_ERR_CUDA;
   }
   dev_free(t->tv.cells);
   dev_free(t->tv.stash);
+  dev_free(t->tv.oldest);
   t->tv = fresh;
   t->key_cells = new_key_cells;
   return MONO_OK;
@@ -1352,8 +1364,9 @@ int mono_audit(mono_table* t, mono_audit_t* host_out) {
   host_out->shared_rows = h.shared_rows;
   host_out->free_rows = h.free_rows;
   host_out->unaccounted_rows = h.unaccounted_rows;
+  host_out->behind_records = h.behind_records > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)h.behind_records;
   const bool leak_ok = h.unaccounted_rows == 0 || d.n_keys_dropped > 0;   // a dropped key may strand its row
-  host_out->ok = (h.misplaced == 0 && h.duplicate_keys == 0 && h.bad_rows == 0 && h.shared_rows == 0 && leak_ok &&
+  host_out->ok = (h.misplaced == 0 && h.duplicate_keys == 0 && h.behind_records == 0 && h.bad_rows == 0 && h.shared_rows == 0 && leak_ok &&
                   h.occupied == d.n_tracked && h.resident_cells == d.n_resident &&
                   h.resident_cells + h.free_rows + h.unaccounted_rows == t->tv.capacity)
                      ? 1u : 0u;

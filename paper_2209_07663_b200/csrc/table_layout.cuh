@@ -35,6 +35,7 @@ constexpr uint32_t kRowMask = 0x3FFFFFFFu;
 constexpr uint32_t kCellsPerBucket = 4;
 constexpr uint32_t kStashCells = 256;      // overflow area scanned only when non-empty
 constexpr uint32_t kMaxChain = 96;         // bound on one insertion's displacement chain
+constexpr uint32_t kNoStamp = 0xFFFFFFFFu; // a bucket's record of its oldest stamp: nothing was put there since the sweep found it empty
 
 // Per-unique "row word" passed from the table phases to the Adagrad phase.
 constexpr uint32_t kNoRow = 0xFFFFFFFFu;
@@ -127,6 +128,8 @@ struct DevState {
 struct TableView {
   Cell* cells;                 // [n_buckets * 4]
   Cell* stash;                 // [kStashCells]
+  uint32_t* oldest;            // [n_buckets]: no entry of the bucket was last seen before this time (kNoStamp:
+                               // none can be there); what the expiry sweep reads instead of the cells
   float* rows;                 // [capacity][2][dim]: weights then accumulator
   uint32_t* free_rows;         // [capacity]
   DevState* st;

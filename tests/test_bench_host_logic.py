@@ -56,15 +56,15 @@ def test_clock_sampler_reports_slowdowns(monkeypatch):
 
 def test_algorithmic_bytes_adds_up():
     n, b, u, ur, ur1, unew, d = 1000, 600, 400, 300, 250, 50, 64
-    per, total = bench.algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=1 << 10)
+    per, total = bench.algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=1 << 10, expired=7)
     assert total == sum(per.values())
     assert per["dedup_tile"] == 32 * n and per["table_lookup"] == 32 * u and per["table_update"] == 64 * u
     assert per["gather_pool"] == 8 * (b + 1) + 8 * n + 4 * d * ur + 4 * d * b
     # a batch that was not announced pays one key-store sector per occurrence inside the lookup instead
-    per_u, total_u = bench.algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=1 << 10, prepared=False)
+    per_u, total_u = bench.algorithmic_bytes(n, b, u, ur, ur1, unew, d, sweep_cells=1 << 10, prepared=False, expired=7)
     assert per_u["table_lookup"] == 0 and per_u["gather_pool"] == per["gather_pool"] + 32 * n
     assert total_u - total == 32 * n - 32 * u
     # the Adagrad phase reads every gradient row once and reads and writes row + accumulator of every ID with a row
     assert per["update_singletons"] + per["reduce_adagrad"] == 16 * d * ur + 4 * d * b
-    assert per["expire"] == 16 << 10
+    assert per["expire"] == 4 * (1 << 8) + 7 * (64 + 32)      # a record per 4-cell bucket, a bucket and a cell per removed entry
     assert set(bench.KERNEL_GROUP) <= set(per) | {"finish_apply"}

@@ -694,6 +694,65 @@ def test_apply_grads_inserts_at_high_load():
     assert st["n_evictions_total"] > 0          # the displacement path really ran
 
 
+def test_sweep_finds_old_entries_that_displacements_moved():
+    """A key store kept near load 0.85 by steady churn: new IDs displace entries of every age into
+    buckets whose other entries are younger, and the sweep, which opens only the buckets its
+    per-bucket record of the oldest stamp points at, has to remove exactly what a sweep over
+    every cell removes -- the oracle's set -- at every sweep, whole or in slices."""
+    cells, ttl = 1 << 14, 9
+    gpu = mb.MonoTable(256, 4, 1000, ttl, key_cells=cells, seed=5)
+    cpu = mo.OracleTable(256, 4, 1000, ttl, seed=5)
+    per_call = int(cells * 0.075) // 2 * 2               # eleven calls' worth of IDs stay alive (a tenth renewed): load 0.85
+    rng = np.random.default_rng(3)
+    evictions = 0
+    for t in range(40):
+        fresh = wl.splitmix64(np.arange(t * per_call, (t + 1) * per_call, dtype=np.uint64))
+        # a tenth of the IDs of the last ten calls come back, which renews their stamps
+        back = wl.splitmix64(rng.integers(max(0, t - 10) * per_call, max(1, t * per_call), per_call // 10 * 2).astype(np.uint64))
+        ids = np.concatenate([fresh, back])
+        off = np.arange(0, ids.size + 1, 2, dtype=np.int64)
+        grad = np.zeros((off.size - 1, 4), f32)
+        gpu.apply_grads(ids, off, grad, t)
+        assert cpu.apply_grads(ids, off, grad, t) == 0
+        if t % 3 == 0:
+            gpu.expire(t)
+        else:
+            for k in range(7):
+                mb.mono_expire_slice(gpu.handle, t, k, 7)
+        cpu.expire(t)
+        st = gpu.status()
+        assert st["error_bits"] == 0 and st["n_keys_dropped"] == 0, f"step {t}: {st}"
+        assert_state_equal(gpu, cpu, f"step {t}")
+        a = assert_audit_ok(gpu, f"step {t}")
+        assert a["behind_records"] == 0
+    st = gpu.status()
+    assert st["error_bits"] == 0 and st["n_keys_dropped"] == 0
+    assert st["n_tracked"] > 0.8 * cells and st["n_expired_total"] > 2 * cells and st["n_evictions_total"] > 1000, st
+
+
+def test_sweep_finds_imported_entries_older_than_their_buckets():
+    """Entries imported with an old last_seen land in buckets whose record was set by recent ones."""
+    ttl = 5
+    gpu = mb.MonoTable(64, 4, 1000, ttl, key_cells=1 << 9, seed=1)
+    cpu = mo.OracleTable(64, 4, 1000, ttl, seed=1)
+    recent = wl.splitmix64(np.arange(0, 150, dtype=np.uint64))
+    off = np.arange(0, recent.size + 1, 2, dtype=np.int64)
+    grad = np.zeros((off.size - 1, 4), f32)
+    gpu.apply_grads(recent, off, grad, 100)
+    cpu.apply_grads(recent, off, grad, 100)
+    gpu.expire(100); cpu.expire(100)                     # every occupied bucket's record is exact: 100
+    old = wl.splitmix64(np.arange(1000, 1060, dtype=np.uint64))
+    seen = np.arange(60, dtype=np.int64) + 60             # 60 .. 119: some stale at 103, some not
+    for side in (gpu, cpu):
+        side.import_entries(old, np.ones(60, np.uint32), seen, np.zeros(60, np.uint8), None, None)
+    assert_audit_ok(gpu)
+    gpu.expire(103); cpu.expire(103)
+    assert_state_equal(gpu, cpu, "after the sweep")
+    left = set(gpu.export(rows=False)["ids"].tolist())
+    assert left == set(recent.tolist()) | set(old[seen >= 98].tolist())
+    assert_audit_ok(gpu)
+
+
 # ---------------------------------------------------------------- overflow conditions (flagged, never fatal)
 
 def test_rows_full_is_flagged_and_table_stays_consistent():
