@@ -78,7 +78,7 @@ __device__ inline void clear_primary_body(const Work& wk, uint32_t vblock, uint3
     *reinterpret_cast<ulonglong2*>(wk.bset + i) = e;
 }
 __global__ void __launch_bounds__(256)
-clear_primary_kernel(Work wk) { clear_primary_body(wk, blockIdx.x, gridDim.x); }
+clear_primary_kernel(Work wk) { after_previous_kernel(); clear_primary_body(wk, blockIdx.x, gridDim.x); }
 
 // Sum of grad rows of bags bag_of_sorted[begin .. end) for the NV column
 // vectors this lane owns.  Eight independent row loads in flight per step.
@@ -149,7 +149,7 @@ __device__ inline void file_segments_body(const Work& wk, long long n_ids, long 
   }
 }
 __global__ void __launch_bounds__(256)
-file_segments_kernel(Work wk, long long n_ids, long long n_bags, uint32_t* __restrict__ occ_row, uint32_t zero_row) {
+file_segments_kernel(Work wk, long long n_ids, long long n_bags, uint32_t* __restrict__ occ_row, uint32_t zero_row) { after_previous_kernel();
   file_segments_body(wk, n_ids, n_bags, occ_row, zero_row, blockIdx.x, gridDim.x);
 }
 
@@ -220,7 +220,7 @@ __device__ inline void update_singletons_body(const TableView& tv, const Work& w
 }
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) {
+update_singletons_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags) { after_previous_kernel();
   update_singletons_body<G, NV>(tv, wk, grad, n_bags, blockIdx.x, gridDim.x);
 }
 
@@ -291,7 +291,7 @@ __device__ inline void reduce_adagrad_body(const TableView& tv, const Work& wk, 
 
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags, int which) {
+reduce_adagrad_kernel(TableView tv, Work wk, const float* __restrict__ grad, long long n_bags, int which) { after_previous_kernel();
   reduce_adagrad_body<G, NV>(tv, wk, grad, n_bags, which, blockIdx.x, gridDim.x);
 }
 
@@ -338,7 +338,7 @@ __device__ inline void fold_partials_body(const TableView& tv, const Work& wk, u
 }
 
 __global__ void __launch_bounds__(256)
-fold_partials_kernel(TableView tv, Work wk) { fold_partials_body(tv, wk, blockIdx.x, gridDim.x); }
+fold_partials_kernel(TableView tv, Work wk) { after_previous_kernel(); fold_partials_body(tv, wk, blockIdx.x, gridDim.x); }
 
 // One block per long ID: the block's threads split into slices of the parts
 // (or, for a very long segment, of the group sums fold_partials_kernel left),
@@ -392,6 +392,6 @@ __device__ inline void combine_adagrad_body(const TableView& tv, const Work& wk,
 }
 
 __global__ void __launch_bounds__(kCombineThreads)
-combine_adagrad_kernel(TableView tv, Work wk) { combine_adagrad_body(tv, wk, blockIdx.x, gridDim.x); }
+combine_adagrad_kernel(TableView tv, Work wk) { after_previous_kernel(); combine_adagrad_body(tv, wk, blockIdx.x, gridDim.x); }
 
 }  // namespace mono

@@ -100,7 +100,7 @@ __device__ inline void fill_occ_bag_body(const long long* __restrict__ offsets, 
 }
 __global__ void __launch_bounds__(256)
 fill_occ_bag_kernel(const long long* __restrict__ offsets, long long n_bags, long long n_ids,
-                    uint32_t* __restrict__ occ_bag, DevState* st) {
+                    uint32_t* __restrict__ occ_bag, DevState* st) { after_previous_kernel();
   fill_occ_bag_body(offsets, n_bags, n_ids, occ_bag, st, blockIdx.x, gridDim.x);
 }
 
@@ -285,7 +285,7 @@ __device__ inline void dedup_tile_body(const Work& wk, const unsigned long long*
 __global__ void __launch_bounds__(kTileThreads, 8)
 dedup_tile_kernel(Work wk, const unsigned long long* __restrict__ ids, long long n_ids,
                   const long long* __restrict__ offsets, long long n_bags, DevState* st,
-                  unsigned long long seed) {
+                  unsigned long long seed) { after_previous_kernel();
   dedup_tile_body(wk, ids, n_ids, offsets, n_bags, st, seed, blockIdx.x);
 }
 

@@ -95,7 +95,7 @@ __device__ inline void probe_rows_body(const TableView& tv, const unsigned long 
 }
 __global__ void __launch_bounds__(256)
 probe_rows_kernel(TableView tv, const unsigned long long* __restrict__ ids, long long n_ids,
-                  uint32_t* __restrict__ occ_row) {
+                  uint32_t* __restrict__ occ_row) { after_previous_kernel();
   probe_rows_body(tv, ids, n_ids, occ_row, blockIdx.x, gridDim.x);
 }
 
@@ -181,7 +181,7 @@ __device__ inline void gather_pool_body(const TableView& tv, const uint32_t* __r
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 gather_pool_kernel(TableView tv, const uint32_t* __restrict__ occ_row, long long n_ids,
-                   const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out) {
+                   const long long* __restrict__ offsets, long long n_bags, float* __restrict__ out) { after_previous_kernel();
   gather_pool_body<G, NV>(tv, occ_row, n_ids, offsets, n_bags, out, blockIdx.x, gridDim.x);
 }
 

@@ -47,6 +47,7 @@ __device__ inline uint32_t find_table(const uint32_t* __restrict__ start, uint32
 }
 
 #define MONO_GROUP_PROLOGUE                                                              \
+  after_previous_kernel();                                                               \
   uint32_t vblock, vgrid;                                                                \
   const GroupItem& it = items[find_table(start, n_tables, blockIdx.x, &vblock, &vgrid)]
 
@@ -128,6 +129,7 @@ group_combine_adagrad_kernel(const GroupItem* __restrict__ items, const uint32_t
 // one block per table
 __global__ void __launch_bounds__(256)
 group_finish_apply_kernel(const GroupItem* __restrict__ items, uint32_t n_tables, int commit) {
+  after_previous_kernel();
   if (blockIdx.x < n_tables && items[blockIdx.x].active) finish_apply_body(items[blockIdx.x].tv.st, items[blockIdx.x].wk.win_count, commit);
 }
 

@@ -226,7 +226,7 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
 // 0.222 ms for look-ups shared within quads, which need twice the registers)
 template <int MODE>
 __global__ void __launch_bounds__(256, 6)
-table_update_kernel(TableView tv, Work wk, uint32_t now) {
+table_update_kernel(TableView tv, Work wk, uint32_t now) { after_previous_kernel();
   table_update_body<MODE>(tv, wk, now, blockIdx.x, gridDim.x);
 }
 
@@ -323,7 +323,7 @@ __device__ inline void sketch_add_body(const TableView& tv, const Work& wk, uint
   }
 }
 __global__ void __launch_bounds__(256)
-sketch_add_kernel(TableView tv, Work wk) { sketch_add_body(tv, wk, blockIdx.x, gridDim.x); }
+sketch_add_kernel(TableView tv, Work wk) { after_previous_kernel(); sketch_add_body(tv, wk, blockIdx.x, gridDim.x); }
 
 // Phase 3 of a push: one thread per ID that phase 2 found unknown to
 // the key store.  Exact filter: it is inserted (with a row straight away when
@@ -374,7 +374,7 @@ __device__ inline void table_insert_body(const TableView& tv, const Work& wk, ui
   }
 }
 __global__ void __launch_bounds__(256)
-table_insert_kernel(TableView tv, Work wk, uint32_t now) {
+table_insert_kernel(TableView tv, Work wk, uint32_t now) { after_previous_kernel();
   table_insert_body(tv, wk, now, blockIdx.x, gridDim.x);
 }
 
@@ -401,7 +401,7 @@ __device__ inline void expand_parts_body(const TableView& tv, const Work& wk, ui
   }
 }
 __global__ void __launch_bounds__(128)
-expand_parts_kernel(TableView tv, Work wk) { expand_parts_body(tv, wk, blockIdx.x, gridDim.x); }
+expand_parts_kernel(TableView tv, Work wk) { after_previous_kernel(); expand_parts_body(tv, wk, blockIdx.x, gridDim.x); }
 
 // The order the parts are reduced in: window by window, so that the parts in flight at any
 // time -- of different IDs -- gather gradient rows of the same stretch of bags, and a row
@@ -438,7 +438,7 @@ __device__ inline void order_parts_body(const TableView& tv, const Work& wk, uin
   }
 }
 __global__ void __launch_bounds__(kWindows)
-order_parts_kernel(TableView tv, Work wk) { order_parts_body(tv, wk, blockIdx.x, gridDim.x); }
+order_parts_kernel(TableView tv, Work wk) { after_previous_kernel(); order_parts_body(tv, wk, blockIdx.x, gridDim.x); }
 
 // End of a mono_apply_grads call: fold the per-call counters into the totals
 // (commit = 0: a grouping that was prepared but never applied is only forgotten).
@@ -458,7 +458,7 @@ __device__ inline void finish_apply_body(DevState* st, uint32_t* win_count, int 
     st->seg_cursor = 0; st->n_multi = 0; st->call_bad_offsets = 0;
   }
 }
-__global__ void finish_apply_kernel(DevState* st, uint32_t* win_count, int commit) {
+__global__ void finish_apply_kernel(DevState* st, uint32_t* win_count, int commit) { after_previous_kernel();
   if (blockIdx.x == 0) finish_apply_body(st, win_count, commit);
 }
 
@@ -575,12 +575,12 @@ __device__ inline void expire_body(const TableView& tv, unsigned long long first
   }
 }
 __global__ void __launch_bounds__(256)
-expire_kernel(TableView tv, unsigned long long first_bkt, unsigned long long last_bkt, int with_stash, long long now) {
+expire_kernel(TableView tv, unsigned long long first_bkt, unsigned long long last_bkt, int with_stash, long long now) { after_previous_kernel();
   expire_body(tv, first_bkt, last_bkt, with_stash != 0, now, blockIdx.x, gridDim.x);
 }
 
 // After a sweep: if the stash has become empty, probes may skip it again.
-__global__ void stash_trim_kernel(TableView tv) {
+__global__ void stash_trim_kernel(TableView tv) { after_previous_kernel();
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     unsigned hw = tv.st->stash_hw;
     while (hw > 0 && tv.stash[hw - 1].key == kEmptyKey) --hw;

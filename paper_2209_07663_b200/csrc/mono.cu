@@ -178,6 +178,29 @@ void launch_end(mono_table* t, int kid, cudaStream_t s) {
     t->open_event = nullptr;
   }
 }
+// Launch with programmatic stream serialisation: the launch may be prepared while the kernel
+// before it on the stream still runs; every kernel launched this way starts with
+// after_previous_kernel(), which waits for that kernel to complete.  What the stream holds
+// before it other than a kernel (a copy, an event wait) is waited for in the ordinary way.
+template <typename... P, typename... A>
+inline void launch_after(void (*kernel)(P...), unsigned grid, unsigned block, cudaStream_t s, A&&... args) {
+#ifdef MONO_PLAIN_LAUNCH
+  kernel<<<grid, block, 0, s>>>(std::forward<A>(args)...);
+#else
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(block, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
+#endif
+}
+
 // Every kernel of the hot calls is launched through this, so that launches can
 // be counted and, on request, timed one by one on the stream it runs on.
 #define LAUNCH_ON(t, s, kid, ...) do { launch_begin((t), (kid), (s)); __VA_ARGS__; launch_end((t), (kid), (s)); } while (0)
@@ -283,7 +306,7 @@ int launch_gather(mono_table* t, const uint32_t* occ_row, int64_t n_ids, const l
     int64_t blocks = (n_bags + groups_per_block - 1) / groups_per_block;
     const int64_t cap = (int64_t)grid_for(t, 8) * 8;
     if (blocks > cap) blocks = cap;
-    LAUNCH(t, K_GATHER, gather_pool_kernel<G, NV><<<(int)blocks, 256, 0, t->stream>>>(t->tv, occ_row, n_ids, off, n_bags, out));
+    LAUNCH(t, K_GATHER, launch_after(gather_pool_kernel<G, NV>, (int)blocks, 256, t->stream, t->tv, occ_row, n_ids, off, n_bags, out));
     CUDA_TRY(t, cudaGetLastError());
     return (int)MONO_OK;
   });
@@ -294,7 +317,7 @@ int launch_probe(mono_table* t, const unsigned long long* ids, int64_t n_ids, ui
   int64_t blocks = (n_ids + 255) / 256;
   const int64_t cap = (int64_t)grid_for(t, 8) * 8;
   if (blocks > cap) blocks = cap;
-  LAUNCH(t, K_PROBE, probe_rows_kernel<<<(int)blocks, 256, 0, t->stream>>>(t->tv, ids, n_ids, occ_row));
+  LAUNCH(t, K_PROBE, launch_after(probe_rows_kernel, (int)blocks, 256, t->stream, t->tv, ids, n_ids, occ_row));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
 }
@@ -305,7 +328,7 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
   if (prepared && n_ids > 0) {
     // every distinct ID of this batch was looked up when it was announced: one pass over the
     // occurrences takes the rows from the per-call set and files the bags for the push
-    LAUNCH(t, K_FILE, file_segments_kernel<<<grid_for(t, 8), 256, 0, t->stream>>>(t->wk, n_ids, n_bags, t->occ_row,
+    LAUNCH(t, K_FILE, launch_after(file_segments_kernel, grid_for(t, 8), 256, t->stream, t->wk, n_ids, n_bags, t->occ_row,
                                                                                   (uint32_t)t->tv.capacity));
     t->prep.filed = true;
   } else {
@@ -321,9 +344,9 @@ int launch_group(mono_table* t, cudaStream_t s, const unsigned long long* ids, i
                  int64_t n_bags) {
   const TableView& tv = t->tv;
   const Work& wk = t->wk;
-  LAUNCH_ON(t, s, K_FILL_BAG, fill_occ_bag_kernel<<<grid_for(t, 8), 256, 0, s>>>(off, n_bags, n_ids, wk.occ_bag, tv.st));
+  LAUNCH_ON(t, s, K_FILL_BAG, launch_after(fill_occ_bag_kernel, grid_for(t, 8), 256, s, off, n_bags, n_ids, wk.occ_bag, tv.st));
   const int tiles = (int)((n_ids + kTileIds - 1) / kTileIds);
-  LAUNCH_ON(t, s, K_DEDUP, dedup_tile_kernel<<<tiles, kTileThreads, 0, s>>>(wk, ids, n_ids, off, n_bags, tv.st,
+  LAUNCH_ON(t, s, K_DEDUP, launch_after(dedup_tile_kernel, tiles, kTileThreads, s, wk, ids, n_ids, off, n_bags, tv.st,
                                                                           tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
@@ -334,7 +357,7 @@ int launch_group(mono_table* t, cudaStream_t s, const unsigned long long* ids, i
 int launch_prepare(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off, int64_t n_bags) {
   int rc = launch_group(t, t->stream, ids, n_ids, off, n_bags);
   if (rc != MONO_OK) return rc;
-  LAUNCH(t, K_LOOKUP, table_update_kernel<kLookUp><<<grid_for(t, 8) * 4, 256, 0, t->stream>>>(t->tv, t->wk, 0u));
+  LAUNCH(t, K_LOOKUP, launch_after(table_update_kernel<kLookUp>, grid_for(t, 8) * 4, 256, t->stream, t->tv, t->wk, 0u));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
 }
@@ -352,17 +375,17 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   if (is_prepared_batch(t, ids, n_ids, off, n_bags)) {
     // grouped and looked up already; filed too, if its lookup has run
     t->prep.valid = false;
-    if (!t->prep.filed) LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags, nullptr, 0u));
-    LAUNCH(t, K_UPDATE, table_update_kernel<kCommit><<<g8 * 4, 256, 0, s>>>(tv, wk, now));
+    if (!t->prep.filed) LAUNCH(t, K_FILE, launch_after(file_segments_kernel, g8, 256, s, wk, n_ids, n_bags, nullptr, 0u));
+    LAUNCH(t, K_UPDATE, launch_after(table_update_kernel<kCommit>, g8 * 4, 256, s, tv, wk, now));
   } else {
     if ((rc0 = discard_prepared(t)) != MONO_OK) return rc0;
     if (n_ids == 0 || n_bags == 0) return MONO_OK;
     if ((rc0 = launch_group(t, s, ids, n_ids, off, n_bags)) != MONO_OK) return rc0;
-    LAUNCH(t, K_UPDATE, table_update_kernel<kLookUp | kCommit><<<g8 * 4, 256, 0, s>>>(tv, wk, now));
-    LAUNCH(t, K_FILE, file_segments_kernel<<<g8, 256, 0, s>>>(wk, n_ids, n_bags, nullptr, 0u));
+    LAUNCH(t, K_UPDATE, launch_after(table_update_kernel<kLookUp | kCommit>, g8 * 4, 256, s, tv, wk, now));
+    LAUNCH(t, K_FILE, launch_after(file_segments_kernel, g8, 256, s, wk, n_ids, n_bags, nullptr, 0u));
   }
-  if (tv.sketch_depth) LAUNCH(t, K_SKETCH, sketch_add_kernel<<<g8, 256, 0, s>>>(tv, wk));
-  LAUNCH(t, K_INSERT, table_insert_kernel<<<g8, 256, 0, s>>>(tv, wk, now));
+  if (tv.sketch_depth) LAUNCH(t, K_SKETCH, launch_after(sketch_add_kernel, g8, 256, s, tv, wk));
+  LAUNCH(t, K_INSERT, launch_after(table_insert_kernel, g8, 256, s, tv, wk, now));
   CUDA_TRY(t, cudaGetLastError());
   // the rest of the call touches rows and scratch only: a sweep may run beside it
   CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
@@ -374,32 +397,32 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   cudaStream_t a = t->timing ? s : t->aux_stream;
   if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_keys, 0));
   // (nobody reads the per-call set after the key-store work: its primary tier is wiped beside the rest)
-  LAUNCH_ON(t, a, K_CLEAR, clear_primary_kernel<<<g8, 256, 0, a>>>(wk));
-  LAUNCH_ON(t, a, K_EXPAND, expand_parts_kernel<<<g8 * 4, 128, 0, a>>>(tv, wk));
-  LAUNCH_ON(t, a, K_ORDER, order_parts_kernel<<<64, kWindows, 0, a>>>(tv, wk));
+  LAUNCH_ON(t, a, K_CLEAR, launch_after(clear_primary_kernel, g8, 256, a, wk));
+  LAUNCH_ON(t, a, K_EXPAND, launch_after(expand_parts_kernel, g8 * 4, 128, a, tv, wk));
+  LAUNCH_ON(t, a, K_ORDER, launch_after(order_parts_kernel, 64, kWindows, a, tv, wk));
   CUDA_TRY(t, cudaGetLastError());
   if (a != s) CUDA_TRY(t, cudaEventRecord(t->ev_parts, a));
   if (grad_ready) CUDA_TRY(t, cudaStreamWaitEvent(s, grad_ready, 0));
   const int rc = dispatch_dim(tv.dim, [&](auto g, auto nv) -> int {
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
-    LAUNCH(t, K_REDUCE, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceShort));
+    LAUNCH(t, K_REDUCE, launch_after(reduce_adagrad_kernel<G, NV>, g8 * 8, 128, s, tv, wk, grad, n_bags, kReduceShort));
     if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_parts, 0));
-    LAUNCH(t, K_REDUCE_PARTS, reduce_adagrad_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags, kReduceParts));
+    LAUNCH(t, K_REDUCE_PARTS, launch_after(reduce_adagrad_kernel<G, NV>, g8 * 8, 128, s, tv, wk, grad, n_bags, kReduceParts));
     if (a != s) {
       CUDA_TRY(t, cudaEventRecord(t->ev_reduced, s));
       CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_reduced, 0));
     }
-    LAUNCH(t, K_SINGLES, update_singletons_kernel<G, NV><<<g8 * 8, 128, 0, s>>>(tv, wk, grad, n_bags));
+    LAUNCH(t, K_SINGLES, launch_after(update_singletons_kernel<G, NV>, g8 * 8, 128, s, tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
-  LAUNCH_ON(t, a, K_FOLD, fold_partials_kernel<<<g4, 256, 0, a>>>(tv, wk));
-  LAUNCH_ON(t, a, K_COMBINE, combine_adagrad_kernel<<<g8, kCombineThreads, 0, a>>>(tv, wk));
+  LAUNCH_ON(t, a, K_FOLD, launch_after(fold_partials_kernel, g4, 256, a, tv, wk));
+  LAUNCH_ON(t, a, K_COMBINE, launch_after(combine_adagrad_kernel, g8, kCombineThreads, a, tv, wk));
   if (a != s) {
     CUDA_TRY(t, cudaEventRecord(t->ev_aux, a));
     CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_aux, 0));
   }
-  LAUNCH(t, K_FINISH, finish_apply_kernel<<<1, 256, 0, s>>>(tv.st, wk.win_count, 1));
+  LAUNCH(t, K_FINISH, launch_after(finish_apply_kernel, 1, 256, s, tv.st, wk.win_count, 1));
   CUDA_TRY(t, cudaGetLastError());
   t->keys_idle = true;
   return MONO_OK;
@@ -583,7 +606,7 @@ int group_upload(GroupPlan& p, mono_table* const* tables) {
   do {                                                                                                    \
     if ((p).grid(gk) > 0) {                                                                               \
       ++(p).owner->launches[kid];                                                                         \
-      kernel<<<(p).grid(gk), (threads), 0, (p).gs>>>((p).d_items, (p).map(gk), (uint32_t)(p).n);           \
+      launch_after(kernel, (p).grid(gk), (threads), (p).gs, (p).d_items, (p).map(gk), (uint32_t)(p).n);    \
     }                                                                                                     \
   } while (0)
 
@@ -864,7 +887,7 @@ int mono_group_apply_grads(int32_t n_tables, mono_table* const* tables, const ui
   GROUP_LAUNCH(p, K_FOLD, GK_FOLD, 256, group_fold_partials_kernel);
   GROUP_LAUNCH(p, K_COMBINE, GK_COMBINE, kCombineThreads, group_combine_adagrad_kernel);
   ++p.owner->launches[K_FINISH];
-  group_finish_apply_kernel<<<(unsigned)n_tables, 256, 0, p.gs>>>(p.d_items, (uint32_t)n_tables, 1);
+  launch_after(group_finish_apply_kernel, (unsigned)n_tables, 256, p.gs, p.d_items, (uint32_t)n_tables, 1);
   CUDA_TRY(p.owner, cudaGetLastError());
   for (int32_t i = 0; i < n_tables; ++i) tables[i]->prep.valid = false;
   return group_end(p, tables);
@@ -906,9 +929,9 @@ static int expire_range(mono_table* t, int64_t now, uint32_t slice, uint32_t n_s
     unsigned long long blocks = (last - first + per_block - 1) / per_block;
     if (blocks < 1) blocks = 1;
     if (blocks > (unsigned long long)grid_for(t, 8)) blocks = grid_for(t, 8);
-    LAUNCH_ON(t, s, K_EXPIRE, expire_kernel<<<(int)blocks, 256, 0, s>>>(t->tv, first, last, is_last ? 1 : 0, (long long)now));
+    LAUNCH_ON(t, s, K_EXPIRE, launch_after(expire_kernel, (int)blocks, 256, s, t->tv, first, last, is_last ? 1 : 0, (long long)now));
   }
-  if (slice + 1 == n_slices) LAUNCH_ON(t, s, K_STASH_TRIM, stash_trim_kernel<<<1, 32, 0, s>>>(t->tv));
+  if (slice + 1 == n_slices) LAUNCH_ON(t, s, K_STASH_TRIM, launch_after(stash_trim_kernel, 1, 32, s, t->tv));
   CUDA_TRY(t, cudaGetLastError());
   CUDA_TRY(t, cudaEventRecord(t->ev_swept, s));
   t->sweep_pending = true;

@@ -124,6 +124,18 @@ struct DevState {
 #define MONO_INDEX_OK(error_bits, i, n) true
 #endif
 
+// First statement of every kernel of the hot path.  These kernels are launched with programmatic
+// stream serialisation, which lets the launch of a kernel be prepared while the kernel before it
+// on the stream is still running; the kernel waits here until that one has completed and its
+// writes are visible, and reads or writes nothing before.  Launched in the ordinary way this is
+// a no-op.  (No kernel releases its successor early: with the successor's blocks placed beside a
+// kernel's last wave, and idle there, the largest configuration measured 0.5 % slower than with
+// ordinary launches; with the wait alone it is 1.2 % faster, and 6-9 % on the configurations
+// whose kernels are short.)
+__device__ __forceinline__ void after_previous_kernel() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Everything a kernel needs to know about a table; passed by value.
 struct TableView {
   Cell* cells;                 // [n_buckets * 4]
