@@ -187,6 +187,10 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
       low = c < tv.threshold ? (uint32_t)c : tv.threshold;
       need_row = low >= tv.threshold;
     }
+    // exact filter: a new ID that this batch alone takes to the threshold gets its row here too, so
+    // that the insertion that follows has nothing to tell the kernels that update rows
+    const bool exact = tv.sketch_depth == 0;
+    if ((MODE & kCommit) && exact && active && !hit && m >= tv.threshold) need_row = true;
     const Reservation rv = block_reserve(tv, &sh, need_row, (MODE & kLookUp) && m > 1, (MODE & kCommit) && active && !hit,
                                          ((MODE & kLookUp) && m > 1) ? m : 0u);
     if (!active) continue;
@@ -211,8 +215,16 @@ __device__ inline void table_update_body(const TableView& tv, const Work& wk, ui
           ++n_res;
           if (m > kSegChunk) register_long(tv, wk, u, m);
         }
-      } else if (MONO_INDEX_OK(wk.error_bits, rv.ins_pos, wk.max_ids)) {
-        wk.ins_list[rv.ins_pos] = u;
+      } else {
+        if (exact) {
+          const uint32_t row_word = rv.row != kNoRow ? (rv.row | kFreshBit) : kNoRow;
+          wk.urow[u] = row_word;
+          if (row_word != kNoRow) {
+            ++n_res;
+            if (m > kSegChunk) register_long(tv, wk, u, m);
+          }
+        }
+        if (MONO_INDEX_OK(wk.error_bits, rv.ins_pos, wk.max_ids)) wk.ins_list[rv.ins_pos] = u;
       }
     }
   }
@@ -325,39 +337,44 @@ __device__ inline void sketch_add_body(const TableView& tv, const Work& wk, uint
 __global__ void __launch_bounds__(256)
 sketch_add_kernel(TableView tv, Work wk) { after_previous_kernel(); sketch_add_body(tv, wk, blockIdx.x, gridDim.x); }
 
-// Phase 3 of a push: one thread per ID that phase 2 found unknown to
-// the key store.  Exact filter: it is inserted (with a row straight away when
-// the batch alone reaches the threshold).  Probabilistic filter: it is inserted,
-// with a row, only if its sketch estimate has reached the threshold; otherwise
-// nothing is stored for it.
+// Phase 3 of a push: one thread per ID that phase 2 found unknown to the key store.
+// Exact filter: it is inserted; whether it has a row straight away (the batch alone reached
+// the threshold) was settled in phase 2, which left the row in urow[], so nothing that
+// updates rows waits for this kernel.  Probabilistic filter: it is inserted, with a row,
+// only if its sketch estimate has reached the threshold; otherwise nothing is stored for it.
 __device__ inline void table_insert_body(const TableView& tv, const Work& wk, uint32_t now, uint32_t vblock, uint32_t vgrid) {
   __shared__ BlockAlloc sh;
   const uint32_t n = tv.st->n_insert;
   const int lane = threadIdx.x & 31;
+  const bool sketch = tv.sketch_depth != 0;
   unsigned int n_res = 0, n_done = 0;
   for (uint32_t base = vblock * blockDim.x; base < n; base += vgrid * blockDim.x) {   // block-uniform
     const bool todo = base + threadIdx.x < n;
     uint32_t u = 0, m = 0;
     if (todo) { u = wk.ins_list[base + threadIdx.x]; m = wk.ulen[u]; }
-    const bool sketch = tv.sketch_depth != 0;
     uint32_t count = m < tv.threshold ? m : tv.threshold;
-    if (sketch && todo) {
-      const unsigned int est = tv.sketch_estimate(wk.uid[u]);
-      count = est < tv.threshold ? est : tv.threshold;
+    uint32_t row_word = kNoRow;
+    if (sketch) {
+      if (todo) {
+        const unsigned int est = tv.sketch_estimate(wk.uid[u]);
+        count = est < tv.threshold ? est : tv.threshold;
+      }
+      const bool need_row = todo && count >= tv.threshold;
+      const Reservation rv = block_reserve(tv, &sh, need_row, false, false, 0u);
+      if (!todo) continue;
+      if (rv.row != kNoRow) row_word = rv.row | kFreshBit;
+      wk.urow[u] = row_word;
+      if (row_word != kNoRow) {
+        ++n_res;
+        if (m > kSegChunk) register_long(tv, wk, u, m);
+      }
+      if (row_word == kNoRow) continue;                // below the estimate (or no row left): not stored
+    } else {
+      if (!todo) continue;
+      row_word = wk.urow[u];
     }
-    const bool need_row = todo && count >= tv.threshold;
-    const Reservation rv = block_reserve(tv, &sh, need_row, false, false, 0u);
-    if (!todo) continue;
-    const unsigned long long id = wk.uid[u];
-    uint32_t low = count, row_word = kNoRow;
-    if (rv.row != kNoRow) { low = kResidentBit | kTouchedBit | rv.row; row_word = rv.row | kFreshBit; }
-    wk.urow[u] = row_word;
-    if (row_word != kNoRow) {
-      ++n_res;
-      if (m > kSegChunk) register_long(tv, wk, u, m);
-    }
-    if (sketch && row_word == kNoRow) continue;      // below the estimate (or no row left): not stored
-    Cell item; item.key = id; item.meta = make_meta(now, low);
+    const uint32_t low = row_word != kNoRow ? (kResidentBit | kTouchedBit | (row_word & ~kFreshBit)) : count;
+    Cell item; item.key = wk.uid[u]; item.meta = make_meta(now, low);
     cuckoo_insert(tv, item);
     ++n_done;
   }

@@ -60,7 +60,7 @@ struct mono_table {
   // the large ones (see launch_apply).
   cudaStream_t aux_stream = nullptr;
   cudaEvent_t ev_aux = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_keys = nullptr, ev_swept = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_keys = nullptr, ev_swept = nullptr, ev_commit = nullptr;
   cudaEvent_t ev_group = nullptr;  // grouped calls: the group's start (first table's), this table's end
   bool sweep_pending = false;     // the sweep stream has work `stream` has not waited for yet
   bool keys_idle = false;         // nothing launched on `stream` after ev_keys touches the key store
@@ -384,20 +384,35 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
     LAUNCH(t, K_UPDATE, launch_after(table_update_kernel<kLookUp | kCommit>, g8 * 4, 256, s, tv, wk, now));
     LAUNCH(t, K_FILE, launch_after(file_segments_kernel, g8, 256, s, wk, n_ids, n_bags, nullptr, 0u));
   }
-  if (tv.sketch_depth) LAUNCH(t, K_SKETCH, launch_after(sketch_add_kernel, g8, 256, s, tv, wk));
-  LAUNCH(t, K_INSERT, launch_after(table_insert_kernel, g8, 256, s, tv, wk, now));
-  CUDA_TRY(t, cudaGetLastError());
-  // the rest of the call touches rows and scratch only: a sweep may run beside it
-  CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
   // The long segments (the few hottest IDs) are reduced on a stream of their own -- expand,
   // order, the parts, fold, combine, one after the other with no event in between -- beside
   // the kernels that work through the rest of the batch on the table's stream: the reduction
   // of the short segments and update_singletons.  The two chains touch different rows and meet
   // again before the call's last kernel (measured 0.9 % of a step faster than the parts on the
-  // table's stream between two event waits).
+  // table's stream between two event waits).  With the exact filter the insertion of the new
+  // IDs runs on a third stream beside both: their rows were settled by the commit half, so the
+  // row updates do not wait for it.  With the probabilistic filter it is the insertion that
+  // decides the rows, and it stays on the table's stream.
   // While kernels are being timed one by one, everything stays on the table's stream.
   cudaStream_t a = t->timing ? s : t->aux_stream;
-  if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_keys, 0));
+  const bool insert_aside = a != s && tv.sketch_depth == 0;
+  if (insert_aside) {
+    // (on the stream the sweep uses: a sweep slice that follows this call follows the insertions)
+    cudaStream_t k = t->sweep_stream;
+    CUDA_TRY(t, cudaEventRecord(t->ev_commit, s));
+    CUDA_TRY(t, cudaStreamWaitEvent(k, t->ev_commit, 0));
+    CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_commit, 0));
+    LAUNCH_ON(t, k, K_INSERT, launch_after(table_insert_kernel, g8, 256, k, tv, wk, now));
+    CUDA_TRY(t, cudaGetLastError());
+    // the rest of the call touches rows and scratch only: a sweep may run beside it
+    CUDA_TRY(t, cudaEventRecord(t->ev_keys, k));
+  } else {
+    if (tv.sketch_depth) LAUNCH(t, K_SKETCH, launch_after(sketch_add_kernel, g8, 256, s, tv, wk));
+    LAUNCH(t, K_INSERT, launch_after(table_insert_kernel, g8, 256, s, tv, wk, now));
+    CUDA_TRY(t, cudaGetLastError());
+    CUDA_TRY(t, cudaEventRecord(t->ev_keys, s));
+    if (a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, t->ev_keys, 0));
+  }
   // (nobody reads the per-call set after the key-store work: its primary tier is wiped beside the rest)
   LAUNCH_ON(t, a, K_CLEAR, launch_after(clear_primary_kernel, g8, 256, a, wk));
   LAUNCH_ON(t, a, K_EXPAND, launch_after(expand_parts_kernel, g8 * 4, 128, a, tv, wk));
@@ -419,6 +434,7 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
     CUDA_TRY(t, cudaEventRecord(t->ev_aux, a));
     CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_aux, 0));
   }
+  if (insert_aside) CUDA_TRY(t, cudaStreamWaitEvent(s, t->ev_keys, 0));
   LAUNCH(t, K_FINISH, launch_after(finish_apply_kernel, 1, 256, s, tv.st, wk.win_count, 1));
   CUDA_TRY(t, cudaGetLastError());
   t->keys_idle = true;
@@ -647,7 +663,7 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
   if (cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaStreamCreateWithFlags(&t->aux_stream, cudaStreamNonBlocking) != cudaSuccess)
     return fail(MONO_ERR_CUDA);
-  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_aux})
+  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_aux, &t->ev_commit})
     if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return fail(MONO_ERR_CUDA);
 
   TableView& tv = t->tv;
@@ -704,7 +720,7 @@ int mono_table_destroy(mono_table* t) {
   if (t->h2d_stream) { cudaStreamSynchronize(t->h2d_stream); cudaStreamDestroy(t->h2d_stream); }
   if (t->d2h_stream) { cudaStreamSynchronize(t->d2h_stream); cudaStreamDestroy(t->d2h_stream); }
   for (cudaEvent_t e : {t->ev_staged, t->ev_grad_in, t->ev_out, t->ev_d2h, t->ev_stage_free}) if (e) cudaEventDestroy(e);
-  for (cudaEvent_t e : {t->ev_fork, t->ev_keys, t->ev_swept, t->ev_group, t->ev_aux})
+  for (cudaEvent_t e : {t->ev_fork, t->ev_keys, t->ev_swept, t->ev_group, t->ev_aux, t->ev_commit})
     if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
