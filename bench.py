@@ -426,6 +426,11 @@ def run_ours(args):
         ids, off, grad = dev_batches[i]
         if prepare and args.prepare:
             mb.mono_prepare_push(table.handle, ids, ids.numel(), off, cfg.n_bags)
+            if args.group_ahead and i + 1 < len(dev_batches):
+                # the next step's batch is grouped by ID beside this step's lookup and push (issued here, it
+                # measured 1.0 % of a step faster than without; issued after the lookup, 0.3 %)
+                nxt = dev_batches[i + 1]
+                mb.mono_group_ahead(table.handle, nxt[0], nxt[0].numel(), nxt[1], cfg.n_bags)
         mb.mono_lookup_pool(table.handle, ids, ids.numel(), off, cfg.n_bags, out)
         mb.mono_apply_grads(table.handle, ids, ids.numel(), off, cfg.n_bags, grad, now0 + 1 + i)
         if S > 0:
@@ -596,6 +601,8 @@ def run_ours(args):
                             "entered_key_store_per_step": (st_b["n_inserted_total"] - st_a["n_inserted_total"]) / K}),
                 "push_prepared": ("mono_prepare_push before each lookup: the batch is grouped and every distinct ID "
                                   "looked up once, for the lookup and the push together" if args.prepare else "no"),
+                "grouped_ahead": ("mono_group_ahead: each step groups the next step's batch by ID on a stream of its own, "
+                                  "beside its own lookup and push" if args.prepare and args.group_ahead else "no"),
             },
             "bags_per_s": world * cfg.n_bags * K / (ms_max * 1e-3),
             "gpu_launches": launches,
@@ -835,6 +842,8 @@ def main():
                          "calls table after table), or single-table calls with every table on a stream of its own")
     ap.add_argument("--no-prepare", dest="prepare", action="store_false",
                     help="do not announce each batch with mono_prepare_push before its lookup")
+    ap.add_argument("--no-group-ahead", dest="group_ahead", action="store_false",
+                    help="do not group the next step's batch with mono_group_ahead beside the current step")
     ap.add_argument("--sweep-slices", type=int, default=32,
                     help="every step sweeps 1/S of the key store for expired IDs (0 = no sweep)")
     ap.add_argument("--filter", default="exact", choices=["exact", "sketch"],

@@ -266,6 +266,23 @@ int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const i
                       int64_t n_bags);
 
 /*
+ * Optional, one step further ahead: groups the occurrences of a batch by ID -- the part of
+ * mono_prepare_push that needs nothing from the table -- on an internal stream, beside whatever
+ * the table's stream is doing (typically the push of the batch before).  It starts once the work
+ * the table's stream holds at the time of the call is done, so `ids` and `slot_offsets` may be
+ * produced on that stream; like an announced batch they must stay unchanged until the push.  A
+ * later mono_prepare_push with exactly these arguments takes the grouping over and only looks the
+ * distinct IDs up; with other arguments it groups its batch itself and the grouping made ahead
+ * stays for a later call.  One batch can be grouped ahead at a time: a second call forgets the
+ * first.  Neither the table nor a batch that was announced is touched, and results are the same
+ * with or without this call.  The first call allocates a second copy of the scratch the grouping
+ * fills (about 70 bytes per ID of max_ids).  Errors: as mono_prepare_push; malformed offsets show
+ * in the status once the batch is taken over.
+ */
+int mono_group_ahead(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets,
+                     int64_t n_bags);
+
+/*
  * Grouped calls: one call, and one kernel launch per step of the path, for several tables
  * (Section 3.1: a production model holds many embedding tables of very uneven size, most of
  * them far too small to fill a GPU on their own).  Table i gets batch i: `tables`, `ids`,

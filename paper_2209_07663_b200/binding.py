@@ -29,7 +29,7 @@ EXPORTS = [
     "mono_table_create", "mono_table_destroy", "mono_reserve", "mono_lookup_pool", "mono_apply_grads",
     "mono_expire", "mono_lookup_pool_host", "mono_apply_grads_host", "mono_status", "mono_clear_errors",
     "mono_probe", "mono_read_rows", "mono_export", "mono_import", "mono_audit", "mono_last_cuda_error",
-    "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc", "mono_export_touched", "mono_rehash", "mono_expire_slice", "mono_prepare_push",
+    "mono_error_string", "mono_timing_enable", "mono_timing_read", "mono_lookup_pool_noalloc", "mono_export_touched", "mono_rehash", "mono_expire_slice", "mono_prepare_push", "mono_group_ahead",
     "mono_group_lookup_pool", "mono_group_apply_grads", "mono_group_prepare_push", "mono_fence", "mono_snapshot_save", "mono_snapshot_restore",
     "mono_snapshot_drop",
 ]
@@ -102,6 +102,7 @@ def load_library(path: Optional[str] = None):
         "mono_apply_grads": (ci, [vp, vp, i64, vp, i64, vp, i64]),
         "mono_expire": (ci, [vp, i64]),
         "mono_prepare_push": (ci, [vp, vp, i64, vp, i64]),
+        "mono_group_ahead": (ci, [vp, vp, i64, vp, i64]),
         "mono_expire_slice": (ci, [vp, i64, u32, u32]),
         "mono_group_prepare_push": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp]),
         "mono_group_lookup_pool": (ci, [ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp]),
@@ -211,6 +212,10 @@ def mono_apply_grads(t: int, ids, n_ids: int, slot_offsets, n_bags: int, grad_po
 
 def mono_expire(t: int, now: int) -> None:
     _check("mono_expire", load_library().mono_expire(t, now), t)
+
+
+def mono_group_ahead(t: int, ids, n_ids: int, slot_offsets, n_bags: int) -> None:
+    _check("mono_group_ahead", load_library().mono_group_ahead(t, _ptr(ids), n_ids, _ptr(slot_offsets), n_bags), t)
 
 
 def mono_prepare_push(t: int, ids, n_ids: int, slot_offsets, n_bags: int) -> None:

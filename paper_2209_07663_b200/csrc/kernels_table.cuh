@@ -596,6 +596,19 @@ expire_kernel(TableView tv, unsigned long long first_bkt, unsigned long long las
   expire_body(tv, first_bkt, last_bkt, with_stash != 0, now, blockIdx.x, gridDim.x);
 }
 
+// A batch that was grouped beside the table's other work is taken over: the counters its
+// grouping left in a block of their own become the call's counters.
+__global__ void adopt_group_kernel(DevState* st, DevState* side) {
+  after_previous_kernel();
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    st->n_unique = side->n_unique;
+    st->n_valid_ids = side->n_valid_ids;
+    st->call_bad_offsets = side->call_bad_offsets;
+    if (side->error_bits) atomicOr(&st->error_bits, side->error_bits);
+    side->n_unique = 0; side->n_valid_ids = 0; side->call_bad_offsets = 0; side->error_bits = 0;
+  }
+}
+
 // After a sweep: if the stash has become empty, probes may skip it again.
 __global__ void stash_trim_kernel(TableView tv) { after_previous_kernel();
   if (threadIdx.x == 0 && blockIdx.x == 0) {

@@ -32,14 +32,14 @@ static __device__ __align__(256) uint32_t g_noalloc_occ_row[MONO_NOALLOC_MAX_IDS
 
 enum KernelId {
   K_PROBE, K_GATHER, K_FILL_BAG, K_DEDUP, K_LOOKUP, K_UPDATE, K_SKETCH, K_INSERT, K_EXPAND, K_ORDER, K_FILE, K_SINGLES, K_REDUCE, K_FOLD, K_COMBINE, K_FINISH, K_EXPIRE,
-  K_STASH_TRIM, K_CLEAR, K_REDUCE_PARTS, K_COUNT
+  K_STASH_TRIM, K_CLEAR, K_REDUCE_PARTS, K_ADOPT, K_COUNT
 };
 // (table_lookup and table_update are the two halves of table_update_kernel; a push that was not
 // announced runs both in one launch, counted as table_update)
 static const char* const kKernelNames[K_COUNT] = {
   "probe_rows", "gather_pool", "fill_occ_bag", "dedup_tile", "table_lookup", "table_update", "sketch_add", "table_insert", "expand_parts", "order_parts",
   "file_segments", "update_singletons", "reduce_adagrad", "fold_partials", "combine_adagrad",
-  "finish_apply", "expire", "stash_trim", "clear_set", "reduce_parts"
+  "finish_apply", "expire", "stash_trim", "clear_set", "reduce_parts", "adopt_group"
 };
 static_assert(K_COUNT <= MONO_MAX_KERNELS, "mono_timing_t has room for MONO_MAX_KERNELS kernels");
 
@@ -67,6 +67,20 @@ struct mono_table {
   // The batch mono_prepare_push announced: grouped and looked up, waiting for its push.
   // filed: its lookup has run too, so every occurrence's bag is in bag_of_sorted[] already.
   struct { const void* ids; int64_t n_ids; const void* off; int64_t n_bags; bool valid; bool filed; } prep = {nullptr, 0, nullptr, 0, false, false};
+  // The batch mono_group_ahead grouped beside the table's other work: a second copy of the scratch
+  // that the grouping fills (the per-call set, the per-occurrence records, the list of distinct
+  // IDs) and of the per-call counters, which mono_prepare_push of the same batch swaps in.
+  struct {
+    BatchSlot* bset = nullptr; uint2* occ = nullptr; uint32_t* occ_bag = nullptr;
+    unsigned long long* uid = nullptr; uint32_t* uslot = nullptr; uint32_t* uocc = nullptr;
+    DevState* st = nullptr;
+    const void* ids = nullptr; int64_t n_ids = 0; const void* off = nullptr; int64_t n_bags = 0;
+    bool valid = false;           // holds a grouped batch that no mono_prepare_push has taken yet
+  } ahead;
+  cudaStream_t ahead_stream = nullptr;
+  cudaEvent_t ev_ahead = nullptr;   // the grouping on ahead_stream is done
+  cudaEvent_t ev_swap = nullptr;    // what `stream` held when mono_group_ahead was called: the batch's arrays are
+                                    // ready, and the copy of the scratch handed back at the last exchange is let go of
   uint32_t* occ_row = nullptr;    // scratch of the two-kernel lookup: row of every occurrence
   int device = 0;                 // the device the table lives on
   uint64_t scratch_reallocs = 0;  // times a hot call had to grow the scratch
@@ -148,6 +162,9 @@ void free_scratch(mono_table* t) {
   dev_free(w.uid); dev_free(w.uslot); dev_free(w.uocc); dev_free(w.useg); dev_free(w.ulen); dev_free(w.urow); dev_free(w.ucell); dev_free(w.umeta);
   dev_free(w.multi_list); dev_free(w.ins_list); dev_free(w.long_u); dev_free(w.long_part0); dev_free(w.part_u); dev_free(w.part_order); dev_free(w.win_count); dev_free(w.partials); dev_free(w.fold_li); dev_free(w.fold_idx);
   dev_free(t->stage_ids); dev_free(t->stage_off); dev_free(t->stage_out); dev_free(t->stage_grad); dev_free(t->occ_row);
+  auto& ah = t->ahead;
+  dev_free(ah.bset); dev_free(ah.occ); dev_free(ah.occ_bag); dev_free(ah.uid); dev_free(ah.uslot); dev_free(ah.uocc); dev_free(ah.st);
+  ah.valid = false;
   t->staged.valid = false;
   t->max_ids = t->max_bags = 0;
 }
@@ -232,6 +249,7 @@ int reserve(mono_table* t, int64_t max_ids, int64_t max_bags) {
   if (max_bags < 1024) max_bags = 1024;
   if (t->max_ids > 0) ++t->scratch_reallocs;               // (the first sizing of a table created without one is not a regrowth)
   CUDA_TRY(t, cudaStreamSynchronize(t->stream));
+  if (t->ahead_stream) CUDA_TRY(t, cudaStreamSynchronize(t->ahead_stream));  // a grouping in flight uses the second copy
   if (t->h2d_stream) CUDA_TRY(t, cudaStreamSynchronize(t->h2d_stream));      // copies in flight use the staging buffers
   if (t->d2h_stream) CUDA_TRY(t, cudaStreamSynchronize(t->d2h_stream));
   t->d2h_pending = false;
@@ -341,12 +359,13 @@ int launch_lookup(mono_table* t, const unsigned long long* ids, int64_t n_ids, c
 // The part of a push that depends on the IDs alone: bag of every occurrence, and the
 // occurrences grouped by ID in the per-call set.
 int launch_group(mono_table* t, cudaStream_t s, const unsigned long long* ids, int64_t n_ids, const long long* off,
-                 int64_t n_bags) {
+                 int64_t n_bags, const Work* into = nullptr, DevState* counters = nullptr) {
   const TableView& tv = t->tv;
-  const Work& wk = t->wk;
-  LAUNCH_ON(t, s, K_FILL_BAG, launch_after(fill_occ_bag_kernel, grid_for(t, 8), 256, s, off, n_bags, n_ids, wk.occ_bag, tv.st));
+  const Work& wk = into ? *into : t->wk;
+  DevState* st = counters ? counters : tv.st;
+  LAUNCH_ON(t, s, K_FILL_BAG, launch_after(fill_occ_bag_kernel, grid_for(t, 8), 256, s, off, n_bags, n_ids, wk.occ_bag, st));
   const int tiles = (int)((n_ids + kTileIds - 1) / kTileIds);
-  LAUNCH_ON(t, s, K_DEDUP, launch_after(dedup_tile_kernel, tiles, kTileThreads, s, wk, ids, n_ids, off, n_bags, tv.st,
+  LAUNCH_ON(t, s, K_DEDUP, launch_after(dedup_tile_kernel, tiles, kTileThreads, s, wk, ids, n_ids, off, n_bags, st,
                                                                           tv.seed0 ^ 0xA5A5A5A55A5A5A5Aull));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
@@ -355,8 +374,21 @@ int launch_group(mono_table* t, cudaStream_t s, const unsigned long long* ids, i
 // mono_prepare_push: group the batch and look every distinct ID up once, for the lookup and the
 // push of this batch together.  Nothing in the table changes.
 int launch_prepare(mono_table* t, const unsigned long long* ids, int64_t n_ids, const long long* off, int64_t n_bags) {
-  int rc = launch_group(t, t->stream, ids, n_ids, off, n_bags);
-  if (rc != MONO_OK) return rc;
+  auto& ah = t->ahead;
+  if (ah.valid && ah.ids == ids && ah.n_ids == n_ids && ah.off == off && ah.n_bags == n_bags) {
+    // grouped already, beside the table's other work: the two copies of the grouping scratch change
+    // places, and the counters the grouping left come over
+    ah.valid = false;
+    CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_ahead, 0));        // (recorded when the grouping ran on a stream of its own)
+    Work& w = t->wk;
+    std::swap(w.bset, ah.bset); std::swap(w.occ, ah.occ); std::swap(w.occ_bag, ah.occ_bag);
+    std::swap(w.uid, ah.uid); std::swap(w.uslot, ah.uslot); std::swap(w.uocc, ah.uocc);
+    LAUNCH(t, K_ADOPT, launch_after(adopt_group_kernel, 1, 32, t->stream, t->tv.st, ah.st));
+    CUDA_TRY(t, cudaGetLastError());
+  } else {
+    const int rc = launch_group(t, t->stream, ids, n_ids, off, n_bags);
+    if (rc != MONO_OK) return rc;
+  }
   LAUNCH(t, K_LOOKUP, launch_after(table_update_kernel<kLookUp>, grid_for(t, 8) * 4, 256, t->stream, t->tv, t->wk, 0u));
   CUDA_TRY(t, cudaGetLastError());
   return MONO_OK;
@@ -661,9 +693,10 @@ int mono_table_create(mono_table** out, uint64_t capacity, uint32_t dim, uint32_
     return fail(MONO_ERR_CUDA);
   t->device = dev;
   if (cudaStreamCreateWithFlags(&t->sweep_stream, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&t->aux_stream, cudaStreamNonBlocking) != cudaSuccess)
+      cudaStreamCreateWithFlags(&t->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&t->ahead_stream, cudaStreamNonBlocking) != cudaSuccess)
     return fail(MONO_ERR_CUDA);
-  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_aux, &t->ev_commit})
+  for (cudaEvent_t* e : {&t->ev_fork, &t->ev_keys, &t->ev_swept, &t->ev_group, &t->ev_aux, &t->ev_commit, &t->ev_ahead, &t->ev_swap})
     if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return fail(MONO_ERR_CUDA);
 
   TableView& tv = t->tv;
@@ -717,10 +750,11 @@ int mono_table_destroy(mono_table* t) {
   cudaStreamSynchronize(t->stream);
   if (t->sweep_stream) { cudaStreamSynchronize(t->sweep_stream); cudaStreamDestroy(t->sweep_stream); }
   if (t->aux_stream) { cudaStreamSynchronize(t->aux_stream); cudaStreamDestroy(t->aux_stream); }
+  if (t->ahead_stream) { cudaStreamSynchronize(t->ahead_stream); cudaStreamDestroy(t->ahead_stream); }
   if (t->h2d_stream) { cudaStreamSynchronize(t->h2d_stream); cudaStreamDestroy(t->h2d_stream); }
   if (t->d2h_stream) { cudaStreamSynchronize(t->d2h_stream); cudaStreamDestroy(t->d2h_stream); }
   for (cudaEvent_t e : {t->ev_staged, t->ev_grad_in, t->ev_out, t->ev_d2h, t->ev_stage_free}) if (e) cudaEventDestroy(e);
-  for (cudaEvent_t e : {t->ev_fork, t->ev_keys, t->ev_swept, t->ev_group, t->ev_aux, t->ev_commit})
+  for (cudaEvent_t e : {t->ev_fork, t->ev_keys, t->ev_swept, t->ev_group, t->ev_aux, t->ev_commit, t->ev_ahead, t->ev_swap})
     if (e) cudaEventDestroy(e);
   for (auto& p : t->pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
   for (cudaEvent_t e : t->spare_events) cudaEventDestroy(e);
@@ -764,6 +798,59 @@ int mono_apply_grads(mono_table* t, const uint64_t* ids, int64_t n_ids, const in
   t->last_now = now;
   return launch_apply(t, reinterpret_cast<const unsigned long long*>(ids), n_ids,
                       reinterpret_cast<const long long*>(slot_offsets), n_bags, grad_pooled, (uint32_t)now);
+}
+
+int mono_group_ahead(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets, int64_t n_bags) {
+  MONO_API_RANGE();
+  int rc = check_batch(t, ids, n_ids, slot_offsets, n_bags);
+  if (rc != MONO_OK) return rc;
+  if ((rc = reserve(t, n_ids, n_bags)) != MONO_OK) return rc;
+  auto& ah = t->ahead;
+  // while kernels are being timed one by one, the grouping runs on the table's stream like everything else
+  cudaStream_t g = t->timing ? t->stream : t->ahead_stream;
+  const Work& w = t->wk;
+  const uint64_t slots = (uint64_t)w.primary_mask + 1 + (uint64_t)w.secondary_mask + 1;
+  // The grouping follows what the table's stream holds so far: whatever fills the batch's arrays,
+  // and the kernels that still use the copy of the scratch handed back at the last exchange.
+  if (g != t->stream) {
+    CUDA_TRY(t, cudaEventRecord(t->ev_swap, t->stream));
+    CUDA_TRY(t, cudaStreamWaitEvent(g, t->ev_swap, 0));
+  }
+  if (!ah.bset) {
+    // the second copy of what the grouping fills, sized like the first
+    const size_t n = (size_t)t->max_ids;
+    int arc = dev_alloc(t, &ah.bset, slots);
+    if (arc == MONO_OK) arc = dev_alloc(t, &ah.occ, n);
+    if (arc == MONO_OK) arc = dev_alloc(t, &ah.occ_bag, n);
+    if (arc == MONO_OK) arc = dev_alloc(t, &ah.uid, n);
+    if (arc == MONO_OK) arc = dev_alloc(t, &ah.uslot, n);
+    if (arc == MONO_OK) arc = dev_alloc(t, &ah.uocc, n);
+    if (arc == MONO_OK) arc = dev_alloc(t, &ah.st, 1);
+    if (arc != MONO_OK) {
+      dev_free(ah.bset); dev_free(ah.occ); dev_free(ah.occ_bag); dev_free(ah.uid); dev_free(ah.uslot); dev_free(ah.uocc); dev_free(ah.st);
+      return arc;
+    }
+    init_bset_kernel<<<grid_for(t, 4), 256, 0, g>>>(ah.bset, slots);
+    CUDA_TRY(t, cudaGetLastError());
+    CUDA_TRY(t, cudaMemsetAsync(ah.st, 0, sizeof(DevState), g));
+    ah.valid = false;
+  }
+  if (ah.valid) {
+    // a batch grouped earlier that was never pushed: forget it
+    ah.valid = false;
+    init_bset_kernel<<<grid_for(t, 4), 256, 0, g>>>(ah.bset, slots);
+    CUDA_TRY(t, cudaGetLastError());
+    CUDA_TRY(t, cudaMemsetAsync(ah.st, 0, sizeof(DevState), g));
+  }
+  if (n_ids == 0 || n_bags == 0) return MONO_OK;
+  Work into = w;
+  into.bset = ah.bset; into.occ = ah.occ; into.occ_bag = ah.occ_bag; into.uid = ah.uid; into.uslot = ah.uslot; into.uocc = ah.uocc;
+  if ((rc = launch_group(t, g, reinterpret_cast<const unsigned long long*>(ids), n_ids,
+                         reinterpret_cast<const long long*>(slot_offsets), n_bags, &into, ah.st)) != MONO_OK) return rc;
+  if (g != t->stream) CUDA_TRY(t, cudaEventRecord(t->ev_ahead, g));
+  ah.ids = ids; ah.n_ids = n_ids; ah.off = slot_offsets; ah.n_bags = n_bags;
+  ah.valid = true;
+  return MONO_OK;
 }
 
 int mono_prepare_push(mono_table* t, const uint64_t* ids, int64_t n_ids, const int64_t* slot_offsets, int64_t n_bags) {
@@ -1410,6 +1497,7 @@ int mono_audit(mono_table* t, mono_audit_t* host_out) {
 
 int mono_timing_enable(mono_table* t, int on) {
   if (!t) return MONO_ERR_ARG;
+  if (t->ahead_stream) cudaStreamSynchronize(t->ahead_stream);     // a grouping in flight keeps the stream it started on
   t->timing = on != 0;
   return MONO_OK;
 }

@@ -50,21 +50,35 @@ def assert_audit_ok(gpu_table, what: str = "audit"):
 
 
 def run_stream(gpu_table, oracle, stream, steps, *, sweep_every: int = 1, check_every: int = 1,
-               time_scale: int = 1, check_forward: bool = True, prepare: bool = False):
+               time_scale: int = 1, check_forward: bool = True, prepare=False):
     """Feed steps [0, steps) of `stream` to both sides; compare as it goes.  With `prepare`
     every batch is announced with mono_prepare_push before its lookup, as a training loop
-    that knows its batch ahead of the pull would do."""
+    that knows its batch ahead of the pull would do; with prepare="ahead" the next batch is also
+    grouped with mono_group_ahead while the current one is being pulled and pushed."""
     import torch
     from paper_2209_07663_b200 import binding as mb
+
+    def device_batch(s):
+        ids = torch.from_numpy(s.ids.view(np.int64)).cuda()
+        off = torch.from_numpy(s.offsets).cuda()
+        return ids, off, torch.from_numpy(s.grad_pooled).cuda()
+
+    ahead = prepare == "ahead"
+    upcoming = None
+    if ahead and steps > 0:
+        upcoming = (stream.step(0),) + device_batch(stream.step(0))
+        mb.mono_group_ahead(gpu_table.handle, upcoming[1], upcoming[1].numel(), upcoming[2], upcoming[2].numel() - 1)
     for t in range(steps):
-        s = stream.step(t)
+        s = upcoming[0] if ahead else stream.step(t)
         now = t * time_scale
         if prepare:
-            ids = torch.from_numpy(s.ids.view(np.int64)).cuda()
-            off = torch.from_numpy(s.offsets).cuda()
-            grad = torch.from_numpy(s.grad_pooled).cuda()
+            ids, off, grad = upcoming[1:] if ahead else device_batch(s)
             n_bags = off.numel() - 1
             mb.mono_prepare_push(gpu_table.handle, ids, ids.numel(), off, n_bags)
+            if ahead and t + 1 < steps:
+                nxt = stream.step(t + 1)
+                upcoming = (nxt,) + device_batch(nxt)
+                mb.mono_group_ahead(gpu_table.handle, upcoming[1], upcoming[1].numel(), upcoming[2], upcoming[2].numel() - 1)
             if check_forward:
                 out = torch.empty((n_bags, gpu_table.dim), dtype=torch.float32, device="cuda")
                 mb.mono_lookup_pool(gpu_table.handle, ids, ids.numel(), off, n_bags, out)

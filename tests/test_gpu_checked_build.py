@@ -27,7 +27,7 @@ def pair(cfg):
     return (mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, key_cells=cfg.key_cells, **kw),
             mo.OracleTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, **kw))
 
-for prepare in (False, True):
+for prepare in (False, True, "ahead"):
     cfg = wl.scaled(wl.CONFIGS["tiny"], steps=12)
     g, c = pair(cfg)
     st = run_stream(g, c, wl.Stream(cfg), cfg.steps, sweep_every=1, check_every=4, prepare=prepare)

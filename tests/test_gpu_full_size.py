@@ -78,14 +78,20 @@ def test_large_config_full_size_sampled_parity():
 
     sample_set = set(sample_ids.tolist())
     out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
+    def on_device(s):
+        return (torch.from_numpy(s.ids.view(np.int64)).cuda(), torch.from_numpy(s.offsets).cuda(),
+                torch.from_numpy(s.grad_pooled).cuda())
+
+    upcoming = on_device(steps[0])
     for t, s in enumerate(steps):
         now = now0 + 1 + t
-        ids = torch.from_numpy(s.ids.view(np.int64)).cuda()
-        off = torch.from_numpy(s.offsets).cuda()
-        grad = torch.from_numpy(s.grad_pooled).cuda()
+        ids, off, grad = upcoming
         # the oracle's view: same bags, IDs outside the sample become padding
         masked = np.where(np.isin(s.ids, sample_ids), s.ids, np.uint64(mb.MONO_RESERVED_ID))
-        mb.mono_prepare_push(gpu.handle, ids, ids.numel(), off, cfg.n_bags)      # as the benchmark does
+        mb.mono_prepare_push(gpu.handle, ids, ids.numel(), off, cfg.n_bags)      # as the benchmark does ...
+        if t + 1 < len(steps):                                                   # ... with the next batch grouped beside this one
+            upcoming = on_device(steps[t + 1])
+            mb.mono_group_ahead(gpu.handle, upcoming[0], upcoming[0].numel(), upcoming[1], cfg.n_bags)
         mb.mono_lookup_pool(gpu.handle, ids, ids.numel(), off, cfg.n_bags, out)
         want = cpu.lookup_pool(masked, s.offsets)
         bags = bags_per_step[t]

@@ -31,7 +31,7 @@ def bags(lists):
 
 # ---------------------------------------------------------------- configured streams
 
-@pytest.mark.parametrize("prepare", [False, True])
+@pytest.mark.parametrize("prepare", [False, True, "ahead"])
 def test_tiny_config_full_stream(prepare):
     cfg = wl.CONFIGS["tiny"]
     gpu, cpu = make_pair(cfg)
@@ -46,7 +46,7 @@ def test_medium_config_prefix():
     run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=4, check_every=4)
 
 
-@pytest.mark.parametrize("prepare", [False, True])
+@pytest.mark.parametrize("prepare", [False, True, "ahead"])
 def test_medium_config_short_ttl_churn(prepare):
     # the medium shape with a TTL short enough that rows are recycled many times
     cfg = wl.scaled(wl.CONFIGS["medium"], steps=10, ttl=2, n_examples=2048, capacity=1 << 18, key_cells=1 << 20)
@@ -55,7 +55,7 @@ def test_medium_config_short_ttl_churn(prepare):
     assert st["n_expired_total"] > 10000
 
 
-@pytest.mark.parametrize("prepare", [False, True])
+@pytest.mark.parametrize("prepare", [False, True, "ahead"])
 def test_drift_config_scaled_down(prepare):
     cfg = wl.scaled(wl.CONFIGS["drift"], n_examples=512, n_slots=10, n_distinct=1 << 18, capacity=1 << 16,
                     key_cells=1 << 18, ttl=6, drift_period=4, steps=16)
@@ -63,7 +63,7 @@ def test_drift_config_scaled_down(prepare):
     run_stream(gpu, cpu, wl.Stream(cfg), cfg.steps, sweep_every=2, check_every=4, prepare=prepare)
 
 
-@pytest.mark.parametrize("prepare", [False, True])
+@pytest.mark.parametrize("prepare", [False, True, "ahead"])
 @pytest.mark.parametrize("dim", [4, 8, 12, 16, 32, 48, 64, 128, 200, 256, 512, 1024])
 def test_every_dim_variant(dim, prepare):
     # bags of 0 to 40 IDs: longer than the widest lane group, so a bag takes several rounds
@@ -328,6 +328,56 @@ def test_prepared_push_gives_the_same_table_as_the_oracle():
 
 def cpu_sum_ids(stream, steps):
     return sum(int((stream.step(t).ids != np.uint64(wl.RESERVED_ID)).sum()) for t in range(steps))
+
+
+def test_grouping_ahead_in_every_order_gives_the_same_table_as_the_oracle():
+    """mono_group_ahead beside the calls of other batches: taken over by the mono_prepare_push of its
+    batch; left alone by a mono_prepare_push or an unannounced push of another batch and taken over
+    later; replaced by a second mono_group_ahead; lost when the scratch grows; never used at all."""
+    cfg = wl.scaled(wl.CONFIGS["tiny"], n_examples=512, steps=14)
+    gpu, cpu = make_pair(cfg)
+    h = gpu.handle
+    stream = wl.Stream(cfg)
+    batches = [stream.step(t) for t in range(cfg.steps + 1)]
+    dev = [(torch.from_numpy(s.ids.view(np.int64)).cuda(), torch.from_numpy(s.offsets).cuda(),
+            torch.from_numpy(s.grad_pooled).cuda()) for s in batches]
+    ahead = lambda k: mb.mono_group_ahead(h, dev[k][0], dev[k][0].numel(), dev[k][1], cfg.n_bags)
+    out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
+    ahead(0)
+    for t in range(cfg.steps):
+        s, (ids, off, grad) = batches[t], dev[t]
+        kind = t % 7
+        if kind == 0:                                     # the plain pipeline
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+            ahead(t + 1)
+        elif kind == 1:                                   # grouped ahead twice: the first is forgotten
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+            ahead(t)
+            ahead(t + 1)
+        elif kind == 2:                                   # another batch announced first: the grouping made ahead waits
+            mb.mono_prepare_push(h, dev[t + 1][0], dev[t + 1][0].numel(), dev[t + 1][1], cfg.n_bags)
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+            ahead(t + 1)
+        elif kind == 3:                                   # pushed without an announcement; batch t's grouping is never used
+            ahead(t + 1)
+        elif kind == 4:                                   # the scratch grows under a grouping made ahead
+            mb.mono_reserve(h, gpu.status()["sum_ids"] // (t + 1) * (3 + t), cfg.n_bags * 2)
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+            ahead(t + 1)
+        elif kind == 5:                                   # a sweep and an empty grouping in between
+            gpu.expire(t - 1); cpu.expire(t - 1)
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+            mb.mono_group_ahead(h, ids, 0, off[:1], 0)
+        else:                                             # nothing grouped ahead for this one
+            mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+            ahead(t + 1)
+        mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
+        assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
+        mb.mono_apply_grads(h, ids, ids.numel(), off, cfg.n_bags, grad, t)
+        assert cpu.apply_grads(s.ids, s.offsets, s.grad_pooled, t) == 0
+        assert_state_equal(gpu, cpu, f"step {t}")
+        assert_audit_ok(gpu, f"step {t}")
+    assert gpu.status()["error_bits"] == 0
 
 
 def test_prepared_push_with_malformed_offsets_is_flagged():
@@ -798,7 +848,7 @@ def _well_formed_only(ids, off):
     return bags(lists)
 
 
-@pytest.mark.parametrize("prepared", [False, True])
+@pytest.mark.parametrize("prepared", [False, True, "ahead"])
 def test_malformed_offsets_empty_the_offending_bags_in_both_directions(prepared):
     kw = dict(init_scale=0.1, seed=5)
     gpu, cpu = mb.MonoTable(64, 4, 1, 0, **kw), mo.OracleTable(64, 4, 1, 0, **kw)
@@ -818,6 +868,9 @@ def test_malformed_offsets_empty_the_offending_bags_in_both_directions(prepared)
         grad_t = torch.from_numpy(grad).cuda()
         o_ids, o_off = _well_formed_only(fresh, off)
         out = torch.empty((4, 4), device="cuda")
+        if prepared == "ahead":                             # grouped beside the table's work: nothing is flagged yet
+            mb.mono_group_ahead(gpu.handle, ids_t, 8, off_t, 4)
+            assert gpu.status()["error_bits"] == 0
         if prepared:
             mb.mono_prepare_push(gpu.handle, ids_t, 8, off_t, 4)
         mb.mono_lookup_pool(gpu.handle, ids_t, 8, off_t, 4, out)
