@@ -386,7 +386,8 @@ int mono_lookup_pool_noalloc(mono_table* t, const uint64_t* ids, int64_t n_ids,
 
 /*
  * Order point for the table's internal streams (the paper has no counterpart).  A hot call may
- * leave work running on streams of the table's own (the sweep of mono_expire*, most of all);
+ * leave work running on streams of the table's own (the sweep of mono_expire*, the grouping of
+ * mono_group_ahead);
  * the next call on the table waits for it by itself.  mono_fence makes the table's stream wait
  * for all of it now, without synchronising the host, so that an event the caller records on
  * the table's stream afterwards marks the end of everything issued so far.

@@ -1196,6 +1196,7 @@ int mono_fence(mono_table* t) {
   if (!t) return MONO_ERR_ARG;
   join_sweep(t);
   if (t->d2h_pending) { CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_d2h, 0)); t->d2h_pending = false; }
+  if (t->ahead.valid) CUDA_TRY(t, cudaStreamWaitEvent(t->stream, t->ev_ahead, 0));     // a batch being grouped ahead
   return MONO_OK;
 }
 
