@@ -53,7 +53,8 @@ def _dev(s):
 
 def test_medium_config_all_200_steps():
     """The whole `medium` stream: 200 steps, a sweep every 10 steps (so the TTL of 100 expires IDs from
-    step 110 on), pooled outputs compared every 20th step, the complete table every 50 steps."""
+    step 110 on), pooled outputs compared every 20th step, the complete table every 50 steps.  Every batch
+    is grouped while the batch before it is pulled and pushed."""
     cfg = wl.CONFIGS["medium"]
     gpu = mb.MonoTable(cfg.capacity, cfg.dim, cfg.filter_threshold, cfg.ttl, key_cells=cfg.key_cells,
                        max_ids=cfg.n_bags * 8, max_bags=cfg.n_bags, **_kw(cfg))
@@ -61,9 +62,18 @@ def test_medium_config_all_200_steps():
     stream = wl.Stream(cfg)
     out = torch.empty((cfg.n_bags, cfg.dim), dtype=torch.float32, device="cuda")
     h = gpu.handle
-    for t, s in enumerate(_steps_ahead(stream, 0, cfg.steps)):
-        ids, off, grad = _dev(s)
+    # as the benchmark runs it: every batch grouped one step ahead, announced, pulled, pushed
+    steps = _steps_ahead(stream, 0, cfg.steps)
+    upcoming = next(steps)
+    upcoming = (upcoming,) + _dev(upcoming)
+    mb.mono_group_ahead(h, upcoming[1], upcoming[1].numel(), upcoming[2], cfg.n_bags)
+    for t in range(cfg.steps):
+        s, ids, off, grad = upcoming
         mb.mono_prepare_push(h, ids, ids.numel(), off, cfg.n_bags)
+        if t + 1 < cfg.steps:
+            upcoming = next(steps)
+            upcoming = (upcoming,) + _dev(upcoming)
+            mb.mono_group_ahead(h, upcoming[1], upcoming[1].numel(), upcoming[2], cfg.n_bags)
         mb.mono_lookup_pool(h, ids, ids.numel(), off, cfg.n_bags, out)
         if t % 20 == 19:
             assert_vectors_close(out.cpu().numpy(), cpu.lookup_pool(s.ids, s.offsets), f"step {t}: pooled output")
