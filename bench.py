@@ -350,6 +350,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
+    if args.stream_priority == "high":
+        torch.cuda.set_stream(torch.cuda.Stream(device=dev, priority=-1))
 
     base = wl.CONFIGS[args.workload]
     cfg = rank_config(base, rank)
@@ -842,6 +844,8 @@ def main():
                          "calls table after table), or single-table calls with every table on a stream of its own")
     ap.add_argument("--no-prepare", dest="prepare", action="store_false",
                     help="do not announce each batch with mono_prepare_push before its lookup")
+    ap.add_argument("--stream-priority", default="default", choices=["default", "high"],
+                    help="priority of the CUDA stream the table is created on (its internal streams have the lowest)")
     ap.add_argument("--no-group-ahead", dest="group_ahead", action="store_false",
                     help="do not group the next step's batch with mono_group_ahead beside the current step")
     ap.add_argument("--sweep-slices", type=int, default=32,
