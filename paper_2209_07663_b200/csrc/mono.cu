@@ -201,9 +201,6 @@ void launch_end(mono_table* t, int kid, cudaStream_t s) {
 // before it other than a kernel (a copy, an event wait) is waited for in the ordinary way.
 template <typename... P, typename... A>
 inline void launch_after(void (*kernel)(P...), unsigned grid, unsigned block, cudaStream_t s, A&&... args) {
-#ifdef MONO_PLAIN_LAUNCH
-  kernel<<<grid, block, 0, s>>>(std::forward<A>(args)...);
-#else
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
   cfg.blockDim = dim3(block, 1, 1);
@@ -215,7 +212,6 @@ inline void launch_after(void (*kernel)(P...), unsigned grid, unsigned block, cu
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
-#endif
 }
 
 // Every kernel of the hot calls is launched through this, so that launches can
