@@ -399,8 +399,10 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
   const TableView& tv = t->tv;
   const Work& wk = t->wk;
   // grids of the grid-stride kernels: several waves of blocks per SM where that measured faster
-  // (shorter tails), one wave elsewhere.  The kernels that update rows run beside one another on
-  // three streams: with four waves each the step measured 1.9 % faster than with eight.
+  // (shorter tails), one wave elsewhere.  The reduction of the short segments runs beside the long
+  // segments' chain and the insertions: with four waves of blocks instead of eight the step measured
+  // 1.9 % faster on the largest configuration (its own time is the same); the parts launch and
+  // update_singletons keep eight.
   const int g4 = grid_for(t, 4), g8 = grid_for(t, 8);
   int rc0 = MONO_OK;
   if (is_prepared_batch(t, ids, n_ids, off, n_bags)) {
@@ -454,8 +456,8 @@ int launch_apply(mono_table* t, const unsigned long long* ids, int64_t n_ids, co
     constexpr int G = decltype(g)::value, NV = decltype(nv)::value;
     LAUNCH(t, K_REDUCE, launch_after(reduce_adagrad_kernel<G, NV>, g8 * 4, 128, s, tv, wk, grad, n_bags, kReduceShort));
     if (grad_ready && a != s) CUDA_TRY(t, cudaStreamWaitEvent(a, grad_ready, 0));
-    LAUNCH_ON(t, a, K_REDUCE_PARTS, launch_after(reduce_adagrad_kernel<G, NV>, g8 * 4, 128, a, tv, wk, grad, n_bags, kReduceParts));
-    LAUNCH(t, K_SINGLES, launch_after(update_singletons_kernel<G, NV>, g8 * 4, 128, s, tv, wk, grad, n_bags));
+    LAUNCH_ON(t, a, K_REDUCE_PARTS, launch_after(reduce_adagrad_kernel<G, NV>, g8 * 8, 128, a, tv, wk, grad, n_bags, kReduceParts));
+    LAUNCH(t, K_SINGLES, launch_after(update_singletons_kernel<G, NV>, g8 * 8, 128, s, tv, wk, grad, n_bags));
     return (int)MONO_OK;
   });
   if (rc != MONO_OK) return rc;
